@@ -1,0 +1,213 @@
+/*
+ * s2moe.h -- C ABI of the B200 (sm_100a) MoE verification layer with reuse-aware
+ * expert gating (S2-MoE, Sec. 4.2) for self-speculative decoding.
+ *
+ * One call verifies one MoE layer for a whole batch or tree of B draft tokens:
+ *
+ *   1. router logits              l_{b,e} = h_b . W_r[e]
+ *   2. reuse-aware expert gating  (Sec. 4.2, Eq. 4 and the two paragraphs after it)
+ *        g_e      = sum_b w_b * l_{b,e}                    cross-token importance
+ *        E*       = the `cap` experts with the largest g_e (ties: lower id)
+ *        lambda_b = alpha * (l_(1) - l_(k+1))              top-1 minus (k+1)-th logit
+ *        l'_{b,e} = l_{b,e} + lambda_b * [e in E*]         soft routing bias
+ *        S_b      = the k experts with the largest l'_{b,e}
+ *                   (ties: larger original logit, then lower id)
+ *        p_{b,e}  = softmax over all E experts of l_b (weight_mode 0) or of l'_b
+ *                   (weight_mode 1), taken at e in S_b, optionally renormalised
+ *   3. union of the batch's choices and the number U of distinct experts
+ *      (the quantity verification cost is proportional to: Sec. 3 "Challenge 2",
+ *      Sec. 4.1 "Routing-aware Cost Estimation"); tokens bucketed by expert
+ *   4. every distinct selected expert's SwiGLU FFN, its weights read from HBM once:
+ *        y_b = sum_{e in S_b} p_{b,e} * W_d[e] ( silu(W_g[e] h_b) .* (W_u[e] h_b) )
+ *            + sum_s c_b * FFN_shared_s(h_b),   c_b = sigmoid(h_b . w_sg) or 1
+ *
+ * The bias is off (standard top-k gating) when alpha == 0, cap >= n_experts or
+ * top_k >= n_experts.  The tree structure of a draft tree is not an argument: the
+ * layer treats tokens independently except through step 2, and ancestry enters only
+ * through the confidences w_b, which the caller computes (Sec. 4.1, prefix
+ * confidence p_i).
+ *
+ * Conventions
+ *   - Every function returns S2MOE_OK (0) or a negative s2moe_status.  No exception
+ *     crosses the boundary and there is no global state.
+ *   - "dev" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *     ordinary host memory.  The library never frees or writes caller weights; it
+ *     borrows the weight pointers for the lifetime of the context.
+ *   - s2moe_verify_layer / s2moe_verify_stack are asynchronous on the given CUDA
+ *     stream (a cudaStream_t passed as void*, NULL = legacy default stream), perform
+ *     no host synchronisation and no allocation, and may be captured in a CUDA graph.
+ *     Outputs are valid once the stream reaches that point.
+ *   - A context may be used by one stream at a time (its workspace is shared by
+ *     calls); it is bound to the device that was current in s2moe_create.
+ *   - All device-side waits are bounded; a wait that gives up stores a non-zero code
+ *     in a device status word that s2moe_last_device_status reads.
+ *
+ * Storage formats (s2moe_dtype)
+ *   S2MOE_F32    IEEE binary32
+ *   S2MOE_BF16   bfloat16
+ *   S2MOE_Q4B32  symmetric block-int4: blocks of 32 weights along the contraction
+ *                (last, contiguous) dimension; 16 bytes per block, weight i of the
+ *                block in nibble i (byte i/2, low nibble for even i) stored as q+8
+ *                with q in [-7,7]; one binary16 scale per block in a separate array;
+ *                value = q * scale.  Weights only (not activations or the router).
+ */
+#ifndef S2MOE_H
+#define S2MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct s2moe_ctx s2moe_ctx;
+
+typedef enum { S2MOE_F32 = 0, S2MOE_BF16 = 1, S2MOE_Q4B32 = 2 } s2moe_dtype;
+
+typedef enum {
+    S2MOE_OK = 0,
+    S2MOE_EINVAL = -1,    /* bad config, shape, null pointer or alignment            */
+    S2MOE_ERANGE = -2,    /* n_tokens > max_tokens, layer index out of range         */
+    S2MOE_ENOMEM = -3,    /* workspace allocation failed                             */
+    S2MOE_ECUDA = -4,     /* a CUDA call failed; see s2moe_last_cuda_error           */
+    S2MOE_ETIMEOUT = -5   /* a bounded device-side wait gave up (device status != 0) */
+} s2moe_status;
+
+#define S2MOE_MAX_TOKENS 64      /* largest draft batch / tree per call       */
+#define S2MOE_MAX_EXPERTS 256    /* largest number of routed experts          */
+#define S2MOE_MAX_TOP_K 16
+
+/* Weights of one layer.  All pointers dev, 16-byte aligned, row-major with the
+ * contraction dimension contiguous. */
+typedef struct {
+    const void *router;    /* [E][d]      router_dtype                                      */
+    const void *w_gate;    /* [E][f][d]   weight_dtype (Q4B32: [E][f][d/2] bytes)           */
+    const void *w_up;      /* [E][f][d]                                                     */
+    const void *w_down;    /* [E][d][f]   (Q4B32: [E][d][f/2] bytes)                        */
+    const void *s_gate;    /* Q4B32 only: binary16 scales [E][f][d/32]; else NULL           */
+    const void *s_up;      /*             [E][f][d/32]                                      */
+    const void *s_down;    /*             [E][d][f/32]                                      */
+    const void *sh_gate;   /* shared experts [n_sh][f_sh][d], NULL when n_shared == 0       */
+    const void *sh_up;     /*                [n_sh][f_sh][d]                                */
+    const void *sh_down;   /*                [n_sh][d][f_sh]                                */
+    const void *sh_s_gate; /* Q4B32 scales of the shared experts, else NULL                 */
+    const void *sh_s_up;
+    const void *sh_s_down;
+    const void *sh_scale;  /* [d] router_dtype: c_b = sigmoid(h_b . sh_scale); NULL: c_b = 1 */
+} s2moe_layer_weights;
+
+typedef struct {
+    int32_t d_model;       /* d, multiple of 64                                             */
+    int32_t d_ff;          /* f, multiple of 32                                             */
+    int32_t n_experts;     /* E <= S2MOE_MAX_EXPERTS                                        */
+    int32_t top_k;         /* 1 <= k <= min(E, S2MOE_MAX_TOP_K)                             */
+    int32_t n_shared;      /* always-on shared experts (0..4)                               */
+    int32_t d_ff_shared;   /* f_sh, multiple of 32 (ignored when n_shared == 0)             */
+    int32_t act_dtype;     /* hidden states: S2MOE_F32 or S2MOE_BF16                        */
+    int32_t router_dtype;  /* S2MOE_F32 or S2MOE_BF16                                       */
+    int32_t weight_dtype;  /* expert weights: any s2moe_dtype                               */
+    int32_t renorm;        /* 1: renormalise the k mixing weights of a token to sum 1       */
+    int32_t cap;           /* |E*|, top_k <= cap <= E; cap == E turns the bias off          */
+    float alpha;           /* lambda_b = alpha * (l_(1) - l_(k+1)); >= 0; 0: bias off       */
+    int32_t weight_mode;   /* 0: mixing weights from l, 1: from l'                          */
+    int32_t max_tokens;    /* 1..S2MOE_MAX_TOKENS: workspace bound for n_tokens             */
+    int32_t n_layers;      /* >= 1                                                          */
+    int32_t kernel_plan;   /* 0: automatic; 1: plain CUDA-core kernels (all dtypes);
+                              2: streaming tensor-core kernels (BF16 / Q4B32 weights)        */
+} s2moe_config;
+
+/*
+ * Create a context for n_layers layers (problem statement of Sec. 4.2: the target
+ * model's gating module and experts are given).  `layers` is a host array of
+ * n_layers structs of dev pointers, copied by the call.  Allocates the workspace
+ * (a few MB) on the current device; no weight is copied or repacked.
+ * Errors: EINVAL (null, config out of the limits above, misaligned or missing
+ * pointer), ENOMEM, ECUDA.  *out is NULL on error.
+ */
+int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, s2moe_ctx **out);
+
+/*
+ * Verify one layer for n_tokens draft tokens (steps 1-4 above; Sec. 4.2).
+ *   hidden   dev [B][d] act_dtype, 16-byte aligned
+ *   conf     dev [B] float w_b >= 0, or NULL for all ones (negative values: undefined)
+ *   out      dev [B][d] float, overwritten with y
+ *   sel_idx  dev [B][k] int32, experts of S_b in selection order (descending l')
+ *   sel_w    dev [B][k] float, mixing weights p_{b,e} in the same order
+ *   n_unique dev int32, U
+ * n_tokens == 0 is a no-op returning S2MOE_OK.
+ * Errors: EINVAL (null ctx/buffer, misaligned hidden/out), ERANGE (layer, n_tokens),
+ * ECUDA (launch failure).
+ */
+int s2moe_verify_layer(s2moe_ctx *ctx, int32_t layer, int32_t n_tokens, const void *hidden,
+                       const float *conf, float *out, int32_t *sel_idx, float *sel_w,
+                       int32_t *n_unique, void *cuda_stream);
+
+/*
+ * Verify all n_layers layers back to back as independent layer problems: layer l reads
+ * hidden + l*B*d elements (conf + l*B) and writes out + l*B*d, sel_idx + l*B*k,
+ * sel_w + l*B*k and n_unique + l.  Same rules and errors as s2moe_verify_layer.
+ */
+int s2moe_verify_stack(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden, const float *conf,
+                       float *out, int32_t *sel_idx, float *sel_w, int32_t *n_unique,
+                       void *cuda_stream);
+
+/*
+ * s2moe_verify_stack with HOST input and output buffers of the same shapes: copies
+ * hidden (and conf, if not NULL) to staging memory the context owns, runs the stack,
+ * copies out, sel_idx, sel_w and n_unique back and synchronises the stream before
+ * returning.  Pinned host memory gives the best transfer rate but is not required.
+ */
+int s2moe_verify_stack_host(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden_host,
+                            const float *conf_host, float *out_host, int32_t *sel_idx_host,
+                            float *sel_w_host, int32_t *n_unique_host, void *cuda_stream);
+
+/* Free the workspace.  NULL is allowed.  The caller's buffers are untouched. */
+int s2moe_destroy(s2moe_ctx *ctx);
+
+/* Static description of a status code. */
+const char *s2moe_strerror(int status);
+
+/* Synchronises the device, stores the device status word (0 = no bounded wait gave
+ * up) in *host_out and clears it.  Returns ETIMEOUT if it was non-zero. */
+int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out);
+
+/* The last cudaError_t a call on this context saw (0 = cudaSuccess). */
+int s2moe_last_cuda_error(const s2moe_ctx *ctx);
+
+/* Kernel launches issued through this context so far (not counting memsets/copies). */
+int64_t s2moe_kernel_launches(const s2moe_ctx *ctx);
+
+/* Unique-expert bytes a layer step reads for U distinct routed experts: expert weight
+ * bytes (with Q4B32 scales) of U routed plus all shared experts. */
+double s2moe_unique_expert_bytes(const s2moe_ctx *ctx, int32_t n_unique);
+
+/*
+ * Per-kernel timing for benchmarks.  Between s2moe_profile_begin and
+ * s2moe_profile_end every kernel the context launches outside a graph capture is
+ * bracketed by CUDA events on its launching stream (up to max_records launches;
+ * later ones run untimed).  s2moe_profile_end synchronises the device and returns,
+ * per kernel class c < n_classes, the summed duration in milliseconds and the
+ * number of timed launches.  s2moe_kernel_class_name gives the kernel's name, or
+ * NULL past the last class.  Do not use during stream capture.
+ */
+#define S2MOE_KERNEL_CLASSES 5
+int s2moe_profile_begin(s2moe_ctx *ctx, int32_t max_records);
+int s2moe_profile_end(s2moe_ctx *ctx, int32_t n_classes, double *ms_out, int64_t *launches_out);
+const char *s2moe_kernel_class_name(int32_t cls);
+
+/*
+ * Diagnostics for tests: after synchronising, copy one workspace array of the LAST
+ * verify call to host memory.  `what`:
+ *   0 logits double [B][E]          1 counts  int32 [E + n_sh]   (tokens per expert)
+ *   2 offsets int32 [E + n_sh + 1]  3 slot_token int32 [n_slots] 4 slot_w float [n_slots]
+ *   5 active  int32 [n_active] (ids of experts with tokens, shared ones as E + s)
+ *   6 header  int32 [4] = {n_active, n_slots, U, B}
+ * n_slots = B*k + n_sh*B.  Returns EINVAL when `bytes` is smaller than the array.
+ */
+int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S2MOE_H */

@@ -1,0 +1,299 @@
+"""ctypes binding of the C ABI declared in ``include/s2moe.h``.
+
+Argument marshalling only: every step of the layer runs in the CUDA library.
+There is no CPU fallback; a missing library raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+F32, BF16, Q4B32 = 0, 1, 2
+OK, EINVAL, ERANGE, ENOMEM, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
+MAX_TOKENS, MAX_EXPERTS, MAX_TOP_K = 64, 256, 16
+
+WEIGHT_FIELDS = ("router", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
+                 "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "sh_scale")
+
+EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_verify_stack_host",
+           "s2moe_destroy", "s2moe_strerror", "s2moe_last_device_status", "s2moe_last_cuda_error",
+           "s2moe_kernel_launches", "s2moe_unique_expert_bytes", "s2moe_debug_read",
+           "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name")
+KERNEL_CLASSES = 5
+
+
+class LayerWeightsC(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_FIELDS]
+
+
+class ConfigC(ctypes.Structure):
+    _fields_ = [
+        ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("n_experts", ctypes.c_int32),
+        ("top_k", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("d_ff_shared", ctypes.c_int32),
+        ("act_dtype", ctypes.c_int32), ("router_dtype", ctypes.c_int32), ("weight_dtype", ctypes.c_int32),
+        ("renorm", ctypes.c_int32), ("cap", ctypes.c_int32), ("alpha", ctypes.c_float),
+        ("weight_mode", ctypes.c_int32), ("max_tokens", ctypes.c_int32), ("n_layers", ctypes.c_int32),
+        ("kernel_plan", ctypes.c_int32),
+    ]
+
+
+class S2MoEError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({strerror(status)}){detail}")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
+    """Load ``libs2moe.so`` (building it with nvcc when it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build_library() if build_if_missing else _build.LIB
+    if not os.path.exists(path):
+        raise RuntimeError(f"CUDA library {path} is missing; run __graft_entry__.build()")
+    lib = ctypes.CDLL(path)
+    vp, i32, fp = ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p
+    lib.s2moe_create.argtypes = [ctypes.POINTER(ConfigC), ctypes.POINTER(LayerWeightsC), ctypes.POINTER(vp)]
+    lib.s2moe_create.restype = ctypes.c_int
+    lib.s2moe_verify_layer.argtypes = [vp, i32, i32, vp, fp, fp, vp, fp, vp, vp]
+    lib.s2moe_verify_layer.restype = ctypes.c_int
+    lib.s2moe_verify_stack.argtypes = [vp, i32, vp, fp, fp, vp, fp, vp, vp]
+    lib.s2moe_verify_stack.restype = ctypes.c_int
+    lib.s2moe_verify_stack_host.argtypes = [vp, i32, vp, fp, fp, vp, fp, vp, vp]
+    lib.s2moe_verify_stack_host.restype = ctypes.c_int
+    lib.s2moe_destroy.argtypes = [vp]
+    lib.s2moe_destroy.restype = ctypes.c_int
+    lib.s2moe_strerror.argtypes = [ctypes.c_int]
+    lib.s2moe_strerror.restype = ctypes.c_char_p
+    lib.s2moe_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.s2moe_last_device_status.restype = ctypes.c_int
+    lib.s2moe_last_cuda_error.argtypes = [vp]
+    lib.s2moe_last_cuda_error.restype = ctypes.c_int
+    lib.s2moe_kernel_launches.argtypes = [vp]
+    lib.s2moe_kernel_launches.restype = ctypes.c_int64
+    lib.s2moe_unique_expert_bytes.argtypes = [vp, i32]
+    lib.s2moe_unique_expert_bytes.restype = ctypes.c_double
+    lib.s2moe_debug_read.argtypes = [vp, i32, vp, ctypes.c_size_t]
+    lib.s2moe_debug_read.restype = ctypes.c_int
+    lib.s2moe_profile_begin.argtypes = [vp, i32]
+    lib.s2moe_profile_begin.restype = ctypes.c_int
+    lib.s2moe_profile_end.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    lib.s2moe_profile_end.restype = ctypes.c_int
+    lib.s2moe_kernel_class_name.argtypes = [i32]
+    lib.s2moe_kernel_class_name.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def strerror(status: int) -> str:
+    return load_library().s2moe_strerror(int(status)).decode()
+
+
+@dataclass
+class Config:
+    d_model: int
+    d_ff: int
+    n_experts: int
+    top_k: int
+    n_shared: int = 0
+    d_ff_shared: int = 0
+    act_dtype: int = BF16
+    router_dtype: int = BF16
+    weight_dtype: int = BF16
+    renorm: int = 0
+    cap: int = 0               # 0 -> n_experts (bias off)
+    alpha: float = 0.5
+    weight_mode: int = 0
+    max_tokens: int = MAX_TOKENS
+    n_layers: int = 1
+    kernel_plan: int = 0
+
+    def c(self) -> ConfigC:
+        cap = self.cap if self.cap > 0 else self.n_experts
+        return ConfigC(self.d_model, self.d_ff, self.n_experts, self.top_k, self.n_shared,
+                       self.d_ff_shared, self.act_dtype, self.router_dtype, self.weight_dtype,
+                       self.renorm, cap, float(self.alpha), self.weight_mode, self.max_tokens,
+                       self.n_layers, self.kernel_plan)
+
+    @staticmethod
+    def from_workload(wl, max_tokens: Optional[int] = None, n_layers: Optional[int] = None,
+                      kernel_plan: int = 0) -> "Config":
+        return Config(wl.d_model, wl.d_ff, wl.n_experts, wl.top_k, wl.n_shared, wl.d_ff_shared,
+                      wl.act_dtype, wl.router_dtype, wl.weight_dtype, wl.renorm, wl.cap, wl.alpha,
+                      wl.weight_mode, max_tokens or MAX_TOKENS, n_layers or wl.n_layers, kernel_plan)
+
+
+def _dptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+@dataclass
+class LayerOutput:
+    out: torch.Tensor        # [..., B, d] float32
+    sel_idx: torch.Tensor    # [..., B, k] int32
+    sel_w: torch.Tensor      # [..., B, k] float32
+    n_unique: torch.Tensor   # [...] int32
+
+
+class S2MoE:
+    """A context of the library: ``n_layers`` MoE layers whose weights stay resident."""
+
+    def __init__(self, config: Config, layers: Sequence[Dict[str, torch.Tensor]]):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p(None)
+        self.config = config
+        if len(layers) != config.n_layers:
+            raise ValueError("one weight dict per layer is required")
+        self._keep = list(layers)          # keeps the caller's tensors alive
+        arr = (LayerWeightsC * config.n_layers)()
+        for i, lw in enumerate(layers):
+            for name in WEIGHT_FIELDS:
+                setattr(arr[i], name, _dptr(lw.get(name)))
+        cfg = config.c()
+        rc = self._lib.s2moe_create(ctypes.byref(cfg), arr, ctypes.byref(self._h))
+        if rc != OK:
+            self._h = ctypes.c_void_p(None)
+            raise S2MoEError(rc, "s2moe_create")
+        self.device = next(iter(layers[0].values())).device
+
+    # -- lifetime
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.s2moe_destroy(self._h)
+            self._h = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- calls
+    def _check(self, rc: int, where: str) -> None:
+        if rc != OK:
+            detail = ""
+            if rc == ECUDA:
+                detail = f" cudaError={self._lib.s2moe_last_cuda_error(self._h)}"
+            raise S2MoEError(rc, where, detail)
+
+    def alloc_outputs(self, n_tokens: int, stack: bool = False) -> LayerOutput:
+        c = self.config
+        lead = (c.n_layers,) if stack else ()
+        dev = self.device
+        return LayerOutput(
+            torch.empty(lead + (n_tokens, c.d_model), dtype=torch.float32, device=dev),
+            torch.empty(lead + (n_tokens, c.top_k), dtype=torch.int32, device=dev),
+            torch.empty(lead + (n_tokens, c.top_k), dtype=torch.float32, device=dev),
+            torch.empty(lead if stack else (1,), dtype=torch.int32, device=dev),
+        )
+
+    def verify_layer(self, layer: int, hidden: torch.Tensor, conf: Optional[torch.Tensor] = None,
+                     outputs: Optional[LayerOutput] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> LayerOutput:
+        B = hidden.shape[0]
+        o = outputs or self.alloc_outputs(B)
+        rc = self._lib.s2moe_verify_layer(self._h, layer, B, _dptr(hidden), _dptr(conf), _dptr(o.out),
+                                          _dptr(o.sel_idx), _dptr(o.sel_w), _dptr(o.n_unique),
+                                          _stream_handle(stream))
+        self._check(rc, "s2moe_verify_layer")
+        return o
+
+    def verify_stack(self, hidden: torch.Tensor, conf: Optional[torch.Tensor] = None,
+                     outputs: Optional[LayerOutput] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> LayerOutput:
+        """hidden [L][B][d]; conf [L][B] or None."""
+        B = hidden.shape[1]
+        o = outputs or self.alloc_outputs(B, stack=True)
+        rc = self._lib.s2moe_verify_stack(self._h, B, _dptr(hidden), _dptr(conf), _dptr(o.out),
+                                          _dptr(o.sel_idx), _dptr(o.sel_w), _dptr(o.n_unique),
+                                          _stream_handle(stream))
+        self._check(rc, "s2moe_verify_stack")
+        return o
+
+    def verify_stack_host(self, hidden: torch.Tensor, conf: Optional[torch.Tensor], out: torch.Tensor,
+                          sel_idx: torch.Tensor, sel_w: torch.Tensor, n_unique: torch.Tensor,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+        """All tensors are HOST tensors (pinned for best speed); returns after the results are there."""
+        for t in (hidden, out, sel_idx, sel_w, n_unique):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("expected contiguous host tensors")
+        B = hidden.shape[1]
+        rc = self._lib.s2moe_verify_stack_host(
+            self._h, B, hidden.data_ptr(), conf.data_ptr() if conf is not None else None, out.data_ptr(),
+            sel_idx.data_ptr(), sel_w.data_ptr(), n_unique.data_ptr(), _stream_handle(stream))
+        self._check(rc, "s2moe_verify_stack_host")
+
+    # -- accounting and diagnostics
+    def kernel_launches(self) -> int:
+        return int(self._lib.s2moe_kernel_launches(self._h))
+
+    def unique_expert_bytes(self, n_unique: int) -> float:
+        return float(self._lib.s2moe_unique_expert_bytes(self._h, int(n_unique)))
+
+    def profile_begin(self, max_records: int) -> None:
+        self._check(self._lib.s2moe_profile_begin(self._h, int(max_records)), "s2moe_profile_begin")
+
+    def profile_end(self) -> Dict[str, Dict[str, float]]:
+        """{kernel name: {"ms": summed duration, "launches": n}} since profile_begin."""
+        ms = (ctypes.c_double * KERNEL_CLASSES)()
+        n = (ctypes.c_int64 * KERNEL_CLASSES)()
+        self._check(self._lib.s2moe_profile_end(self._h, KERNEL_CLASSES, ms, n), "s2moe_profile_end")
+        out = {}
+        for c in range(KERNEL_CLASSES):
+            name = self._lib.s2moe_kernel_class_name(c)
+            if name is not None and n[c] > 0:
+                out[name.decode()] = {"ms": float(ms[c]), "launches": int(n[c])}
+        return out
+
+    def device_status(self) -> int:
+        v = ctypes.c_int32(0)
+        rc = self._lib.s2moe_last_device_status(self._h, ctypes.byref(v))
+        if rc not in (OK, ETIMEOUT):
+            self._check(rc, "s2moe_last_device_status")
+        return int(v.value)
+
+    def debug_read(self, what: int, count: int, dtype: torch.dtype) -> torch.Tensor:
+        t = torch.zeros(max(count, 1), dtype=dtype)
+        rc = self._lib.s2moe_debug_read(self._h, what, t.data_ptr(), t.numel() * t.element_size())
+        self._check(rc, "s2moe_debug_read")
+        return t[:count]
+
+    def debug_lists(self) -> Dict[str, torch.Tensor]:
+        """Bucketing arrays of the last call (host tensors)."""
+        c = self.config
+        G = c.n_experts + c.n_shared
+        hdr = self.debug_read(6, 4, torch.int32)
+        n_active, n_slots, U, B = (int(x) for x in hdr)
+        return dict(
+            n_active=n_active, n_slots=n_slots, U=U, B=B,
+            logits=self.debug_read(0, B * c.n_experts, torch.float64).reshape(B, c.n_experts),
+            counts=self.debug_read(1, G, torch.int32), offsets=self.debug_read(2, G + 1, torch.int32),
+            slot_token=self.debug_read(3, n_slots, torch.int32), slot_w=self.debug_read(4, n_slots, torch.float32),
+            active=self.debug_read(5, n_active, torch.int32))

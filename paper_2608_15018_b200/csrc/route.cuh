@@ -1,0 +1,244 @@
+// Router logits and reuse-aware expert gating (Sec. 4.2) for one draft batch.
+//
+//   router_logits_kernel : l_{b,e} = h_b . W_r[e]  (and the shared-expert gate logit),
+//                          float64 accumulation so that the discrete choices below
+//                          do not depend on the summation order.
+//   gating_kernel        : Eq. 4 aggregation, TopCap, lambda_b, biased top-k, mixing
+//                          weights, union / unique count, token->expert bucketing.
+#pragma once
+
+#include "common.cuh"
+
+namespace s2moe {
+
+constexpr int kRouteWarps = 8;
+constexpr int kGateThreads = 1024;
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_max(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// One warp per router row (row E is the shared-expert gate vector), all B tokens.
+template <int ACT, int RT>
+__global__ void __launch_bounds__(kRouteWarps * 32)
+router_logits_kernel(Shape sh, int B, const void *__restrict__ hidden, const void *__restrict__ router,
+                     const void *__restrict__ sh_scale, double *__restrict__ logits,
+                     double *__restrict__ gate_logit)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kRouteWarps + warp;
+    const int n_rows = sh.E + (sh_scale ? 1 : 0);
+    if (row >= n_rows) return;
+    const int d = sh.d;
+    const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
+    const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
+                                     : reinterpret_cast<const uint8_t *>(sh_scale);
+    for (int b0 = 0; b0 < B; b0 += 8) {
+        double acc[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) acc[t] = 0.0;
+        for (int c = lane * 8; c < d; c += 256) {
+            float w[8];
+            load8_plain<RT>(wrow, c, w);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                if (b0 + t < B) {
+                    float x[8];
+                    load8_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)(b0 + t) * d * ab, c, x);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[t] = fma((double)w[i], (double)x[i], acc[t]);
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            double s = warp_sum(acc[t]);
+            if (lane == 0 && b0 + t < B) {
+                if (row < sh.E) logits[(size_t)(b0 + t) * sh.E + row] = s;
+                else gate_logit[b0 + t] = s;
+            }
+        }
+    }
+}
+
+// order (value descending, id ascending): is a before b?
+__device__ __forceinline__ bool before1(double va, int a, double vb, int b)
+{
+    return va > vb || (va == vb && a < b);
+}
+// order (l' descending, l descending, id ascending)
+__device__ __forceinline__ bool before2(double l2a, double la, int a, double l2b, double lb, int b)
+{
+    if (l2a != l2b) return l2a > l2b;
+    if (la != lb) return la > lb;
+    return a < b;
+}
+
+// One block.  Dynamic shared memory: B*E doubles (the logits).
+__global__ void __launch_bounds__(kGateThreads)
+gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int has_gate,
+              int32_t *__restrict__ sel_idx, float *__restrict__ sel_w, int32_t *__restrict__ n_unique)
+{
+    extern __shared__ double s_l[];  // [B][E]
+    __shared__ double s_g[kMaxExperts];
+    __shared__ unsigned char s_star[kMaxExperts];
+    __shared__ double s_w[kMaxTokens], s_top1[kMaxTokens], s_kth[kMaxTokens], s_lam[kMaxTokens];
+    __shared__ int s_sel[kMaxTokens * kMaxTopK];
+    __shared__ float s_pw[kMaxTokens * kMaxTopK];
+    __shared__ unsigned long long s_mask[kMaxExperts];
+    __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_pos[kMaxExperts];
+    __shared__ int s_U;
+
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int E = sh.E, k = sh.k, cap = sh.cap;
+    const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
+
+    for (int i = tid; i < B * E; i += nt) s_l[i] = ws.logits[i];
+    for (int b = tid; b < B; b += nt) {
+        s_w[b] = conf ? (double)conf[b] : 1.0;
+        s_lam[b] = 0.0;
+    }
+    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
+    __syncthreads();
+
+    if (bias_on) {
+        // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
+        for (int e = tid; e < E; e += nt) {
+            double g = 0.0;
+            for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
+            s_g[e] = g;
+        }
+        __syncthreads();
+        // TopCap by rank
+        for (int e = tid; e < E; e += nt) {
+            int rank = 0;
+            const double ge = s_g[e];
+            for (int o = 0; o < E; ++o) rank += before1(s_g[o], o, ge, e);
+            s_star[e] = rank < cap;
+        }
+        // order statistics of the original logits: top-1 and (k+1)-th
+        for (int i = tid; i < B * E; i += nt) {
+            const int b = i / E, e = i - b * E;
+            const double le = s_l[i];
+            int rank = 0;
+            for (int o = 0; o < E; ++o) rank += before1(s_l[b * E + o], o, le, e);
+            if (rank == 0) s_top1[b] = le;
+            if (rank == k) s_kth[b] = le;
+        }
+        __syncthreads();
+        for (int b = tid; b < B; b += nt) s_lam[b] = sh.alpha * (s_top1[b] - s_kth[b]);
+        __syncthreads();
+    }
+
+    // biased top-k by rank
+    for (int i = tid; i < B * E; i += nt) {
+        const int b = i / E, e = i - b * E;
+        const double lam = s_lam[b];
+        const double le = s_l[i];
+        const double l2e = s_star[e] ? le + lam : le;
+        int rank = 0;
+        for (int o = 0; o < E; ++o) {
+            const double lo = s_l[b * E + o];
+            const double l2o = s_star[o] ? lo + lam : lo;
+            rank += before2(l2o, lo, o, l2e, le, e);
+        }
+        if (rank < k) s_sel[b * k + rank] = e;
+    }
+    __syncthreads();
+
+    // mixing weights: one warp per token
+    {
+        const int warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
+        for (int b = warp; b < B; b += nw) {
+            const double lam = sh.weight_mode ? s_lam[b] : 0.0;
+            double zmax = -1.0e300;
+            for (int e = lane; e < E; e += 32) {
+                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
+                zmax = fmax(zmax, z);
+            }
+            zmax = warp_max(zmax);
+            double den = 0.0;
+            for (int e = lane; e < E; e += 32) {
+                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
+                den += exp(z - zmax);
+            }
+            den = warp_sum(den);
+            double p = 0.0;
+            int e = 0;
+            if (lane < k) {
+                e = s_sel[b * k + lane];
+                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
+                p = exp(z - zmax) / den;
+            }
+            if (sh.renorm) {
+                const double tot = warp_sum(p);
+                p /= tot;
+            }
+            if (lane < k) {
+                s_pw[b * k + lane] = (float)p;
+                sel_idx[b * k + lane] = e;
+                sel_w[b * k + lane] = (float)p;
+                atomicOr(&s_mask[e], 1ull << b);
+            }
+        }
+    }
+    __syncthreads();
+
+    // union, unique count, exclusive scan, list of active experts
+    for (int e = tid; e < E; e += nt) s_cnt[e] = __popcll(s_mask[e]);
+    __syncthreads();
+    for (int e = tid; e < E; e += nt) {
+        int off = 0, pos = 0;
+        for (int o = 0; o < e; ++o) { off += s_cnt[o]; pos += s_cnt[o] > 0; }
+        s_off[e] = off;
+        s_pos[e] = pos;
+        if (e == E - 1) { s_off[E] = off + s_cnt[e]; s_U = pos + (s_cnt[e] > 0); }
+    }
+    __syncthreads();
+    const int U = s_U, n_routed = B * k;
+    for (int e = tid; e < E; e += nt) {
+        ws.counts[e] = s_cnt[e];
+        ws.offsets[e] = s_off[e];
+        if (s_cnt[e] > 0) ws.active[s_pos[e]] = e;
+    }
+    // bucket the (token, choice) pairs: tokens ascending inside an expert
+    for (int i = tid; i < n_routed; i += nt) {
+        const int b = i / k;
+        const int e = s_sel[i];
+        const int pos = s_off[e] + __popcll(s_mask[e] & ((1ull << b) - 1ull));
+        ws.slot_token[pos] = b;
+        ws.slot_w[pos] = s_pw[i];
+    }
+    // shared experts: every token, weight c_b
+    for (int i = tid; i < sh.n_sh * B; i += nt) {
+        const int s = i / B, b = i - s * B;
+        float c = 1.0f;
+        if (has_gate) c = (float)(1.0 / (1.0 + exp(-ws.gate_logit[b])));
+        ws.slot_token[n_routed + i] = b;
+        ws.slot_w[n_routed + i] = c;
+        if (b == 0) {
+            ws.counts[E + s] = B;
+            ws.offsets[E + s] = n_routed + s * B;
+            ws.active[U + s] = E + s;
+        }
+    }
+    if (tid == 0) {
+        ws.offsets[E + sh.n_sh] = n_routed + sh.n_sh * B;
+        ws.header[0] = U + sh.n_sh;
+        ws.header[1] = n_routed + sh.n_sh * B;
+        ws.header[2] = U;
+        ws.header[3] = B;
+        *n_unique = U;
+    }
+}
+
+}  // namespace s2moe

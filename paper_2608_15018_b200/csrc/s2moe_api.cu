@@ -1,0 +1,458 @@
+// C ABI of the MoE verification library: context, validation, kernel dispatch.
+// See include/s2moe.h for the contract of every entry point.
+#include "../../include/s2moe.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "ffn_simple.cuh"
+#include "route.cuh"
+
+using namespace s2moe;
+
+struct s2moe_ctx {
+    s2moe_config cfg;
+    Shape shape;
+    std::vector<LayerPtrs> layers;
+    Workspace ws;
+    void *slab = nullptr;          // one allocation behind ws
+    size_t slab_bytes = 0;
+    // staging for the host-buffer entry point
+    void *st_hidden = nullptr;
+    float *st_conf = nullptr, *st_out = nullptr, *st_selw = nullptr;
+    int32_t *st_sel = nullptr, *st_nu = nullptr;
+    int device = 0;
+    int plan = 1;
+    int last_cuda = 0;
+    int64_t launches = 0;
+    int last_B = 0;
+    // optional per-kernel timing (CUDA events on the launching stream)
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_ev;   // 2 per record
+    std::vector<int> prof_cls;
+    size_t prof_cap = 0;
+};
+
+enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_COUNT = 5 };
+
+namespace {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(s2moe_ctx *ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda = (int)e;
+    return S2MOE_ECUDA;
+}
+
+#define CU(ctx, call)                                       \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail((ctx), e_); \
+    } while (0)
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Brackets one kernel launch: counts it and, when timing is on, records an event
+// before and after it on the launching stream.
+struct LaunchScope {
+    s2moe_ctx *ctx;
+    cudaStream_t st;
+    long rec = -1;
+    LaunchScope(s2moe_ctx *c, int cls, cudaStream_t s) : ctx(c), st(s)
+    {
+        ctx->launches++;
+        if (ctx->prof_on && ctx->prof_cls.size() < ctx->prof_cap) {
+            rec = (long)ctx->prof_cls.size();
+            ctx->prof_cls.push_back(cls);
+            cudaEventRecord(ctx->prof_ev[2 * rec], st);
+        }
+    }
+    ~LaunchScope()
+    {
+        if (rec >= 0) cudaEventRecord(ctx->prof_ev[2 * rec + 1], st);
+    }
+};
+
+int validate_config(const s2moe_config *c)
+{
+    if (!c) return S2MOE_EINVAL;
+    if (c->d_model < 64 || c->d_model % 64) return S2MOE_EINVAL;
+    if (c->d_ff < 32 || c->d_ff % 32) return S2MOE_EINVAL;
+    if (c->n_experts < 1 || c->n_experts > S2MOE_MAX_EXPERTS) return S2MOE_EINVAL;
+    if (c->top_k < 1 || c->top_k > c->n_experts || c->top_k > S2MOE_MAX_TOP_K) return S2MOE_EINVAL;
+    if (c->n_shared < 0 || c->n_shared > kMaxShared) return S2MOE_EINVAL;
+    if (c->n_shared > 0 && (c->d_ff_shared < 32 || c->d_ff_shared % 32)) return S2MOE_EINVAL;
+    if (c->act_dtype != S2MOE_F32 && c->act_dtype != S2MOE_BF16) return S2MOE_EINVAL;
+    if (c->router_dtype != S2MOE_F32 && c->router_dtype != S2MOE_BF16) return S2MOE_EINVAL;
+    if (c->weight_dtype < S2MOE_F32 || c->weight_dtype > S2MOE_Q4B32) return S2MOE_EINVAL;
+    if (c->renorm != 0 && c->renorm != 1) return S2MOE_EINVAL;
+    if (c->cap < c->top_k || c->cap > c->n_experts) return S2MOE_EINVAL;
+    if (!(c->alpha >= 0.0f)) return S2MOE_EINVAL;
+    if (c->weight_mode != 0 && c->weight_mode != 1) return S2MOE_EINVAL;
+    if (c->max_tokens < 1 || c->max_tokens > S2MOE_MAX_TOKENS) return S2MOE_EINVAL;
+    if (c->n_layers < 1) return S2MOE_EINVAL;
+    if (c->kernel_plan < 0 || c->kernel_plan > 2) return S2MOE_EINVAL;
+    if (c->kernel_plan == 2 && c->weight_dtype == S2MOE_F32) return S2MOE_EINVAL;
+    return S2MOE_OK;
+}
+
+int validate_layer(const s2moe_config *c, const s2moe_layer_weights *w)
+{
+    const void *need[] = {w->router, w->w_gate, w->w_up, w->w_down};
+    for (const void *p : need)
+        if (!p || !aligned16(p)) return S2MOE_EINVAL;
+    if (c->weight_dtype == S2MOE_Q4B32) {
+        const void *sc[] = {w->s_gate, w->s_up, w->s_down};
+        for (const void *p : sc)
+            if (!p || !aligned16(p)) return S2MOE_EINVAL;
+    }
+    if (c->n_shared > 0) {
+        const void *shp[] = {w->sh_gate, w->sh_up, w->sh_down};
+        for (const void *p : shp)
+            if (!p || !aligned16(p)) return S2MOE_EINVAL;
+        if (c->weight_dtype == S2MOE_Q4B32) {
+            const void *sc[] = {w->sh_s_gate, w->sh_s_up, w->sh_s_down};
+            for (const void *p : sc)
+                if (!p || !aligned16(p)) return S2MOE_EINVAL;
+        }
+        if (w->sh_scale && !aligned16(w->sh_scale)) return S2MOE_EINVAL;
+    }
+    return S2MOE_OK;
+}
+
+// ---- dispatch over storage formats ------------------------------------------
+
+template <int ACT>
+void launch_router(s2moe_ctx *ctx, const LayerPtrs &lp, int B, const void *hidden, cudaStream_t st)
+{
+    const int rows = ctx->shape.E + (lp.sh_scale ? 1 : 0);
+    const dim3 grid((rows + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
+    LaunchScope scope(ctx, KC_ROUTER, st);
+    if (ctx->shape.router_dtype == DT_F32)
+        router_logits_kernel<ACT, DT_F32><<<grid, block, 0, st>>>(ctx->shape, B, hidden, lp.router, lp.sh_scale,
+                                                                  ctx->ws.logits, ctx->ws.gate_logit);
+    else
+        router_logits_kernel<ACT, DT_BF16><<<grid, block, 0, st>>>(ctx->shape, B, hidden, lp.router, lp.sh_scale,
+                                                                   ctx->ws.logits, ctx->ws.gate_logit);
+}
+
+constexpr size_t kSimpleSmem = (size_t)kSimpleTokChunk * kSimpleKChunk * sizeof(float);
+
+template <int WT, int ACT>
+void launch_simple(s2moe_ctx *ctx, const LayerPtrs &lp, const void *hidden, float *out, cudaStream_t st)
+{
+    const Shape &sh = ctx->shape;
+    const int groups = sh.E + sh.n_sh;
+    const int fmax = sh.n_sh > 0 && sh.f_sh > sh.f ? sh.f_sh : sh.f;
+    const dim3 block(kSimpleWarps * 32);
+    const dim3 g1((fmax + kSimpleWarps - 1) / kSimpleWarps, groups);
+    const dim3 g2((sh.d + kSimpleWarps - 1) / kSimpleWarps, groups);
+    {
+        LaunchScope scope(ctx, KC_GATEUP, st);
+        ffn_gateup_simple<WT, ACT><<<g1, block, kSimpleSmem, st>>>(sh, lp, ctx->ws, hidden);
+    }
+    {
+        LaunchScope scope(ctx, KC_DOWN, st);
+        ffn_down_simple<WT><<<g2, block, kSimpleSmem, st>>>(sh, lp, ctx->ws, out);
+    }
+}
+
+template <int WT, int ACT>
+cudaError_t prepare_simple()
+{
+    cudaError_t e = cudaFuncSetAttribute(ffn_gateup_simple<WT, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSimpleSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(ffn_down_simple<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSimpleSmem);
+}
+
+#define DISPATCH_WT_ACT(ctx, FN, ...)                                                    \
+    do {                                                                                 \
+        const int wt_ = (ctx)->shape.weight_dtype, at_ = (ctx)->shape.act_dtype;         \
+        if (wt_ == DT_F32 && at_ == DT_F32) FN<DT_F32, DT_F32>(__VA_ARGS__);             \
+        else if (wt_ == DT_F32) FN<DT_F32, DT_BF16>(__VA_ARGS__);                        \
+        else if (wt_ == DT_BF16 && at_ == DT_F32) FN<DT_BF16, DT_F32>(__VA_ARGS__);      \
+        else if (wt_ == DT_BF16) FN<DT_BF16, DT_BF16>(__VA_ARGS__);                      \
+        else if (at_ == DT_F32) FN<DT_Q4B32, DT_F32>(__VA_ARGS__);                       \
+        else FN<DT_Q4B32, DT_BF16>(__VA_ARGS__);                                         \
+    } while (0)
+
+int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float *conf, float *out,
+               int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
+{
+    const Shape &sh = ctx->shape;
+    const LayerPtrs &lp = ctx->layers[layer];
+    CU(ctx, cudaMemsetAsync(out, 0, (size_t)B * sh.d * sizeof(float), st));
+    if (sh.act_dtype == DT_F32) launch_router<DT_F32>(ctx, lp, B, hidden, st);
+    else launch_router<DT_BF16>(ctx, lp, B, hidden, st);
+    {
+        LaunchScope scope(ctx, KC_GATING, st);
+        gating_kernel<<<1, kGateThreads, (size_t)B * sh.E * sizeof(double), st>>>(
+            sh, B, ctx->ws, conf, lp.sh_scale ? 1 : 0, sel_idx, sel_w, n_unique);
+    }
+    DISPATCH_WT_ACT(ctx, launch_simple, ctx, lp, hidden, out, st);
+    ctx->last_B = B;
+    CU(ctx, cudaGetLastError());
+    return S2MOE_OK;
+}
+
+int check_call(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden, float *out, int32_t *sel_idx, float *sel_w,
+               int32_t *n_unique)
+{
+    if (!ctx) return S2MOE_EINVAL;
+    if (n_tokens < 0 || n_tokens > ctx->cfg.max_tokens) return S2MOE_ERANGE;
+    if (n_tokens == 0) return S2MOE_OK;
+    if (!hidden || !out || !sel_idx || !sel_w || !n_unique) return S2MOE_EINVAL;
+    if (!aligned16(hidden) || !aligned16(out)) return S2MOE_EINVAL;
+    return S2MOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, s2moe_ctx **out)
+{
+    if (out) *out = nullptr;
+    if (!config || !layers || !out) return S2MOE_EINVAL;
+    int rc = validate_config(config);
+    if (rc != S2MOE_OK) return rc;
+    for (int l = 0; l < config->n_layers; ++l) {
+        rc = validate_layer(config, &layers[l]);
+        if (rc != S2MOE_OK) return rc;
+    }
+    s2moe_ctx *ctx = new (std::nothrow) s2moe_ctx();
+    if (!ctx) return S2MOE_ENOMEM;
+    ctx->cfg = *config;
+    Shape &sh = ctx->shape;
+    sh.d = config->d_model; sh.f = config->d_ff; sh.E = config->n_experts; sh.k = config->top_k;
+    sh.n_sh = config->n_shared; sh.f_sh = config->n_shared ? config->d_ff_shared : 0;
+    sh.act_dtype = config->act_dtype; sh.router_dtype = config->router_dtype;
+    sh.weight_dtype = config->weight_dtype;
+    sh.renorm = config->renorm; sh.cap = config->cap; sh.weight_mode = config->weight_mode;
+    sh.alpha = (double)config->alpha;
+    ctx->layers.resize(config->n_layers);
+    static_assert(sizeof(LayerPtrs) == sizeof(s2moe_layer_weights), "layout");
+    std::memcpy(ctx->layers.data(), layers, sizeof(LayerPtrs) * (size_t)config->n_layers);
+    ctx->plan = 1;
+
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e != cudaSuccess) { delete ctx; return S2MOE_ECUDA; }
+
+    const int T = config->max_tokens, E = sh.E, G = E + sh.n_sh, L = config->n_layers;
+    const size_t n_slots = (size_t)T * sh.k + (size_t)sh.n_sh * T;
+    const size_t act_floats = (size_t)T * sh.k * sh.f + (size_t)sh.n_sh * T * sh.f_sh;
+    const size_t ab = sh.act_dtype == DT_F32 ? 4 : 2;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_logits = take(sizeof(double) * T * E), o_gl = take(sizeof(double) * T);
+    const size_t o_ticket = take(256), o_status = take(256), o_header = take(256);
+    const size_t o_counts = take(4 * (size_t)G), o_offsets = take(4 * (size_t)(G + 1));
+    const size_t o_stok = take(4 * n_slots), o_sw = take(4 * n_slots), o_active = take(4 * (size_t)G);
+    const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(G + 64));
+    const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
+    const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
+    const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
+    ctx->slab_bytes = off;
+    e = cudaMalloc(&ctx->slab, ctx->slab_bytes);
+    if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? S2MOE_ENOMEM : S2MOE_ECUDA; }
+    e = cudaMemset(ctx->slab, 0, ctx->slab_bytes);
+    if (e == cudaSuccess) DISPATCH_WT_ACT(ctx, e = prepare_simple);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gating_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(sizeof(double) * kMaxTokens * kMaxExperts));
+    if (e != cudaSuccess) { cudaFree(ctx->slab); delete ctx; return S2MOE_ECUDA; }
+    uint8_t *base = (uint8_t *)ctx->slab;
+    Workspace &ws = ctx->ws;
+    ws.logits = (double *)(base + o_logits); ws.gate_logit = (double *)(base + o_gl);
+    ws.ticket = (unsigned int *)(base + o_ticket); ws.status = (int32_t *)(base + o_status);
+    ws.header = (int32_t *)(base + o_header); ws.counts = (int32_t *)(base + o_counts);
+    ws.offsets = (int32_t *)(base + o_offsets); ws.slot_token = (int32_t *)(base + o_stok);
+    ws.slot_w = (float *)(base + o_sw); ws.active = (int32_t *)(base + o_active);
+    ws.act = (float *)(base + o_act); ws.sync = (int32_t *)(base + o_sync);
+    ctx->st_hidden = base + o_sth; ctx->st_conf = (float *)(base + o_stc);
+    ctx->st_out = (float *)(base + o_sto); ctx->st_sel = (int32_t *)(base + o_sts);
+    ctx->st_selw = (float *)(base + o_stw); ctx->st_nu = (int32_t *)(base + o_stn);
+    *out = ctx;
+    return S2MOE_OK;
+}
+
+int s2moe_verify_layer(s2moe_ctx *ctx, int32_t layer, int32_t n_tokens, const void *hidden, const float *conf,
+                       float *out, int32_t *sel_idx, float *sel_w, int32_t *n_unique, void *cuda_stream)
+{
+    int rc = check_call(ctx, n_tokens, hidden, out, sel_idx, sel_w, n_unique);
+    if (rc != S2MOE_OK) return rc;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return S2MOE_ERANGE;
+    if (n_tokens == 0) return S2MOE_OK;
+    return verify_one(ctx, layer, n_tokens, hidden, conf, out, sel_idx, sel_w, n_unique,
+                      (cudaStream_t)cuda_stream);
+}
+
+int s2moe_verify_stack(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden, const float *conf, float *out,
+                       int32_t *sel_idx, float *sel_w, int32_t *n_unique, void *cuda_stream)
+{
+    int rc = check_call(ctx, n_tokens, hidden, out, sel_idx, sel_w, n_unique);
+    if (rc != S2MOE_OK || n_tokens == 0) return rc;
+    const Shape &sh = ctx->shape;
+    const size_t ab = sh.act_dtype == DT_F32 ? 4 : 2, B = (size_t)n_tokens;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+        rc = verify_one(ctx, l, n_tokens, (const uint8_t *)hidden + (size_t)l * B * sh.d * ab,
+                        conf ? conf + (size_t)l * B : nullptr, out + (size_t)l * B * sh.d,
+                        sel_idx + (size_t)l * B * sh.k, sel_w + (size_t)l * B * sh.k, n_unique + l,
+                        (cudaStream_t)cuda_stream);
+        if (rc != S2MOE_OK) return rc;
+    }
+    return S2MOE_OK;
+}
+
+int s2moe_verify_stack_host(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden_host, const float *conf_host,
+                            float *out_host, int32_t *sel_idx_host, float *sel_w_host, int32_t *n_unique_host,
+                            void *cuda_stream)
+{
+    if (!ctx) return S2MOE_EINVAL;
+    if (n_tokens < 0 || n_tokens > ctx->cfg.max_tokens) return S2MOE_ERANGE;
+    if (n_tokens == 0) return S2MOE_OK;
+    if (!hidden_host || !out_host || !sel_idx_host || !sel_w_host || !n_unique_host) return S2MOE_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const Shape &sh = ctx->shape;
+    const size_t ab = sh.act_dtype == DT_F32 ? 4 : 2, L = (size_t)ctx->cfg.n_layers, B = (size_t)n_tokens;
+    CU(ctx, cudaMemcpyAsync(ctx->st_hidden, hidden_host, L * B * sh.d * ab, cudaMemcpyHostToDevice, st));
+    if (conf_host) CU(ctx, cudaMemcpyAsync(ctx->st_conf, conf_host, L * B * 4, cudaMemcpyHostToDevice, st));
+    int rc = s2moe_verify_stack(ctx, n_tokens, ctx->st_hidden, conf_host ? ctx->st_conf : nullptr, ctx->st_out,
+                                ctx->st_sel, ctx->st_selw, ctx->st_nu, cuda_stream);
+    if (rc != S2MOE_OK) return rc;
+    CU(ctx, cudaMemcpyAsync(out_host, ctx->st_out, L * B * sh.d * 4, cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaMemcpyAsync(sel_idx_host, ctx->st_sel, L * B * sh.k * 4, cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaMemcpyAsync(sel_w_host, ctx->st_selw, L * B * sh.k * 4, cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaMemcpyAsync(n_unique_host, ctx->st_nu, L * 4, cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaStreamSynchronize(st));
+    return S2MOE_OK;
+}
+
+int s2moe_destroy(s2moe_ctx *ctx)
+{
+    if (!ctx) return S2MOE_OK;
+    cudaError_t e = cudaSuccess;
+    if (ctx->slab) e = cudaFree(ctx->slab);
+    for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
+    delete ctx;
+    return e == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
+}
+
+const char *s2moe_strerror(int status)
+{
+    switch (status) {
+        case S2MOE_OK: return "ok";
+        case S2MOE_EINVAL: return "invalid argument (config, shape, null pointer or alignment)";
+        case S2MOE_ERANGE: return "n_tokens or layer out of range";
+        case S2MOE_ENOMEM: return "out of device memory";
+        case S2MOE_ECUDA: return "CUDA call failed";
+        case S2MOE_ETIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out)
+{
+    if (!ctx || !host_out) return S2MOE_EINVAL;
+    CU(ctx, cudaDeviceSynchronize());
+    CU(ctx, cudaMemcpy(host_out, ctx->ws.status, 4, cudaMemcpyDeviceToHost));
+    if (*host_out != 0) {
+        CU(ctx, cudaMemset(ctx->ws.status, 0, 4));
+        return S2MOE_ETIMEOUT;
+    }
+    return S2MOE_OK;
+}
+
+int s2moe_last_cuda_error(const s2moe_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int64_t s2moe_kernel_launches(const s2moe_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+double s2moe_unique_expert_bytes(const s2moe_ctx *ctx, int32_t n_unique)
+{
+    if (!ctx) return 0.0;
+    const Shape &sh = ctx->shape;
+    auto mat = [&](int rows, int K) {
+        double b = (double)rows * (double)row_bytes(sh.weight_dtype, K);
+        if (sh.weight_dtype == DT_Q4B32) b += (double)rows * (K / 32) * 2.0;
+        return b;
+    };
+    const double routed = 2.0 * mat(sh.f, sh.d) + mat(sh.d, sh.f);
+    const double shared = sh.n_sh ? sh.n_sh * (2.0 * mat(sh.f_sh, sh.d) + mat(sh.d, sh.f_sh)) : 0.0;
+    return (double)n_unique * routed + shared;
+}
+
+int s2moe_profile_begin(s2moe_ctx *ctx, int32_t max_records)
+{
+    if (!ctx || max_records < 0) return S2MOE_EINVAL;
+    while (ctx->prof_ev.size() < 2 * (size_t)max_records) {
+        cudaEvent_t ev;
+        CU(ctx, cudaEventCreate(&ev));
+        ctx->prof_ev.push_back(ev);
+    }
+    ctx->prof_cap = (size_t)max_records;
+    ctx->prof_cls.clear();
+    ctx->prof_on = true;
+    return S2MOE_OK;
+}
+
+int s2moe_profile_end(s2moe_ctx *ctx, int32_t n_classes, double *ms_out, int64_t *launches_out)
+{
+    if (!ctx || !ms_out || !launches_out || n_classes < 1) return S2MOE_EINVAL;
+    ctx->prof_on = false;
+    CU(ctx, cudaDeviceSynchronize());
+    for (int c = 0; c < n_classes; ++c) { ms_out[c] = 0.0; launches_out[c] = 0; }
+    for (size_t r = 0; r < ctx->prof_cls.size(); ++r) {
+        float ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&ms, ctx->prof_ev[2 * r], ctx->prof_ev[2 * r + 1]));
+        const int c = ctx->prof_cls[r];
+        if (c < n_classes) { ms_out[c] += ms; launches_out[c] += 1; }
+    }
+    ctx->prof_cls.clear();
+    return S2MOE_OK;
+}
+
+const char *s2moe_kernel_class_name(int32_t cls)
+{
+    switch (cls) {
+        case KC_ROUTER: return "router_logits_kernel";
+        case KC_GATING: return "gating_kernel";
+        case KC_GATEUP: return "ffn_gateup_simple";
+        case KC_DOWN: return "ffn_down_simple";
+        case KC_STREAM: return "ffn_stream_kernel";
+        default: return nullptr;
+    }
+}
+
+int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
+{
+    if (!ctx || !host_out) return S2MOE_EINVAL;
+    CU(ctx, cudaDeviceSynchronize());
+    int32_t hdr[4];
+    CU(ctx, cudaMemcpy(hdr, ctx->ws.header, sizeof(hdr), cudaMemcpyDeviceToHost));
+    const Shape &sh = ctx->shape;
+    const int G = sh.E + sh.n_sh, B = ctx->last_B;
+    const void *src = nullptr;
+    size_t need = 0;
+    switch (what) {
+        case 0: src = ctx->ws.logits; need = sizeof(double) * (size_t)B * sh.E; break;
+        case 1: src = ctx->ws.counts; need = 4 * (size_t)G; break;
+        case 2: src = ctx->ws.offsets; need = 4 * (size_t)(G + 1); break;
+        case 3: src = ctx->ws.slot_token; need = 4 * (size_t)hdr[1]; break;
+        case 4: src = ctx->ws.slot_w; need = 4 * (size_t)hdr[1]; break;
+        case 5: src = ctx->ws.active; need = 4 * (size_t)hdr[0]; break;
+        case 6: src = ctx->ws.header; need = 16; break;
+        default: return S2MOE_EINVAL;
+    }
+    if (bytes < need) return S2MOE_EINVAL;
+    CU(ctx, cudaMemcpy(host_out, src, need, cudaMemcpyDeviceToHost));
+    return S2MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,34 @@
+"""Helpers of the GPU parity tests: run one layer through the C ABI and check it."""
+import numpy as np
+import torch
+
+from oracle import parity
+from paper_2608_15018_b200 import binding, workloads
+
+TOL = {workloads.F32: 2e-3, workloads.BF16: 2e-3, workloads.Q4B32: 1e-2}
+
+
+def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
+             hidden=None, conf=None, check_lists=True):
+    dev = torch.device("cuda", 0)
+    T = workloads.layer_weights(wl, layer, dev)
+    H = workloads.hidden_states(wl, layer, n_tokens, sigma, dev) if hidden is None else hidden.to(dev)
+    if conf is None and use_conf:
+        conf = workloads.confidences(wl, layer, H.shape[0], dev)
+    cfg = binding.Config.from_workload(wl, n_layers=1, kernel_plan=plan)
+    with binding.S2MoE(cfg, [T]) as m:
+        o = m.verify_layer(0, H, conf)
+        torch.cuda.synchronize()
+        assert m.device_status() == 0
+        lists = m.debug_lists() if check_lists else None
+        launches = m.kernel_launches()
+    assert launches > 0
+    ocfg, ow = parity.from_workload(wl, T)
+    sel = o.sel_idx.cpu().numpy()
+    w = o.sel_w.cpu().numpy()
+    rep = parity.check_layer(ocfg, ow, workloads.raw_numpy(H), None if conf is None else conf.cpu().numpy(),
+                             o.out.cpu().numpy(), sel, w, int(o.n_unique.item()),
+                             TOL[wl.weight_dtype], tok_list=tok_list)
+    if lists is not None:
+        parity.check_bucketing(lists, sel, w, wl.n_experts, wl.n_shared)
+    return rep, o

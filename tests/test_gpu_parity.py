@@ -1,0 +1,202 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 oracle, element by element.
+
+Tolerances (max over tokens of max|y - y_ref| / max|y_ref|): 2e-3 for fp32 and bf16
+weights, 1e-2 for block-int4 weights; expert indices and the unique-expert count are
+exact up to router ties below 1e-6, which the checker reports (see oracle/parity.py).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_15018_b200 import binding, workloads
+from paper_2608_15018_b200.workloads import BF16, CONFIGS, F32, Q4B32
+
+from gpu_util import run_case
+
+pytestmark = pytest.mark.gpu
+
+# reduced shapes of the five workload families: same structure, several row tiles and
+# ragged tails, small enough for the oracle to finish in seconds
+SMALL = {
+    "cfg1": CONFIGS["cfg1"],
+    "cfg2": CONFIGS["cfg2"].with_(d_model=512, d_ff=320),
+    "cfg3": CONFIGS["cfg3"].with_(d_model=512, d_ff=352, d_ff_shared=736),
+    "cfg4": CONFIGS["cfg4"].with_(d_model=1024, d_ff=1824),
+    "cfg5": CONFIGS["cfg5"].with_(d_model=512, d_ff=352, d_ff_shared=352),
+}
+PLANS = [1]
+
+
+def plans_for(wl):
+    return [1] if wl.weight_dtype == F32 else PLANS
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+@pytest.mark.parametrize("plan", PLANS)
+def test_small_configs(name, plan):
+    wl = SMALL[name]
+    if plan not in plans_for(wl):
+        pytest.skip("fp32 weights run on the CUDA-core plan")
+    for layer in range(2):
+        rep, _ = run_case(wl, layer=layer, plan=plan)
+        assert rep.tokens_checked == wl.n_tokens
+
+
+@pytest.mark.parametrize("plan", PLANS)
+@pytest.mark.parametrize("renorm,mode,alpha", [(0, 0, 0.5), (1, 0, 0.25), (0, 1, 1.0), (1, 1, 0.5), (0, 0, 0.0)])
+def test_gating_variants(plan, renorm, mode, alpha):
+    wl = SMALL["cfg2"].with_(renorm=renorm, weight_mode=mode, alpha=alpha)
+    run_case(wl, plan=plan)
+    run_case(wl, plan=plan, use_conf=False)
+
+
+@pytest.mark.parametrize("plan", PLANS)
+@pytest.mark.parametrize("B", [1, 2, 4, 8, 16, 32])
+def test_cfg4_batch_sweep(plan, B):
+    run_case(SMALL["cfg4"], n_tokens=B, plan=plan)
+
+
+@pytest.mark.parametrize("plan", PLANS)
+@pytest.mark.parametrize("B,sigma", [(1, 0.3), (2, 1.0), (7, 0.5), (16, 0.1), (33, 0.7), (64, 1.0), (64, 0.1)])
+def test_cfg5_tree_sweep(plan, B, sigma):
+    rep, o = run_case(SMALL["cfg5"], n_tokens=B, sigma=sigma, plan=plan)
+    assert SMALL["cfg5"].top_k <= rep.n_unique <= 64
+
+
+@pytest.mark.parametrize("plan", PLANS)
+def test_degenerate_cases(plan):
+    base = SMALL["cfg5"]
+    run_case(base.with_(top_k=4, cap=64), plan=plan)                      # cap = E: bias off
+    run_case(base.with_(n_experts=8, top_k=8, cap=8), plan=plan)          # k = E: dense sum
+    run_case(base.with_(n_experts=256, top_k=16, cap=40), n_tokens=64, plan=plan)   # limits
+    run_case(base.with_(n_shared=0, d_ff_shared=0), plan=plan)
+    # identical tokens: U = k, reuse ratio 1/B
+    H = workloads.hidden_states(base, 0, 1, device="cuda").repeat(8, 1)
+    rep, _ = run_case(base, hidden=H, plan=plan)
+    assert rep.n_unique == base.top_k
+    # all-zero confidences: E* falls back to the lowest ids
+    run_case(base, conf=torch.zeros(16, device="cuda"), plan=plan)
+    # uncorrelated tokens reach (almost) every expert
+    Hr = torch.randn(64, base.d_model, device="cuda", generator=torch.Generator("cuda").manual_seed(5)).to(torch.bfloat16)
+    rep, _ = run_case(base, hidden=Hr, plan=plan)
+    assert rep.n_unique > 48
+
+
+@pytest.mark.parametrize("plan", PLANS)
+def test_mixed_storage_formats(plan):
+    run_case(SMALL["cfg2"].with_(act_dtype=F32, router_dtype=F32), plan=plan)
+    run_case(SMALL["cfg4"].with_(act_dtype=F32), plan=plan)
+    run_case(SMALL["cfg3"].with_(weight_dtype=Q4B32, d_ff_shared=704), plan=plan)
+    if plan == 1:
+        run_case(SMALL["cfg2"].with_(weight_dtype=F32), plan=plan)
+
+
+@pytest.mark.parametrize("name,tokens", [("cfg2", [0, 7]), ("cfg3", [0, 15]), ("cfg4", [3]), ("cfg5", [9])])
+def test_full_size_layer_sampled_tokens(name, tokens):
+    """Full-size shapes in the plan the benchmark times; the oracle evaluates sampled tokens."""
+    wl = CONFIGS[name]
+    rep, _ = run_case(wl, layer=1, plan=0, tok_list=tokens)
+    assert rep.tokens_checked == len(tokens)
+    torch.cuda.empty_cache()
+
+
+def _ctx(wl, n_layers, plan=0, max_tokens=64):
+    dev = torch.device("cuda", 0)
+    T = [workloads.layer_weights(wl, l, dev) for l in range(n_layers)]
+    cfg = binding.Config.from_workload(wl, n_layers=n_layers, kernel_plan=plan, max_tokens=max_tokens)
+    return binding.S2MoE(cfg, T), T
+
+
+@pytest.mark.parametrize("plan", PLANS)
+def test_stack_host_and_graph_agree_with_single_calls(plan):
+    wl = SMALL["cfg3"]
+    L, B = 3, wl.n_tokens
+    m, T = _ctx(wl, L, plan)
+    dev = torch.device("cuda", 0)
+    H = torch.stack([workloads.hidden_states(wl, l, device=dev) for l in range(L)])
+    C = torch.stack([workloads.confidences(wl, l, device=dev) for l in range(L)])
+    single = [m.verify_layer(l, H[l], C[l]) for l in range(L)]
+    torch.cuda.synchronize()
+    ref_out = torch.stack([s.out for s in single]).cpu()
+    ref_sel = torch.stack([s.sel_idx for s in single]).cpu()
+    ref_w = torch.stack([s.sel_w for s in single]).cpu()
+    ref_u = torch.cat([s.n_unique for s in single]).cpu()
+    scale = ref_out.abs().max().item()
+
+    o = m.verify_stack(H, C)
+    torch.cuda.synchronize()
+    assert torch.equal(o.sel_idx.cpu(), ref_sel) and torch.equal(o.n_unique.cpu(), ref_u)
+    assert torch.equal(o.sel_w.cpu(), ref_w)
+    assert (o.out.cpu() - ref_out).abs().max().item() <= 1e-5 * scale   # atomics reorder fp32 sums
+
+    # host buffers in, host buffers out
+    hh, hc = H.cpu().pin_memory(), C.cpu().pin_memory()
+    ho = torch.empty_like(ref_out).pin_memory(); hs = torch.empty_like(ref_sel).pin_memory()
+    hw = torch.empty_like(ref_w).pin_memory(); hu = torch.empty_like(ref_u).pin_memory()
+    m.verify_stack_host(hh, hc, ho, hs, hw, hu)
+    assert torch.equal(hs, ref_sel) and torch.equal(hu, ref_u) and torch.equal(hw, ref_w)
+    assert (ho - ref_out).abs().max().item() <= 1e-5 * scale
+
+    # CUDA graph capture and replay of the whole stack
+    o2 = m.alloc_outputs(B, stack=True)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.verify_stack(H, C, o2, stream=s)          # warm-up on the capture stream
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.verify_stack(H, C, o2, stream=torch.cuda.current_stream())
+    o2.out.zero_(); o2.sel_idx.zero_()
+    torch.cuda.synchronize()
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(o2.sel_idx.cpu(), ref_sel) and torch.equal(o2.n_unique.cpu(), ref_u)
+    assert (o2.out.cpu() - ref_out).abs().max().item() <= 1e-5 * scale
+    assert m.device_status() == 0
+    m.close()
+
+
+def test_argument_errors_on_device():
+    wl = SMALL["cfg1"]
+    m, T = _ctx(wl, 1, max_tokens=8)
+    dev = torch.device("cuda", 0)
+    H = workloads.hidden_states(wl, 0, 8, device=dev)
+    o = m.alloc_outputs(8)
+    lib = m._lib
+    args = lambda layer, B, h: (m._h, layer, B, h, None, o.out.data_ptr(), o.sel_idx.data_ptr(),
+                                o.sel_w.data_ptr(), o.n_unique.data_ptr(), None)
+    assert lib.s2moe_verify_layer(*args(0, 9, H.data_ptr())) == binding.ERANGE
+    assert lib.s2moe_verify_layer(*args(1, 4, H.data_ptr())) == binding.ERANGE
+    assert lib.s2moe_verify_layer(*args(-1, 4, H.data_ptr())) == binding.ERANGE
+    assert lib.s2moe_verify_layer(*args(0, 4, None)) == binding.EINVAL
+    assert lib.s2moe_verify_layer(*args(0, 4, H.data_ptr() + 4)) == binding.EINVAL
+    assert lib.s2moe_verify_layer(*args(0, 0, None)) == binding.OK            # empty batch: no-op
+    before = m.kernel_launches()
+    assert lib.s2moe_verify_layer(*args(0, 0, H.data_ptr())) == binding.OK
+    assert m.kernel_launches() == before
+    assert lib.s2moe_verify_layer(None, 0, 4, H.data_ptr(), None, None, None, None, None, None) == binding.EINVAL
+    # a good call still works afterwards
+    m.verify_layer(0, H[:4], None, m.alloc_outputs(4))
+    torch.cuda.synchronize()
+    assert m.device_status() == 0
+    assert m.unique_expert_bytes(3) == 3 * 3 * wl.d_model * wl.d_ff * 4
+    m.close()
+
+
+def test_reuse_aware_gating_lowers_unique_experts_on_average():
+    """Direction of the effect the paper reports for the reuse ratio (its Table on
+    expert reuse): over the synthetic routing the bias does not raise the mean
+    number of unique experts."""
+    wl = SMALL["cfg2"]
+    L = 8
+    m1, T = _ctx(wl, L)
+    cfg0 = binding.Config.from_workload(wl.with_(alpha=0.0), n_layers=L)
+    m0 = binding.S2MoE(cfg0, T)
+    dev = torch.device("cuda", 0)
+    H = torch.stack([workloads.hidden_states(wl, l, device=dev) for l in range(L)])
+    C = torch.stack([workloads.confidences(wl, l, device=dev) for l in range(L)])
+    u1 = m1.verify_stack(H, C).n_unique.float().mean().item()
+    u0 = m0.verify_stack(H, C).n_unique.float().mean().item()
+    assert u1 <= u0
+    m0.close(); m1.close()
