@@ -175,6 +175,9 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out);
 /* The last cudaError_t a call on this context saw (0 = cudaSuccess). */
 int s2moe_last_cuda_error(const s2moe_ctx *ctx);
 
+/* The kernel plan in effect (1 or 2; see s2moe_config.kernel_plan), 0 for a NULL context. */
+int s2moe_kernel_plan(const s2moe_ctx *ctx);
+
 /* Kernel launches issued through this context so far (not counting memsets/copies). */
 int64_t s2moe_kernel_launches(const s2moe_ctx *ctx);
 

@@ -24,7 +24,7 @@ WEIGHT_FIELDS = ("router", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down
 EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_verify_stack_host",
            "s2moe_destroy", "s2moe_strerror", "s2moe_last_device_status", "s2moe_last_cuda_error",
            "s2moe_kernel_launches", "s2moe_unique_expert_bytes", "s2moe_debug_read",
-           "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name")
+           "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan")
 KERNEL_CLASSES = 5
 
 
@@ -82,6 +82,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_last_device_status.restype = ctypes.c_int
     lib.s2moe_last_cuda_error.argtypes = [vp]
     lib.s2moe_last_cuda_error.restype = ctypes.c_int
+    lib.s2moe_kernel_plan.argtypes = [vp]
+    lib.s2moe_kernel_plan.restype = ctypes.c_int
     lib.s2moe_kernel_launches.argtypes = [vp]
     lib.s2moe_kernel_launches.restype = ctypes.c_int64
     lib.s2moe_unique_expert_bytes.argtypes = [vp, i32]
@@ -251,6 +253,9 @@ class S2MoE:
         self._check(rc, "s2moe_verify_stack_host")
 
     # -- accounting and diagnostics
+    def kernel_plan(self) -> int:
+        return int(self._lib.s2moe_kernel_plan(self._h))
+
     def kernel_launches(self) -> int:
         return int(self._lib.s2moe_kernel_launches(self._h))
 

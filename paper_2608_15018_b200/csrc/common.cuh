@@ -34,6 +34,7 @@ struct Shape {
     int d, f, E, k, n_sh, f_sh;
     int act_dtype, router_dtype, weight_dtype;
     int renorm, cap, weight_mode;
+    int plan;              // 1: CUDA-core kernels, 2: streaming kernel (unit tables are built)
     double alpha;
 };
 
@@ -53,7 +54,9 @@ struct Workspace {
     int32_t *active;       // [n_active] groups that have tokens, ascending
     float *act;            // SwiGLU activations: routed slot s at s*f, shared slot at
                            // B*k*f + (s - B*k)*f_sh
-    int32_t *sync;         // counters used by the streaming kernels
+    int32_t *sync;         // streaming kernel: finished phase-1 units per active group, then total
+    int32_t *upfx1;        // [n_active + 1] first phase-1 unit of each active group
+    int32_t *upfx2;        // [n_active + 1] first phase-2 unit of each active group
 };
 
 __device__ __forceinline__ size_t act_offset(int slot, int n_routed_slots, int f, int f_sh)

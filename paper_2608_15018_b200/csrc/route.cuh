@@ -8,6 +8,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ffn_stream.cuh"
 
 namespace s2moe {
 
@@ -229,6 +230,23 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
             ws.counts[E + s] = B;
             ws.offsets[E + s] = n_routed + s * B;
             ws.active[U + s] = E + s;
+        }
+    }
+    if (sh.plan == 2) {
+        // unit tables of the streaming kernel: per active group, first phase-1 unit
+        // (8 gate + 8 up rows each) and first phase-2 unit (32 down rows x one K-slice)
+        const int u1r = sh.f / 8, u2r = (sh.d / 32) * st_nks2(sh.f);
+        const int u1s = sh.n_sh ? sh.f_sh / 8 : 0, u2s = sh.n_sh ? (sh.d / 32) * st_nks2(sh.f_sh) : 0;
+        for (int a = tid; a <= U + sh.n_sh; a += nt) {
+            const int r = a < U ? a : U, s = a < U ? 0 : a - U;
+            ws.upfx1[a] = r * u1r + s * u1s;
+            ws.upfx2[a] = r * u2r + s * u2s;
+            ws.sync[a] = 0;
+        }
+        if (tid == 0) {
+            ws.header[4] = U * u1r + sh.n_sh * u1s;
+            ws.header[5] = U * u2r + sh.n_sh * u2s;
+            ws.sync[kStMaxGroups] = 0;
         }
     }
     if (tid == 0) {

@@ -11,6 +11,7 @@
 
 #include "common.cuh"
 #include "ffn_simple.cuh"
+#include "ffn_stream.cuh"
 #include "route.cuh"
 
 using namespace s2moe;
@@ -28,6 +29,8 @@ struct s2moe_ctx {
     int32_t *st_sel = nullptr, *st_nu = nullptr;
     int device = 0;
     int plan = 1;
+    int n_sm = 0;
+    __nv_bfloat16 *act_hi = nullptr, *act_lo = nullptr;
     int last_cuda = 0;
     int64_t launches = 0;
     int last_B = 0;
@@ -98,7 +101,8 @@ int validate_config(const s2moe_config *c)
     if (c->max_tokens < 1 || c->max_tokens > S2MOE_MAX_TOKENS) return S2MOE_EINVAL;
     if (c->n_layers < 1) return S2MOE_EINVAL;
     if (c->kernel_plan < 0 || c->kernel_plan > 2) return S2MOE_EINVAL;
-    if (c->kernel_plan == 2 && c->weight_dtype == S2MOE_F32) return S2MOE_EINVAL;
+    // the streaming plan covers bf16 weights with bf16 activations
+    if (c->kernel_plan == 2 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     return S2MOE_OK;
 }
 
@@ -196,7 +200,15 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         gating_kernel<<<1, kGateThreads, (size_t)B * sh.E * sizeof(double), st>>>(
             sh, B, ctx->ws, conf, lp.sh_scale ? 1 : 0, sel_idx, sel_w, n_unique);
     }
-    DISPATCH_WT_ACT(ctx, launch_simple, ctx, lp, hidden, out, st);
+    if (ctx->plan == 2) {
+        StreamArgs a;
+        a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.hidden = hidden; a.y = out;
+        a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo;
+        LaunchScope scope(ctx, KC_STREAM, st);
+        ffn_stream_kernel<<<ctx->n_sm, kStThreads, kStSmemBytes, st>>>(a);
+    } else {
+        DISPATCH_WT_ACT(ctx, launch_simple, ctx, lp, hidden, out, st);
+    }
     ctx->last_B = B;
     CU(ctx, cudaGetLastError());
     return S2MOE_OK;
@@ -240,7 +252,9 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ctx->layers.resize(config->n_layers);
     static_assert(sizeof(LayerPtrs) == sizeof(s2moe_layer_weights), "layout");
     std::memcpy(ctx->layers.data(), layers, sizeof(LayerPtrs) * (size_t)config->n_layers);
-    ctx->plan = 1;
+    ctx->plan = config->kernel_plan;
+    if (ctx->plan == 0) ctx->plan = (sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16) ? 2 : 1;
+    sh.plan = ctx->plan;
 
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e != cudaSuccess) { delete ctx; return S2MOE_ECUDA; }
@@ -255,7 +269,9 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_ticket = take(256), o_status = take(256), o_header = take(256);
     const size_t o_counts = take(4 * (size_t)G), o_offsets = take(4 * (size_t)(G + 1));
     const size_t o_stok = take(4 * n_slots), o_sw = take(4 * n_slots), o_active = take(4 * (size_t)G);
-    const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(G + 64));
+    const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(kStMaxGroups + 64));
+    const size_t o_ahi = take(2 * act_floats), o_alo = take(2 * act_floats);
+    const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
@@ -264,6 +280,9 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? S2MOE_ENOMEM : S2MOE_ECUDA; }
     e = cudaMemset(ctx->slab, 0, ctx->slab_bytes);
     if (e == cudaSuccess) DISPATCH_WT_ACT(ctx, e = prepare_simple);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e == cudaSuccess && ctx->plan == 2)
+        e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(gating_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)(sizeof(double) * kMaxTokens * kMaxExperts));
@@ -276,6 +295,8 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ws.offsets = (int32_t *)(base + o_offsets); ws.slot_token = (int32_t *)(base + o_stok);
     ws.slot_w = (float *)(base + o_sw); ws.active = (int32_t *)(base + o_active);
     ws.act = (float *)(base + o_act); ws.sync = (int32_t *)(base + o_sync);
+    ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
+    ctx->act_hi = (__nv_bfloat16 *)(base + o_ahi); ctx->act_lo = (__nv_bfloat16 *)(base + o_alo);
     ctx->st_hidden = base + o_sth; ctx->st_conf = (float *)(base + o_stc);
     ctx->st_out = (float *)(base + o_sto); ctx->st_sel = (int32_t *)(base + o_sts);
     ctx->st_selw = (float *)(base + o_stw); ctx->st_nu = (int32_t *)(base + o_stn);
@@ -371,6 +392,8 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out)
 }
 
 int s2moe_last_cuda_error(const s2moe_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int s2moe_kernel_plan(const s2moe_ctx *ctx) { return ctx ? ctx->plan : 0; }
 
 int64_t s2moe_kernel_launches(const s2moe_ctx *ctx) { return ctx ? ctx->launches : 0; }
 

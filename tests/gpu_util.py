@@ -8,8 +8,15 @@ from paper_2608_15018_b200 import binding, workloads
 TOL = {workloads.F32: 2e-3, workloads.BF16: 2e-3, workloads.Q4B32: 1e-2}
 
 
+def supports(wl, plan):
+    """Kernel plan 2 (streaming tensor-core kernel) covers bf16 weights with bf16 activations."""
+    return plan != 2 or (wl.weight_dtype == workloads.BF16 and wl.act_dtype == workloads.BF16)
+
+
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
              hidden=None, conf=None, check_lists=True):
+    if not supports(wl, plan):
+        return None, None
     dev = torch.device("cuda", 0)
     T = workloads.layer_weights(wl, layer, dev)
     H = workloads.hidden_states(wl, layer, n_tokens, sigma, dev) if hidden is None else hidden.to(dev)

@@ -11,7 +11,7 @@ import torch
 from paper_2608_15018_b200 import binding, workloads
 from paper_2608_15018_b200.workloads import BF16, CONFIGS, F32, Q4B32
 
-from gpu_util import run_case
+from gpu_util import run_case, supports
 
 pytestmark = pytest.mark.gpu
 
@@ -24,19 +24,15 @@ SMALL = {
     "cfg4": CONFIGS["cfg4"].with_(d_model=1024, d_ff=1824),
     "cfg5": CONFIGS["cfg5"].with_(d_model=512, d_ff=352, d_ff_shared=352),
 }
-PLANS = [1]
-
-
-def plans_for(wl):
-    return [1] if wl.weight_dtype == F32 else PLANS
+PLANS = [1, 2]
 
 
 @pytest.mark.parametrize("name", sorted(SMALL))
 @pytest.mark.parametrize("plan", PLANS)
 def test_small_configs(name, plan):
     wl = SMALL[name]
-    if plan not in plans_for(wl):
-        pytest.skip("fp32 weights run on the CUDA-core plan")
+    if not supports(wl, plan):
+        pytest.skip("the streaming plan covers bf16 weights with bf16 activations")
     for layer in range(2):
         rep, _ = run_case(wl, layer=layer, plan=plan)
         assert rep.tokens_checked == wl.n_tokens
@@ -53,6 +49,8 @@ def test_gating_variants(plan, renorm, mode, alpha):
 @pytest.mark.parametrize("plan", PLANS)
 @pytest.mark.parametrize("B", [1, 2, 4, 8, 16, 32])
 def test_cfg4_batch_sweep(plan, B):
+    if not supports(SMALL["cfg4"], plan):
+        pytest.skip("the streaming plan covers bf16 weights with bf16 activations")
     run_case(SMALL["cfg4"], n_tokens=B, plan=plan)
 
 
@@ -112,6 +110,7 @@ def test_stack_host_and_graph_agree_with_single_calls(plan):
     wl = SMALL["cfg3"]
     L, B = 3, wl.n_tokens
     m, T = _ctx(wl, L, plan)
+    assert m.kernel_plan() == plan
     dev = torch.device("cuda", 0)
     H = torch.stack([workloads.hidden_states(wl, l, device=dev) for l in range(L)])
     C = torch.stack([workloads.confidences(wl, l, device=dev) for l in range(L)])
