@@ -113,8 +113,9 @@ typedef struct {
     int32_t weight_mode;   /* 0: mixing weights from l, 1: from l'                          */
     int32_t max_tokens;    /* 1..S2MOE_MAX_TOKENS: workspace bound for n_tokens             */
     int32_t n_layers;      /* >= 1                                                          */
-    int32_t kernel_plan;   /* 0: automatic; 1: plain CUDA-core kernels (all dtypes);
-                              2: streaming tensor-core kernels (BF16 / Q4B32 weights)        */
+    int32_t kernel_plan;   /* 0: automatic (plan 2 where it applies, else plan 1);
+                              1: plain CUDA-core kernels (every format and batch size);
+                              2: streaming tensor-core kernel (bf16 weights and activations) */
 } s2moe_config;
 
 /*
@@ -175,8 +176,10 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out);
 /* The last cudaError_t a call on this context saw (0 = cudaSuccess). */
 int s2moe_last_cuda_error(const s2moe_ctx *ctx);
 
-/* The kernel plan in effect (1 or 2; see s2moe_config.kernel_plan), 0 for a NULL context. */
-int s2moe_kernel_plan(const s2moe_ctx *ctx);
+/* The kernel plan a batch of n_tokens runs with (1 or 2; see s2moe_config.kernel_plan).
+ * 0: NULL context, n_tokens out of range, or plan 2 was demanded and this batch size
+ * does not fit its shared-memory layout (s2moe_verify_layer then returns EINVAL). */
+int s2moe_kernel_plan(const s2moe_ctx *ctx, int32_t n_tokens);
 
 /* Kernel launches issued through this context so far (not counting memsets/copies). */
 int64_t s2moe_kernel_launches(const s2moe_ctx *ctx);

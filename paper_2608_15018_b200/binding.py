@@ -82,7 +82,7 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_last_device_status.restype = ctypes.c_int
     lib.s2moe_last_cuda_error.argtypes = [vp]
     lib.s2moe_last_cuda_error.restype = ctypes.c_int
-    lib.s2moe_kernel_plan.argtypes = [vp]
+    lib.s2moe_kernel_plan.argtypes = [vp, i32]
     lib.s2moe_kernel_plan.restype = ctypes.c_int
     lib.s2moe_kernel_launches.argtypes = [vp]
     lib.s2moe_kernel_launches.restype = ctypes.c_int64
@@ -253,8 +253,9 @@ class S2MoE:
         self._check(rc, "s2moe_verify_stack_host")
 
     # -- accounting and diagnostics
-    def kernel_plan(self) -> int:
-        return int(self._lib.s2moe_kernel_plan(self._h))
+    def kernel_plan(self, n_tokens: int) -> int:
+        """Kernel plan a batch of ``n_tokens`` runs with (0: demanded plan not runnable)."""
+        return int(self._lib.s2moe_kernel_plan(self._h, int(n_tokens)))
 
     def kernel_launches(self) -> int:
         return int(self._lib.s2moe_kernel_launches(self._h))

@@ -34,7 +34,8 @@ struct Shape {
     int d, f, E, k, n_sh, f_sh;
     int act_dtype, router_dtype, weight_dtype;
     int renorm, cap, weight_mode;
-    int plan;              // 1: CUDA-core kernels, 2: streaming kernel (unit tables are built)
+    int plan;              // 1: CUDA-core kernels, 2: streaming kernel (stage tables are built)
+    int op_cap;            // streaming kernel: capacity of the phase-2 operand region, bytes
     double alpha;
 };
 
@@ -54,9 +55,10 @@ struct Workspace {
     int32_t *active;       // [n_active] groups that have tokens, ascending
     float *act;            // SwiGLU activations: routed slot s at s*f, shared slot at
                            // B*k*f + (s - B*k)*f_sh
-    int32_t *sync;         // streaming kernel: finished phase-1 units per active group, then total
-    int32_t *upfx1;        // [n_active + 1] first phase-1 unit of each active group
-    int32_t *upfx2;        // [n_active + 1] first phase-2 unit of each active group
+    int32_t *sync;         // streaming kernel: finished phase-1 stages per active group
+    int32_t *upfx1;        // [n_active + 1] first phase-1 stage of each active group
+    int32_t *upfx2;        // [n_active + 1] first phase-2 stage of each active group
+    unsigned long long *tokmask;   // [E + n_sh] bit b set: token b is bucketed to the group
 };
 
 __device__ __forceinline__ size_t act_offset(int slot, int n_routed_slots, int f, int f_sh)

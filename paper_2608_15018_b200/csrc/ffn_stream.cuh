@@ -1,21 +1,26 @@
 // Streaming expert kernel (kernel plan 2): one persistent CTA per SM reads every
 // selected expert's weights from HBM exactly once through a ring of TMA bulk copies
-// and contracts them with the tokens bucketed to that expert on the tensor cores.
+// and contracts them with the draft tokens on the tensor cores.
 //
-// Work is cut into units of equal cost, taken round-robin by the CTAs:
-//   phase 1 unit: 8 gate rows + 8 up rows of one expert (all of K = d)
-//                 -> a[slot][j] = silu(g) * u, stored as bf16 hi + lo parts
-//   phase 2 unit: 32 down rows of one expert, one K-slice of f
-//                 -> y[token][r] += p * (W_d[r] . a[slot])        (red.add, fp32)
-// All phase-1 units precede all phase-2 units; a phase-2 unit of an expert waits on a
-// counter of that expert's finished phase-1 units (bounded wait).
+// Work items are "stages": the bytes one consumer warp turns into finished outputs.
+//   phase 1 stage: 4 gate rows + 4 up rows of one expert, all of K = d (two contiguous
+//                  copies).  The hidden states of ALL B tokens stay resident in shared
+//                  memory, the contraction runs over all of them, and only the tokens
+//                  bucketed to this expert store a = silu(g) * u (as bf16 hi + lo).
+//   phase 2 stage: 8 down rows of one expert over one K-slice of f, contracted with
+//                  the expert's activations (resident operand), y += p * result.
+// Phase-1 stages are dealt round-robin to the CTAs; phase-2 stages are split into one
+// contiguous range per CTA so that a CTA needs the activations of one or two experts
+// only.  A phase-2 operand load waits on a counter of that expert's finished phase-1
+// stages.  Every wait in the kernel is bounded and reports through the status word.
 //
-// Inside a CTA one producer warp issues the copies (one cp.async.bulk per weight row
-// chunk and per token row chunk, completing on an mbarrier) and eight consumer warps
-// split each staged chunk along K.  The contraction is mma.sync m16n8k16 with the
-// tokens as the M operand and eight weight rows as the N operand; the K index inside
-// every 32-wide step is permuted identically for both operands so that each lane feeds
-// the tensor core straight from one 128-bit shared-memory load per row.
+// Inside a CTA one producer warp issues the copies; each of the eight consumer warps
+// takes every eighth stage and finishes it alone (no CTA-wide barrier anywhere).
+// The contraction is mma.sync m16n8k16 with tokens as the M operand and eight weight
+// rows as the N operand.  The K index inside every 32-wide step is permuted identically
+// for both operands, so each lane feeds the tensor core from one 128-bit shared-memory
+// load per row; the two 4-row halves of a stage are placed 64 bytes apart modulo 128 so
+// that those loads are free of bank conflicts.
 #pragma once
 
 #include "common.cuh"
@@ -24,29 +29,100 @@ namespace s2moe {
 
 constexpr int kStConsumerWarps = 8;
 constexpr int kStThreads = (kStConsumerWarps + 1) * 32;
-constexpr int kStStages = 5;
-constexpr int kStRegion = 18432;                       // bytes per operand / weight region of a slot
-constexpr int kStSlotBytes = 2 * kStRegion;
-constexpr int kStScratchBytes = 16384;
+constexpr int kStMaxStages = 8;
 constexpr int kStMaxGroups = kMaxExperts + kMaxShared;
-constexpr size_t kStSmemBytes = (size_t)kStStages * kStSlotBytes + kStScratchBytes;
-constexpr unsigned kStSpinLimit = 1u << 22;            // bounded waits (each poll ~ 50-100 ns)
+constexpr unsigned kStSpinLimit = 1u << 22;   // bounded waits (a poll takes some tens of ns)
+constexpr int kStMaxSmem = 232448 - 2048;     // dynamic shared memory the kernel may use
+
+// Per-call plan, computed on the host (st_make_plan) and passed by value.
+struct StPlan {
+    int feasible;
+    int n_cta;
+    int stages;       // ring slots
+    int slot_bytes;   // bytes per ring slot
+    int x_pitch;      // bytes per token row of the resident hidden states (d*2 + 64)
+    int x_bytes;      // pad8(B) * x_pitch
+    int op_cap;       // capacity of the phase-2 operand region
+    int alias;        // 1: the operand region is the hidden-state region (drained first)
+    int tab_bytes;    // group and slot tables
+    int smem_bytes;   // total dynamic shared memory
+};
+
+struct StGroup {      // one active group, in shared memory
+    unsigned long long mask;   // tokens of the batch bucketed to this group
+    int group, T, off, f;      // group id, tokens, first slot, inner dim
+    int p1, p2;                // first phase-1 / phase-2 stage of the group
+    int nks, ksl;              // K-slices of a phase-2 row and their length
+};
 
 struct StageDesc {
-    int unit, chunk, nchunks, group_slot;   // group_slot: index into the active list
-    int phase, tile, T, off;                // tokens of the group, first slot
-    int klen, pitch_w, pitch_o, tpad8;      // this chunk's K length, row pitches, padded tokens
-    int f_g, k_begin, group, pad_;
+    int phase, gslot, tile, ks;   // gslot: index into the active list
+    int klen, op_gen, rc, pad_;   // K elements, operand generation, row chunk bytes
 };
 
 struct StreamArgs {
     Shape sh;
     LayerPtrs lp;
     Workspace ws;
+    StPlan plan;
     const void *hidden;
     float *y;
     __nv_bfloat16 *act_hi, *act_lo;
+    int B;
 };
+
+// ---- shapes shared by the host planner, the gating kernel and this kernel ----------
+
+__host__ __device__ __forceinline__ int st_pad8(int t) { return (t + 7) & ~7; }
+
+// number of K-slices of a phase-2 row of inner dim f for T tokens, given the operand
+// capacity: hi and lo rows of pad8(T) tokens, each row padded by 64 bytes
+__host__ __device__ __forceinline__ int st_nks(int f, int T, int op_cap)
+{
+    const int rows = 2 * st_pad8(T);
+    int kmax = ((op_cap / rows - 64) / 2) & ~31;
+    if (kmax < 32) kmax = 32;
+    return (f + kmax - 1) / kmax;
+}
+__host__ __device__ __forceinline__ int st_ksl(int f, int nks) { return ((f / 32 + nks - 1) / nks) * 32; }
+
+inline StPlan st_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
+{
+    StPlan p{};
+    const int G = sh.E + sh.n_sh;
+    p.n_cta = n_sm;
+    p.x_pitch = sh.d * 2 + 64;
+    p.x_bytes = st_pad8(B) * p.x_pitch;
+    const int fmax = sh.n_sh && sh.f_sh > sh.f ? sh.f_sh : sh.f;
+    const int stage1 = 8 * sh.d * 2 + 128;
+    p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 127) & ~127;
+    const int avail = kStMaxSmem - p.tab_bytes;
+    const int op_full = 2 * st_pad8(B) * (fmax * 2 + 64);
+    const int op_min = 2 * st_pad8(B) * (256 * 2 + 64);
+    p.slot_bytes = stage1;
+    p.stages = 4;
+    const int left = avail - p.x_bytes - p.stages * p.slot_bytes;
+    if (left >= op_min) {
+        p.alias = 0;
+        p.op_cap = left < op_full ? left : op_full;
+    } else {
+        p.alias = 1;
+        p.op_cap = avail - p.stages * p.slot_bytes;
+        if (p.op_cap < p.x_bytes || p.op_cap < op_min) {
+            p.stages = 3;
+            p.op_cap = avail - p.stages * p.slot_bytes;
+        }
+    }
+    p.op_cap = (p.op_cap + 127) & ~127;
+    if (p.op_cap > avail) p.op_cap = avail & ~127;
+    // a phase-2 stage (8 rows of one K-slice) must fit a ring slot
+    const int ksl_max = st_ksl(fmax, st_nks(fmax, B, p.op_cap));
+    p.smem_bytes = p.tab_bytes + (p.alias ? p.op_cap : p.x_bytes + p.op_cap) + p.stages * p.slot_bytes;
+    const bool fits = p.op_cap >= op_min && (!p.alias || p.op_cap >= p.x_bytes) &&
+                      8 * ksl_max * 2 + 128 <= p.slot_bytes && p.smem_bytes <= kStMaxSmem && B <= kMaxTokens;
+    p.feasible = fits && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16;
+    return p;
+}
 
 // ---- PTX helpers ---------------------------------------------------------------
 
@@ -99,17 +175,6 @@ __device__ __forceinline__ int ld_acquire(const int *p)
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// Barrier among the consumer warps built on an mbarrier so that the wait is bounded
-// (a hardware bar.sync would hang for ever if a warp had left after a time-out).
-// `phase` is the caller's running parity bit.  Returns false when it gave up.
-__device__ __forceinline__ bool consumer_bar(uint64_t *bar, uint32_t &phase, int lane)
-{
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar);
-    const bool ok = mbar_wait(bar, phase);
-    phase ^= 1u;
-    return ok;
-}
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1)
 {
@@ -120,349 +185,367 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// row pitch in shared memory: consecutive rows must differ by 64 bytes modulo 128 so
-// that the 128-bit loads of a quarter warp (two rows x 64 bytes) hit distinct banks
-__host__ __device__ __forceinline__ int st_pitch(int chunk_bytes)
+__device__ __forceinline__ int upper_group1(const StGroup *g, int n, int u)
 {
-    return (chunk_bytes % 128 == 64) ? chunk_bytes : chunk_bytes + 64;
-}
-
-// K elements staged per chunk for a group with tpad8 padded tokens
-__host__ __device__ __forceinline__ int st_kc(int phase, int tpad8)
-{
-    const int rows_w = phase == 1 ? 16 : 32;
-    const int rows_o = phase == 1 ? tpad8 : 2 * tpad8;
-    int kc = phase == 1 ? 512 : 256;
-    while (kc > 32 && (rows_w * st_pitch(kc * 2) > kStRegion || rows_o * st_pitch(kc * 2) > kStRegion)) kc >>= 1;
-    return kc;
-}
-
-// number of K-slices of a phase-2 unit so that a unit holds at most 64 KiB of weights
-__host__ __device__ __forceinline__ int st_nks2(int f_g)
-{
-    const int n = (32 * f_g * 2 + 65535) / 65536;
-    return n < 1 ? 1 : n;
-}
-__host__ __device__ __forceinline__ int st_kslice2(int f_g) { return ((f_g / 32 + st_nks2(f_g) - 1) / st_nks2(f_g)) * 32; }
-
-__device__ __forceinline__ int upper_group(const int *pfx, int n, int u)
-{
-    int lo = 0, hi = n;                 // largest a with pfx[a] <= u
+    int lo = 0, hi = n;   // largest a with g[a].p1 <= u
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (pfx[mid] <= u) lo = mid; else hi = mid;
+        if (g[mid].p1 <= u) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+__device__ __forceinline__ int upper_group2(const StGroup *g, int n, int u)
+{
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (g[mid].p2 <= u) lo = mid; else hi = mid;
     }
     return lo;
 }
 
-// ---- the kernel -----------------------------------------------------------------
+// ---- consumer side ----------------------------------------------------------------
 
-template <int MT, int PHASE>
-__device__ __forceinline__ bool consume_unit(const StreamArgs &p, uint8_t *slots, float *scratch, uint64_t *full_bar,
-                                             uint64_t *empty_bar, const StageDesc *desc, unsigned &it, int warp,
-                                             int lane, int ctid, uint64_t *cbar, uint32_t &cphase)
+// One phase-1 stage: D[token][gate/up row pairs] over all of K, then SwiGLU and store.
+template <int MT>
+__device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGroup &grp, const StageDesc &d,
+                                               const uint8_t *wreg, const uint8_t *xreg, int lane)
 {
-    constexpr int NT = PHASE == 1 ? 2 : 4;
     const int g = lane >> 2, t = lane & 3;
-    float acc[MT][NT][4];
+    const int rowbytes = p.sh.d * 2;
+    const uint8_t *wrow = wreg + (size_t)(g >> 1) * rowbytes + (size_t)(g & 1) * (4 * rowbytes + 64) + t * 16;
+    const int bpad = st_pad8(p.B);
+    float acc[MT][4];
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int n = 0; n < NT; ++n)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) acc[m][n][q] = 0.f;
-
-    StageDesc d;
-    while (true) {
-        const int slot = it % kStStages;
-        const uint32_t parity = (it / kStStages) & 1u;
-        if (!mbar_wait(&full_bar[slot], parity)) return false;
-        d = desc[slot];
-        const uint8_t *wreg = slots + (size_t)slot * kStSlotBytes;
-        const uint8_t *oreg = wreg + kStRegion;
-        const int nsteps = d.klen >> 5;
-        for (int s = warp; s < nsteps; s += kStConsumerWarps) {
-            const int boff = s * 64 + t * 16;
-            uint4 xa[MT], xb[MT], la[MT], lb[MT];
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                const int r0 = m * 16 + g, r1 = r0 + 8;
-                xa[m] = *reinterpret_cast<const uint4 *>(oreg + (size_t)r0 * d.pitch_o + boff);
-                xb[m] = r1 < d.tpad8 ? *reinterpret_cast<const uint4 *>(oreg + (size_t)r1 * d.pitch_o + boff)
-                                     : make_uint4(0, 0, 0, 0);
-                if (PHASE == 2) {
-                    la[m] = *reinterpret_cast<const uint4 *>(oreg + (size_t)(d.tpad8 + r0) * d.pitch_o + boff);
-                    lb[m] = r1 < d.tpad8
-                                ? *reinterpret_cast<const uint4 *>(oreg + (size_t)(d.tpad8 + r1) * d.pitch_o + boff)
-                                : make_uint4(0, 0, 0, 0);
-                }
-            }
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                const uint4 w = *reinterpret_cast<const uint4 *>(wreg + (size_t)(n * 8 + g) * d.pitch_w + boff);
-#pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    mma_bf16(acc[m][n], xa[m].x, xb[m].x, xa[m].y, xb[m].y, w.x, w.y);
-                    mma_bf16(acc[m][n], xa[m].z, xb[m].z, xa[m].w, xb[m].w, w.z, w.w);
-                    if (PHASE == 2) {
-                        mma_bf16(acc[m][n], la[m].x, lb[m].x, la[m].y, lb[m].y, w.x, w.y);
-                        mma_bf16(acc[m][n], la[m].z, lb[m].z, la[m].w, lb[m].w, w.z, w.w);
-                    }
-                }
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[slot]);
-        ++it;
-        if (d.chunk == d.nchunks - 1) break;
-    }
-
-    // cross-warp reduction and epilogue, one m-tile (16 tokens) per round
-    constexpr int COLS = NT * 8;
-    const int n_routed = p.ws.header[3] * p.sh.k;
+        for (int q = 0; q < 4; ++q) acc[m][q] = 0.f;
+    const uint8_t *xrow[MT];
+    bool has1[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) {
-        float *mine = scratch + (size_t)warp * 16 * COLS;
+        xrow[m] = xreg + (size_t)(m * 16 + g) * p.plan.x_pitch + t * 16;
+        has1[m] = m * 16 + g + 8 < bpad;
+    }
+    const size_t x8 = (size_t)8 * p.plan.x_pitch;
+    const int nsteps = p.sh.d >> 5;
+#pragma unroll 4
+    for (int s = 0; s < nsteps; ++s) {
+        const uint4 w = *reinterpret_cast<const uint4 *>(wrow + s * 64);
 #pragma unroll
-        for (int n = 0; n < NT; ++n) {
-            *reinterpret_cast<float2 *>(&mine[g * COLS + n * 8 + 2 * t]) = make_float2(acc[m][n][0], acc[m][n][1]);
-            *reinterpret_cast<float2 *>(&mine[(g + 8) * COLS + n * 8 + 2 * t]) =
-                make_float2(acc[m][n][2], acc[m][n][3]);
+        for (int m = 0; m < MT; ++m) {
+            const uint4 xa = *reinterpret_cast<const uint4 *>(xrow[m] + s * 64);
+            const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(xrow[m] + x8 + s * 64) : make_uint4(0, 0, 0, 0);
+            mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+            mma_bf16(acc[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
         }
-        if (!consumer_bar(cbar, cphase, lane)) return false;
-        if (PHASE == 1) {
-            if (ctid < 128) {
-                const int tt = ctid >> 3, j = ctid & 7;
-                const int ti = m * 16 + tt;
-                float sg = 0.f, su = 0.f;
+    }
+    // lane (g, t) holds (gate row t, up row t) of tokens g and g + 8 of every m-tile
+    const int n_routed = p.B * p.sh.k;
 #pragma unroll
-                for (int w = 0; w < kStConsumerWarps; ++w) {
-                    sg += scratch[(size_t)w * 16 * COLS + tt * COLS + j];
-                    su += scratch[(size_t)w * 16 * COLS + tt * COLS + 8 + j];
-                }
-                if (ti < d.T) {
-                    const float a = silu_mul(sg, su);
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-                    const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
-                    const size_t o = act_offset(d.off + ti, n_routed, p.sh.f, p.sh.f_sh) + (size_t)d.tile * 8 + j;
-                    p.act_hi[o] = hi;
-                    p.act_lo[o] = lo;
-                }
-            }
-            __threadfence();
-            fence_proxy_async();
-        } else {
-            const int tt = ctid >> 4, c0 = (ctid & 15) * 2;
-            const int ti = m * 16 + tt;
-            float s0 = 0.f, s1 = 0.f;
+    for (int m = 0; m < MT; ++m) {
 #pragma unroll
-            for (int w = 0; w < kStConsumerWarps; ++w) {
-                const float2 v = *reinterpret_cast<const float2 *>(&scratch[(size_t)w * 16 * COLS + tt * COLS + c0]);
-                s0 += v.x;
-                s1 += v.y;
-            }
-            if (ti < d.T) {
-                const int slot = d.off + ti;
-                const float pw = p.ws.slot_w[slot];
-                float *dst = p.y + (size_t)p.ws.slot_token[slot] * p.sh.d + (size_t)d.tile * 32 + c0;
-                atomicAdd(dst, pw * s0);
-                atomicAdd(dst + 1, pw * s1);
+        for (int h = 0; h < 2; ++h) {
+            const int b = m * 16 + g + 8 * h;
+            if (b < p.B && ((grp.mask >> b) & 1ull)) {
+                const int slot = grp.off + __popcll(grp.mask & ((1ull << b) - 1ull));
+                const float a = silu_mul(acc[m][2 * h], acc[m][2 * h + 1]);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(a);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+                const size_t o = act_offset(slot, n_routed, p.sh.f, p.sh.f_sh) + (size_t)d.tile * 4 + t;
+                p.act_hi[o] = hi;
+                p.act_lo[o] = lo;
             }
         }
-        if (!consumer_bar(cbar, cphase, lane)) return false;
     }
-    if (PHASE == 1 && ctid == 0) {
-        atomicAdd(&p.ws.sync[d.group_slot], 1);
-        atomicAdd(&p.ws.sync[kStMaxGroups], 1);
-    }
-    return true;
+    // release: this warp's stores, then one count for the stage
+    __threadfence();
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) atomicAdd(&p.ws.sync[d.gslot], 1);
 }
+
+// One phase-2 stage: D[slot][8 down rows] over one K-slice, y += p * D.
+template <int MT>
+__device__ __forceinline__ void consume_phase2(const StreamArgs &p, const StGroup &grp, const StageDesc &d,
+                                               const uint8_t *wreg, const uint8_t *oreg, const int *slot_token,
+                                               const float *slot_w, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const int rc = d.rc;                       // bytes of one weight row chunk
+    const int opitch = d.klen * 2 + 64;        // operand row pitch
+    const int tpad = st_pad8(grp.T);
+    const uint8_t *wrow = wreg + (size_t)(g >> 1) * rc + (size_t)(g & 1) * (4 * rc + 64) + t * 16;
+    float acc[MT][4];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[m][q] = 0.f;
+    const uint8_t *hrow[MT];
+    bool has1[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        hrow[m] = oreg + (size_t)(m * 16 + g) * opitch + t * 16;
+        has1[m] = m * 16 + g + 8 < tpad;
+    }
+    const size_t o8 = (size_t)8 * opitch;
+    const size_t lo_off = (size_t)tpad * opitch;
+    const int nsteps = d.klen >> 5;
+#pragma unroll 2
+    for (int s = 0; s < nsteps; ++s) {
+        const uint4 w = *reinterpret_cast<const uint4 *>(wrow + s * 64);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            const uint4 z = make_uint4(0, 0, 0, 0);
+            const uint4 xa = *reinterpret_cast<const uint4 *>(hrow[m] + s * 64);
+            const uint4 la = *reinterpret_cast<const uint4 *>(hrow[m] + lo_off + s * 64);
+            const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + s * 64) : z;
+            const uint4 lb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + lo_off + s * 64) : z;
+            mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+            mma_bf16(acc[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+            mma_bf16(acc[m], la.x, lb.x, la.y, lb.y, w.x, w.y);
+            mma_bf16(acc[m], la.z, lb.z, la.w, lb.w, w.z, w.w);
+        }
+    }
+    // lane (g, t): columns 2t, 2t+1 are down rows t and 4 + t of the stage
+    const int r0 = d.tile * 8 + t;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int ti = m * 16 + g + 8 * h;
+            if (ti < grp.T) {
+                const int slot = grp.off + ti;
+                const float pw = slot_w[slot];
+                float *dst = p.y + (size_t)slot_token[slot] * p.sh.d + r0;
+                atomicAdd(dst, pw * acc[m][2 * h]);
+                atomicAdd(dst + 4, pw * acc[m][2 * h + 1]);
+            }
+        }
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------
 
 __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
 {
     extern __shared__ __align__(128) uint8_t st_smem[];
-    __shared__ __align__(8) uint64_t full_bar[kStStages];
-    __shared__ __align__(8) uint64_t empty_bar[kStStages];
-    __shared__ __align__(8) uint64_t cbar;
-    __shared__ StageDesc desc[kStStages];
-    __shared__ int s_pfx1[kStMaxGroups + 1], s_pfx2[kStMaxGroups + 1];
+    __shared__ __align__(8) uint64_t full_bar[kStMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStMaxStages];
+    __shared__ __align__(8) uint64_t x_bar, op_bar;
+    __shared__ StageDesc desc[kStMaxStages];
 
-    uint8_t *slots = st_smem;
-    float *scratch = reinterpret_cast<float *>(st_smem + (size_t)kStStages * kStSlotBytes);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const StPlan &pl = p.plan;
+    const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
-    const int n_active = ws.header[0];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_active = ws.header[0], n_slots = ws.header[1];
     const int total1 = ws.header[4], total2 = ws.header[5];
-    const int total = total1 + total2;
+    const int G = sh.E + sh.n_sh;
 
-    for (int i = tid; i <= n_active; i += blockDim.x) {
-        s_pfx1[i] = ws.upfx1[i];
-        s_pfx2[i] = ws.upfx2[i];
+    // shared memory: [group table | slot_token | slot_w | hidden states | operand | ring]
+    StGroup *groups = reinterpret_cast<StGroup *>(st_smem);
+    const int tab_rest = pl.tab_bytes - (int)sizeof(StGroup) * (G + 1);
+    int *s_slot_token = reinterpret_cast<int *>(st_smem + sizeof(StGroup) * (G + 1));
+    float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
+    uint8_t *xreg = st_smem + pl.tab_bytes;
+    uint8_t *oreg = pl.alias ? xreg : xreg + pl.x_bytes;
+    uint8_t *ring = oreg + pl.op_cap;
+
+    for (int a = tid; a < n_active; a += blockDim.x) {
+        StGroup gr;
+        gr.group = ws.active[a];
+        gr.T = ws.counts[gr.group];
+        gr.off = ws.offsets[gr.group];
+        gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
+        gr.mask = ws.tokmask[gr.group];
+        gr.p1 = ws.upfx1[a];
+        gr.p2 = ws.upfx2[a];
+        gr.nks = st_nks(gr.f, gr.T, pl.op_cap);
+        gr.ksl = st_ksl(gr.f, gr.nks);
+        groups[a] = gr;
+    }
+    for (int i = tid; i < n_slots; i += blockDim.x) {
+        s_slot_token[i] = ws.slot_token[i];
+        s_slot_w[i] = ws.slot_w[i];
     }
     if (tid == 0) {
-        for (int s = 0; s < kStStages; ++s) {
+        for (int s = 0; s < pl.stages; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], kStConsumerWarps);
+            mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&cbar, kStConsumerWarps);
+        mbar_init(&x_bar, 1);
+        mbar_init(&op_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    const Shape &sh = p.sh;
+    // this CTA's work: phase-1 stages blockIdx.x, +gridDim.x, ...; phase-2 stages [lo2, hi2)
+    const int P = gridDim.x;
+    const int n1_mine = total1 > (int)blockIdx.x ? (total1 - 1 - (int)blockIdx.x) / P + 1 : 0;
+    const int lo2 = (int)(((long long)total2 * blockIdx.x) / P);
+    const int hi2 = (int)(((long long)total2 * (blockIdx.x + 1)) / P);
+    const int n_mine = n1_mine + (hi2 - lo2);
+    const int S = pl.stages;
+
     if (warp == kStConsumerWarps) {
         // ------------------------------------------------------------ producer warp
-        unsigned it = 0;
-        bool all_ready = false, alive = true;
-        for (int u = blockIdx.x; u < total && alive; u += gridDim.x) {
+        bool alive = true;
+        // hidden states of all tokens, one copy per token row
+        if (lane == 0) mbar_expect_tx(&x_bar, (uint32_t)p.B * sh.d * 2);
+        __syncwarp();
+        for (int b = lane; b < p.B; b += 32)
+            bulk_g2s(xreg + (size_t)b * pl.x_pitch, (const uint8_t *)p.hidden + (size_t)b * sh.d * 2, sh.d * 2, &x_bar);
+
+        int cur_a = -1, cur_ks = -1, op_gen = 0;
+        for (int n = 0; n < n_mine && alive; ++n) {
             StageDesc d;
-            d.unit = u;
-            d.phase = u < total1 ? 1 : 2;
-            int ks = 0;
-            if (d.phase == 1) {
-                d.group_slot = upper_group(s_pfx1, n_active, u);
-                d.tile = u - s_pfx1[d.group_slot];
+            const uint8_t *src0, *src1;   // the two 4-row halves
+            size_t rstride;
+            if (n < n1_mine) {
+                const int u = blockIdx.x + n * P;
+                d.phase = 1;
+                d.gslot = upper_group1(groups, n_active, u);
+                const StGroup &gr = groups[d.gslot];
+                d.tile = u - gr.p1;
+                d.ks = 0;
+                d.klen = sh.d;
+                d.op_gen = 0;
+                d.rc = sh.d * 2;
+                rstride = (size_t)sh.d * 2;
+                const bool shared = gr.group >= sh.E;
+                const size_t e = shared ? gr.group - sh.E : gr.group;
+                const size_t r0 = (e * gr.f + (size_t)d.tile * 4) * rstride;
+                src0 = (const uint8_t *)(shared ? p.lp.sh_gate : p.lp.w_gate) + r0;
+                src1 = (const uint8_t *)(shared ? p.lp.sh_up : p.lp.w_up) + r0;
             } else {
-                const int v = u - total1;
-                d.group_slot = upper_group(s_pfx2, n_active, v);
-                d.tile = v - s_pfx2[d.group_slot];
-            }
-            d.group = ws.active[d.group_slot];
-            d.T = ws.counts[d.group];
-            d.off = ws.offsets[d.group];
-            d.tpad8 = (d.T + 7) & ~7;
-            const bool shared = d.group >= sh.E;
-            d.f_g = shared ? sh.f_sh : sh.f;
-            const int e = shared ? d.group - sh.E : d.group;
-            const int kc = st_kc(d.phase, d.tpad8);
-            int klen_unit;
-            const uint8_t *wrow0, *wrow1 = nullptr;   // first row of the unit (gate / down), up rows
-            size_t row_stride;
-            if (d.phase == 1) {
-                d.k_begin = 0;
-                klen_unit = sh.d;
-                row_stride = (size_t)sh.d * 2;
-                const size_t r0 = ((size_t)e * d.f_g + (size_t)d.tile * 8) * row_stride;
-                wrow0 = (const uint8_t *)(shared ? p.lp.sh_gate : p.lp.w_gate) + r0;
-                wrow1 = (const uint8_t *)(shared ? p.lp.sh_up : p.lp.w_up) + r0;
-            } else {
-                const int nks = st_nks2(d.f_g), ksl = st_kslice2(d.f_g);
-                ks = d.tile % nks;
-                d.tile = d.tile / nks;
-                d.k_begin = ks * ksl;
-                klen_unit = min(ksl, d.f_g - d.k_begin);
-                row_stride = (size_t)d.f_g * 2;
-                wrow0 = (const uint8_t *)(shared ? p.lp.sh_down : p.lp.w_down) +
-                        ((size_t)e * sh.d + (size_t)d.tile * 32) * row_stride;
-                // wait until every phase-1 unit of this group has stored its activations
-                if (!all_ready) {
-                    int ok = 0;
+                const int v = lo2 + (n - n1_mine);
+                d.phase = 2;
+                d.gslot = upper_group2(groups, n_active, v);
+                const StGroup &gr = groups[d.gslot];
+                const int local = v - gr.p2, tiles = sh.d / 8;
+                d.ks = local / tiles;
+                d.tile = local - d.ks * tiles;
+                d.klen = min(gr.ksl, gr.f - d.ks * gr.ksl);
+                d.rc = d.klen * 2;
+                rstride = (size_t)gr.f * 2;
+                const bool shared = gr.group >= sh.E;
+                const size_t e = shared ? gr.group - sh.E : gr.group;
+                src0 = (const uint8_t *)(shared ? p.lp.sh_down : p.lp.w_down) +
+                       (e * sh.d + (size_t)d.tile * 8) * rstride + (size_t)d.ks * gr.ksl * 2;
+                src1 = src0 + 4 * rstride;
+                if (d.gslot != cur_a || d.ks != cur_ks) {
+                    // new operand: (1) every stage issued so far must have been consumed (it may still
+                    // read the old operand, or the hidden states the operand region aliases)
+                    int ok = 1;
                     if (lane == 0) {
-                        const int need = s_pfx1[d.group_slot + 1] - s_pfx1[d.group_slot];
-                        for (unsigned i = 0; i < (kStSpinLimit >> 2); ++i) {
-                            if (ld_acquire(&ws.sync[kStMaxGroups]) >= total1) { ok = 2; break; }
-                            if (ld_acquire(&ws.sync[d.group_slot]) >= need) { ok = 1; break; }
-                            __nanosleep(64);
+                        for (int back = 1; back <= S && back <= n && ok; ++back) {
+                            const int m = n - back;
+                            if (m < n1_mine && !pl.alias) break;   // phase-1 stages never read the operand
+                            ok = mbar_wait(&empty_bar[m % S], (uint32_t)(m / S) & 1u) ? 1 : 0;
                         }
-                        if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+                        if (!ok) atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                        // (2) every phase-1 stage of this group must have stored its activations
+                        if (ok && d.gslot != cur_a) {
+                            const int need = gr.f / 4;
+                            ok = 0;
+                            for (unsigned i = 0; i < (kStSpinLimit >> 2); ++i) {
+                                if (ld_acquire(&ws.sync[d.gslot]) >= need) { ok = 1; break; }
+                                __nanosleep(40);
+                            }
+                            if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+                        }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) { alive = false; break; }
-                    if (ok == 2) all_ready = true;
                     fence_proxy_async();
+                    cur_a = d.gslot;
+                    cur_ks = d.ks;
+                    ++op_gen;
+                    const int tpad = st_pad8(gr.T), opitch = d.klen * 2 + 64;
+                    if (lane == 0) mbar_expect_tx(&op_bar, (uint32_t)(2 * gr.T) * d.rc);
+                    __syncwarp();
+                    const size_t n_routed = (size_t)p.B * sh.k;
+                    for (int r = lane; r < 2 * gr.T; r += 32) {
+                        const int ti = r < gr.T ? r : r - gr.T;
+                        const __nv_bfloat16 *base = r < gr.T ? p.act_hi : p.act_lo;
+                        const size_t o = act_offset(gr.off + ti, (int)n_routed, sh.f, sh.f_sh) + (size_t)d.ks * gr.ksl;
+                        const int srow = r < gr.T ? ti : tpad + ti;
+                        bulk_g2s(oreg + (size_t)srow * opitch, base + o, d.rc, &op_bar);
+                    }
                 }
+                d.op_gen = op_gen;
             }
-            d.nchunks = (klen_unit + kc - 1) / kc;
-            const int rows_w = d.phase == 1 ? 16 : 32;
-            const size_t n_routed = (size_t)ws.header[3] * sh.k;
-            for (int c = 0; c < d.nchunks; ++c) {
-                const int slot = it % kStStages;
-                const uint32_t parity = ((it / kStStages) & 1u) ^ 1u;
-                int ok = 1;
-                if (lane == 0) ok = mbar_wait(&empty_bar[slot], parity) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) {
-                    if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
-                    alive = false;
-                    break;
-                }
-                d.chunk = c;
-                d.klen = min(kc, klen_unit - c * kc);
-                const int cbytes = d.klen * 2;
-                d.pitch_w = st_pitch(cbytes);
-                d.pitch_o = d.pitch_w;
-                uint8_t *wreg = slots + (size_t)slot * kStSlotBytes;
-                uint8_t *oreg = wreg + kStRegion;
-                const size_t kbyte = (size_t)(d.k_begin + c * kc) * 2;
-                if (lane == 0) {
-                    desc[slot] = d;
-                    const uint32_t total_bytes = (uint32_t)(rows_w + (d.phase == 1 ? d.T : 2 * d.T)) * cbytes;
-                    mbar_expect_tx(&full_bar[slot], total_bytes);
-                }
-                __syncwarp();
-                for (int r = lane; r < rows_w; r += 32) {
-                    const uint8_t *src;
-                    if (d.phase == 1) src = (r < 8 ? wrow0 + (size_t)r * row_stride : wrow1 + (size_t)(r - 8) * row_stride);
-                    else src = wrow0 + (size_t)r * row_stride;
-                    bulk_g2s(wreg + (size_t)r * d.pitch_w, src + kbyte, cbytes, &full_bar[slot]);
-                }
-                if (d.phase == 1) {
-                    for (int r = lane; r < d.T; r += 32) {
-                        const int tok = ws.slot_token[d.off + r];
-                        bulk_g2s(oreg + (size_t)r * d.pitch_o,
-                                 (const uint8_t *)p.hidden + ((size_t)tok * sh.d) * 2 + kbyte, cbytes, &full_bar[slot]);
-                    }
-                } else {
-                    for (int r = lane; r < 2 * d.T; r += 32) {
-                        const int ti = r < d.T ? r : r - d.T;
-                        const __nv_bfloat16 *base = r < d.T ? p.act_hi : p.act_lo;
-                        const size_t o = act_offset(d.off + ti, (int)n_routed, sh.f, sh.f_sh);
-                        const int srow = r < d.T ? ti : d.tpad8 + ti;
-                        bulk_g2s(oreg + (size_t)srow * d.pitch_o, (const uint8_t *)(base + o) + kbyte, cbytes,
-                                 &full_bar[slot]);
-                    }
-                }
-                ++it;
+            const int slot = n % S;
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(&empty_bar[slot], (((uint32_t)(n / S)) & 1u) ^ 1u) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) {
+                if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                alive = false;
+                break;
+            }
+            uint8_t *wreg = ring + (size_t)slot * pl.slot_bytes;
+            const bool contiguous = (size_t)d.rc == rstride;
+            if (lane == 0) {
+                desc[slot] = d;
+                mbar_expect_tx(&full_bar[slot], (uint32_t)8 * d.rc);
+            }
+            __syncwarp();
+            if (contiguous) {
+                if (lane == 0) bulk_g2s(wreg, src0, 4 * d.rc, &full_bar[slot]);
+                if (lane == 1) bulk_g2s(wreg + 4 * d.rc + 64, src1, 4 * d.rc, &full_bar[slot]);
+            } else if (lane < 8) {
+                const uint8_t *src = (lane < 4 ? src0 : src1) + (size_t)(lane & 3) * rstride;
+                bulk_g2s(wreg + (size_t)(lane & 3) * d.rc + (lane < 4 ? 0 : 4 * d.rc + 64), src, d.rc, &full_bar[slot]);
             }
         }
-        // let every copy that was issued land before the CTA may exit
         if (!alive && lane == 0) {
-            for (int s = 0; s < kStStages; ++s) {
-                // a slot whose full barrier is pending completes when its bytes arrive; bounded wait
-                for (unsigned i = 0; i < (1u << 16); ++i)
-                    if (mbar_try_wait(&full_bar[s], 0) || mbar_try_wait(&full_bar[s], 1)) break;
-            }
+            // let the copies that were issued land before the CTA may exit (bounded)
+            for (unsigned i = 0; i < (1u << 20); ++i) __nanosleep(20);
         }
     } else {
         // ------------------------------------------------------------ consumer warps
-        unsigned it = 0;
-        uint32_t cphase = 0;
-        const int ctid = tid;
-        for (int u = blockIdx.x; u < total; u += gridDim.x) {
-            const int slot = it % kStStages;
-            const uint32_t parity = (it / kStStages) & 1u;
-            if (!mbar_wait(&full_bar[slot], parity)) {
+        const int mt_all = (st_pad8(p.B) + 15) >> 4;
+        bool x_ready = false;
+        for (int n = warp; n < n_mine; n += kStConsumerWarps) {
+            const int slot = n % S;
+            if (!mbar_wait(&full_bar[slot], ((uint32_t)(n / S)) & 1u)) {
                 if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 break;
             }
-            const StageDesc d0 = desc[slot];
-            const int mt = (d0.tpad8 + 15) >> 4;
-            bool ok;
-            if (d0.phase == 1) {
-                if (mt == 1) ok = consume_unit<1, 1>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else if (mt == 2) ok = consume_unit<2, 1>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else if (mt == 3) ok = consume_unit<3, 1>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else ok = consume_unit<4, 1>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
+            const StageDesc d = desc[slot];
+            const StGroup &gr = groups[d.gslot];
+            const uint8_t *wreg = ring + (size_t)slot * pl.slot_bytes;
+            bool ok = true;
+            if (d.phase == 1) {
+                if (!x_ready) {
+                    ok = mbar_wait(&x_bar, 0);
+                    x_ready = ok;
+                }
+                if (ok) {
+                    if (mt_all == 1) consume_phase1<1>(p, gr, d, wreg, xreg, lane);
+                    else if (mt_all == 2) consume_phase1<2>(p, gr, d, wreg, xreg, lane);
+                    else if (mt_all == 3) consume_phase1<3>(p, gr, d, wreg, xreg, lane);
+                    else consume_phase1<4>(p, gr, d, wreg, xreg, lane);
+                }
             } else {
-                if (mt == 1) ok = consume_unit<1, 2>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else if (mt == 2) ok = consume_unit<2, 2>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else if (mt == 3) ok = consume_unit<3, 2>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
-                else ok = consume_unit<4, 2>(p, slots, scratch, full_bar, empty_bar, desc, it, warp, lane, ctid, &cbar, cphase);
+                // generation g of the operand completes phase g - 1 of its barrier
+                ok = mbar_wait(&op_bar, (uint32_t)(d.op_gen - 1) & 1u);
+                if (ok) {
+                    const int mt = (st_pad8(gr.T) + 15) >> 4;
+                    if (mt == 1) consume_phase2<1>(p, gr, d, wreg, oreg, s_slot_token, s_slot_w, lane);
+                    else if (mt == 2) consume_phase2<2>(p, gr, d, wreg, oreg, s_slot_token, s_slot_w, lane);
+                    else if (mt == 3) consume_phase2<3>(p, gr, d, wreg, oreg, s_slot_token, s_slot_w, lane);
+                    else consume_phase2<4>(p, gr, d, wreg, oreg, s_slot_token, s_slot_w, lane);
+                }
             }
             if (!ok) {
                 if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 break;
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[slot]);
         }
     }
 }

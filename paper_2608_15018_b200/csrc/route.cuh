@@ -232,21 +232,40 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
             ws.active[U + s] = E + s;
         }
     }
+    for (int e = tid; e < E; e += nt) ws.tokmask[e] = s_mask[e];
+    for (int s = tid; s < sh.n_sh; s += nt) ws.tokmask[E + s] = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
     if (sh.plan == 2) {
-        // unit tables of the streaming kernel: per active group, first phase-1 unit
-        // (8 gate + 8 up rows each) and first phase-2 unit (32 down rows x one K-slice)
-        const int u1r = sh.f / 8, u2r = (sh.d / 32) * st_nks2(sh.f);
-        const int u1s = sh.n_sh ? sh.f_sh / 8 : 0, u2s = sh.n_sh ? (sh.d / 32) * st_nks2(sh.f_sh) : 0;
-        for (int a = tid; a <= U + sh.n_sh; a += nt) {
-            const int r = a < U ? a : U, s = a < U ? 0 : a - U;
-            ws.upfx1[a] = r * u1r + s * u1s;
-            ws.upfx2[a] = r * u2r + s * u2s;
-            ws.sync[a] = 0;
+        // stage tables of the streaming kernel: per active group, its first phase-1 stage
+        // (4 gate + 4 up rows each) and first phase-2 stage (8 down rows x one K-slice)
+        __syncthreads();
+        for (int e = tid; e < E; e += nt)
+            s_cnt[e] = s_cnt[e] > 0 ? st_nks(sh.f, s_cnt[e], sh.op_cap) * (sh.d / 8) : 0;   // phase-2 stages
+        __syncthreads();
+        for (int e = tid; e < E; e += nt) {
+            if (s_mask[e]) {
+                int pre = 0;
+                for (int o = 0; o < e; ++o) pre += s_cnt[o];
+                const int a = s_pos[e];
+                ws.upfx1[a] = a * (sh.f / 4);
+                ws.upfx2[a] = pre;
+                ws.sync[a] = 0;
+                if (a == U - 1) s_off[0] = pre + s_cnt[e];   // all routed phase-2 stages
+            }
         }
+        __syncthreads();
         if (tid == 0) {
-            ws.header[4] = U * u1r + sh.n_sh * u1s;
-            ws.header[5] = U * u2r + sh.n_sh * u2s;
-            ws.sync[kStMaxGroups] = 0;
+            int t1 = U * (sh.f / 4), t2 = s_off[0];
+            for (int s = 0; s <= sh.n_sh; ++s) {
+                ws.upfx1[U + s] = t1;
+                ws.upfx2[U + s] = t2;
+                ws.sync[U + s] = 0;
+                if (s < sh.n_sh) {
+                    t1 += sh.f_sh / 4;
+                    t2 += st_nks(sh.f_sh, B, sh.op_cap) * (sh.d / 8);
+                }
+            }
+            ws.header[4] = t1;
+            ws.header[5] = t2;
         }
     }
     if (tid == 0) {

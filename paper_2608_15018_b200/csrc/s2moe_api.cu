@@ -187,11 +187,28 @@ cudaError_t prepare_simple()
         else FN<DT_Q4B32, DT_BF16>(__VA_ARGS__);                                         \
     } while (0)
 
+// The plan a batch of B tokens runs with: the streaming kernel when it is allowed and its
+// shared-memory layout fits, else the CUDA-core kernels; 0 when plan 2 was demanded and does not fit.
+int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
+{
+    const Shape &s0 = ctx->shape;
+    if (ctx->cfg.kernel_plan == 1) return 1;
+    const StPlan pl = st_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
+    if (out) *out = pl;
+    if (pl.feasible) return 2;
+    return ctx->cfg.kernel_plan == 2 ? 0 : 1;
+}
+
 int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float *conf, float *out,
                int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
 {
-    const Shape &sh = ctx->shape;
+    Shape sh = ctx->shape;
     const LayerPtrs &lp = ctx->layers[layer];
+    StPlan pl{};
+    const int plan = plan_for(ctx, B, &pl);
+    if (plan == 0) return S2MOE_EINVAL;
+    sh.plan = plan;
+    sh.op_cap = pl.op_cap;
     CU(ctx, cudaMemsetAsync(out, 0, (size_t)B * sh.d * sizeof(float), st));
     if (sh.act_dtype == DT_F32) launch_router<DT_F32>(ctx, lp, B, hidden, st);
     else launch_router<DT_BF16>(ctx, lp, B, hidden, st);
@@ -200,12 +217,12 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         gating_kernel<<<1, kGateThreads, (size_t)B * sh.E * sizeof(double), st>>>(
             sh, B, ctx->ws, conf, lp.sh_scale ? 1 : 0, sel_idx, sel_w, n_unique);
     }
-    if (ctx->plan == 2) {
+    if (plan == 2) {
         StreamArgs a;
-        a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.hidden = hidden; a.y = out;
-        a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo;
+        a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
+        a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
         LaunchScope scope(ctx, KC_STREAM, st);
-        ffn_stream_kernel<<<ctx->n_sm, kStThreads, kStSmemBytes, st>>>(a);
+        ffn_stream_kernel<<<pl.n_cta, kStThreads, pl.smem_bytes, st>>>(a);
     } else {
         DISPATCH_WT_ACT(ctx, launch_simple, ctx, lp, hidden, out, st);
     }
@@ -253,8 +270,8 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     static_assert(sizeof(LayerPtrs) == sizeof(s2moe_layer_weights), "layout");
     std::memcpy(ctx->layers.data(), layers, sizeof(LayerPtrs) * (size_t)config->n_layers);
     ctx->plan = config->kernel_plan;
-    if (ctx->plan == 0) ctx->plan = (sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16) ? 2 : 1;
-    sh.plan = ctx->plan;
+    sh.plan = 1;
+    sh.op_cap = 0;
 
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e != cudaSuccess) { delete ctx; return S2MOE_ECUDA; }
@@ -272,6 +289,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(kStMaxGroups + 64));
     const size_t o_ahi = take(2 * act_floats), o_alo = take(2 * act_floats);
     const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
+    const size_t o_tm = take(8 * (size_t)G);
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
@@ -281,8 +299,8 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     e = cudaMemset(ctx->slab, 0, ctx->slab_bytes);
     if (e == cudaSuccess) DISPATCH_WT_ACT(ctx, e = prepare_simple);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device);
-    if (e == cudaSuccess && ctx->plan == 2)
-        e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBytes);
+    if (e == cudaSuccess && ctx->plan != 1)
+        e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStMaxSmem);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(gating_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)(sizeof(double) * kMaxTokens * kMaxExperts));
@@ -296,6 +314,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ws.slot_w = (float *)(base + o_sw); ws.active = (int32_t *)(base + o_active);
     ws.act = (float *)(base + o_act); ws.sync = (int32_t *)(base + o_sync);
     ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
+    ws.tokmask = (unsigned long long *)(base + o_tm);
     ctx->act_hi = (__nv_bfloat16 *)(base + o_ahi); ctx->act_lo = (__nv_bfloat16 *)(base + o_alo);
     ctx->st_hidden = base + o_sth; ctx->st_conf = (float *)(base + o_stc);
     ctx->st_out = (float *)(base + o_sto); ctx->st_sel = (int32_t *)(base + o_sts);
@@ -393,7 +412,11 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out)
 
 int s2moe_last_cuda_error(const s2moe_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
 
-int s2moe_kernel_plan(const s2moe_ctx *ctx) { return ctx ? ctx->plan : 0; }
+int s2moe_kernel_plan(const s2moe_ctx *ctx, int32_t n_tokens)
+{
+    if (!ctx || n_tokens < 1 || n_tokens > ctx->cfg.max_tokens) return 0;
+    return plan_for(ctx, n_tokens, nullptr);
+}
 
 int64_t s2moe_kernel_launches(const s2moe_ctx *ctx) { return ctx ? ctx->launches : 0; }
 

@@ -15,6 +15,8 @@ def supports(wl, plan):
 
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
              hidden=None, conf=None, check_lists=True):
+    """Returns (report, outputs), or (None, None) when the demanded plan does not cover the case
+    (format not covered, or the batch does not fit the streaming kernel's shared memory)."""
     if not supports(wl, plan):
         return None, None
     dev = torch.device("cuda", 0)
@@ -24,6 +26,10 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
         conf = workloads.confidences(wl, layer, H.shape[0], dev)
     cfg = binding.Config.from_workload(wl, n_layers=1, kernel_plan=plan)
     with binding.S2MoE(cfg, [T]) as m:
+        used = m.kernel_plan(H.shape[0])
+        if plan == 2 and used != 2:
+            return None, None
+        assert used in (1, 2) and (plan == 0 or used == plan)
         o = m.verify_layer(0, H, conf)
         torch.cuda.synchronize()
         assert m.device_status() == 0
@@ -38,4 +44,5 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
                              TOL[wl.weight_dtype], tok_list=tok_list)
     if lists is not None:
         parity.check_bucketing(lists, sel, w, wl.n_experts, wl.n_shared)
+    rep.plan = used
     return rep, o
