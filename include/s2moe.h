@@ -209,6 +209,8 @@ const char *s2moe_kernel_class_name(int32_t cls);
  *   2 offsets int32 [E + n_sh + 1]  3 slot_token int32 [n_slots] 4 slot_w float [n_slots]
  *   5 active  int32 [n_active] (ids of experts with tokens, shared ones as E + s)
  *   6 header  int32 [4] = {n_active, n_slots, U, B}
+ *   7 check   int32 [8]: first violation seen by a self-checking build of the kernels
+ *             ({code, value, limit, block, ...}; all zero in the normal build)
  * n_slots = B*k + n_sh*B.  Returns EINVAL when `bytes` is smaller than the array.
  */
 int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes);

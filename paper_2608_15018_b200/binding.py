@@ -61,7 +61,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.build_library() if build_if_missing else _build.LIB
+    override = os.environ.get("S2MOE_LIBRARY")     # e.g. a self-checking build of the same sources
+    path = override or (_build.build_library() if build_if_missing else _build.LIB)
     if not os.path.exists(path):
         raise RuntimeError(f"CUDA library {path} is missing; run __graft_entry__.build()")
     lib = ctypes.CDLL(path)

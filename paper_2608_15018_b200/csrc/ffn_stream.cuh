@@ -14,8 +14,8 @@
 // only.  A phase-2 operand load waits on a counter of that expert's finished phase-1
 // stages.  Every wait in the kernel is bounded and reports through the status word.
 //
-// Inside a CTA one producer warp issues the copies; each of the eight consumer warps
-// takes every eighth stage and finishes it alone (no CTA-wide barrier anywhere).
+// Inside a CTA one producer warp issues the copies; every ring slot belongs to one consumer
+// warp, which finishes the stages landing there alone (no CTA-wide barrier anywhere).
 // The contraction is mma.sync m16n8k16 with tokens as the M operand and eight weight
 // rows as the N operand.  The K index inside every 32-wide step is permuted identically
 // for both operands, so each lane feeds the tensor core from one 128-bit shared-memory
@@ -69,6 +69,7 @@ struct StreamArgs {
     float *y;
     __nv_bfloat16 *act_hi, *act_lo;
     int B;
+    size_t act_elems;   // elements of act_hi / act_lo
 };
 
 // ---- shapes shared by the host planner, the gating kernel and this kernel ----------
@@ -76,11 +77,13 @@ struct StreamArgs {
 __host__ __device__ __forceinline__ int st_pad8(int t) { return (t + 7) & ~7; }
 
 // number of K-slices of a phase-2 row of inner dim f for T tokens, given the operand
-// capacity: hi and lo rows of pad8(T) tokens, each row padded by 64 bytes
-__host__ __device__ __forceinline__ int st_nks(int f, int T, int op_cap)
+// capacity (hi and lo rows of pad8(T) tokens, each row padded by 64 bytes) and the longest
+// slice a ring slot takes (kcap = d: a phase-2 stage is never larger than a phase-1 stage)
+__host__ __device__ __forceinline__ int st_nks(int f, int T, int op_cap, int kcap)
 {
     const int rows = 2 * st_pad8(T);
     int kmax = ((op_cap / rows - 64) / 2) & ~31;
+    if (kmax > kcap) kmax = kcap & ~31;
     if (kmax < 32) kmax = 32;
     return (f + kmax - 1) / kmax;
 }
@@ -94,32 +97,42 @@ inline StPlan st_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.x_pitch = sh.d * 2 + 64;
     p.x_bytes = st_pad8(B) * p.x_pitch;
     const int fmax = sh.n_sh && sh.f_sh > sh.f ? sh.f_sh : sh.f;
-    const int stage1 = 8 * sh.d * 2 + 128;
     p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 127) & ~127;
     const int avail = kStMaxSmem - p.tab_bytes;
     const int op_full = 2 * st_pad8(B) * (fmax * 2 + 64);
     const int op_min = 2 * st_pad8(B) * (256 * 2 + 64);
-    p.slot_bytes = stage1;
-    p.stages = 4;
-    const int left = avail - p.x_bytes - p.stages * p.slot_bytes;
-    if (left >= op_min) {
-        p.alias = 0;
-        p.op_cap = left < op_full ? left : op_full;
-    } else {
-        p.alias = 1;
-        p.op_cap = avail - p.stages * p.slot_bytes;
-        if (p.op_cap < p.x_bytes || p.op_cap < op_min) {
-            p.stages = 3;
+    // a ring slot holds a phase-1 stage (8 rows of d) or a phase-2 stage (8 rows of one K-slice);
+    // two rounds: the K-slice length depends on the operand capacity, which depends on the slot
+    p.slot_bytes = 8 * sh.d * 2 + 128;
+    bool fits = false;
+    for (int round = 0; round < 2; ++round) {
+        // one consumer warp per ring slot: as many slots (up to 8) as leave room for the whole
+        // phase-2 operand next to the hidden states; at least 4, then the operand takes over the
+        // hidden-state region once phase 1 has drained (alias)
+        p.stages = 8;
+        while (p.stages > 4 && avail - p.x_bytes - p.stages * p.slot_bytes < op_full) --p.stages;
+        const int left = avail - p.x_bytes - p.stages * p.slot_bytes;
+        if (left >= op_full) {
+            p.alias = 0;
+            p.op_cap = op_full;
+        } else {
+            p.alias = 1;
             p.op_cap = avail - p.stages * p.slot_bytes;
+            if (p.op_cap < p.x_bytes || p.op_cap < op_min) {
+                p.stages = 3;
+                p.op_cap = avail - p.stages * p.slot_bytes;
+            }
+            if (p.op_cap > op_full && op_full >= p.x_bytes) p.op_cap = op_full;
         }
+        p.op_cap &= ~127;
+        const int ksl_max = st_ksl(fmax, st_nks(fmax, 1, p.op_cap, sh.d));   // longest slice: fewest tokens
+        const int stage2 = 8 * ksl_max * 2 + 128;
+        p.smem_bytes = p.tab_bytes + (p.alias ? p.op_cap : p.x_bytes + p.op_cap) + p.stages * p.slot_bytes;
+        fits = p.op_cap >= op_min && (!p.alias || p.op_cap >= p.x_bytes) && stage2 <= p.slot_bytes &&
+               p.smem_bytes <= kStMaxSmem && B <= kMaxTokens;
+        if (fits || stage2 <= p.slot_bytes) break;
+        p.slot_bytes = stage2;
     }
-    p.op_cap = (p.op_cap + 127) & ~127;
-    if (p.op_cap > avail) p.op_cap = avail & ~127;
-    // a phase-2 stage (8 rows of one K-slice) must fit a ring slot
-    const int ksl_max = st_ksl(fmax, st_nks(fmax, B, p.op_cap));
-    p.smem_bytes = p.tab_bytes + (p.alias ? p.op_cap : p.x_bytes + p.op_cap) + p.stages * p.slot_bytes;
-    const bool fits = p.op_cap >= op_min && (!p.alias || p.op_cap >= p.x_bytes) &&
-                      8 * ksl_max * 2 + 128 <= p.slot_bytes && p.smem_bytes <= kStMaxSmem && B <= kMaxTokens;
     p.feasible = fits && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16;
     return p;
 }
@@ -168,6 +181,18 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
         "l"(src), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
+#ifdef S2MOE_SELFCHECK
+#define ST_BULK(ws, smem0, smem_bytes, dst, src, bytes, bar, g0, gbytes, code)                                      \
+    do {                                                                                                           \
+        const long long so_ = (const uint8_t *)(dst) - (const uint8_t *)(smem0);                                   \
+        const long long go_ = (const uint8_t *)(src) - (const uint8_t *)(g0);                                      \
+        if (st_check(ws, so_ >= 0 && so_ + (long long)(bytes) <= (long long)(smem_bytes) && (so_ & 15) == 0, (code), so_, (smem_bytes)) && \
+            st_check(ws, go_ >= 0 && go_ + (long long)(bytes) <= (long long)(gbytes) && (go_ & 15) == 0 && ((bytes) & 15) == 0, (code) + 100, go_, (gbytes))) \
+            bulk_g2s(dst, src, bytes, bar);                                                                        \
+    } while (0)
+#else
+#define ST_BULK(ws, smem0, smem_bytes, dst, src, bytes, bar, g0, gbytes, code) bulk_g2s(dst, src, bytes, bar)
+#endif
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ int ld_acquire(const int *p)
 {
@@ -204,6 +229,25 @@ __device__ __forceinline__ int upper_group2(const StGroup *g, int n, int u)
     return lo;
 }
 
+// Optional self-check build (-DS2MOE_SELFCHECK): every global access and bulk copy of the
+// kernel is bounds-checked; the first violation is recorded in header[8..11] as
+// {code, value, limit, block} and the access is skipped.
+#ifdef S2MOE_SELFCHECK
+__device__ __forceinline__ bool st_check(const Workspace &ws, bool ok, int code, long long v, long long lim)
+{
+    if (!ok && atomicCAS(&ws.header[8], 0, code) == 0) {
+        ws.header[9] = (int)v;
+        ws.header[10] = (int)lim;
+        ws.header[11] = (int)blockIdx.x;
+        ws.header[12] = (int)(v >> 32);
+    }
+    return ok;
+}
+#define ST_CHECK(ws, cond, code, v, lim) st_check(ws, cond, code, (long long)(v), (long long)(lim))
+#else
+#define ST_CHECK(ws, cond, code, v, lim) true
+#endif
+
 // ---- consumer side ----------------------------------------------------------------
 
 // One phase-1 stage: D[token][gate/up row pairs] over all of K, then SwiGLU and store.
@@ -229,6 +273,12 @@ __device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGrou
     }
     const size_t x8 = (size_t)8 * p.plan.x_pitch;
     const int nsteps = p.sh.d >> 5;
+    // two accumulator sets per m-tile shorten the dependent chain of tensor-core instructions
+    float acc2[MT][4];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc2[m][q] = 0.f;
 #pragma unroll 4
     for (int s = 0; s < nsteps; ++s) {
         const uint4 w = *reinterpret_cast<const uint4 *>(wrow + s * 64);
@@ -237,9 +287,13 @@ __device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGrou
             const uint4 xa = *reinterpret_cast<const uint4 *>(xrow[m] + s * 64);
             const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(xrow[m] + x8 + s * 64) : make_uint4(0, 0, 0, 0);
             mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-            mma_bf16(acc[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+            mma_bf16(acc2[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
         }
     }
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[m][q] += acc2[m][q];
     // lane (g, t) holds (gate row t, up row t) of tokens g and g + 8 of every m-tile
     const int n_routed = p.B * p.sh.k;
 #pragma unroll
@@ -253,8 +307,10 @@ __device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGrou
                 const __nv_bfloat16 hi = __float2bfloat16_rn(a);
                 const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
                 const size_t o = act_offset(slot, n_routed, p.sh.f, p.sh.f_sh) + (size_t)d.tile * 4 + t;
-                p.act_hi[o] = hi;
-                p.act_lo[o] = lo;
+                if (ST_CHECK(p.ws, o < p.act_elems && slot < p.ws.header[1], 1, o, p.act_elems)) {
+                    p.act_hi[o] = hi;
+                    p.act_lo[o] = lo;
+                }
             }
         }
     }
@@ -262,7 +318,8 @@ __device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGrou
     __threadfence();
     fence_proxy_async();
     __syncwarp();
-    if (lane == 0) atomicAdd(&p.ws.sync[d.gslot], 1);
+    if (lane == 0 && ST_CHECK(p.ws, d.gslot >= 0 && d.gslot < kStMaxGroups, 2, d.gslot, kStMaxGroups))
+        atomicAdd(&p.ws.sync[d.gslot], 1);
 }
 
 // One phase-2 stage: D[slot][8 down rows] over one K-slice, y += p * D.
@@ -290,6 +347,11 @@ __device__ __forceinline__ void consume_phase2(const StreamArgs &p, const StGrou
     }
     const size_t o8 = (size_t)8 * opitch;
     const size_t lo_off = (size_t)tpad * opitch;
+    float acc2[MT][4], acc3[MT][4], acc4[MT][4];   // independent chains: hi/lo parts, even/odd halves
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc2[m][q] = acc3[m][q] = acc4[m][q] = 0.f;
     const int nsteps = d.klen >> 5;
 #pragma unroll 2
     for (int s = 0; s < nsteps; ++s) {
@@ -302,11 +364,15 @@ __device__ __forceinline__ void consume_phase2(const StreamArgs &p, const StGrou
             const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + s * 64) : z;
             const uint4 lb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + lo_off + s * 64) : z;
             mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-            mma_bf16(acc[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
-            mma_bf16(acc[m], la.x, lb.x, la.y, lb.y, w.x, w.y);
-            mma_bf16(acc[m], la.z, lb.z, la.w, lb.w, w.z, w.w);
+            mma_bf16(acc2[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+            mma_bf16(acc3[m], la.x, lb.x, la.y, lb.y, w.x, w.y);
+            mma_bf16(acc4[m], la.z, lb.z, la.w, lb.w, w.z, w.w);
         }
     }
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[m][q] += acc2[m][q] + (acc3[m][q] + acc4[m][q]);
     // lane (g, t): columns 2t, 2t+1 are down rows t and 4 + t of the stage
     const int r0 = d.tile * 8 + t;
 #pragma unroll
@@ -317,9 +383,12 @@ __device__ __forceinline__ void consume_phase2(const StreamArgs &p, const StGrou
             if (ti < grp.T) {
                 const int slot = grp.off + ti;
                 const float pw = slot_w[slot];
-                float *dst = p.y + (size_t)slot_token[slot] * p.sh.d + r0;
-                atomicAdd(dst, pw * acc[m][2 * h]);
-                atomicAdd(dst + 4, pw * acc[m][2 * h + 1]);
+                const size_t yo = (size_t)slot_token[slot] * p.sh.d + r0;
+                float *dst = p.y + yo;
+                if (ST_CHECK(p.ws, yo + 4 < (size_t)p.B * p.sh.d && slot < p.ws.header[1], 3, yo, p.B * p.sh.d)) {
+                    atomicAdd(dst, pw * acc[m][2 * h]);
+                    atomicAdd(dst + 4, pw * acc[m][2 * h + 1]);
+                }
             }
         }
     }
@@ -361,7 +430,7 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
         gr.mask = ws.tokmask[gr.group];
         gr.p1 = ws.upfx1[a];
         gr.p2 = ws.upfx2[a];
-        gr.nks = st_nks(gr.f, gr.T, pl.op_cap);
+        gr.nks = st_nks(gr.f, gr.T, pl.op_cap, sh.d);
         gr.ksl = st_ksl(gr.f, gr.nks);
         groups[a] = gr;
     }
@@ -395,13 +464,16 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
         if (lane == 0) mbar_expect_tx(&x_bar, (uint32_t)p.B * sh.d * 2);
         __syncwarp();
         for (int b = lane; b < p.B; b += 32)
-            bulk_g2s(xreg + (size_t)b * pl.x_pitch, (const uint8_t *)p.hidden + (size_t)b * sh.d * 2, sh.d * 2, &x_bar);
+            ST_BULK(ws, st_smem, pl.smem_bytes, xreg + (size_t)b * pl.x_pitch,
+                    (const uint8_t *)p.hidden + (size_t)b * sh.d * 2, sh.d * 2, &x_bar, p.hidden,
+                    (size_t)p.B * sh.d * 2, 10);
 
         int cur_a = -1, cur_ks = -1, op_gen = 0;
         for (int n = 0; n < n_mine && alive; ++n) {
             StageDesc d;
             const uint8_t *src0, *src1;   // the two 4-row halves
-            size_t rstride;
+            const uint8_t *wbase0, *wbase1;   // tensors the halves come from (self-check build only)
+            size_t rstride, wbytes = 0;
             if (n < n1_mine) {
                 const int u = blockIdx.x + n * P;
                 d.phase = 1;
@@ -416,8 +488,11 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
                 const bool shared = gr.group >= sh.E;
                 const size_t e = shared ? gr.group - sh.E : gr.group;
                 const size_t r0 = (e * gr.f + (size_t)d.tile * 4) * rstride;
-                src0 = (const uint8_t *)(shared ? p.lp.sh_gate : p.lp.w_gate) + r0;
-                src1 = (const uint8_t *)(shared ? p.lp.sh_up : p.lp.w_up) + r0;
+                wbase0 = (const uint8_t *)(shared ? p.lp.sh_gate : p.lp.w_gate);
+                wbase1 = (const uint8_t *)(shared ? p.lp.sh_up : p.lp.w_up);
+                wbytes = (size_t)(shared ? sh.n_sh : sh.E) * gr.f * rstride;   // self-check build only
+                src0 = wbase0 + r0;
+                src1 = wbase1 + r0;
             } else {
                 const int v = lo2 + (n - n1_mine);
                 d.phase = 2;
@@ -431,8 +506,9 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
                 rstride = (size_t)gr.f * 2;
                 const bool shared = gr.group >= sh.E;
                 const size_t e = shared ? gr.group - sh.E : gr.group;
-                src0 = (const uint8_t *)(shared ? p.lp.sh_down : p.lp.w_down) +
-                       (e * sh.d + (size_t)d.tile * 8) * rstride + (size_t)d.ks * gr.ksl * 2;
+                wbase0 = wbase1 = (const uint8_t *)(shared ? p.lp.sh_down : p.lp.w_down);
+                wbytes = (size_t)(shared ? sh.n_sh : sh.E) * sh.d * rstride;
+                src0 = wbase0 + (e * sh.d + (size_t)d.tile * 8) * rstride + (size_t)d.ks * gr.ksl * 2;
                 src1 = src0 + 4 * rstride;
                 if (d.gslot != cur_a || d.ks != cur_ks) {
                     // new operand: (1) every stage issued so far must have been consumed (it may still
@@ -471,7 +547,8 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
                         const __nv_bfloat16 *base = r < gr.T ? p.act_hi : p.act_lo;
                         const size_t o = act_offset(gr.off + ti, (int)n_routed, sh.f, sh.f_sh) + (size_t)d.ks * gr.ksl;
                         const int srow = r < gr.T ? ti : tpad + ti;
-                        bulk_g2s(oreg + (size_t)srow * opitch, base + o, d.rc, &op_bar);
+                        ST_BULK(ws, st_smem, pl.smem_bytes, oreg + (size_t)srow * opitch, base + o, d.rc, &op_bar, base,
+                                p.act_elems * 2, 20);
                     }
                 }
                 d.op_gen = op_gen;
@@ -487,17 +564,20 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
             }
             uint8_t *wreg = ring + (size_t)slot * pl.slot_bytes;
             const bool contiguous = (size_t)d.rc == rstride;
+            (void)wbytes; (void)wbase0; (void)wbase1;
             if (lane == 0) {
                 desc[slot] = d;
                 mbar_expect_tx(&full_bar[slot], (uint32_t)8 * d.rc);
             }
             __syncwarp();
             if (contiguous) {
-                if (lane == 0) bulk_g2s(wreg, src0, 4 * d.rc, &full_bar[slot]);
-                if (lane == 1) bulk_g2s(wreg + 4 * d.rc + 64, src1, 4 * d.rc, &full_bar[slot]);
+                if (lane == 0) ST_BULK(ws, st_smem, pl.smem_bytes, wreg, src0, 4 * d.rc, &full_bar[slot], wbase0, wbytes, 30);
+                if (lane == 1)
+                    ST_BULK(ws, st_smem, pl.smem_bytes, wreg + 4 * d.rc + 64, src1, 4 * d.rc, &full_bar[slot], wbase1, wbytes, 40);
             } else if (lane < 8) {
                 const uint8_t *src = (lane < 4 ? src0 : src1) + (size_t)(lane & 3) * rstride;
-                bulk_g2s(wreg + (size_t)(lane & 3) * d.rc + (lane < 4 ? 0 : 4 * d.rc + 64), src, d.rc, &full_bar[slot]);
+                ST_BULK(ws, st_smem, pl.smem_bytes, wreg + (size_t)(lane & 3) * d.rc + (lane < 4 ? 0 : 4 * d.rc + 64), src,
+                        d.rc, &full_bar[slot], lane < 4 ? wbase0 : wbase1, wbytes, 50);
             }
         }
         if (!alive && lane == 0) {
@@ -506,10 +586,13 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
         }
     } else {
         // ------------------------------------------------------------ consumer warps
+        // Consumer warp w owns ring slot w and takes the stages n = w, w + S, ...  One waiter per
+        // barrier: a parity wait is only meaningful for the phase that follows the one the
+        // waiter saw complete, so two warps must never poll the same slot for different uses.
         const int mt_all = (st_pad8(p.B) + 15) >> 4;
         bool x_ready = false;
-        for (int n = warp; n < n_mine; n += kStConsumerWarps) {
-            const int slot = n % S;
+        for (int n = warp; n < n_mine && warp < S; n += S) {
+            const int slot = warp;
             if (!mbar_wait(&full_bar[slot], ((uint32_t)(n / S)) & 1u)) {
                 if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 break;

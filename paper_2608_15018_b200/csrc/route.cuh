@@ -239,7 +239,7 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
         // (4 gate + 4 up rows each) and first phase-2 stage (8 down rows x one K-slice)
         __syncthreads();
         for (int e = tid; e < E; e += nt)
-            s_cnt[e] = s_cnt[e] > 0 ? st_nks(sh.f, s_cnt[e], sh.op_cap) * (sh.d / 8) : 0;   // phase-2 stages
+            s_cnt[e] = s_cnt[e] > 0 ? st_nks(sh.f, s_cnt[e], sh.op_cap, sh.d) * (sh.d / 8) : 0;   // phase-2 stages
         __syncthreads();
         for (int e = tid; e < E; e += nt) {
             if (s_mask[e]) {
@@ -261,7 +261,7 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
                 ws.sync[U + s] = 0;
                 if (s < sh.n_sh) {
                     t1 += sh.f_sh / 4;
-                    t2 += st_nks(sh.f_sh, B, sh.op_cap) * (sh.d / 8);
+                    t2 += st_nks(sh.f_sh, B, sh.op_cap, sh.d) * (sh.d / 8);
                 }
             }
             ws.header[4] = t1;

@@ -31,6 +31,7 @@ struct s2moe_ctx {
     int plan = 1;
     int n_sm = 0;
     __nv_bfloat16 *act_hi = nullptr, *act_lo = nullptr;
+    size_t act_elems = 0;
     int last_cuda = 0;
     int64_t launches = 0;
     int last_B = 0;
@@ -221,6 +222,7 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         StreamArgs a;
         a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
         a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
+        a.act_elems = ctx->act_elems;
         LaunchScope scope(ctx, KC_STREAM, st);
         ffn_stream_kernel<<<pl.n_cta, kStThreads, pl.smem_bytes, st>>>(a);
     } else {
@@ -294,6 +296,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
     ctx->slab_bytes = off;
+    ctx->act_elems = act_floats;
     e = cudaMalloc(&ctx->slab, ctx->slab_bytes);
     if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? S2MOE_ENOMEM : S2MOE_ECUDA; }
     e = cudaMemset(ctx->slab, 0, ctx->slab_bytes);
@@ -494,6 +497,7 @@ int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
         case 4: src = ctx->ws.slot_w; need = 4 * (size_t)hdr[1]; break;
         case 5: src = ctx->ws.active; need = 4 * (size_t)hdr[0]; break;
         case 6: src = ctx->ws.header; need = 16; break;
+        case 7: src = ctx->ws.header + 8; need = 32; break;
         default: return S2MOE_EINVAL;
     }
     if (bytes < need) return S2MOE_EINVAL;
