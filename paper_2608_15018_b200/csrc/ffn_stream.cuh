@@ -27,7 +27,7 @@
 
 namespace s2moe {
 
-constexpr int kStConsumerWarps = 8;
+constexpr int kStConsumerWarps = 7;   // + 1 producer warp = 256 threads, so a thread may use 255 registers
 constexpr int kStThreads = (kStConsumerWarps + 1) * 32;
 constexpr int kStMaxStages = 8;
 constexpr int kStMaxGroups = kMaxExperts + kMaxShared;
@@ -106,10 +106,10 @@ inline StPlan st_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.slot_bytes = 8 * sh.d * 2 + 128;
     bool fits = false;
     for (int round = 0; round < 2; ++round) {
-        // one consumer warp per ring slot: as many slots (up to 8) as leave room for the whole
+        // one consumer warp per ring slot: as many slots (up to 7) as leave room for the whole
         // phase-2 operand next to the hidden states; at least 4, then the operand takes over the
         // hidden-state region once phase 1 has drained (alias)
-        p.stages = 8;
+        p.stages = kStConsumerWarps;
         while (p.stages > 4 && avail - p.x_bytes - p.stages * p.slot_bytes < op_full) --p.stages;
         const int left = avail - p.x_bytes - p.stages * p.slot_bytes;
         if (left >= op_full) {
@@ -273,27 +273,79 @@ __device__ __forceinline__ void consume_phase1(const StreamArgs &p, const StGrou
     }
     const size_t x8 = (size_t)8 * p.plan.x_pitch;
     const int nsteps = p.sh.d >> 5;
-    // two accumulator sets per m-tile shorten the dependent chain of tensor-core instructions
-    float acc2[MT][4];
+    // A single warp has to hide its own latencies: work in blocks of BS K-steps, load the next
+    // block's operands while the current block's tensor-core instructions run, and keep
+    // 2 * BS independent accumulator chains per m-tile.
+    constexpr int BS = MT == 1 ? 4 : (MT == 2 ? 2 : 1);
+    constexpr int NB = MT <= 2 ? 2 : 1;   // operand buffers: double-buffered while registers allow
+    float ch[MT][2 * BS][4];
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc2[m][q] = 0.f;
-#pragma unroll 4
-    for (int s = 0; s < nsteps; ++s) {
-        const uint4 w = *reinterpret_cast<const uint4 *>(wrow + s * 64);
+        for (int c = 0; c < 2 * BS; ++c)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) ch[m][c][q] = 0.f;
+    uint4 w[NB][BS], xa[NB][BS][MT], xb[NB][BS][MT];
+    auto load_block = [&](int buf, int s0) {
+#pragma unroll
+        for (int i = 0; i < BS; ++i) {
+            w[buf][i] = *reinterpret_cast<const uint4 *>(wrow + (s0 + i) * 64);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                xa[buf][i][m] = *reinterpret_cast<const uint4 *>(xrow[m] + (s0 + i) * 64);
+                xb[buf][i][m] = has1[m] ? *reinterpret_cast<const uint4 *>(xrow[m] + x8 + (s0 + i) * 64)
+                                        : make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+    auto mma_block = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < BS; ++i)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                mma_bf16(ch[m][2 * i], xa[buf][i][m].x, xb[buf][i][m].x, xa[buf][i][m].y, xb[buf][i][m].y,
+                         w[buf][i].x, w[buf][i].y);
+                mma_bf16(ch[m][2 * i + 1], xa[buf][i][m].z, xb[buf][i][m].z, xa[buf][i][m].w, xb[buf][i][m].w,
+                         w[buf][i].z, w[buf][i].w);
+            }
+    };
+    const int nblk = nsteps / BS;          // d is a multiple of 64, BS divides nsteps when d % 128 == 0
+    if (NB == 2) {
+        load_block(0, 0);
+#pragma unroll 1
+        for (int blk = 0; blk + 1 < nblk; blk += 2) {
+            load_block(NB - 1, (blk + 1) * BS);
+            mma_block(0);
+            if (blk + 2 < nblk) load_block(0, (blk + 2) * BS);
+            mma_block(NB - 1);
+        }
+        if (nblk & 1) mma_block(0);
+    } else {
+#pragma unroll 1
+        for (int blk = 0; blk < nblk; ++blk) {
+            load_block(0, blk * BS);
+            mma_block(0);
+        }
+    }
+    for (int s = nblk * BS; s < nsteps; ++s) {     // tail steps when BS does not divide nsteps
+        const uint4 wv = *reinterpret_cast<const uint4 *>(wrow + s * 64);
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
-            const uint4 xa = *reinterpret_cast<const uint4 *>(xrow[m] + s * 64);
-            const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(xrow[m] + x8 + s * 64) : make_uint4(0, 0, 0, 0);
-            mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-            mma_bf16(acc2[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+            const uint4 va = *reinterpret_cast<const uint4 *>(xrow[m] + s * 64);
+            const uint4 vb = has1[m] ? *reinterpret_cast<const uint4 *>(xrow[m] + x8 + s * 64) : make_uint4(0, 0, 0, 0);
+            mma_bf16(ch[m][0], va.x, vb.x, va.y, vb.y, wv.x, wv.y);
+            mma_bf16(ch[m][1], va.z, vb.z, va.w, vb.w, wv.z, wv.w);
         }
     }
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[m][q] += acc2[m][q];
+        for (int q = 0; q < 4; ++q) {
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2 * BS; ++c) sum += ch[m][c][q];
+            acc[m][q] = sum;
+        }
     // lane (g, t) holds (gate row t, up row t) of tokens g and g + 8 of every m-tile
     const int n_routed = p.B * p.sh.k;
 #pragma unroll
@@ -347,32 +399,89 @@ __device__ __forceinline__ void consume_phase2(const StreamArgs &p, const StGrou
     }
     const size_t o8 = (size_t)8 * opitch;
     const size_t lo_off = (size_t)tpad * opitch;
-    float acc2[MT][4], acc3[MT][4], acc4[MT][4];   // independent chains: hi/lo parts, even/odd halves
+    const int nsteps = d.klen >> 5;
+    // blocks of two K-steps, next block's loads in flight during the current block's
+    // tensor-core instructions; four chains per step (hi / lo parts, two halves of the step)
+    constexpr int BS = MT == 1 ? 2 : 1;
+    constexpr int NB = MT <= 2 ? 2 : 1;
+    float ch[MT][4 * BS][4];
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc2[m][q] = acc3[m][q] = acc4[m][q] = 0.f;
-    const int nsteps = d.klen >> 5;
-#pragma unroll 2
-    for (int s = 0; s < nsteps; ++s) {
-        const uint4 w = *reinterpret_cast<const uint4 *>(wrow + s * 64);
+        for (int c = 0; c < 4 * BS; ++c)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) ch[m][c][q] = 0.f;
+    uint4 w[NB][BS], xa[NB][BS][MT], xb[NB][BS][MT], la[NB][BS][MT], lb[NB][BS][MT];
+    auto load_block = [&](int buf, int s0) {
+#pragma unroll
+        for (int i = 0; i < BS; ++i) {
+            const int o = (s0 + i) * 64;
+            w[buf][i] = *reinterpret_cast<const uint4 *>(wrow + o);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                const uint4 z = make_uint4(0, 0, 0, 0);
+                xa[buf][i][m] = *reinterpret_cast<const uint4 *>(hrow[m] + o);
+                la[buf][i][m] = *reinterpret_cast<const uint4 *>(hrow[m] + lo_off + o);
+                xb[buf][i][m] = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + o) : z;
+                lb[buf][i][m] = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + lo_off + o) : z;
+            }
+        }
+    };
+    auto mma_block = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < BS; ++i)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                const uint4 &A = xa[buf][i][m], &Bq = xb[buf][i][m], &L = la[buf][i][m], &M = lb[buf][i][m];
+                mma_bf16(ch[m][4 * i], A.x, Bq.x, A.y, Bq.y, w[buf][i].x, w[buf][i].y);
+                mma_bf16(ch[m][4 * i + 1], A.z, Bq.z, A.w, Bq.w, w[buf][i].z, w[buf][i].w);
+                mma_bf16(ch[m][4 * i + 2], L.x, M.x, L.y, M.y, w[buf][i].x, w[buf][i].y);
+                mma_bf16(ch[m][4 * i + 3], L.z, M.z, L.w, M.w, w[buf][i].z, w[buf][i].w);
+            }
+    };
+    const int nblk = nsteps / BS;
+    if (NB == 2) {
+        if (nblk > 0) load_block(0, 0);
+#pragma unroll 1
+        for (int blk = 0; blk + 1 < nblk; blk += 2) {
+            load_block(NB - 1, (blk + 1) * BS);
+            mma_block(0);
+            if (blk + 2 < nblk) load_block(0, (blk + 2) * BS);
+            mma_block(NB - 1);
+        }
+        if (nblk & 1) mma_block(0);
+    } else {
+#pragma unroll 1
+        for (int blk = 0; blk < nblk; ++blk) {
+            load_block(0, blk * BS);
+            mma_block(0);
+        }
+    }
+    for (int s = nblk * BS; s < nsteps; ++s) {
+        const int o = s * 64;
+        const uint4 wv = *reinterpret_cast<const uint4 *>(wrow + o);
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
             const uint4 z = make_uint4(0, 0, 0, 0);
-            const uint4 xa = *reinterpret_cast<const uint4 *>(hrow[m] + s * 64);
-            const uint4 la = *reinterpret_cast<const uint4 *>(hrow[m] + lo_off + s * 64);
-            const uint4 xb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + s * 64) : z;
-            const uint4 lb = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + lo_off + s * 64) : z;
-            mma_bf16(acc[m], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-            mma_bf16(acc2[m], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
-            mma_bf16(acc3[m], la.x, lb.x, la.y, lb.y, w.x, w.y);
-            mma_bf16(acc4[m], la.z, lb.z, la.w, lb.w, w.z, w.w);
+            const uint4 A = *reinterpret_cast<const uint4 *>(hrow[m] + o);
+            const uint4 L = *reinterpret_cast<const uint4 *>(hrow[m] + lo_off + o);
+            const uint4 Bq = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + o) : z;
+            const uint4 M = has1[m] ? *reinterpret_cast<const uint4 *>(hrow[m] + o8 + lo_off + o) : z;
+            mma_bf16(ch[m][0], A.x, Bq.x, A.y, Bq.y, wv.x, wv.y);
+            mma_bf16(ch[m][1], A.z, Bq.z, A.w, Bq.w, wv.z, wv.w);
+            mma_bf16(ch[m][2], L.x, M.x, L.y, M.y, wv.x, wv.y);
+            mma_bf16(ch[m][3], L.z, M.z, L.w, M.w, wv.z, wv.w);
         }
     }
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[m][q] += acc2[m][q] + (acc3[m][q] + acc4[m][q]);
+        for (int q = 0; q < 4; ++q) {
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4 * BS; ++c) sum += ch[m][c][q];
+            acc[m][q] = sum;
+        }
     // lane (g, t): columns 2t, 2t+1 are down rows t and 4 + t of the stage
     const int r0 = d.tile * 8 + t;
 #pragma unroll
