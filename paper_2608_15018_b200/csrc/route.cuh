@@ -1,10 +1,10 @@
 // Router logits and reuse-aware expert gating (Sec. 4.2) for one draft batch.
 //
-//   router_logits_kernel : l_{b,e} = h_b . W_r[e]  (and the shared-expert gate logit),
-//                          float64 accumulation so that the discrete choices below
-//                          do not depend on the summation order.
-//   gating_kernel        : Eq. 4 aggregation, TopCap, lambda_b, biased top-k, mixing
-//                          weights, union / unique count, token->expert bucketing.
+//   route_kernel : l_{b,e} = h_b . W_r[e] (and the shared-expert gate logit) in float64, so
+//                  that the discrete choices below do not depend on the summation order;
+//                  the last block to finish then runs gating_block:
+//   gating_block : Eq. 4 aggregation, TopCap, lambda_b, biased top-k, mixing weights,
+//                  union / unique count, token->expert bucketing, stage tables.
 #pragma once
 
 #include "common.cuh"
@@ -12,8 +12,6 @@
 
 namespace s2moe {
 
-constexpr int kRouteWarps = 8;
-constexpr int kGateThreads = 1024;
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -26,49 +24,6 @@ __device__ __forceinline__ double warp_max(double v)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
     return v;
-}
-
-// One warp per router row (row E is the shared-expert gate vector), all B tokens.
-template <int ACT, int RT>
-__global__ void __launch_bounds__(kRouteWarps * 32)
-router_logits_kernel(Shape sh, int B, const void *__restrict__ hidden, const void *__restrict__ router,
-                     const void *__restrict__ sh_scale, double *__restrict__ logits,
-                     double *__restrict__ gate_logit)
-{
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = blockIdx.x * kRouteWarps + warp;
-    const int n_rows = sh.E + (sh_scale ? 1 : 0);
-    if (row >= n_rows) return;
-    const int d = sh.d;
-    const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
-    const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
-                                     : reinterpret_cast<const uint8_t *>(sh_scale);
-    for (int b0 = 0; b0 < B; b0 += 8) {
-        double acc[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) acc[t] = 0.0;
-        for (int c = lane * 8; c < d; c += 256) {
-            float w[8];
-            load8_plain<RT>(wrow, c, w);
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                if (b0 + t < B) {
-                    float x[8];
-                    load8_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)(b0 + t) * d * ab, c, x);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[t] = fma((double)w[i], (double)x[i], acc[t]);
-                }
-            }
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            double s = warp_sum(acc[t]);
-            if (lane == 0 && b0 + t < B) {
-                if (row < sh.E) logits[(size_t)(b0 + t) * sh.E + row] = s;
-                else gate_logit[b0 + t] = s;
-            }
-        }
-    }
 }
 
 // order (value descending, id ascending): is a before b?
@@ -84,12 +39,12 @@ __device__ __forceinline__ bool before2(double l2a, double la, int a, double l2b
     return a < b;
 }
 
-// One block.  Dynamic shared memory: B*E doubles (the logits).
-__global__ void __launch_bounds__(kGateThreads)
-gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int has_gate,
-              int32_t *__restrict__ sel_idx, float *__restrict__ sel_w, int32_t *__restrict__ n_unique)
+// Gating of one batch by one thread block (any block size that is a multiple of 32).
+// s_l: shared memory for B*E doubles (the logits, copied from the workspace).
+__device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
+                                             int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
+                                             int32_t *__restrict__ n_unique, double *s_l)
 {
-    extern __shared__ double s_l[];  // [B][E]
     __shared__ double s_g[kMaxExperts];
     __shared__ unsigned char s_star[kMaxExperts];
     __shared__ double s_w[kMaxTokens], s_top1[kMaxTokens], s_kth[kMaxTokens], s_lam[kMaxTokens];
@@ -103,7 +58,7 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
     const int E = sh.E, k = sh.k, cap = sh.cap;
     const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
 
-    for (int i = tid; i < B * E; i += nt) s_l[i] = ws.logits[i];
+    for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
     for (int b = tid; b < B; b += nt) {
         s_w[b] = conf ? (double)conf[b] : 1.0;
         s_lam[b] = 0.0;
@@ -223,7 +178,7 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
     for (int i = tid; i < sh.n_sh * B; i += nt) {
         const int s = i / B, b = i - s * B;
         float c = 1.0f;
-        if (has_gate) c = (float)(1.0 / (1.0 + exp(-ws.gate_logit[b])));
+        if (has_gate) c = (float)(1.0 / (1.0 + exp(-__ldcg(&ws.gate_logit[b]))));
         ws.slot_token[n_routed + i] = b;
         ws.slot_w[n_routed + i] = c;
         if (b == 0) {
@@ -276,6 +231,86 @@ gating_kernel(Shape sh, int B, Workspace ws, const float *__restrict__ conf, int
         ws.header[3] = B;
         *n_unique = U;
     }
+}
+
+// 4 consecutive elements of a plain (f32 / bf16) row starting at column c (c % 4 == 0)
+template <int DT>
+__device__ __forceinline__ void load4_plain(const void *row, int c, float (&v)[4])
+{
+    if (DT == DT_F32) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(row) + c));
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    } else {
+        const uint2 a = __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(row) + c));
+        v[0] = bf16_lo(a.x); v[1] = bf16_hi(a.x); v[2] = bf16_lo(a.y); v[3] = bf16_hi(a.y);
+    }
+}
+
+constexpr int kRouteThreads = 512;
+constexpr int kRouteTok = 16;   // tokens accumulated per pass
+
+// Router logits and gating in one launch.  Block r computes row r of the router (row E is the
+// shared-expert gate vector) against all B tokens in float64; the block that finishes last
+// (atomic ticket, nobody waits) then runs the gating for the whole batch.
+// Dynamic shared memory: max(B * E, 16 * kRouteTok) doubles.
+template <int ACT, int RT>
+__global__ void __launch_bounds__(kRouteThreads)
+route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
+             const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
+             float *__restrict__ sel_w, int32_t *__restrict__ n_unique)
+{
+    extern __shared__ double s_dyn[];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int row = blockIdx.x, d = sh.d;
+    const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
+    const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
+                                     : reinterpret_cast<const uint8_t *>(sh_scale);
+    for (int b0 = 0; b0 < B; b0 += kRouteTok) {
+        double acc[kRouteTok];
+#pragma unroll
+        for (int t = 0; t < kRouteTok; ++t) acc[t] = 0.0;
+        for (int c = tid * 4; c < d; c += kRouteThreads * 4) {
+            float w[4];
+            load4_plain<RT>(wrow, c, w);
+#pragma unroll
+            for (int t = 0; t < kRouteTok; ++t) {
+                if (b0 + t < B) {
+                    float x[4];
+                    load4_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)(b0 + t) * d * ab, c, x);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[i], acc[t]);
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < kRouteTok; ++t) {
+            if (b0 + t < B) {           // uniform across the block
+                const double s = warp_sum(acc[t]);
+                if (lane == 0) s_dyn[warp * kRouteTok + t] = s;
+            }
+        }
+        __syncthreads();
+        if (tid < kRouteTok && b0 + tid < B) {
+            double s = 0.0;
+            for (int w = 0; w < kRouteThreads / 32; ++w) s += s_dyn[w * kRouteTok + tid];
+            if (row < sh.E) ws.logits[(size_t)(b0 + tid) * sh.E + row] = s;
+            else ws.gate_logit[b0 + tid] = s;
+        }
+        __syncthreads();
+    }
+    // the block that arrives last sees every row (release by fence + ticket, acquire by fence)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned t = atomicAdd(ws.ticket, 1u);
+        s_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) *ws.ticket = 0u;
+    gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
 }
 
 }  // namespace s2moe

@@ -133,18 +133,40 @@ int validate_layer(const s2moe_config *c, const s2moe_layer_weights *w)
 
 // ---- dispatch over storage formats ------------------------------------------
 
-template <int ACT>
-void launch_router(s2moe_ctx *ctx, const LayerPtrs &lp, int B, const void *hidden, cudaStream_t st)
+size_t route_smem(int B, int E)
 {
-    const int rows = ctx->shape.E + (lp.sh_scale ? 1 : 0);
-    const dim3 grid((rows + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
+    const size_t a = (size_t)B * E, b = (size_t)(kRouteThreads / 32) * kRouteTok;
+    return sizeof(double) * (a > b ? a : b);
+}
+
+template <int ACT, int RT>
+void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
+                    int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
+{
+    const int rows = sh.E + (lp.sh_scale ? 1 : 0);
     LaunchScope scope(ctx, KC_ROUTER, st);
-    if (ctx->shape.router_dtype == DT_F32)
-        router_logits_kernel<ACT, DT_F32><<<grid, block, 0, st>>>(ctx->shape, B, hidden, lp.router, lp.sh_scale,
-                                                                  ctx->ws.logits, ctx->ws.gate_logit);
-    else
-        router_logits_kernel<ACT, DT_BF16><<<grid, block, 0, st>>>(ctx->shape, B, hidden, lp.router, lp.sh_scale,
-                                                                   ctx->ws.logits, ctx->ws.gate_logit);
+    route_kernel<ACT, RT><<<rows, kRouteThreads, route_smem(B, sh.E), st>>>(sh, B, ctx->ws, hidden, lp.router, lp.sh_scale,
+                                                                            conf, sel_idx, sel_w, n_unique);
+}
+
+void launch_route(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
+                  int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
+{
+    const bool af = sh.act_dtype == DT_F32, rf = sh.router_dtype == DT_F32;
+    if (af && rf) launch_route_t<DT_F32, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+    else if (af) launch_route_t<DT_F32, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+    else if (rf) launch_route_t<DT_BF16, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+    else launch_route_t<DT_BF16, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+}
+
+cudaError_t prepare_route()
+{
+    const int bytes = (int)(sizeof(double) * kMaxTokens * kMaxExperts);
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<DT_F32, DT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_F32, DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_BF16, DT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_BF16, DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
 }
 
 constexpr size_t kSimpleSmem = (size_t)kSimpleTokChunk * kSimpleKChunk * sizeof(float);
@@ -211,13 +233,7 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     sh.plan = plan;
     sh.op_cap = pl.op_cap;
     CU(ctx, cudaMemsetAsync(out, 0, (size_t)B * sh.d * sizeof(float), st));
-    if (sh.act_dtype == DT_F32) launch_router<DT_F32>(ctx, lp, B, hidden, st);
-    else launch_router<DT_BF16>(ctx, lp, B, hidden, st);
-    {
-        LaunchScope scope(ctx, KC_GATING, st);
-        gating_kernel<<<1, kGateThreads, (size_t)B * sh.E * sizeof(double), st>>>(
-            sh, B, ctx->ws, conf, lp.sh_scale ? 1 : 0, sel_idx, sel_w, n_unique);
-    }
+    launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
     if (plan == 2) {
         StreamArgs a;
         a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
@@ -304,9 +320,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e == cudaSuccess && ctx->plan != 1)
         e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStMaxSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gating_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(double) * kMaxTokens * kMaxExperts));
+    if (e == cudaSuccess) e = prepare_route();
     if (e != cudaSuccess) { cudaFree(ctx->slab); delete ctx; return S2MOE_ECUDA; }
     uint8_t *base = (uint8_t *)ctx->slab;
     Workspace &ws = ctx->ws;
@@ -470,8 +484,8 @@ int s2moe_profile_end(s2moe_ctx *ctx, int32_t n_classes, double *ms_out, int64_t
 const char *s2moe_kernel_class_name(int32_t cls)
 {
     switch (cls) {
-        case KC_ROUTER: return "router_logits_kernel";
-        case KC_GATING: return "gating_kernel";
+        case KC_ROUTER: return "route_kernel";
+        case KC_GATING: return "(unused)";
         case KC_GATEUP: return "ffn_gateup_simple";
         case KC_DOWN: return "ffn_down_simple";
         case KC_STREAM: return "ffn_stream_kernel";
@@ -498,6 +512,7 @@ int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
         case 5: src = ctx->ws.active; need = 4 * (size_t)hdr[0]; break;
         case 6: src = ctx->ws.header; need = 16; break;
         case 7: src = ctx->ws.header + 8; need = 32; break;
+        case 8: src = ctx->ws.act; need = bytes; break;   // timing build: per-warp cycle counters
         default: return S2MOE_EINVAL;
     }
     if (bytes < need) return S2MOE_EINVAL;
