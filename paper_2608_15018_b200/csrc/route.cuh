@@ -57,6 +57,14 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     const int tid = threadIdx.x, nt = blockDim.x;
     const int E = sh.E, k = sh.k, cap = sh.cap;
     const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
+#ifdef S2MOE_TIMING
+    long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64;
+    int tmi = 0;
+#define GATE_MARK() do { __syncthreads(); if (tid == 0) tm[tmi] = clock64(); ++tmi; } while (0)
+#else
+#define GATE_MARK() do { } while (0)
+#endif
+    GATE_MARK();
 
     for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
     for (int b = tid; b < B; b += nt) {
@@ -66,6 +74,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
     __syncthreads();
 
+    GATE_MARK();
     if (bias_on) {
         // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
         for (int e = tid; e < E; e += nt) {
@@ -95,6 +104,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         __syncthreads();
     }
 
+    GATE_MARK();
     // biased top-k by rank
     for (int i = tid; i < B * E; i += nt) {
         const int b = i / E, e = i - b * E;
@@ -111,6 +121,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     __syncthreads();
 
+    GATE_MARK();
     // mixing weights: one warp per token
     {
         const int warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
@@ -149,6 +160,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     __syncthreads();
 
+    GATE_MARK();
     // union, unique count, exclusive scan, list of active experts
     for (int e = tid; e < E; e += nt) s_cnt[e] = __popcll(s_mask[e]);
     __syncthreads();
@@ -187,6 +199,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             ws.active[U + s] = E + s;
         }
     }
+    GATE_MARK();
     for (int e = tid; e < E; e += nt) ws.tokmask[e] = s_mask[e];
     for (int s = tid; s < sh.n_sh; s += nt) ws.tokmask[E + s] = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
     if (sh.plan == 2) {
@@ -223,6 +236,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             ws.header[5] = t2;
         }
     }
+    GATE_MARK();
     if (tid == 0) {
         ws.offsets[E + sh.n_sh] = n_routed + sh.n_sh * B;
         ws.header[0] = U + sh.n_sh;
@@ -262,6 +276,9 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     extern __shared__ double s_dyn[];
     __shared__ int s_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef S2MOE_TIMING
+    const long long t_start = clock64();
+#endif
     const int row = blockIdx.x, d = sh.d;
     const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
     const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
@@ -310,6 +327,9 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     if (!s_last) return;
     __threadfence();
     if (tid == 0) *ws.ticket = 0u;
+#ifdef S2MOE_TIMING
+    if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[15] = t_start; tm[14] = clock64(); }
+#endif
     gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
 }
 
