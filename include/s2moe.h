@@ -215,6 +215,43 @@ const char *s2moe_kernel_class_name(int32_t cls);
  */
 int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes);
 
+/*
+ * Routing without any allocation (the paper has no counterpart; this is a convenience of
+ * this library).  Some callers must not allocate device memory while they run: a serving
+ * loop that has handed the whole device to its own memory pool, code that runs while a
+ * framework's allocator is locked or a stream capture is open, or a latency-critical
+ * path where a cudaMalloc (which may synchronise the device) is not acceptable.
+ * s2moe_create allocates a workspace, so it is closed to them.  This entry point runs
+ * steps 1-3 of the layer (router logits, reuse-aware gating, the unique-expert count)
+ * with its scratch memory in a fixed array that is part of the library image: every GPU
+ * that loads the library holds S2MOE_NOALLOC_SCRATCH_BYTES of it until the process exits.
+ *
+ *   cfg      the fields d_model, n_experts, top_k, act_dtype, router_dtype, renorm, cap,
+ *            alpha and weight_mode are used, with the limits of s2moe_config; the rest
+ *            is ignored
+ *   router   dev [E][d] router_dtype          gate_vec  dev [d] router_dtype or NULL
+ *   hidden   dev [B][d] act_dtype             conf      dev [B] float or NULL
+ *   sel_idx  dev [B][k] int32, sel_w dev [B][k] float, n_unique dev int32: as in
+ *            s2moe_verify_layer
+ *   gate_out dev [B] float or NULL: sigmoid(h_b . gate_vec) when gate_vec is given
+ *
+ * Limits: n_tokens <= S2MOE_NOALLOC_MAX_TOKENS, n_experts <= S2MOE_NOALLOC_MAX_EXPERTS;
+ * larger sizes return ERANGE and launch nothing.  The call is asynchronous on the stream
+ * and calls no cudaMalloc, cudaFree or other allocating routine.  The first call on a
+ * device looks up the scratch array's device address and raises the kernel's shared-memory
+ * limit (once per device, with that device current); make that first call outside any
+ * stream capture.  All calls on a device share the one scratch array: the call clears the
+ * words that must start at zero, the rest keeps the previous call's contents, and two
+ * calls that overlap on the GPU (different streams, no ordering between them) race.
+ * Errors: EINVAL (null pointer, bad config, misaligned hidden or router), ERANGE, ECUDA.
+ */
+#define S2MOE_NOALLOC_MAX_TOKENS 64
+#define S2MOE_NOALLOC_MAX_EXPERTS 128
+#define S2MOE_NOALLOC_SCRATCH_BYTES (96 * 1024)
+int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *router, const void *gate_vec,
+                        const void *hidden, const float *conf, int32_t *sel_idx, float *sel_w,
+                        int32_t *n_unique, float *gate_out, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,9 @@ WEIGHT_FIELDS = ("router", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down
 EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_verify_stack_host",
            "s2moe_destroy", "s2moe_strerror", "s2moe_last_device_status", "s2moe_last_cuda_error",
            "s2moe_kernel_launches", "s2moe_unique_expert_bytes", "s2moe_debug_read",
-           "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan")
+           "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan",
+           "s2moe_route_noalloc")
+NOALLOC_MAX_TOKENS, NOALLOC_MAX_EXPERTS = 64, 128
 KERNEL_CLASSES = 5
 
 
@@ -91,6 +93,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_unique_expert_bytes.restype = ctypes.c_double
     lib.s2moe_debug_read.argtypes = [vp, i32, vp, ctypes.c_size_t]
     lib.s2moe_debug_read.restype = ctypes.c_int
+    lib.s2moe_route_noalloc.argtypes = [ctypes.POINTER(ConfigC), i32, vp, vp, vp, fp, vp, fp, vp, fp, vp]
+    lib.s2moe_route_noalloc.restype = ctypes.c_int
     lib.s2moe_profile_begin.argtypes = [vp, i32]
     lib.s2moe_profile_begin.restype = ctypes.c_int
     lib.s2moe_profile_end.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
@@ -304,3 +308,25 @@ class S2MoE:
             counts=self.debug_read(1, G, torch.int32), offsets=self.debug_read(2, G + 1, torch.int32),
             slot_token=self.debug_read(3, n_slots, torch.int32), slot_w=self.debug_read(4, n_slots, torch.float32),
             active=self.debug_read(5, n_active, torch.int32))
+
+
+def route_noalloc(config: Config, hidden: torch.Tensor, router: torch.Tensor,
+                  conf: Optional[torch.Tensor] = None, gate_vec: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None):
+    """Router logits, reuse-aware gating and the unique-expert count through
+    ``s2moe_route_noalloc``: the library allocates nothing (its scratch is a fixed array in
+    the library image).  For callers that may not allocate device memory while they run;
+    the output tensors here are the caller's.  Returns (sel_idx, sel_w, n_unique, gate)."""
+    lib = load_library()
+    B = hidden.shape[0]
+    dev = hidden.device
+    sel_idx = torch.empty((B, config.top_k), dtype=torch.int32, device=dev)
+    sel_w = torch.empty((B, config.top_k), dtype=torch.float32, device=dev)
+    n_unique = torch.empty((1,), dtype=torch.int32, device=dev)
+    gate = torch.empty((B,), dtype=torch.float32, device=dev) if gate_vec is not None else None
+    cfg = config.c()
+    rc = lib.s2moe_route_noalloc(ctypes.byref(cfg), B, _dptr(router), _dptr(gate_vec), _dptr(hidden), _dptr(conf),
+                                 _dptr(sel_idx), _dptr(sel_w), _dptr(n_unique), _dptr(gate), _stream_handle(stream))
+    if rc != OK:
+        raise S2MoEError(rc, "s2moe_route_noalloc")
+    return sel_idx, sel_w, n_unique, gate

@@ -520,4 +520,99 @@ int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
     return S2MOE_OK;
 }
 
+// ---- routing without allocation -------------------------------------------------------
+
+namespace {
+
+// Scratch of s2moe_route_noalloc.  In host code this name is only a handle for
+// cudaGetSymbolAddress; kernels get the device address that call returns.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[S2MOE_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kNoallocMaxDevices = 64;
+void *g_noalloc_ptr[kNoallocMaxDevices] = {};
+
+__global__ void noalloc_gate_out_kernel(const double *__restrict__ gate_logit, float *__restrict__ gate_out, int B)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) gate_out[b] = (float)(1.0 / (1.0 + exp(-gate_logit[b])));
+}
+
+}  // namespace
+
+int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *router, const void *gate_vec,
+                        const void *hidden, const float *conf, int32_t *sel_idx, float *sel_w,
+                        int32_t *n_unique, float *gate_out, void *cuda_stream)
+{
+    if (!cfg || !router || !hidden || !sel_idx || !sel_w || !n_unique) return S2MOE_EINVAL;
+    if (cfg->d_model < 64 || cfg->d_model % 64) return S2MOE_EINVAL;
+    if (cfg->n_experts < 1 || cfg->top_k < 1 || cfg->top_k > cfg->n_experts || cfg->top_k > S2MOE_MAX_TOP_K)
+        return S2MOE_EINVAL;
+    if (cfg->act_dtype != S2MOE_F32 && cfg->act_dtype != S2MOE_BF16) return S2MOE_EINVAL;
+    if (cfg->router_dtype != S2MOE_F32 && cfg->router_dtype != S2MOE_BF16) return S2MOE_EINVAL;
+    if ((cfg->renorm != 0 && cfg->renorm != 1) || (cfg->weight_mode != 0 && cfg->weight_mode != 1)) return S2MOE_EINVAL;
+    if (cfg->cap < cfg->top_k || cfg->cap > cfg->n_experts || !(cfg->alpha >= 0.0f)) return S2MOE_EINVAL;
+    if (!aligned16(router) || !aligned16(hidden) || (gate_vec && !aligned16(gate_vec))) return S2MOE_EINVAL;
+    if (n_tokens < 0 || n_tokens > S2MOE_NOALLOC_MAX_TOKENS || cfg->n_experts > S2MOE_NOALLOC_MAX_EXPERTS)
+        return S2MOE_ERANGE;
+    if (n_tokens == 0) return S2MOE_OK;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    // once per device: the scratch array's device address, and the kernels' shared-memory limit
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoallocMaxDevices) return S2MOE_ECUDA;
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return S2MOE_ECUDA;
+        if (prepare_route() != cudaSuccess) return S2MOE_ECUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    uint8_t *base = (uint8_t *)g_noalloc_ptr[dev];
+
+    // carve the scratch: the routing kernel's workspace for E <= 128 experts, B <= 64 tokens
+    const int T = S2MOE_NOALLOC_MAX_TOKENS, E = S2MOE_NOALLOC_MAX_EXPERTS, K = S2MOE_MAX_TOP_K;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    Workspace ws{};
+    ws.logits = (double *)(base + take(sizeof(double) * T * E));
+    ws.gate_logit = (double *)(base + take(sizeof(double) * T));
+    uint8_t *zero_begin = base + off;                       // words that must start at zero
+    ws.ticket = (unsigned int *)(base + take(256));
+    ws.status = (int32_t *)(base + take(256));
+    uint8_t *zero_end = base + off;
+    ws.header = (int32_t *)(base + take(256));
+    ws.counts = (int32_t *)(base + take(4 * (size_t)E));
+    ws.offsets = (int32_t *)(base + take(4 * (size_t)(E + 1)));
+    ws.slot_token = (int32_t *)(base + take(4 * (size_t)T * K));
+    ws.slot_w = (float *)(base + take(4 * (size_t)T * K));
+    ws.active = (int32_t *)(base + take(4 * (size_t)E));
+    ws.tokmask = (unsigned long long *)(base + take(8 * (size_t)E));
+    static_assert(sizeof(double) * S2MOE_NOALLOC_MAX_TOKENS * S2MOE_NOALLOC_MAX_EXPERTS + 24 * 1024 <=
+                      S2MOE_NOALLOC_SCRATCH_BYTES, "scratch too small");
+    if (off > S2MOE_NOALLOC_SCRATCH_BYTES) return S2MOE_ERANGE;
+
+    Shape sh{};
+    sh.d = cfg->d_model; sh.f = 0; sh.E = cfg->n_experts; sh.k = cfg->top_k; sh.n_sh = 0; sh.f_sh = 0;
+    sh.act_dtype = cfg->act_dtype; sh.router_dtype = cfg->router_dtype; sh.weight_dtype = DT_BF16;
+    sh.renorm = cfg->renorm; sh.cap = cfg->cap; sh.weight_mode = cfg->weight_mode; sh.plan = 1; sh.op_cap = 0;
+    sh.alpha = (double)cfg->alpha;
+    if (cudaMemsetAsync(zero_begin, 0, (size_t)(zero_end - zero_begin), st) != cudaSuccess) return S2MOE_ECUDA;
+    const int rows = sh.E + (gate_vec ? 1 : 0);
+    const size_t smem = route_smem(n_tokens, sh.E);
+    const bool af = sh.act_dtype == DT_F32, rf = sh.router_dtype == DT_F32;
+    if (af && rf)
+        route_kernel<DT_F32, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
+                                                                        sel_idx, sel_w, n_unique);
+    else if (af)
+        route_kernel<DT_F32, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
+                                                                         sel_idx, sel_w, n_unique);
+    else if (rf)
+        route_kernel<DT_BF16, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
+                                                                         sel_idx, sel_w, n_unique);
+    else
+        route_kernel<DT_BF16, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
+                                                                          sel_idx, sel_w, n_unique);
+    if (gate_vec && gate_out) noalloc_gate_out_kernel<<<1, 64, 0, st>>>(ws.gate_logit, gate_out, n_tokens);
+    return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
+}
+
 }  // extern "C"
