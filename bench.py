@@ -176,7 +176,7 @@ def run_own(args, wl, B, sigma):
     import torch
     import torch.distributed as dist
 
-    from paper_2608_15018_b200 import binding, workloads
+    from paper_2608_15018_b200 import binding, replicas, workloads
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -186,7 +186,7 @@ def run_own(args, wl, B, sigma):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     L = args.layers or wl.n_layers
-    wl_r = wl.with_(seed=wl.seed + 1000 * rank, n_layers=L)      # replicas: independent requests
+    wl_r = replicas.replica_workload(wl, rank).with_(n_layers=L)      # replicas: independent requests
 
     weights = [workloads.layer_weights(wl_r, l, dev) for l in range(L)]
     H = torch.stack([workloads.hidden_states(wl_r, l, B, sigma, dev) for l in range(L)]).contiguous()
@@ -270,13 +270,10 @@ def run_own(args, wl, B, sigma):
     d2h = ho.numel() * 4 + hs.numel() * 4 + hw.numel() * 4 + hu.numel() * 4
 
     # ---- max over ranks
-    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_total = times.tolist()
+    ms_total, e2e_ms_total = replicas.max_over_ranks([ms_total, e2e_s * 1e3], device=dev)
     ms_step = ms_total / args.steps
-    value = world * B * L / (ms_step * 1e-3)                 # tokens/s per layer, all ranks
-    e2e_value = world * B * L / (e2e_ms_total / args.steps * 1e-3)
+    value = replicas.aggregate_tokens_per_s(world, B, L, ms_step)          # tokens/s per layer, all ranks
+    e2e_value = replicas.aggregate_tokens_per_s(world, B, L, e2e_ms_total / args.steps)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
