@@ -115,7 +115,8 @@ typedef struct {
     int32_t n_layers;      /* >= 1                                                          */
     int32_t kernel_plan;   /* 0: automatic (plan 2 where it applies, else plan 1);
                               1: plain CUDA-core kernels (every format and batch size);
-                              2: streaming tensor-core kernel (bf16 weights and activations) */
+                              2: streaming mma.sync kernel (bf16 weights and activations);
+                              3: streaming tcgen05 kernel (bf16 weights and activations)      */
 } s2moe_config;
 
 /*
@@ -176,8 +177,8 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out);
 /* The last cudaError_t a call on this context saw (0 = cudaSuccess). */
 int s2moe_last_cuda_error(const s2moe_ctx *ctx);
 
-/* The kernel plan a batch of n_tokens runs with (1 or 2; see s2moe_config.kernel_plan).
- * 0: NULL context, n_tokens out of range, or plan 2 was demanded and this batch size
+/* The kernel plan a batch of n_tokens runs with (1, 2 or 3; see s2moe_config.kernel_plan).
+ * 0: NULL context, n_tokens out of range, or plan 2 / 3 was demanded and this batch size
  * does not fit its shared-memory layout (s2moe_verify_layer then returns EINVAL). */
 int s2moe_kernel_plan(const s2moe_ctx *ctx, int32_t n_tokens);
 
@@ -197,7 +198,7 @@ double s2moe_unique_expert_bytes(const s2moe_ctx *ctx, int32_t n_unique);
  * number of timed launches.  s2moe_kernel_class_name gives the kernel's name, or
  * NULL past the last class.  Do not use during stream capture.
  */
-#define S2MOE_KERNEL_CLASSES 5
+#define S2MOE_KERNEL_CLASSES 6
 int s2moe_profile_begin(s2moe_ctx *ctx, int32_t max_records);
 int s2moe_profile_end(s2moe_ctx *ctx, int32_t n_classes, double *ms_out, int64_t *launches_out);
 const char *s2moe_kernel_class_name(int32_t cls);

@@ -27,7 +27,7 @@ EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_ve
            "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan",
            "s2moe_route_noalloc")
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_EXPERTS = 64, 128
-KERNEL_CLASSES = 5
+KERNEL_CLASSES = 6
 
 
 class LayerWeightsC(ctypes.Structure):

@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "ffn_simple.cuh"
 #include "ffn_stream.cuh"
+#include "ffn_tc.cuh"
 #include "route.cuh"
 
 using namespace s2moe;
@@ -32,6 +33,9 @@ struct s2moe_ctx {
     int n_sm = 0;
     __nv_bfloat16 *act_hi = nullptr, *act_lo = nullptr;
     size_t act_elems = 0;
+    float *pre = nullptr;                 // plan 3: fp32 pre-activations [slot][2][f]
+    std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
+    void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
     int last_cuda = 0;
     int64_t launches = 0;
     int last_B = 0;
@@ -42,7 +46,7 @@ struct s2moe_ctx {
     size_t prof_cap = 0;
 };
 
-enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_COUNT = 5 };
+enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_TC = 5, KC_COUNT = 6 };
 
 namespace {
 
@@ -101,7 +105,8 @@ int validate_config(const s2moe_config *c)
     if (c->weight_mode != 0 && c->weight_mode != 1) return S2MOE_EINVAL;
     if (c->max_tokens < 1 || c->max_tokens > S2MOE_MAX_TOKENS) return S2MOE_EINVAL;
     if (c->n_layers < 1) return S2MOE_EINVAL;
-    if (c->kernel_plan < 0 || c->kernel_plan > 2) return S2MOE_EINVAL;
+    if (c->kernel_plan < 0 || c->kernel_plan > 3) return S2MOE_EINVAL;
+    if (c->kernel_plan == 3 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     // the streaming plan covers bf16 weights with bf16 activations
     if (c->kernel_plan == 2 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     return S2MOE_OK;
@@ -210,16 +215,41 @@ cudaError_t prepare_simple()
         else FN<DT_Q4B32, DT_BF16>(__VA_ARGS__);                                         \
     } while (0)
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box = 64 columns x box_rows rows, 128-byte swizzle,
+// out-of-range elements read as zero
+bool make_map(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    if (!ctx->encode_tiled || !base || rows == 0) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The plan a batch of B tokens runs with: the streaming kernel when it is allowed and its
 // shared-memory layout fits, else the CUDA-core kernels; 0 when plan 2 was demanded and does not fit.
 int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
 {
     const Shape &s0 = ctx->shape;
-    if (ctx->cfg.kernel_plan == 1) return 1;
+    const int want = ctx->cfg.kernel_plan;
+    if (want == 1) return 1;
+    if (want == 0 || want == 3) {
+        const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
+        if (tp.feasible && !ctx->tc_maps.empty()) return 3;
+        if (want == 3) return 0;
+    }
     const StPlan pl = st_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
     if (out) *out = pl;
     if (pl.feasible) return 2;
-    return ctx->cfg.kernel_plan == 2 ? 0 : 1;
+    return want == 2 ? 0 : 1;
 }
 
 int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float *conf, float *out,
@@ -233,8 +263,29 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     sh.plan = plan;
     sh.op_cap = pl.op_cap;
     CU(ctx, cudaMemsetAsync(out, 0, (size_t)B * sh.d * sizeof(float), st));
+    if (plan == 3) {
+        const size_t used = (size_t)B * sh.k * sh.f + (size_t)sh.n_sh * B * sh.f_sh;
+        CU(ctx, cudaMemsetAsync(ctx->pre, 0, used * 2 * sizeof(float), st));
+        CU(ctx, cudaMemsetAsync(ctx->ws.sync, 0, 4 * (size_t)(kTcReady + kStMaxGroups), st));
+    }
     launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
-    if (plan == 2) {
+    if (plan == 3) {
+        const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
+        TcMaps maps = ctx->tc_maps[layer];
+        const size_t n_routed = (size_t)B * sh.k;
+        bool ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
+                  make_map(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, 16) &&
+                  make_map(ctx, &maps.m[8], ctx->act_lo, n_routed, (uint64_t)sh.f, 16);
+        if (ok && sh.n_sh)
+            ok = make_map(ctx, &maps.m[9], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, 16) &&
+                 make_map(ctx, &maps.m[10], ctx->act_lo + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, 16);
+        if (!ok) return S2MOE_ECUDA;
+        TcArgs a;
+        a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
+        a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
+        LaunchScope scope(ctx, KC_TC, st);
+        ffn_tc_kernel<<<tp.n_cta, kTcThreads, tp.smem_bytes, st>>>(maps, a);
+    } else if (plan == 2) {
         StreamArgs a;
         a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
         a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
@@ -304,7 +355,8 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_ticket = take(256), o_status = take(256), o_header = take(256);
     const size_t o_counts = take(4 * (size_t)G), o_offsets = take(4 * (size_t)(G + 1));
     const size_t o_stok = take(4 * n_slots), o_sw = take(4 * n_slots), o_active = take(4 * (size_t)G);
-    const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(kStMaxGroups + 64));
+    const size_t o_act = take(4 * act_floats), o_sync = take(4 * (size_t)(kTcReady + kStMaxGroups + 64));
+    const size_t o_pre = take(8 * act_floats);
     const size_t o_ahi = take(2 * act_floats), o_alo = take(2 * act_floats);
     const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
     const size_t o_tm = take(8 * (size_t)G);
@@ -332,6 +384,32 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ws.act = (float *)(base + o_act); ws.sync = (int32_t *)(base + o_sync);
     ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
     ws.tokmask = (unsigned long long *)(base + o_tm);
+    ctx->pre = (float *)(base + o_pre);
+    // plan 3: tensor maps of the weights (one set per layer); without the driver entry point or
+    // for other formats the plan is simply not offered
+    if (ctx->plan != 1 && ctx->plan != 2 && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16) {
+        cudaDriverEntryPointQueryResult qres;
+        void *fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && fn) {
+            ctx->encode_tiled = fn;
+            ctx->tc_maps.resize(config->n_layers);
+            bool ok = cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
+            for (int l = 0; l < config->n_layers && ok; ++l) {
+                const LayerPtrs &lp = ctx->layers[l];
+                TcMaps &m = ctx->tc_maps[l];
+                std::memset(&m, 0, sizeof(m));
+                ok = make_map(ctx, &m.m[0], lp.w_gate, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
+                     make_map(ctx, &m.m[1], lp.w_up, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
+                     make_map(ctx, &m.m[2], lp.w_down, (uint64_t)sh.E * sh.d, (uint64_t)sh.f, 128);
+                if (ok && sh.n_sh)
+                    ok = make_map(ctx, &m.m[3], lp.sh_gate, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
+                         make_map(ctx, &m.m[4], lp.sh_up, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
+                         make_map(ctx, &m.m[5], lp.sh_down, (uint64_t)sh.n_sh * sh.d, (uint64_t)sh.f_sh, 128);
+            }
+            if (!ok) ctx->tc_maps.clear();
+        }
+    }
     ctx->act_hi = (__nv_bfloat16 *)(base + o_ahi); ctx->act_lo = (__nv_bfloat16 *)(base + o_alo);
     ctx->st_hidden = base + o_sth; ctx->st_conf = (float *)(base + o_stc);
     ctx->st_out = (float *)(base + o_sto); ctx->st_sel = (int32_t *)(base + o_sts);
@@ -489,6 +567,7 @@ const char *s2moe_kernel_class_name(int32_t cls)
         case KC_GATEUP: return "ffn_gateup_simple";
         case KC_DOWN: return "ffn_down_simple";
         case KC_STREAM: return "ffn_stream_kernel";
+        case KC_TC: return "ffn_tc_kernel";
         default: return nullptr;
     }
 }

@@ -9,8 +9,8 @@ TOL = {workloads.F32: 2e-3, workloads.BF16: 2e-3, workloads.Q4B32: 1e-2}
 
 
 def supports(wl, plan):
-    """Kernel plan 2 (streaming tensor-core kernel) covers bf16 weights with bf16 activations."""
-    return plan != 2 or (wl.weight_dtype == workloads.BF16 and wl.act_dtype == workloads.BF16)
+    """Kernel plans 2 and 3 (streaming tensor-core kernels) cover bf16 weights with bf16 activations."""
+    return plan not in (2, 3) or (wl.weight_dtype == workloads.BF16 and wl.act_dtype == workloads.BF16)
 
 
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
@@ -27,12 +27,13 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
     cfg = binding.Config.from_workload(wl, n_layers=1, kernel_plan=plan)
     with binding.S2MoE(cfg, [T]) as m:
         used = m.kernel_plan(H.shape[0])
-        if plan == 2 and used != 2:
+        if plan in (2, 3) and used != plan:
             return None, None
-        assert used in (1, 2) and (plan == 0 or used == plan)
+        assert used in (1, 2, 3) and (plan == 0 or used == plan)
         o = m.verify_layer(0, H, conf)
         torch.cuda.synchronize()
-        assert m.device_status() == 0
+        status = m.device_status()
+        assert status == 0, f"device status {status}"
         lists = m.debug_lists() if check_lists else None
         launches = m.kernel_launches()
     assert launches > 0

@@ -24,7 +24,7 @@ SMALL = {
     "cfg4": CONFIGS["cfg4"].with_(d_model=1024, d_ff=1824),
     "cfg5": CONFIGS["cfg5"].with_(d_model=512, d_ff=352, d_ff_shared=352),
 }
-PLANS = [1, 2]
+PLANS = [1, 2, 3]
 
 
 @pytest.mark.parametrize("name", sorted(SMALL))
@@ -98,7 +98,7 @@ def test_full_size_layer_sampled_tokens(name, tokens):
     rep, _ = run_case(wl, layer=1, plan=0, tok_list=tokens)
     assert rep.tokens_checked == len(tokens)
     if wl.weight_dtype == BF16:
-        assert rep.plan == 2          # the plan the benchmark times
+        assert rep.plan in (2, 3)     # a streaming plan, as the benchmark times
     torch.cuda.empty_cache()
 
 
