@@ -9,9 +9,11 @@
 //   phase 2 unit: 128 rows of W_down of one expert x KT k-tiles of 64
 //                 D[row][slot] = W[rows, k-range] . a[slots, k-range]^T, a as bf16 hi + lo
 //                 -> y[token][row] += p * D                 (red.add, fp32)
-// The unit that completes an expert's phase 1 (counter) turns pre into a = silu(g) * u
-// (bf16 hi + lo parts) and raises the expert's ready flag, which phase-2 units wait for
-// (bounded).  Units are dealt round-robin to one persistent CTA per SM.
+// Between the phases every CTA arrives on a grid-wide counter (bounded wait; one CTA per SM,
+// so all are resident), then each turns its slice of pre into a = silu(g) * u (bf16 hi + lo
+// parts) and arrives on a second counter, which the phase-2 token tiles wait for; the weight
+// tiles of the first phase-2 units are fetched meanwhile.  Units are dealt round-robin to one
+// persistent CTA per SM.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = epilogue (TMEM -> registers -> red.add).  A ring of stages, each one weight
@@ -25,6 +27,13 @@
 #include "common.cuh"
 #include "ffn_stream.cuh"
 
+// cycle-counter statements, compiled only with -DS2MOE_TIMING
+#ifdef S2MOE_TIMING
+#define TCT(...) __VA_ARGS__
+#else
+#define TCT(...)
+#endif
+
 namespace s2moe {
 
 constexpr int kTcThreads = 192;
@@ -33,7 +42,7 @@ constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 K
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
 constexpr int kTcMaxSmem = 232448 - 4096;
 constexpr unsigned kTcSpinLimit = 1u << 22;
-constexpr int kTcReady = 512;                  // ws.sync[kTcReady + a]: activations of active group a are written
+constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 2], [kTcReady - 1]: the two grid-wide counters
 
 struct TcPlan {
     int feasible;
@@ -69,7 +78,7 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
     if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
     p.tmem_cols = 32;
-    while (p.tmem_cols < 2 * p.n1) p.tmem_cols <<= 1;
+    while (p.tmem_cols < 4 * p.n1) p.tmem_cols <<= 1;   // two accumulators of up to 2 * n1 columns
     p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align the ring to 1024
     p.feasible = p.stages >= 4 && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
                  sh.d % 64 == 0;
@@ -118,6 +127,18 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 // K-major, 128-byte swizzle: rows 128 bytes apart, 8-row groups 1024 bytes apart
 __device__ __forceinline__ uint64_t tc_smem_desc(const void *p)
@@ -258,7 +279,36 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             unsigned it = 0;
-            bool alive = true;
+            bool alive = true, ready = false;
+            // phase-2 stages whose weight tile is in flight but whose token tiles wait for the
+            // activations (second grid-wide counter)
+            int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
+                pend_tn[kTcMaxStages];
+            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
+            auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
+                uint8_t *op = ring + (size_t)s * pl.stage_bytes + kTcWTile;
+                const CUtensorMap *hi = &maps.m[shared ? 9 : 7], *lo = &maps.m[shared ? 10 : 8];
+                for (int r = 0; r < tn; r += 16) {
+                    tma_load_2d(op + r * 128, hi, kt * 64, srow + r, &full_bar[s]);
+                    tma_load_2d(op + (tn + r) * 128, lo, kt * 64, srow + r, &full_bar[s]);
+                }
+            };
+            auto wait_ready = [&]() -> bool {
+                TCT(long long c0 = clock64();)
+                bool ok = false;
+                for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
+                    if (ld_acquire(&ws.sync[kTcReady - 1]) >= (int)gridDim.x) { ok = true; break; }
+                    __nanosleep(40);
+                }
+                TCT(tp_ready += clock64() - c0;)
+                if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); return false; }
+                fence_proxy_async();
+                for (int i = 0; i < pend_n; ++i) load_tokens2(pend_stage[i], pend_kt[i], pend_row[i], pend_shared[i], pend_tn[i]);
+                pend_n = 0;
+                ready = true;
+                return true;
+            };
+            const int n_routed = p.B * sh.k;
             for (int u = blockIdx.x; u < total && alive; u += P) {
                 const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
                 const StGroup &g = groups[t.a];
@@ -267,160 +317,208 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 const CUtensorMap *wmap = &maps.m[(shared ? 3 : 0) + t.mat];
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
-                if (t.phase == 2) {
-                    // the expert's activations must have been written
-                    bool ok = false;
-                    for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
-                        if (ld_acquire(&ws.sync[kTcReady + t.a]) != 0) { ok = true; break; }
-                        __nanosleep(40);
-                    }
-                    if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); alive = false; break; }
-                    fence_proxy_async();
-                }
-                const int n_routed = p.B * sh.k;
-                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it) {
+                const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared activation array
+                if (t.phase == 2 && !ready && ld_acquire(&ws.sync[kTcReady - 1]) >= (int)gridDim.x) alive = wait_ready();
+                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it) {
                     const int s = it % S;
+                    if (t.phase == 2 && !ready && pend_n == S) {
+                        if (!wait_ready()) { alive = false; break; }     // every slot waits for tokens
+                    }
+                    TCT(long long c1 = clock64();)
                     if (!mbar_wait(&empty_bar[s], ((it / S) & 1u) ^ 1u)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
                     }
+                    TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint32_t op_bytes = (uint32_t)t.n * 128u * (t.phase == 1 ? 1u : 2u);
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
                     tma_load_2d(stage, wmap, kt * 64, row0, &full_bar[s]);
-                    uint8_t *op = stage + kTcWTile;
                     if (t.phase == 1) {
+                        uint8_t *op = stage + kTcWTile;
                         for (int r = 0; r < t.n; r += 16) tma_load_2d(op + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
+                    } else if (ready) {
+                        load_tokens2(s, kt, srow, shared, t.n);
                     } else {
-                        const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared act array
-                        const CUtensorMap *hi = &maps.m[shared ? 9 : 7], *lo = &maps.m[shared ? 10 : 8];
-                        for (int r = 0; r < t.n; r += 16) {
-                            tma_load_2d(op + r * 128, hi, kt * 64, srow + r, &full_bar[s]);
-                            tma_load_2d(op + (t.n + r) * 128, lo, kt * 64, srow + r, &full_bar[s]);
-                        }
+                        pend_stage[pend_n] = s; pend_kt[pend_n] = kt; pend_row[pend_n] = srow;
+                        pend_shared[pend_n] = shared; pend_tn[pend_n] = t.n;
+                        ++pend_n;
                     }
+                    TCT(tp_issue += clock64() - c2;)
                 }
             }
+            if (alive && pend_n > 0) wait_ready();
+            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0;)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             unsigned it = 0, ui = 0;
             bool alive = true;
+            TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0; const long long tm0 = clock64();)
             for (int u = blockIdx.x; u < total && alive; u += P, ++ui) {
                 const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
                 const int buf = ui & 1;
+                TCT(long long c0 = clock64();)
                 if (!mbar_wait(&acc_empty[buf], ((ui >> 1) & 1u) ^ 1u)) {
                     atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     break;
                 }
+                TCT(tm_acc += clock64() - c0;)
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * pl.n1);
-                const uint32_t idesc = tc_idesc(t.n);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * pl.n1);
+                // phase 2: the hi and lo token tiles lie back to back, one MMA of N = 2n covers both;
+                // the epilogue adds the two halves
+                const uint32_t idesc = tc_idesc(t.phase == 1 ? t.n : 2 * t.n);
                 uint32_t acc = 0;
                 for (int kt = t.kt0; kt < t.kt1; ++kt, ++it) {
                     const int s = it % S;
+                    TCT(long long c1 = clock64();)
                     if (!mbar_wait(&full_bar[s], (it / S) & 1u)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
                     }
+                    TCT(long long c2 = clock64(); tm_full += c2 - c1;)
                     tc_fence_after();
                     const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint64_t ad = tc_smem_desc(stage);
                     const uint64_t bd = tc_smem_desc(stage + kTcWTile);
-                    const uint64_t ld = tc_smem_desc(stage + kTcWTile + t.n * 128);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {      // 4 x K=16 inside the 64-wide tile: +32 bytes each
                         tc_mma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, acc);
                         acc = 1;
-                        if (t.phase == 2) tc_mma_bf16(d_tmem, ad + 2 * k, ld + 2 * k, idesc, 1);
                     }
                     tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
+                    TCT(tm_mma += clock64() - c2;)
                 }
                 if (alive) tc_commit(&acc_full[buf]);
             }
+            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0;)
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;                        // TMEM lane quarter this warp may read
+        const int et = tid - 64;                       // 0..127 among the epilogue threads
         unsigned ui = 0;
         uint32_t ep_phase = 0;
         const int n_routed = p.B * sh.k;
         bool alive = true;
-        for (int u = blockIdx.x; u < total && alive; u += P, ++ui) {
-            const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
-            const StGroup &g = groups[t.a];
-            const int buf = ui & 1;
-            if (!mbar_wait(&acc_full[buf], (ui >> 1) & 1u)) {
-                if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
-                break;
-            }
-            tc_fence_after();
-            const int row = t.rb * 128 + q * 32 + lane;           // row of the matrix inside the expert
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * pl.n1);
-            if (t.phase == 1) {
-                const bool row_ok = row < g.f;
-                for (int c = 0; c < t.n; c += 8) {
-                    float v[8];
-                    tc_ld8(taddr + c, v);
+        TCT(long long te_wait = 0, te_red = 0, te_sync = 0, te_conv = 0; const long long te0 = clock64();)
+        int u = blockIdx.x;
+        for (int pass = 1; pass <= 2 && alive; ++pass) {
+            const int end = pass == 1 ? total1 : total;
+            for (; u < end && alive; u += P, ++ui) {
+                const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
+                const StGroup &g = groups[t.a];
+                const int buf = ui & 1;
+                TCT(long long c0 = clock64();)
+                if (!mbar_wait(&acc_full[buf], (ui >> 1) & 1u)) {
+                    if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                    alive = false;
+                    break;
+                }
+                TCT(long long c1 = clock64(); te_wait += c1 - c0;)
+                tc_fence_after();
+                const int row = t.rb * 128 + q * 32 + lane;           // row of the matrix inside the expert
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * pl.n1);
+                if (t.phase == 1) {
+                    const bool row_ok = row < g.f;
+                    // slot of the expert's i-th token = g.off + i; walk its tokens in ascending order
+                    float *dst = p.pre + 2 * act_offset(g.off, n_routed, sh.f, sh.f_sh) + (size_t)t.mat * g.f + row;
+                    const size_t slot_stride = 2 * (size_t)g.f;
+                    for (int c = 0; c < t.n; c += 16) {
+                        float v[16];
+                        tc_ld16(taddr + c, v);
+                        const unsigned m16 = (unsigned)((g.mask >> c) & 0xffffull);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int b = c + i;
-                        if (b < p.B && ((g.mask >> b) & 1ull) && row_ok) {
-                            const int slot = g.off + __popcll(g.mask & ((1ull << b) - 1ull));
-                            atomicAdd(&p.pre[2 * act_offset(slot, n_routed, sh.f, sh.f_sh) + (size_t)t.mat * g.f + row], v[i]);
+                        for (int i = 0; i < 16; ++i) {
+                            if (((m16 >> i) & 1u) && row_ok) {
+                                const int rank = __popcll(g.mask & ((1ull << (c + i)) - 1ull));
+                                atomicAdd(dst + rank * slot_stride, v[i]);
+                            }
+                        }
+                    }
+                } else {
+                    const bool row_ok = row < sh.d;
+                    for (int c = 0; c < t.n; c += 16) {
+                        float v[16], w[16];
+                        tc_ld16(taddr + c, v);
+                        tc_ld16(taddr + t.n + c, w);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int ti = c + i;
+                            if (ti < g.T && row_ok) {
+                                const int slot = g.off + ti;
+                                atomicAdd(&p.y[(size_t)s_slot_token[slot] * sh.d + row], s_slot_w[slot] * (v[i] + w[i]));
+                            }
                         }
                     }
                 }
-            } else {
-                const bool row_ok = row < sh.d;
-                for (int c = 0; c < t.n; c += 8) {
-                    float v[8];
-                    tc_ld8(taddr + c, v);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int ti = c + i;
-                        if (ti < g.T && row_ok) {
-                            const int slot = g.off + ti;
-                            atomicAdd(&p.y[(size_t)s_slot_token[slot] * sh.d + row], s_slot_w[slot] * v[i]);
-                        }
-                    }
-                }
+                // the accumulator may be overwritten
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                TCT(te_red += clock64() - c1;)
             }
-            // the accumulator may be overwritten
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (t.phase == 1) {
-                // count the unit; whoever completes the expert's phase 1 writes its activations
+            if (pass == 1 && alive) {
+                // ---- between the phases: grid-wide arrival, this CTA's slice of the activations, arrival
+                TCT(long long c2 = clock64();)
+                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
+                if (et == 0) {
+                    __threadfence();                     // the CTA's reductions, ordered by the barrier above
+                    atomicAdd(&ws.sync[kTcReady - 2], 1);
+                    bool ok = false;
+                    for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
+                        if (ld_acquire(&ws.sync[kTcReady - 2]) >= (int)gridDim.x) { ok = true; break; }
+                        __nanosleep(40);
+                    }
+                    if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+                    s_flag = ok;
+                }
+                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
+                if (!s_flag) { alive = false; break; }
                 __threadfence();
-                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                if (warp == 2 && lane == 0) {
-                    const int done = atomicAdd(&ws.sync[t.a], 1) + 1;
-                    s_flag = done == tc_units1(g.f, sh.d);
-                }
-                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                if (s_flag) {
-                    __threadfence();
-                    const int et = tid - 64;                      // 0..127
-                    for (int i = et; i < g.T * g.f; i += 128) {
-                        const int ti = i / g.f, j = i - ti * g.f;
-                        const size_t o = act_offset(g.off + ti, n_routed, sh.f, sh.f_sh);
-                        const float gv = __ldcg(&p.pre[2 * o + j]), uv = __ldcg(&p.pre[2 * o + g.f + j]);
-                        const float a = silu_mul(gv, uv);
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-                        p.act_hi[o + j] = hi;
-                        p.act_lo[o + j] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                TCT(long long c3 = clock64(); te_sync += c3 - c2;)
+                // activations are stored flat exactly like act_offset(slot) + j: convert a contiguous slice
+                const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
+                const long long lo_i = n_el * blockIdx.x / gridDim.x, hi_i = n_el * (blockIdx.x + 1) / gridDim.x;
+                const long long split = (long long)n_routed * sh.f;
+                for (long long i0 = lo_i + et; i0 < hi_i; i0 += 128 * 4) {
+                    float gv[4], uv[4];
+                    long long idx[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const long long i = i0 + (long long)r * 128;
+                        idx[r] = i;
+                        if (i < hi_i) {
+                            const int fg = i < split ? sh.f : sh.f_sh;
+                            const long long rel = i < split ? i : i - split;
+                            const long long j = rel % fg;
+                            const long long base = 2 * (i - j) + j;      // pre holds [gate f_g][up f_g] per slot
+                            gv[r] = __ldcg(&p.pre[base]);
+                            uv[r] = __ldcg(&p.pre[base + fg]);
+                        }
                     }
-                    __threadfence();
-                    fence_proxy_async();
-                    if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                    if (warp == 2 && lane == 0) atomicExch(&ws.sync[kTcReady + t.a], 1);
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        if (idx[r] < hi_i) {
+                            const float a = silu_mul(gv[r], uv[r]);
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(a);
+                            p.act_hi[idx[r]] = hi;
+                            p.act_lo[idx[r]] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                        }
+                    }
                 }
+                __threadfence();
+                fence_proxy_async();
+                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
+                if (et == 0) atomicAdd(&ws.sync[kTcReady - 1], 1);
+                TCT(te_conv += clock64() - c3;)
             }
         }
+        TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 16; o[0] = te_wait; o[1] = te_red; o[2] = te_sync; o[3] = te_conv; o[4] = clock64() - te0; })
     }
     // every path ends here (all waits above are bounded), so the TMEM is always returned
     tc_fence_before();
