@@ -36,12 +36,13 @@
 
 namespace s2moe {
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 224;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1
 constexpr int kTcMaxStages = 12;
 constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 KiB of weights
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
-constexpr int kTcMaxSmem = 232448 - 4096;
+constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
 constexpr unsigned kTcSpinLimit = 1u << 22;
+constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
 constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 2], [kTcReady - 1]: the two grid-wide counters
 
 struct TcPlan {
@@ -52,6 +53,7 @@ struct TcPlan {
     int n1;            // tokens padded to 16 (phase-1 N)
     int tmem_cols;     // power of two >= 32
     int tab_bytes;
+    int x_bytes;       // > 0: the hidden states stay resident in shared memory (all k-tiles)
     int smem_bytes;
 };
 
@@ -75,11 +77,15 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.stage_bytes = kTcWTile + 2 * p.n1 * 128;
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
     p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
-    p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
+    // hidden states resident (one token tile per k-tile) when at least 6 stages remain: every CTA
+    // needs every token tile in phase 1, and fetching them per stage makes a few L2 lines a hot spot
+    p.x_bytes = ((sh.d + 63) / 64) * p.n1 * 128;
+    if ((kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes < 6) p.x_bytes = 0;
+    p.stages = (kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes;
     if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
     p.tmem_cols = 32;
-    while (p.tmem_cols < 4 * p.n1) p.tmem_cols <<= 1;   // two accumulators of up to 2 * n1 columns
-    p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align the ring to 1024
+    while (p.tmem_cols < 8 * p.n1) p.tmem_cols <<= 1;   // 2 buffers x 2 issuers x up to 2 * n1 columns
+    p.smem_bytes = p.tab_bytes + p.x_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align to 1024
     p.feasible = p.stages >= 4 && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
                  sh.d % 64 == 0;
     return p;
@@ -97,6 +103,13 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -197,19 +210,21 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
     return t;
 }
 
-// tensor maps: 0 gate, 1 up, 2 down, 3 sh_gate, 4 sh_up, 5 sh_down, 6 hidden, 7/8 act hi/lo routed,
-// 9/10 act hi/lo shared
+// tensor maps: 0 gate, 1 up, 2 down, 3 sh_gate, 4 sh_up, 5 sh_down, 6 hidden, 7 activations of the
+// routed slots, 8 of the shared slots: 3-D {k, slot, hi|lo}, so that one copy of box {64, 16, 2}
+// lands the hi tile and, right behind it, the lo tile of 16 slots
 struct TcMaps {
-    CUtensorMap m[11];
+    CUtensorMap m[9];
 };
 
 __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar;
+    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar;
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
+    __shared__ TcUnit s_units[kTcMaxUnits];
 
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
@@ -222,8 +237,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     const int tab_rest = pl.tab_bytes - (int)sizeof(StGroup) * (G + 1);
     int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(StGroup) * (G + 1));
     float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
-    uint8_t *ring = tc_smem + pl.tab_bytes;
-    ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(ring) + 1023) & ~(uintptr_t)1023);
+    uint8_t *xres = tc_smem + pl.tab_bytes;
+    xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
+    uint8_t *ring = xres + pl.x_bytes;
 
     // group table; stage prefixes follow from the active list alone (routed groups first)
     const int U = ws.header[2];
@@ -250,16 +266,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     const int total1 = U * u1r + sh.n_sh * u1s, total2 = U * u2r + sh.n_sh * u2s;
     const int total = total1 + total2;
     const int S = pl.stages;
+    const int P = gridDim.x;
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
+            mbar_init(&empty_bar[s], 2);      // one commit from each MMA issuer
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_full[b], 2);
             mbar_init(&acc_empty[b], 4);
         }
         mbar_init(&ep_bar, 4);
+        mbar_init(&x_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -273,13 +291,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem;
-    const int P = gridDim.x;
+    // this CTA's units (u = blockIdx.x + i * P), decoded once by all threads: the single-thread
+    // roles below then read a unit with two shared-memory loads instead of dividing
+    const int n_units = total > (int)blockIdx.x ? (total - 1 - (int)blockIdx.x) / P + 1 : 0;
+    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x)
+        s_units[i] = tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
+    __syncthreads();
+    auto unit_at = [&](int i) -> TcUnit {
+        return i < kTcMaxUnits ? s_units[i] : tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             unsigned it = 0;
+#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
+            bool alive = true, ready = true;
+#else
             bool alive = true, ready = false;
+#endif
             // phase-2 stages whose weight tile is in flight but whose token tiles wait for the
             // activations (second grid-wide counter)
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
@@ -287,11 +317,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 uint8_t *op = ring + (size_t)s * pl.stage_bytes + kTcWTile;
-                const CUtensorMap *hi = &maps.m[shared ? 9 : 7], *lo = &maps.m[shared ? 10 : 8];
-                for (int r = 0; r < tn; r += 16) {
-                    tma_load_2d(op + r * 128, hi, kt * 64, srow + r, &full_bar[s]);
-                    tma_load_2d(op + (tn + r) * 128, lo, kt * 64, srow + r, &full_bar[s]);
-                }
+                const CUtensorMap *am = &maps.m[shared ? 8 : 7];
+                // one copy per 16 slots: their hi tile (2 KiB) and, right behind it, their lo tile
+                for (int r = 0; r < tn; r += 16) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
             auto wait_ready = [&]() -> bool {
                 TCT(long long c0 = clock64();)
@@ -309,8 +337,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 return true;
             };
             const int n_routed = p.B * sh.k;
-            for (int u = blockIdx.x; u < total && alive; u += P) {
-                const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
+            if (pl.x_bytes) {
+                // all token tiles of the hidden states, once
+                mbar_expect_tx(&x_bar, (uint32_t)pl.x_bytes);
+                for (int kt = 0; kt < (sh.d + 63) / 64; ++kt)
+                    for (int r = 0; r < pl.n1; r += 16)
+                        tma_load_2d(xres + ((size_t)kt * pl.n1 + r) * 128, &maps.m[6], kt * 64, r, &x_bar);
+            }
+            for (int i = 0; i < n_units && alive; ++i) {
+                const TcUnit t = unit_at(i);
                 const StGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
                 const int e = shared ? g.group - sh.E : g.group;
@@ -332,12 +367,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     }
                     TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
-                    const uint32_t op_bytes = (uint32_t)t.n * 128u * (t.phase == 1 ? 1u : 2u);
+                    const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 256u;
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
                     tma_load_2d(stage, wmap, kt * 64, row0, &full_bar[s]);
                     if (t.phase == 1) {
                         uint8_t *op = stage + kTcWTile;
-                        for (int r = 0; r < t.n; r += 16) tma_load_2d(op + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
+                        if (!pl.x_bytes)
+                            for (int r = 0; r < t.n; r += 16) tma_load_2d(op + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
                     } else if (ready) {
                         load_tokens2(s, kt, srow, shared, t.n);
                     } else {
@@ -351,14 +387,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             if (alive && pend_n > 0) wait_ready();
             TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0;)
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 6) {
+        // ------------------------------------------------------------------ MMA issuers
+        // Issuing one tcgen05.mma costs a thread on the order of 100 cycles whatever its shape, and
+        // with N = 16 every instruction covers only 4 KiB of weights, so two warps share the work:
+        // issuer h takes K-steps 2h and 2h + 1 of every k-tile and accumulates into its own TMEM
+        // columns; the epilogue adds the two partial accumulators.
+        const int half = warp == 1 ? 0 : 1;
         if (lane == 0) {
             unsigned it = 0, ui = 0;
             bool alive = true;
+            if (pl.x_bytes && !mbar_wait(&x_bar, 0)) {
+                atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                alive = false;
+            }
             TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0; const long long tm0 = clock64();)
-            for (int u = blockIdx.x; u < total && alive; u += P, ++ui) {
-                const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
+            for (; (int)ui < n_units && alive; ++ui) {
+                const TcUnit t = unit_at((int)ui);
                 const int buf = ui & 1;
                 TCT(long long c0 = clock64();)
                 if (!mbar_wait(&acc_empty[buf], ((ui >> 1) & 1u) ^ 1u)) {
@@ -367,7 +412,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 }
                 TCT(tm_acc += clock64() - c0;)
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * pl.n1);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 4 * pl.n1 + half * 2 * pl.n1);
                 // phase 2: the hi and lo token tiles lie back to back, one MMA of N = 2n covers both;
                 // the epilogue adds the two halves
                 const uint32_t idesc = tc_idesc(t.phase == 1 ? t.n : 2 * t.n);
@@ -384,18 +429,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     tc_fence_after();
                     const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint64_t ad = tc_smem_desc(stage);
-                    const uint64_t bd = tc_smem_desc(stage + kTcWTile);
+                    const uint64_t bd = (t.phase == 1 && pl.x_bytes) ? tc_smem_desc(xres + (size_t)kt * pl.n1 * 128)
+                                                                     : tc_smem_desc(stage + kTcWTile);
+#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {      // 4 x K=16 inside the 64-wide tile: +32 bytes each
+                    for (int k = 2 * half; k < 2 * half + 2; ++k) {   // K = 16 steps inside the 64-wide tile: +32 bytes each
                         tc_mma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, acc);
                         acc = 1;
                     }
+#else
+                    (void)ad; (void)bd; (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
+#endif
                     tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
                     TCT(tm_mma += clock64() - c2;)
                 }
                 if (alive) tc_commit(&acc_full[buf]);
             }
-            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0;)
+            TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; })
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -406,11 +456,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         const int n_routed = p.B * sh.k;
         bool alive = true;
         TCT(long long te_wait = 0, te_red = 0, te_sync = 0, te_conv = 0; const long long te0 = clock64();)
-        int u = blockIdx.x;
+        const int n_units1 = total1 > (int)blockIdx.x ? (total1 - 1 - (int)blockIdx.x) / P + 1 : 0;
         for (int pass = 1; pass <= 2 && alive; ++pass) {
-            const int end = pass == 1 ? total1 : total;
-            for (; u < end && alive; u += P, ++ui) {
-                const TcUnit t = tc_decode(groups, n_active, total1, u, sh.d, pl.n1);
+            const int end = pass == 1 ? n_units1 : n_units;
+            for (; (int)ui < end && alive; ++ui) {
+                const TcUnit t = unit_at((int)ui);
                 const StGroup &g = groups[t.a];
                 const int buf = ui & 1;
                 TCT(long long c0 = clock64();)
@@ -421,16 +471,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 }
                 TCT(long long c1 = clock64(); te_wait += c1 - c0;)
                 tc_fence_after();
+#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 2)
+                if (false)
+#endif
+                {
                 const int row = t.rb * 128 + q * 32 + lane;           // row of the matrix inside the expert
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * pl.n1);
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 4 * pl.n1);
+                const uint32_t other = (uint32_t)(2 * pl.n1);      // the second issuer's partial accumulator
                 if (t.phase == 1) {
                     const bool row_ok = row < g.f;
                     // slot of the expert's i-th token = g.off + i; walk its tokens in ascending order
                     float *dst = p.pre + 2 * act_offset(g.off, n_routed, sh.f, sh.f_sh) + (size_t)t.mat * g.f + row;
                     const size_t slot_stride = 2 * (size_t)g.f;
                     for (int c = 0; c < t.n; c += 16) {
-                        float v[16];
+                        float v[16], v2[16];
                         tc_ld16(taddr + c, v);
+                        tc_ld16(taddr + other + c, v2);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] += v2[i];
                         const unsigned m16 = (unsigned)((g.mask >> c) & 0xffffull);
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
@@ -443,9 +501,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 } else {
                     const bool row_ok = row < sh.d;
                     for (int c = 0; c < t.n; c += 16) {
-                        float v[16], w[16];
-                        tc_ld16(taddr + c, v);
-                        tc_ld16(taddr + t.n + c, w);
+                        float v[16], w[16];                       // columns: 16 hi, 16 lo, 16 hi, ...
+                        float v2[16], w2[16];
+                        tc_ld16(taddr + 2 * c, v);
+                        tc_ld16(taddr + 2 * c + 16, w);
+                        tc_ld16(taddr + other + 2 * c, v2);
+                        tc_ld16(taddr + other + 2 * c + 16, w2);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { v[i] += v2[i]; w[i] += w2[i]; }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const int ti = c + i;
@@ -456,15 +519,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                         }
                     }
                 }
+                }
                 // the accumulator may be overwritten
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 TCT(te_red += clock64() - c1;)
             }
+#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
+            if (false) {
+#else
             if (pass == 1 && alive) {
+#endif
                 // ---- between the phases: grid-wide arrival, this CTA's slice of the activations, arrival
                 TCT(long long c2 = clock64();)
+                TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 24; o[0] = c2 - te0; o[2] = ui; })
                 if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
                 if (et == 0) {
                     __threadfence();                     // the CTA's reductions, ordered by the barrier above
@@ -516,6 +585,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
                 if (et == 0) atomicAdd(&ws.sync[kTcReady - 1], 1);
                 TCT(te_conv += clock64() - c3;)
+                TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 24; o[1] = clock64() - te0; })
             }
         }
         TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 16; o[0] = te_wait; o[1] = te_red; o[2] = te_sync; o[3] = te_conv; o[4] = clock64() - te0; })

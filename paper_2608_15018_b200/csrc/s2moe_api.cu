@@ -234,6 +234,22 @@ bool make_map(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t
                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D bf16 tensor {cols, rows, 2}: the hi array and, `plane_bytes` further, the lo array of the
+// activations; box = 64 columns x 16 rows x both planes
+bool make_map_hilo(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                   uint64_t plane_bytes)
+{
+    if (!ctx->encode_tiled || !base || rows == 0) return false;
+    const cuuint64_t dims[3] = {cols, rows, 2};
+    const cuuint64_t strides[2] = {cols * 2, plane_bytes};
+    const cuuint32_t box[3] = {64, 16, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The plan a batch of B tokens runs with: the streaming kernel when it is allowed and its
 // shared-memory layout fits, else the CUDA-core kernels; 0 when plan 2 was demanded and does not fit.
 int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
@@ -273,12 +289,11 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
         TcMaps maps = ctx->tc_maps[layer];
         const size_t n_routed = (size_t)B * sh.k;
+        const uint64_t plane = (uint64_t)((const uint8_t *)ctx->act_lo - (const uint8_t *)ctx->act_hi);
         bool ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
-                  make_map(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, 16) &&
-                  make_map(ctx, &maps.m[8], ctx->act_lo, n_routed, (uint64_t)sh.f, 16);
+                  make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
         if (ok && sh.n_sh)
-            ok = make_map(ctx, &maps.m[9], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, 16) &&
-                 make_map(ctx, &maps.m[10], ctx->act_lo + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, 16);
+            ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
         if (!ok) return S2MOE_ECUDA;
         TcArgs a;
         a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
