@@ -9,11 +9,13 @@
 //   phase 2 unit: 128 rows of W_down of one expert x KT k-tiles of 64
 //                 D[row][slot] = W[rows, k-range] . a[slots, k-range]^T, a as bf16 hi + lo
 //                 -> y[token][row] += p * D                 (red.add, fp32)
-// Between the phases every CTA arrives on a grid-wide counter (bounded wait; one CTA per SM,
-// so all are resident), then each turns its slice of pre into a = silu(g) * u (bf16 hi + lo
-// parts) and arrives on a second counter, which the phase-2 token tiles wait for; the weight
-// tiles of the first phase-2 units are fetched meanwhile.  Units are dealt round-robin to one
-// persistent CTA per SM.
+// The experts are split into two waves.  When a CTA has finished its phase-1 units of a wave
+// it arrives on that wave's grid-wide counter and carries on (nobody waits there); a couple
+// of units later it waits (bounded) until all CTAs have arrived, turns its slice of the wave's
+// pre into a = silu(g) * u (bf16 hi + lo parts) and arrives on the wave's second counter, which
+// the phase-2 token tiles of that wave wait for.  So the hand-over between the projections
+// of one wave hides behind the other wave's work.  Units are dealt round-robin to one
+// persistent CTA per SM (all resident: one CTA per SM).
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = epilogue (TMEM -> registers -> red.add).  A ring of stages, each one weight
@@ -36,14 +38,14 @@
 
 namespace s2moe {
 
-constexpr int kTcThreads = 224;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1
+constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
 constexpr int kTcMaxStages = 12;
 constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 KiB of weights
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
 constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
 constexpr unsigned kTcSpinLimit = 1u << 22;
 constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
-constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 2], [kTcReady - 1]: the two grid-wide counters
+constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 8 + w], [kTcReady - 4 + w]: the two counters of wave w
 
 struct TcPlan {
     int feasible;
@@ -221,10 +223,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar;
+    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
+    __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
 
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
@@ -268,6 +271,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     const int S = pl.stages;
     const int P = gridDim.x;
     if (tid == 0) {
+        // wave 1 starts at the first group whose phase-1 units begin in the second half
+        int sp = n_active;
+        if (n_active >= 2) {
+            sp = 1;
+            while (sp < n_active - 1) {
+                const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
+                if (r * u1r + q * u1s >= total1 / 2) break;
+                ++sp;
+            }
+        }
+        s_split = sp;
+    }
+    if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 2);      // one commit from each MMA issuer
@@ -278,6 +294,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         }
         mbar_init(&ep_bar, 4);
         mbar_init(&x_bar, 1);
+        mbar_init(&cv_bar, 4);
+        mbar_init(&conv_go[0], 1);
+        mbar_init(&conv_go[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -297,6 +316,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x)
         s_units[i] = tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
     __syncthreads();
+    const int a_split = s_split;
+    const int W = a_split < n_active ? 2 : 1;
+    // first phase-1 / phase-2 unit of wave 1, and the segment of a global unit index:
+    // 0: phase 1 wave 0, 1: phase 1 wave 1, 2: phase 2 wave 0, 3: phase 2 wave 1, 4: past the end
+    const int split1 = W == 2 ? groups[a_split].p1 : total1;
+    const int split2 = W == 2 ? groups[a_split].p2 : total2;
+    auto seg_of_unit = [&](int i) -> int {
+        const long long u = (long long)blockIdx.x + (long long)i * P;
+        if (u >= total) return 4;
+        if (u < total1) return u < split1 ? 0 : 1;
+        return (u - total1) < split2 ? 2 : 3;
+    };
     auto unit_at = [&](int i) -> TcUnit {
         return i < kTcMaxUnits ? s_units[i] : tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
     };
@@ -305,13 +336,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             unsigned it = 0;
+            bool alive = true;
 #if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
-            bool alive = true, ready = true;
+            int ready_w = 2;                     // waves whose activations are known to be written
 #else
-            bool alive = true, ready = false;
+            int ready_w = 0;
 #endif
             // phase-2 stages whose weight tile is in flight but whose token tiles wait for the
             // activations (second grid-wide counter)
+            int pend_wave = 0;
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
                 pend_tn[kTcMaxStages];
             TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
@@ -321,11 +354,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 // one copy per 16 slots: their hi tile (2 KiB) and, right behind it, their lo tile
                 for (int r = 0; r < tn; r += 16) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
-            auto wait_ready = [&]() -> bool {
+            auto wait_ready = [&](int w) -> bool {
                 TCT(long long c0 = clock64();)
                 bool ok = false;
                 for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
-                    if (ld_acquire(&ws.sync[kTcReady - 1]) >= (int)gridDim.x) { ok = true; break; }
+                    if (ld_acquire(&ws.sync[kTcReady - 4 + w]) >= (int)gridDim.x) { ok = true; break; }
                     __nanosleep(40);
                 }
                 TCT(tp_ready += clock64() - c0;)
@@ -333,7 +366,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 fence_proxy_async();
                 for (int i = 0; i < pend_n; ++i) load_tokens2(pend_stage[i], pend_kt[i], pend_row[i], pend_shared[i], pend_tn[i]);
                 pend_n = 0;
-                ready = true;
+                ready_w = w + 1;
                 return true;
             };
             const int n_routed = p.B * sh.k;
@@ -353,11 +386,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
                 const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared activation array
-                if (t.phase == 2 && !ready && ld_acquire(&ws.sync[kTcReady - 1]) >= (int)gridDim.x) alive = wait_ready();
+                const int wv = t.a >= a_split ? 1 : 0;
+                bool ready = t.phase == 1 || wv < ready_w;
+                if (!ready) {
+                    // tiles still pending belong to an earlier wave only if that wave is not ready either
+                    if (pend_n > 0 && wv > ready_w) { if (!wait_ready(ready_w)) { alive = false; break; } }
+                    if (ld_acquire(&ws.sync[kTcReady - 4 + wv]) >= (int)gridDim.x) {
+                        alive = wait_ready(wv);
+                        ready = alive;
+                    }
+                }
                 for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it) {
                     const int s = it % S;
-                    if (t.phase == 2 && !ready && pend_n == S) {
-                        if (!wait_ready()) { alive = false; break; }     // every slot waits for tokens
+                    if (!ready && pend_n == S) {
+                        if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
+                        ready = true;
                     }
                     TCT(long long c1 = clock64();)
                     if (!mbar_wait(&empty_bar[s], ((it / S) & 1u) ^ 1u)) {
@@ -379,12 +422,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     } else {
                         pend_stage[pend_n] = s; pend_kt[pend_n] = kt; pend_row[pend_n] = srow;
                         pend_shared[pend_n] = shared; pend_tn[pend_n] = t.n;
+                        pend_wave = wv;
                         ++pend_n;
                     }
                     TCT(tp_issue += clock64() - c2;)
                 }
             }
-            if (alive && pend_n > 0) wait_ready();
+            if (alive && pend_n > 0) wait_ready(pend_wave);
             TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0;)
         }
     } else if (warp == 1 || warp == 6) {
@@ -447,6 +491,86 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             }
             TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; })
         }
+    } else if (warp >= 7) {
+        // ------------------------------------------------------------------ converter warps
+        // per wave: wait for this CTA's hand-over, arrive on the wave's grid-wide counter, wait
+        // (bounded) for all CTAs, convert this CTA's slice of the wave, arrive on the second counter
+        const int et = tid - 224;                      // 0..127 among the converter threads
+        const int n_routed = p.B * sh.k;
+        uint32_t ep_phase = 0;                         // running parity of cv_bar
+        uint64_t *ep_bar_p = &cv_bar;
+        const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
+        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
+        TCT(long long te_sync = 0, te_conv = 0;)
+        auto wave_convert = [&](int w) -> bool {
+            TCT(long long c2 = clock64();)
+            if (et == 0) {
+                bool ok = false;
+                for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
+                    if (ld_acquire(&ws.sync[kTcReady - 8 + w]) >= (int)gridDim.x) { ok = true; break; }
+                    __nanosleep(40);
+                }
+                if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+                s_flag = ok;
+            }
+            if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
+            if (!s_flag) return false;
+            __threadfence();
+            TCT(long long c3 = clock64(); te_sync += c3 - c2;)
+            // activations are stored flat exactly like act_offset(slot) + j: this CTA converts a
+            // contiguous slice of the wave's range
+            const long long w_lo = w == 0 ? 0 : el_split, w_hi = (w == 0 && W == 2) ? el_split : n_el;
+            const long long lo_i = w_lo + (w_hi - w_lo) * blockIdx.x / gridDim.x;
+            const long long hi_i = w_lo + (w_hi - w_lo) * (blockIdx.x + 1) / gridDim.x;
+            const long long split = (long long)n_routed * sh.f;
+            for (long long i0 = lo_i + et; i0 < hi_i; i0 += 128 * 4) {
+                float gv[4], uv[4];
+                long long idx[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const long long i = i0 + (long long)r * 128;
+                    idx[r] = i;
+                    if (i < hi_i) {
+                        const int fg = i < split ? sh.f : sh.f_sh;
+                        const long long rel = i < split ? i : i - split;
+                        const long long j = rel % fg;
+                        const long long base = 2 * (i - j) + j;      // pre holds [gate f_g][up f_g] per slot
+                        gv[r] = __ldcg(&p.pre[base]);
+                        uv[r] = __ldcg(&p.pre[base + fg]);
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (idx[r] < hi_i) {
+                        const float a = silu_mul(gv[r], uv[r]);
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(a);
+                        p.act_hi[idx[r]] = hi;
+                        p.act_lo[idx[r]] = __float2bfloat16_rn(a - __bfloat162float(hi));
+                    }
+                }
+            }
+            __threadfence();
+            fence_proxy_async();
+            if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
+            if (et == 0) atomicAdd(&ws.sync[kTcReady - 4 + w], 1);
+            TCT(te_conv += clock64() - c3;)
+            return true;
+        };
+
+#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 4)
+        for (int w = 0; w < W; ++w) {
+            // the hand-over may come late in the kernel: a long but bounded wait
+            bool ok = false;
+            for (unsigned i = 0; i < (1u << 22); ++i) {
+                if (mbar_try_wait(&conv_go[w], 0)) { ok = true; break; }
+                __nanosleep(64);
+            }
+            if (!ok) { if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
+            if (et == 0) atomicAdd(&ws.sync[kTcReady - 8 + w], 1);
+            if (!wave_convert(w)) break;
+        }
+#endif
+        TCT(if (et == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 28; o[0] = te_sync; o[1] = te_conv; })
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;                        // TMEM lane quarter this warp may read
@@ -456,10 +580,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         const int n_routed = p.B * sh.k;
         bool alive = true;
         TCT(long long te_wait = 0, te_red = 0, te_sync = 0, te_conv = 0; const long long te0 = clock64();)
-        const int n_units1 = total1 > (int)blockIdx.x ? (total1 - 1 - (int)blockIdx.x) / P + 1 : 0;
-        for (int pass = 1; pass <= 2 && alive; ++pass) {
-            const int end = pass == 1 ? n_units1 : n_units;
-            for (; (int)ui < end && alive; ++ui) {
+        // ---- hand-over between the projections, per wave (see the header comment)
+        const int n_routed_el = n_routed;   // (alias used below)
+        (void)n_routed_el;
+        const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
+        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
+        int next_arrive = 0;
+        auto wave_arrive = [&](int w) -> bool {
+            // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps
+            if (!tc_bar(&ep_bar, ep_phase, lane)) return false;
+            if (et == 0) {
+                __threadfence();                     // the CTA's reductions, ordered by the barrier above
+                mbar_arrive(&conv_go[w]);
+            }
+            return true;
+        };
+        // called before every unit (and once at the end): hand a wave over once this CTA's phase-1
+        // units of it are all done
+        auto service = [&](int upcoming_seg) -> bool {
+            const int seg_wave1 = W == 2 ? 1 : 2;        // first segment that lies after phase 1 of wave 0
+            while (next_arrive < W && upcoming_seg >= (next_arrive == 0 ? seg_wave1 : 2)) {
+                if (!wave_arrive(next_arrive)) return false;
+                ++next_arrive;
+            }
+            return true;
+        };
+#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
+        next_arrive = W;
+#endif
+        {
+            for (; (int)ui < n_units && alive; ++ui) {
+                if (!service(seg_of_unit((int)ui))) { alive = false; break; }
                 const TcUnit t = unit_at((int)ui);
                 const StGroup &g = groups[t.a];
                 const int buf = ui & 1;
@@ -526,67 +677,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 TCT(te_red += clock64() - c1;)
             }
-#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
-            if (false) {
-#else
-            if (pass == 1 && alive) {
-#endif
-                // ---- between the phases: grid-wide arrival, this CTA's slice of the activations, arrival
-                TCT(long long c2 = clock64();)
-                TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 24; o[0] = c2 - te0; o[2] = ui; })
-                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                if (et == 0) {
-                    __threadfence();                     // the CTA's reductions, ordered by the barrier above
-                    atomicAdd(&ws.sync[kTcReady - 2], 1);
-                    bool ok = false;
-                    for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
-                        if (ld_acquire(&ws.sync[kTcReady - 2]) >= (int)gridDim.x) { ok = true; break; }
-                        __nanosleep(40);
-                    }
-                    if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
-                    s_flag = ok;
-                }
-                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                if (!s_flag) { alive = false; break; }
-                __threadfence();
-                TCT(long long c3 = clock64(); te_sync += c3 - c2;)
-                // activations are stored flat exactly like act_offset(slot) + j: convert a contiguous slice
-                const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
-                const long long lo_i = n_el * blockIdx.x / gridDim.x, hi_i = n_el * (blockIdx.x + 1) / gridDim.x;
-                const long long split = (long long)n_routed * sh.f;
-                for (long long i0 = lo_i + et; i0 < hi_i; i0 += 128 * 4) {
-                    float gv[4], uv[4];
-                    long long idx[4];
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const long long i = i0 + (long long)r * 128;
-                        idx[r] = i;
-                        if (i < hi_i) {
-                            const int fg = i < split ? sh.f : sh.f_sh;
-                            const long long rel = i < split ? i : i - split;
-                            const long long j = rel % fg;
-                            const long long base = 2 * (i - j) + j;      // pre holds [gate f_g][up f_g] per slot
-                            gv[r] = __ldcg(&p.pre[base]);
-                            uv[r] = __ldcg(&p.pre[base + fg]);
-                        }
-                    }
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        if (idx[r] < hi_i) {
-                            const float a = silu_mul(gv[r], uv[r]);
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-                            p.act_hi[idx[r]] = hi;
-                            p.act_lo[idx[r]] = __float2bfloat16_rn(a - __bfloat162float(hi));
-                        }
-                    }
-                }
-                __threadfence();
-                fence_proxy_async();
-                if (!tc_bar(&ep_bar, ep_phase, lane)) { alive = false; break; }
-                if (et == 0) atomicAdd(&ws.sync[kTcReady - 1], 1);
-                TCT(te_conv += clock64() - c3;)
-                TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 24; o[1] = clock64() - te0; })
-            }
+            if (alive && !service(4)) alive = false;
         }
         TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 16; o[0] = te_wait; o[1] = te_red; o[2] = te_sync; o[3] = te_conv; o[4] = clock64() - te0; })
     }
