@@ -29,14 +29,12 @@ __device__ __forceinline__ double warp_max(double v)
 // order (value descending, id ascending): is a before b?
 __device__ __forceinline__ bool before1(double va, int a, double vb, int b)
 {
-    return va > vb || (va == vb && a < b);
+    return (va > vb) | ((va == vb) & (a < b));
 }
 // order (l' descending, l descending, id ascending)
 __device__ __forceinline__ bool before2(double l2a, double la, int a, double l2b, double lb, int b)
 {
-    if (l2a != l2b) return l2a > l2b;
-    if (la != lb) return la > lb;
-    return a < b;
+    return (l2a > l2b) | ((l2a == l2b) & ((la > lb) | ((la == lb) & (a < b))));
 }
 
 // Gating of one batch by one thread block (any block size that is a multiple of 32).
@@ -87,6 +85,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         for (int e = tid; e < E; e += nt) {
             int rank = 0;
             const double ge = s_g[e];
+#pragma unroll 8
             for (int o = 0; o < E; ++o) rank += before1(s_g[o], o, ge, e);
             s_star[e] = rank < cap;
         }
@@ -95,6 +94,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             const int b = i / E, e = i - b * E;
             const double le = s_l[i];
             int rank = 0;
+#pragma unroll 8
             for (int o = 0; o < E; ++o) rank += before1(s_l[b * E + o], o, le, e);
             if (rank == 0) s_top1[b] = le;
             if (rank == k) s_kth[b] = le;
@@ -112,6 +112,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         const double le = s_l[i];
         const double l2e = s_star[e] ? le + lam : le;
         int rank = 0;
+#pragma unroll 8
         for (int o = 0; o < E; ++o) {
             const double lo = s_l[b * E + o];
             const double l2o = s_star[o] ? lo + lam : lo;
@@ -166,6 +167,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     __syncthreads();
     for (int e = tid; e < E; e += nt) {
         int off = 0, pos = 0;
+#pragma unroll 8
         for (int o = 0; o < e; ++o) { off += s_cnt[o]; pos += s_cnt[o] > 0; }
         s_off[e] = off;
         s_pos[e] = pos;
