@@ -29,10 +29,16 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
 
+# DRAM bytes (read + write) per algorithmic byte, from the ncu captures summarised under profiles/
+# (ffn_tc_kernel_cfg2_2layers.md, ffn_stream_kernel_cfg2_2layers.md); traffic grows with the
+# number of distinct experts exactly as the algorithmic bytes do.
+TRAFFIC_RATIO = {"ffn_tc_kernel": 1.03, "ffn_stream_kernel": 1.005}
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="cfg2")
@@ -202,7 +208,7 @@ def run_own(args, wl, B, sigma):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident steps: stream launches through the C ABI, per-kernel events on
+    # ---- warm-up, launch count, clock sampler
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
             m.verify_stack(H, C, out, stream=stream)
@@ -211,45 +217,53 @@ def run_own(args, wl, B, sigma):
         m.verify_stack(H, C, out, stream=stream)
         stream.synchronize()
         launches_per_step = m.kernel_launches() - launches_before
-        sampler = ClockSampler(local)
-        sampler.start()
-        time.sleep(0.3)
-        barrier()
-        m.profile_begin(launches_per_step * args.steps)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0 = time.perf_counter()
-        e0.record(stream)
-        for _ in range(args.steps):
-            m.verify_stack(H, C, out, stream=stream)
-        e1.record(stream)
-        barrier()
-        t1 = time.perf_counter()
-        ms_total = e0.elapsed_time(e1)
-        kernels = m.profile_end()
-        clocks = sampler.stop(t0, t1)
-    status = m.device_status()
-    n_unique = out.n_unique.cpu().tolist()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    t_host0 = time.perf_counter()
 
-    # ---- CUDA-graph replay of the same stack (reported beside the stream-launch figure)
-    graph_ms = None
+    # ---- timed region A (the headline): K steps, each one replay of a CUDA graph that holds one
+    # s2moe_verify_stack call (every layer's kernels, nothing else); falls back to plain stream launches
+    graph_ms_total = None
+    timed_path = "stream launches of s2moe_verify_stack"
     try:
         with torch.cuda.stream(stream):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
                 m.verify_stack(H, C, out, stream=torch.cuda.current_stream())
-            for _ in range(3):
+            for _ in range(max(args.warmup, 3)):
                 g.replay()
-            stream.synchronize()
+            barrier()
             g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             g0.record(stream)
             for _ in range(args.steps):
                 g.replay()
             g1.record(stream)
-            stream.synchronize()
-            graph_ms = g0.elapsed_time(g1) / args.steps
+            barrier()
+            graph_ms_total = g0.elapsed_time(g1)
+            timed_path = "CUDA graph replay of one s2moe_verify_stack call per step"
     except Exception as exc:  # pragma: no cover
-        graph_ms = None
+        graph_ms_total = None
         print(f"graph replay skipped: {exc}", file=sys.stderr)
+
+    # ---- timed region B: the same K steps as plain stream launches with an event pair around every
+    # kernel (per-kernel durations for the roofline; the event pairs cost a few per cent)
+    with torch.cuda.stream(stream):
+        barrier()
+        m.profile_begin(launches_per_step * args.steps)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            m.verify_stack(H, C, out, stream=stream)
+        e1.record(stream)
+        barrier()
+        stream_ms_total = e0.elapsed_time(e1)
+        kernels = m.profile_end()
+    t_host1 = time.perf_counter()
+    clocks = sampler.stop(t_host0, t_host1)
+    status = m.device_status()
+    n_unique = out.n_unique.cpu().tolist()
+    ms_total = graph_ms_total if graph_ms_total is not None else stream_ms_total
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region
     hH, hC = H.cpu().pin_memory(), C.cpu().pin_memory()
@@ -270,7 +284,8 @@ def run_own(args, wl, B, sigma):
     d2h = ho.numel() * 4 + hs.numel() * 4 + hw.numel() * 4 + hu.numel() * 4
 
     # ---- max over ranks
-    ms_total, e2e_ms_total = replicas.max_over_ranks([ms_total, e2e_s * 1e3], device=dev)
+    ms_total, e2e_ms_total, stream_ms_total = replicas.max_over_ranks(
+        [ms_total, e2e_s * 1e3, stream_ms_total], device=dev)
     ms_step = ms_total / args.steps
     value = replicas.aggregate_tokens_per_s(world, B, L, ms_step)          # tokens/s per layer, all ranks
     e2e_value = replicas.aggregate_tokens_per_s(world, B, L, e2e_ms_total / args.steps)
@@ -291,7 +306,9 @@ def run_own(args, wl, B, sigma):
             bytes_per_launch = share * step_bytes / L / max(launches_per_layer, 1e-9)
             achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
             roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                    "traffic": TRAFFIC_RATIO[dom] * bytes_per_launch if dom in TRAFFIC_RATIO else None,
+                    "traffic_source": "ncu capture of a 2-layer case, scaled by algorithmic bytes",
                     "bytes_per_launch": bytes_per_launch, "us_per_launch": per_launch_ms * 1e3}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -309,7 +326,8 @@ def run_own(args, wl, B, sigma):
             "unique_expert_gbs": world * step_bytes / (ms_step * 1e-3) / 1e9,
             "unique_expert_frac_of_8tbs": step_bytes / (ms_step * 1e-3) / 8e12,
             "unique_expert_frac_of_measured": step_bytes / (ms_step * 1e-3) / (peak * 1e9),
-            "graph_ms_per_step": graph_ms,
+            "timed_path": timed_path,
+            "stream_ms_per_step_with_kernel_events": stream_ms_total / args.steps,
             "kernels": kernels,
             "roofline": roof,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
