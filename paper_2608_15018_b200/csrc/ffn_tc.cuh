@@ -107,6 +107,23 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
 }
+// Weight tiles are read once: mark their L2 lines evict-first, so that the stream does not push
+// out what is reused across layers (kernel code, bucketing arrays, activations).
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d_stream(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar,
+                                                   uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, uint64_t *bar)
 {
     asm volatile(
@@ -333,6 +350,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     };
 
     if (warp == 0) {
+        const uint64_t wpolicy = l2_evict_first_policy();
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             unsigned it = 0;
@@ -412,7 +430,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 256u;
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
-                    tma_load_2d(stage, wmap, kt * 64, row0, &full_bar[s]);
+                    tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
                     if (t.phase == 1) {
                         uint8_t *op = stage + kTcWTile;
                         if (!pl.x_bytes)

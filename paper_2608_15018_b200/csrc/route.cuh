@@ -26,15 +26,157 @@ __device__ __forceinline__ double warp_max(double v)
     return v;
 }
 
-// order (value descending, id ascending): is a before b?
-__device__ __forceinline__ bool before1(double va, int a, double vb, int b)
+// Monotone map from doubles (no NaN) to unsigned integers: a < b  <=>  dkey(a) < dkey(b), and
+// equal doubles (-0 included) have equal keys.  Keys of finite values are never 0.
+__device__ __forceinline__ unsigned long long dkey(double x)
 {
-    return (va > vb) | ((va == vb) & (a < b));
+    const long long b = __double_as_longlong(x + 0.0);
+    return (unsigned long long)(b ^ ((b >> 63) | (long long)0x8000000000000000ull));
 }
-// order (l' descending, l descending, id ascending)
-__device__ __forceinline__ bool before2(double l2a, double la, int a, double l2b, double lb, int b)
+__device__ __forceinline__ double dkey_value(unsigned long long k)
 {
-    return (l2a > l2b) | ((l2a == l2b) & ((la > lb) | ((la == lb) & (a < b))));
+    const long long b = (long long)k;
+    return __longlong_as_double(b < 0 ? (b ^ (long long)0x8000000000000000ull) : ~b);
+}
+// maximum of a 64-bit key over the warp: two 32-bit warp reductions
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k)
+{
+    const unsigned hi = (unsigned)(k >> 32);
+    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? (unsigned)k : 0u);
+    return ((unsigned long long)mh << 32) | ml;
+}
+
+#ifdef S2MOE_TIMING
+__device__ long long g_gt_marks[8];
+#define GT_MARK(i) do { if (tid == 0) g_gt_marks[i] = clock64(); } while (0)
+#else
+#define GT_MARK(i) do { } while (0)
+#endif
+
+// Per-token part of the gating, one warp per token: lane owns experts lane, lane + 32, ...
+// (J per lane, in registers).  lambda_b from the top-1 and (k+1)-th original logit, the k
+// experts of largest biased logit in the order (l' descending, l descending, id ascending),
+// softmax mixing weights.  Selection runs k (+ k + 1) rounds of a warp-wide maximum over
+// integer keys instead of ranking all E x E pairs.
+template <int J>
+__device__ __forceinline__ void gate_tokens(const Shape &sh, int B, bool bias_on, const double *s_l,
+                                            const unsigned char *s_star, int *s_sel, float *s_pw,
+                                            unsigned long long *s_mask, int32_t *__restrict__ sel_idx,
+                                            float *__restrict__ sel_w, int tid, int nt)
+{
+    const unsigned full = 0xffffffffu;
+    const int warp = tid >> 5, lane = tid & 31, nw = nt >> 5, E = sh.E, k = sh.k;
+    for (int b = warp; b < B; b += nw) {
+        GT_MARK(0);
+        double l[J];
+        unsigned long long k1[J];
+        unsigned valid = 0, star = 0;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int e = lane + 32 * j;
+            l[j] = 0.0;
+            k1[j] = 0ull;
+            if (e < E) {
+                l[j] = s_l[b * E + e] + 0.0;
+                k1[j] = dkey(l[j]);
+                valid |= 1u << j;
+                star |= (unsigned)s_star[e] << j;
+            }
+        }
+        GT_MARK(1);
+        // order statistics of the original logits: top-1 and (k+1)-th value (with multiplicity)
+        double lam = 0.0;
+        if (bias_on) {
+            unsigned alive = valid;
+            unsigned long long top1 = 0ull, m = 0ull;
+            for (int r = 0; r <= k; ++r) {
+                unsigned long long lm = 0ull;
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+                    if (((alive >> j) & 1u) && k1[j] > lm) lm = k1[j];
+                m = warp_max_key(lm);
+                if (r == 0) top1 = m;
+                const unsigned hb = __ballot_sync(full, alive != 0u && lm == m);
+                if (lane == __ffs(hb) - 1) {            // drop one instance of the maximum
+                    bool done = false;
+#pragma unroll
+                    for (int j = 0; j < J; ++j)
+                        if (!done && ((alive >> j) & 1u) && k1[j] == m) { alive &= ~(1u << j); done = true; }
+                }
+            }
+            lam = sh.alpha * (dkey_value(top1) - dkey_value(m));
+        }
+        GT_MARK(2);
+        unsigned long long k2[J];
+#pragma unroll
+        for (int j = 0; j < J; ++j) k2[j] = ((star >> j) & 1u) ? dkey(l[j] + lam) : k1[j];
+        // biased top-k, one winner per round
+        unsigned alive = valid;
+        int my_sel = 0;
+        for (int r = 0; r < k; ++r) {
+            unsigned long long b2 = 0ull, b1 = 0ull;
+            int bj = -1;
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                if ((alive >> j) & 1u) {
+                    const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
+                    if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
+                }
+            }
+            const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
+            const unsigned long long m2 = warp_max_key(b2);
+            bool hold = bj >= 0 && b2 == m2;
+            unsigned hb = __ballot_sync(full, hold);
+            if (__popc(hb) > 1) {                       // equal biased logits: larger original logit first
+                const unsigned long long m1 = warp_max_key(hold ? b1 : 0ull);
+                hold = hold && b1 == m1;
+                hb = __ballot_sync(full, hold);
+                if (__popc(hb) > 1) {                   // still equal: lower expert id first
+                    const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
+                    hold = hold && my_e == me;
+                    hb = __ballot_sync(full, hold);
+                }
+            }
+            const int wl = __ffs(hb) - 1;
+            const int we = (int)__shfl_sync(full, my_e, wl);
+            if (lane == wl) alive &= ~(1u << bj);
+            if (lane == r) my_sel = we;
+        }
+        GT_MARK(3);
+        // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
+        const double lamw = sh.weight_mode ? lam : 0.0;
+        double z[J];
+        unsigned long long zk = 0ull;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            z[j] = l[j] + (((star >> j) & 1u) ? lamw : 0.0);
+            if ((valid >> j) & 1u) { const unsigned long long q = dkey(z[j]); zk = q > zk ? q : zk; }
+        }
+        const double zmax = dkey_value(warp_max_key(zk));
+        double den = 0.0;
+#pragma unroll
+        for (int j = 0; j < J; ++j)
+            if ((valid >> j) & 1u) den += exp(z[j] - zmax);
+        den = warp_sum(den);
+        double p = 0.0;
+        if (lane < k) {
+            const double zs = s_l[b * E + my_sel] + (s_star[my_sel] ? lamw : 0.0);
+            p = exp(zs - zmax) / den;
+        }
+        if (sh.renorm) {
+            const double tot = warp_sum(p);
+            p /= tot;
+        }
+        if (lane < k) {
+            s_sel[b * k + lane] = my_sel;
+            s_pw[b * k + lane] = (float)p;
+            sel_idx[b * k + lane] = my_sel;
+            sel_w[b * k + lane] = (float)p;
+            atomicOr(&s_mask[my_sel], 1ull << b);
+        }
+        GT_MARK(4);
+    }
 }
 
 // Gating of one batch by one thread block (any block size that is a multiple of 32).
@@ -43,9 +185,10 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
                                              int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
                                              int32_t *__restrict__ n_unique, double *s_l)
 {
-    __shared__ double s_g[kMaxExperts];
+    __shared__ unsigned long long s_gk[kMaxExperts];
+    __shared__ int s_rank[kMaxExperts];
     __shared__ unsigned char s_star[kMaxExperts];
-    __shared__ double s_w[kMaxTokens], s_top1[kMaxTokens], s_kth[kMaxTokens], s_lam[kMaxTokens];
+    __shared__ double s_w[kMaxTokens];
     __shared__ int s_sel[kMaxTokens * kMaxTopK];
     __shared__ float s_pw[kMaxTokens * kMaxTopK];
     __shared__ unsigned long long s_mask[kMaxExperts];
@@ -65,11 +208,8 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     GATE_MARK();
 
     for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
-    for (int b = tid; b < B; b += nt) {
-        s_w[b] = conf ? (double)conf[b] : 1.0;
-        s_lam[b] = 0.0;
-    }
-    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
+    for (int b = tid; b < B; b += nt) s_w[b] = conf ? (double)conf[b] : 1.0;
+    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; s_rank[e] = 0; }
     __syncthreads();
 
     GATE_MARK();
@@ -78,108 +218,82 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         for (int e = tid; e < E; e += nt) {
             double g = 0.0;
             for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
-            s_g[e] = g;
+            s_gk[e] = dkey(g);
         }
         __syncthreads();
-        // TopCap by rank
-        for (int e = tid; e < E; e += nt) {
+        // TopCap by rank in the order (g descending, id ascending); P threads share an expert
+        int P = 1;
+        while (P < 8 && E * (P * 2) <= nt) P *= 2;
+        for (int i = tid; i < E * P; i += nt) {
+            const int e = i / P, part = i - e * P;
+            const unsigned long long ge = s_gk[e];
             int rank = 0;
-            const double ge = s_g[e];
-#pragma unroll 8
-            for (int o = 0; o < E; ++o) rank += before1(s_g[o], o, ge, e);
-            s_star[e] = rank < cap;
-        }
-        // order statistics of the original logits: top-1 and (k+1)-th
-        for (int i = tid; i < B * E; i += nt) {
-            const int b = i / E, e = i - b * E;
-            const double le = s_l[i];
-            int rank = 0;
-#pragma unroll 8
-            for (int o = 0; o < E; ++o) rank += before1(s_l[b * E + o], o, le, e);
-            if (rank == 0) s_top1[b] = le;
-            if (rank == k) s_kth[b] = le;
+            for (int o = part; o < E; o += P) {
+                const unsigned long long go = s_gk[o];
+                rank += (go > ge) | ((go == ge) & (o < e));
+            }
+            if (rank) atomicAdd(&s_rank[e], rank);
         }
         __syncthreads();
-        for (int b = tid; b < B; b += nt) s_lam[b] = sh.alpha * (s_top1[b] - s_kth[b]);
+        for (int e = tid; e < E; e += nt) s_star[e] = s_rank[e] < cap;
         __syncthreads();
     }
 
     GATE_MARK();
-    // biased top-k by rank
-    for (int i = tid; i < B * E; i += nt) {
-        const int b = i / E, e = i - b * E;
-        const double lam = s_lam[b];
-        const double le = s_l[i];
-        const double l2e = s_star[e] ? le + lam : le;
-        int rank = 0;
-#pragma unroll 8
-        for (int o = 0; o < E; ++o) {
-            const double lo = s_l[b * E + o];
-            const double l2o = s_star[o] ? lo + lam : lo;
-            rank += before2(l2o, lo, o, l2e, le, e);
-        }
-        if (rank < k) s_sel[b * k + rank] = e;
-    }
+    if (E <= 64) gate_tokens<2>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
+    else if (E <= 128) gate_tokens<4>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
+    else gate_tokens<8>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
     __syncthreads();
 
     GATE_MARK();
-    // mixing weights: one warp per token
-    {
-        const int warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
-        for (int b = warp; b < B; b += nw) {
-            const double lam = sh.weight_mode ? s_lam[b] : 0.0;
-            double zmax = -1.0e300;
-            for (int e = lane; e < E; e += 32) {
-                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
-                zmax = fmax(zmax, z);
-            }
-            zmax = warp_max(zmax);
-            double den = 0.0;
-            for (int e = lane; e < E; e += 32) {
-                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
-                den += exp(z - zmax);
-            }
-            den = warp_sum(den);
-            double p = 0.0;
-            int e = 0;
-            if (lane < k) {
-                e = s_sel[b * k + lane];
-                const double z = s_l[b * E + e] + (s_star[e] ? lam : 0.0);
-                p = exp(z - zmax) / den;
-            }
-            if (sh.renorm) {
-                const double tot = warp_sum(p);
-                p /= tot;
-            }
-            if (lane < k) {
-                s_pw[b * k + lane] = (float)p;
-                sel_idx[b * k + lane] = e;
-                sel_w[b * k + lane] = (float)p;
-                atomicOr(&s_mask[e], 1ull << b);
+    // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts
+#ifdef S2MOE_TIMING
+#pragma unroll 1
+    for (int rep = 0; rep < 2; ++rep) {
+    if (rep == 1) GATE_MARK();
+#endif
+    if (tid < 32) {
+        const int C = (E + 31) >> 5, e0 = tid * C;
+        int sum = 0, act = 0;
+        for (int i = 0; i < C; ++i) {
+            const int e = e0 + i;
+            if (e < E) {
+                const int c = __popcll(s_mask[e]);
+                s_cnt[e] = c;
+                sum += c;
+                act += c > 0;
             }
         }
+        int xs = sum, xa = act;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, xs, o), u = __shfl_up_sync(0xffffffffu, xa, o);
+            if (tid >= o) { xs += t; xa += u; }
+        }
+        int off = xs - sum, pos = xa - act;
+        for (int i = 0; i < C; ++i) {
+            const int e = e0 + i;
+            if (e < E) {
+                s_off[e] = off;
+                s_pos[e] = pos;
+                off += s_cnt[e];
+                pos += s_cnt[e] > 0;
+            }
+        }
+        if (tid == 31) { s_off[E] = xs; s_U = xa; }
     }
+#ifdef S2MOE_TIMING
+    }
+#endif
     __syncthreads();
-
     GATE_MARK();
-    // union, unique count, exclusive scan, list of active experts
-    for (int e = tid; e < E; e += nt) s_cnt[e] = __popcll(s_mask[e]);
-    __syncthreads();
-    for (int e = tid; e < E; e += nt) {
-        int off = 0, pos = 0;
-#pragma unroll 8
-        for (int o = 0; o < e; ++o) { off += s_cnt[o]; pos += s_cnt[o] > 0; }
-        s_off[e] = off;
-        s_pos[e] = pos;
-        if (e == E - 1) { s_off[E] = off + s_cnt[e]; s_U = pos + (s_cnt[e] > 0); }
-    }
-    __syncthreads();
     const int U = s_U, n_routed = B * k;
     for (int e = tid; e < E; e += nt) {
         ws.counts[e] = s_cnt[e];
         ws.offsets[e] = s_off[e];
         if (s_cnt[e] > 0) ws.active[s_pos[e]] = e;
     }
+    GATE_MARK();
     // bucket the (token, choice) pairs: tokens ascending inside an expert
     for (int i = tid; i < n_routed; i += nt) {
         const int b = i / k;
@@ -188,6 +302,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         ws.slot_token[pos] = b;
         ws.slot_w[pos] = s_pw[i];
     }
+    GATE_MARK();
     // shared experts: every token, weight c_b
     for (int i = tid; i < sh.n_sh * B; i += nt) {
         const int s = i / B, b = i - s * B;
@@ -239,6 +354,9 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         }
     }
     GATE_MARK();
+#ifdef S2MOE_TIMING
+    if (tid == 0) for (int i = 0; i < 5; ++i) tm[20 + i] = g_gt_marks[i];
+#endif
     if (tid == 0) {
         ws.offsets[E + sh.n_sh] = n_routed + sh.n_sh * B;
         ws.header[0] = U + sh.n_sh;
@@ -263,7 +381,54 @@ __device__ __forceinline__ void load4_plain(const void *row, int c, float (&v)[4
 }
 
 constexpr int kRouteThreads = 512;
-constexpr int kRouteTok = 16;   // tokens accumulated per pass
+constexpr int kRouteTok = 16;   // most tokens accumulated per pass
+
+// Buffers that the layer's later kernels accumulate into and that must start at zero; the
+// routing blocks clear them (16-byte units) so that no separate fill precedes the layer.
+struct ZeroList {
+    void *ptr[3];
+    unsigned long long n16[3];
+};
+
+// One pass of a router row over NT tokens b0 .. b0 + NT - 1 (indices past B - 1 repeat token
+// B - 1, so that every load is unconditional and issued before the first use).
+template <int ACT, int RT, int NT>
+__device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const Workspace &ws, const uint8_t *wrow,
+                                           const void *__restrict__ hidden, double *s_part)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, d = sh.d, row = blockIdx.x;
+    const size_t ab = ACT == DT_F32 ? 4 : 2;
+    double acc[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) acc[t] = 0.0;
+    for (int c = tid * 4; c < d; c += kRouteThreads * 4) {
+        float w[4], x[NT][4];
+        load4_plain<RT>(wrow, c, w);
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const int bt = min(b0 + t, B - 1);
+            load4_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)bt * d * ab, c, x[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[t][i], acc[t]);
+    }
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+        const double s = warp_sum(acc[t]);
+        if (lane == 0) s_part[warp * kRouteTok + t] = s;
+    }
+    __syncthreads();
+    if (tid < NT && b0 + tid < B) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kRouteThreads / 32; ++w) s += s_part[w * kRouteTok + tid];
+        if (row < sh.E) ws.logits[(size_t)(b0 + tid) * sh.E + row] = s;
+        else ws.gate_logit[b0 + tid] = s;
+    }
+    __syncthreads();
+}
 
 // Router logits and gating in one launch.  Block r computes row r of the router (row E is the
 // shared-expert gate vector) against all B tokens in float64; the block that finishes last
@@ -273,50 +438,30 @@ template <int ACT, int RT>
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
              const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
-             float *__restrict__ sel_w, int32_t *__restrict__ n_unique)
+             float *__restrict__ sel_w, int32_t *__restrict__ n_unique, ZeroList zl)
 {
     extern __shared__ double s_dyn[];
     __shared__ int s_last;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x;
 #ifdef S2MOE_TIMING
     const long long t_start = clock64();
 #endif
+#pragma unroll
+    for (int z = 0; z < 3; ++z) {
+        uint4 *p = reinterpret_cast<uint4 *>(zl.ptr[z]);
+        for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.n16[z];
+             i += (unsigned long long)gridDim.x * kRouteThreads)
+            p[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
     const int row = blockIdx.x, d = sh.d;
-    const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
+    const size_t rb = RT == DT_F32 ? 4 : 2;
     const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
                                      : reinterpret_cast<const uint8_t *>(sh_scale);
-    for (int b0 = 0; b0 < B; b0 += kRouteTok) {
-        double acc[kRouteTok];
-#pragma unroll
-        for (int t = 0; t < kRouteTok; ++t) acc[t] = 0.0;
-        for (int c = tid * 4; c < d; c += kRouteThreads * 4) {
-            float w[4];
-            load4_plain<RT>(wrow, c, w);
-#pragma unroll
-            for (int t = 0; t < kRouteTok; ++t) {
-                if (b0 + t < B) {
-                    float x[4];
-                    load4_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)(b0 + t) * d * ab, c, x);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[i], acc[t]);
-                }
-            }
-        }
-#pragma unroll
-        for (int t = 0; t < kRouteTok; ++t) {
-            if (b0 + t < B) {           // uniform across the block
-                const double s = warp_sum(acc[t]);
-                if (lane == 0) s_dyn[warp * kRouteTok + t] = s;
-            }
-        }
-        __syncthreads();
-        if (tid < kRouteTok && b0 + tid < B) {
-            double s = 0.0;
-            for (int w = 0; w < kRouteThreads / 32; ++w) s += s_dyn[w * kRouteTok + tid];
-            if (row < sh.E) ws.logits[(size_t)(b0 + tid) * sh.E + row] = s;
-            else ws.gate_logit[b0 + tid] = s;
-        }
-        __syncthreads();
+    for (int b0 = 0; b0 < B;) {
+        const int left = B - b0;
+        if (left > 8) { route_pass<ACT, RT, 16>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 16; }
+        else if (left > 4) { route_pass<ACT, RT, 8>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 8; }
+        else { route_pass<ACT, RT, 4>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 4; }
     }
     // the block that arrives last sees every row (release by fence + ticket, acquire by fence)
     __threadfence();

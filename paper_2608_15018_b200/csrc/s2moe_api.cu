@@ -146,22 +146,22 @@ size_t route_smem(int B, int E)
 
 template <int ACT, int RT>
 void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
-                    int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
+                    int32_t *sel_idx, float *sel_w, int32_t *n_unique, const ZeroList &zl, cudaStream_t st)
 {
     const int rows = sh.E + (lp.sh_scale ? 1 : 0);
     LaunchScope scope(ctx, KC_ROUTER, st);
     route_kernel<ACT, RT><<<rows, kRouteThreads, route_smem(B, sh.E), st>>>(sh, B, ctx->ws, hidden, lp.router, lp.sh_scale,
-                                                                            conf, sel_idx, sel_w, n_unique);
+                                                                            conf, sel_idx, sel_w, n_unique, zl);
 }
 
 void launch_route(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
-                  int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
+                  int32_t *sel_idx, float *sel_w, int32_t *n_unique, const ZeroList &zl, cudaStream_t st)
 {
     const bool af = sh.act_dtype == DT_F32, rf = sh.router_dtype == DT_F32;
-    if (af && rf) launch_route_t<DT_F32, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
-    else if (af) launch_route_t<DT_F32, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
-    else if (rf) launch_route_t<DT_BF16, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
-    else launch_route_t<DT_BF16, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+    if (af && rf) launch_route_t<DT_F32, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
+    else if (af) launch_route_t<DT_F32, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
+    else if (rf) launch_route_t<DT_BF16, DT_F32>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
+    else launch_route_t<DT_BF16, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
 }
 
 cudaError_t prepare_route()
@@ -278,13 +278,18 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     if (plan == 0) return S2MOE_EINVAL;
     sh.plan = plan;
     sh.op_cap = pl.op_cap;
-    CU(ctx, cudaMemsetAsync(out, 0, (size_t)B * sh.d * sizeof(float), st));
+    // what the FFN kernels accumulate into is cleared by the routing kernel's blocks
+    ZeroList zl{};
+    zl.ptr[0] = out;
+    zl.n16[0] = (size_t)B * sh.d * sizeof(float) / 16;
     if (plan == 3) {
         const size_t used = (size_t)B * sh.k * sh.f + (size_t)sh.n_sh * B * sh.f_sh;
-        CU(ctx, cudaMemsetAsync(ctx->pre, 0, used * 2 * sizeof(float), st));
-        CU(ctx, cudaMemsetAsync(ctx->ws.sync, 0, 4 * (size_t)(kTcReady + kStMaxGroups), st));
+        zl.ptr[1] = ctx->pre;
+        zl.n16[1] = used * 2 * sizeof(float) / 16;
+        zl.ptr[2] = ctx->ws.sync + (kTcReady - 8);      // the hand-over counters of the two waves
+        zl.n16[2] = 8 * sizeof(int32_t) / 16;
     }
-    launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, st);
+    launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
     if (plan == 3) {
         const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
         TcMaps maps = ctx->tc_maps[layer];
@@ -695,16 +700,16 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
     const bool af = sh.act_dtype == DT_F32, rf = sh.router_dtype == DT_F32;
     if (af && rf)
         route_kernel<DT_F32, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                        sel_idx, sel_w, n_unique);
+                                                                        sel_idx, sel_w, n_unique, ZeroList{});
     else if (af)
         route_kernel<DT_F32, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                         sel_idx, sel_w, n_unique);
+                                                                         sel_idx, sel_w, n_unique, ZeroList{});
     else if (rf)
         route_kernel<DT_BF16, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                         sel_idx, sel_w, n_unique);
+                                                                         sel_idx, sel_w, n_unique, ZeroList{});
     else
         route_kernel<DT_BF16, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                          sel_idx, sel_w, n_unique);
+                                                                          sel_idx, sel_w, n_unique, ZeroList{});
     if (gate_vec && gate_out) noalloc_gate_out_kernel<<<1, 64, 0, st>>>(ws.gate_logit, gate_out, n_tokens);
     return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
 }
