@@ -5,23 +5,24 @@
 // Both projections are cut into split-K tiles ("units") of equal cost:
 //   phase 1 unit: 128 rows of W_gate or W_up of one expert x KT k-tiles of 64
 //                 D[row][token] = W[rows, k-range] . h[tokens, k-range]^T       (all B tokens)
-//                 -> red.add into pre[slot][gate|up][row]   (only the expert's tokens)
+//                 -> red.add into pre[gate|up][slot][row]   (only the expert's tokens)
 //   phase 2 unit: 128 rows of W_down of one expert x KT k-tiles of 64
 //                 D[row][slot] = W[rows, k-range] . a[slots, k-range]^T, a as bf16 hi + lo
 //                 -> y[token][row] += p * D                 (red.add, fp32)
 // The experts are split into two waves.  When a CTA has finished its phase-1 units of a wave
-// it arrives on that wave's grid-wide counter and carries on (nobody waits there); a couple
-// of units later it waits (bounded) until all CTAs have arrived, turns its slice of the wave's
-// pre into a = silu(g) * u (bf16 hi + lo parts) and arrives on the wave's second counter, which
+// its epilogue hands the wave over to the CTA's converter warps, which arrive on the wave's
+// grid-wide counter, wait (bounded) until all CTAs have arrived, turn their slice of the wave's
+// pre into a = silu(g) * u (bf16 hi + lo parts) and arrive on the wave's second counter, which
 // the phase-2 token tiles of that wave wait for.  So the hand-over between the projections
-// of one wave hides behind the other wave's work.  Units are dealt round-robin to one
-// persistent CTA per SM (all resident: one CTA per SM).
+// of one wave hides behind the other wave's work.  One persistent CTA per SM; of each of the
+// four segments (phase 1 / 2 of wave 0 / 1) a CTA takes one contiguous run of units, so that
+// consecutive k-pieces of a row block accumulate in TMEM and are reduced to memory once.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (TMEM -> registers -> red.add).  A ring of stages, each one weight
-// k-tile (128 x 64 bf16 = 16 KiB) plus the matching token k-tile(s); accumulators are
-// double-buffered in TMEM.  tcgen05.mma: M = 128 weight rows, N = tokens padded to 16,
-// K = 16 per instruction, fp32 accumulate.
+// Warp roles (352 threads): warp 0 = TMA producer; warps 1 and 6 = MMA issuers (warp 1 owns the
+// TMEM allocation); warps 2..5 = epilogue (TMEM -> registers -> red.add); warps 7..10 =
+// converters.  A ring of stages, each one weight k-tile (128 x 64 bf16 = 16 KiB) plus, in phase
+// 2, the matching token k-tiles; accumulators are double-buffered in TMEM.  tcgen05.mma:
+// M = 128 weight rows, N = tokens padded to 16, K = 16 per instruction, fp32 accumulate.
 #pragma once
 
 #include <cuda.h>
@@ -32,8 +33,10 @@
 // cycle-counter statements, compiled only with -DS2MOE_TIMING
 #ifdef S2MOE_TIMING
 #define TCT(...) __VA_ARGS__
+#define TCG(slot) do { unsigned long long g_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_)); (reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32)[slot] = (long long)g_; } while (0)
 #else
 #define TCT(...)
+#define TCG(slot) do { } while (0)
 #endif
 
 namespace s2moe {
@@ -45,6 +48,11 @@ constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in 
 constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
 constexpr unsigned kTcSpinLimit = 1u << 22;
 constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
+#ifndef S2MOE_SPLIT_NUM
+#define S2MOE_SPLIT_NUM 1
+#define S2MOE_SPLIT_DEN 2
+#endif
+constexpr int kTcSplitNum = S2MOE_SPLIT_NUM, kTcSplitDen = S2MOE_SPLIT_DEN;   // share of the experts in wave 0
 constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 8 + w], [kTcReady - 4 + w]: the two counters of wave w
 
 struct TcPlan {
@@ -64,7 +72,7 @@ struct TcArgs {
     Workspace ws;
     TcPlan plan;
     float *y;
-    float *pre;                       // [slot][2][f_g] fp32 pre-activations (zeroed before the launch)
+    float *pre;                       // [gate|up][slot][f_g] fp32 pre-activations (zeroed by the routing kernel)
     __nv_bfloat16 *act_hi, *act_lo;   // [slot][f_g]
     int B;
 };
@@ -79,10 +87,12 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.stage_bytes = kTcWTile + 2 * p.n1 * 128;
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
     p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
-    // hidden states resident (one token tile per k-tile) when at least 6 stages remain: every CTA
-    // needs every token tile in phase 1, and fetching them per stage makes a few L2 lines a hot spot
+    // The ring is what keeps HBM busy (bytes in flight = stages x 16 KiB per SM, against a loaded
+    // latency of 2-3 us), so shared memory goes to stages first: the hidden-state tiles stay
+    // resident only if the ring reaches its maximum depth anyway, otherwise every stage fetches
+    // its token k-tile (2 KiB per 16 tokens, an L2 hit) next to the weight k-tile.
     p.x_bytes = ((sh.d + 63) / 64) * p.n1 * 128;
-    if ((kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes < 6) p.x_bytes = 0;
+    if ((kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes < kTcMaxStages) p.x_bytes = 0;
     p.stages = (kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes;
     if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
     p.tmem_cols = 32;
@@ -194,9 +204,17 @@ __device__ __forceinline__ bool tc_bar(uint64_t *bar, uint32_t &phase, int lane)
     return ok;
 }
 
+// next slot of the ring; the parity flips on wrap-around
+__device__ __forceinline__ void tc_ring_next(int &s, uint32_t &parity, int S)
+{
+    if (++s == S) { s = 0; parity ^= 1u; }
+}
+
 struct TcUnit {
     int phase, a, mat, rb, kt0, kt1;   // group slot, matrix (0 gate, 1 up, 2 down), row block, k-tile range
     int n;                             // MMA N (tokens padded to 16)
+    int seg;                           // 0 / 1: phase 1 of wave 0 / 1, 2 / 3: phase 2 of wave 0 / 1
+    int first, last;                   // first / last unit of an accumulation run (see the kernel)
 };
 
 __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active, int total1, int u, int d, int n1)
@@ -245,11 +263,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
     __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
+    __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
 
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
     const TcPlan &pl = p.plan;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    TCT(const long long t_entry = clock64(); unsigned long long g_entry; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_entry));)
     const int n_active = ws.header[0], n_slots = ws.header[1];
     const int G = sh.E + sh.n_sh;
 
@@ -294,11 +314,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             sp = 1;
             while (sp < n_active - 1) {
                 const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
-                if (r * u1r + q * u1s >= total1 / 2) break;
+                if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)total1 * kTcSplitNum) break;
                 ++sp;
             }
         }
         s_split = sp;
+        s_ready[0] = 0;
+        s_ready[1] = 0;
     }
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -311,7 +333,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         }
         mbar_init(&ep_bar, 4);
         mbar_init(&x_bar, 1);
-        mbar_init(&cv_bar, 4);
+        mbar_init(&cv_bar, 3);
         mbar_init(&conv_go[0], 1);
         mbar_init(&conv_go[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -327,28 +349,52 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem;
-    // this CTA's units (u = blockIdx.x + i * P), decoded once by all threads: the single-thread
-    // roles below then read a unit with two shared-memory loads instead of dividing
-    const int n_units = total > (int)blockIdx.x ? (total - 1 - (int)blockIdx.x) / P + 1 : 0;
-    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x)
-        s_units[i] = tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
-    __syncthreads();
     const int a_split = s_split;
     const int W = a_split < n_active ? 2 : 1;
-    // first phase-1 / phase-2 unit of wave 1, and the segment of a global unit index:
-    // 0: phase 1 wave 0, 1: phase 1 wave 1, 2: phase 2 wave 0, 3: phase 2 wave 1, 4: past the end
+    // Four segments in time order: phase 1 of wave 0, of wave 1, phase 2 of wave 0, of wave 1.
+    // Every CTA takes one contiguous run of units of each segment (sizes differ by at most one;
+    // the CTAs that get the extra unit rotate from segment to segment, so the totals differ by at
+    // most one as well).  Contiguous units are consecutive k-pieces of one 128-row block, so a CTA
+    // accumulates them in one TMEM accumulator and the epilogue runs once per run of k-pieces
+    // instead of once per unit; only row blocks cut by a CTA boundary are reduced from two CTAs.
     const int split1 = W == 2 ? groups[a_split].p1 : total1;
     const int split2 = W == 2 ? groups[a_split].p2 : total2;
-    auto seg_of_unit = [&](int i) -> int {
-        const long long u = (long long)blockIdx.x + (long long)i * P;
-        if (u >= total) return 4;
-        if (u < total1) return u < split1 ? 0 : 1;
-        return (u - total1) < split2 ? 2 : 3;
+    int my_start0, my_start1, my_start2, my_start3, my_cnt0, my_cnt1, my_cnt2, my_cnt3;
+    {
+        int rot = 0;
+        auto share = [&](int begin, int n, int &start, int &cnt) {
+            const int q = n / P, r = n - q * P;
+            const int c = ((int)blockIdx.x + P - rot) % P;
+            cnt = q + (c < r ? 1 : 0);
+            start = begin + c * q + min(c, r);
+            rot = (rot + r) % P;
+        };
+        share(0, split1, my_start0, my_cnt0);
+        share(split1, total1 - split1, my_start1, my_cnt1);
+        share(total1, split2, my_start2, my_cnt2);
+        share(total1 + split2, total2 - split2, my_start3, my_cnt3);
+    }
+    const int n_units = my_cnt0 + my_cnt1 + my_cnt2 + my_cnt3;
+    auto unit_make = [&](int i) -> TcUnit {
+        int seg = 0, j = i, start = my_start0, cnt = my_cnt0;
+        if (j >= cnt) { j -= cnt; seg = 1; start = my_start1; cnt = my_cnt1; }
+        if (seg == 1 && j >= cnt) { j -= cnt; seg = 2; start = my_start2; cnt = my_cnt2; }
+        if (seg == 2 && j >= cnt) { j -= cnt; seg = 3; start = my_start3; cnt = my_cnt3; }
+        TcUnit t = tc_decode(groups, n_active, total1, start + j, sh.d, pl.n1);
+        const int K = t.phase == 1 ? sh.d : groups[t.a].f;
+        t.seg = seg;
+        t.first = (j == 0 || t.kt0 == 0) ? 1 : 0;
+        t.last = (j == cnt - 1 || t.kt1 == (K + 63) / 64) ? 1 : 0;
+        return t;
     };
-    auto unit_at = [&](int i) -> TcUnit {
-        return i < kTcMaxUnits ? s_units[i] : tc_decode(groups, n_active, total1, blockIdx.x + i * P, sh.d, pl.n1);
-    };
+    // decoded once by all threads: the single-thread roles below then read a unit from shared
+    // memory instead of dividing
+    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x) s_units[i] = unit_make(i);
+    __syncthreads();
+    auto unit_at = [&](int i) -> TcUnit { return i < kTcMaxUnits ? s_units[i] : unit_make(i); };
+    auto seg_of_unit = [&](int i) -> int { return i < n_units ? unit_at(i).seg : 4; };
 
+    TCT(const long long t_roles = clock64();)
     if (warp == 0) {
         const uint64_t wpolicy = l2_evict_first_policy();
         // ------------------------------------------------------------------ TMA producer
@@ -365,7 +411,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             int pend_wave = 0;
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
                 pend_tn[kTcMaxStages];
-            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
+            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0, tp_x = 0, tp_unit = 0; const long long tp0 = clock64();)
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 uint8_t *op = ring + (size_t)s * pl.stage_bytes + kTcWTile;
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
@@ -374,13 +420,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             };
             auto wait_ready = [&](int w) -> bool {
                 TCT(long long c0 = clock64();)
+                TCG(30 + w);
                 bool ok = false;
-                for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
-                    if (ld_acquire(&ws.sync[kTcReady - 4 + w]) >= (int)gridDim.x) { ok = true; break; }
-                    __nanosleep(40);
+                for (unsigned i = 0; i < kTcSpinLimit; ++i) {
+                    if (s_ready[w]) { ok = true; break; }
+                    __nanosleep(32);
                 }
                 TCT(tp_ready += clock64() - c0;)
                 if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); return false; }
+                __threadfence_block();
                 fence_proxy_async();
                 for (int i = 0; i < pend_n; ++i) load_tokens2(pend_stage[i], pend_kt[i], pend_row[i], pend_shared[i], pend_tn[i]);
                 pend_n = 0;
@@ -388,14 +436,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 return true;
             };
             const int n_routed = p.B * sh.k;
-            if (pl.x_bytes) {
-                // all token tiles of the hidden states, once
-                mbar_expect_tx(&x_bar, (uint32_t)pl.x_bytes);
-                for (int kt = 0; kt < (sh.d + 63) / 64; ++kt)
-                    for (int r = 0; r < pl.n1; r += 16)
-                        tma_load_2d(xres + ((size_t)kt * pl.n1 + r) * 128, &maps.m[6], kt * 64, r, &x_bar);
-            }
+            int s = 0;                                   // ring slot of the next k-tile
+            uint32_t ring_par = 1;                       // parity to wait for on its empty barrier
+            TCT(tp_x = clock64() - tp0;)
             for (int i = 0; i < n_units && alive; ++i) {
+                TCT(const long long cu = clock64();)
                 const TcUnit t = unit_at(i);
                 const StGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
@@ -409,19 +454,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 if (!ready) {
                     // tiles still pending belong to an earlier wave only if that wave is not ready either
                     if (pend_n > 0 && wv > ready_w) { if (!wait_ready(ready_w)) { alive = false; break; } }
-                    if (ld_acquire(&ws.sync[kTcReady - 4 + wv]) >= (int)gridDim.x) {
+                    if (s_ready[wv]) {
                         alive = wait_ready(wv);
                         ready = alive;
                     }
                 }
-                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it) {
-                    const int s = it % S;
+                TCT(tp_unit += clock64() - cu;)
+                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     if (!ready && pend_n == S) {
                         if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
                         ready = true;
                     }
                     TCT(long long c1 = clock64();)
-                    if (!mbar_wait(&empty_bar[s], ((it / S) & 1u) ^ 1u)) {
+                    if (!mbar_wait(&empty_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
@@ -447,7 +492,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 }
             }
             if (alive && pend_n > 0) wait_ready(pend_wave);
-            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0;)
+            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry; o[5] = tp_x; o[6] = tp_unit;)
         }
     } else if (warp == 1 || warp == 6) {
         // ------------------------------------------------------------------ MMA issuers
@@ -457,8 +502,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         // columns; the epilogue adds the two partial accumulators.
         const int half = warp == 1 ? 0 : 1;
         if (lane == 0) {
-            unsigned it = 0, ui = 0;
+            unsigned it = 0, ui = 0, run = 0;
+            uint32_t acc = 0;
             bool alive = true;
+            int s = 0;
+            uint32_t ring_par = 0;
+            if (pl.x_bytes && half == 0) {
+                // all token tiles of the hidden states, once (this thread has nothing to issue before they land)
+                mbar_expect_tx(&x_bar, (uint32_t)pl.x_bytes);
+                for (int kt = 0; kt < (sh.d + 63) / 64; ++kt)
+                    for (int r = 0; r < pl.n1; r += 16)
+                        tma_load_2d(xres + ((size_t)kt * pl.n1 + r) * 128, &maps.m[6], kt * 64, r, &x_bar);
+            }
             if (pl.x_bytes && !mbar_wait(&x_bar, 0)) {
                 atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 alive = false;
@@ -466,23 +521,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0; const long long tm0 = clock64();)
             for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
-                const int buf = ui & 1;
-                TCT(long long c0 = clock64();)
-                if (!mbar_wait(&acc_empty[buf], ((ui >> 1) & 1u) ^ 1u)) {
-                    atomicExch(ws.status, ST_MBAR_TIMEOUT);
-                    break;
+                const int buf = run & 1;
+                if (t.first) {
+                    TCT(long long c0 = clock64();)
+                    if (!mbar_wait(&acc_empty[buf], ((run >> 1) & 1u) ^ 1u)) {
+                        atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                        break;
+                    }
+                    TCT(tm_acc += clock64() - c0;)
+                    tc_fence_after();
+                    acc = 0;
                 }
-                TCT(tm_acc += clock64() - c0;)
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 4 * pl.n1 + half * 2 * pl.n1);
                 // phase 2: the hi and lo token tiles lie back to back, one MMA of N = 2n covers both;
                 // the epilogue adds the two halves
                 const uint32_t idesc = tc_idesc(t.phase == 1 ? t.n : 2 * t.n);
-                uint32_t acc = 0;
-                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it) {
-                    const int s = it % S;
+                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
-                    if (!mbar_wait(&full_bar[s], (it / S) & 1u)) {
+                    if (!mbar_wait(&full_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
@@ -505,15 +561,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
                     TCT(tm_mma += clock64() - c2;)
                 }
-                if (alive) tc_commit(&acc_full[buf]);
+                if (alive && t.last) {
+                    tc_commit(&acc_full[buf]);
+                    ++run;
+                }
             }
             TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; })
         }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------------ watcher
+        // polls the waves' second counters (all CTAs have written their slice of the activations)
+        // and publishes them in shared memory, so that the producer never waits on global memory
+#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 4)
+        if (lane == 0) {
+            for (int w = 0; w < W; ++w) {
+                bool ok = false;
+                for (unsigned i = 0; i < (1u << 21); ++i) {
+                    if (ld_acquire(&ws.sync[kTcReady - 4 + w]) >= (int)gridDim.x) { ok = true; break; }
+                    __nanosleep(100);
+                }
+                if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); break; }
+                __threadfence_block();
+                s_ready[w] = 1;
+                TCG(25 + w);
+            }
+        }
+#endif
     } else if (warp >= 7) {
         // ------------------------------------------------------------------ converter warps
         // per wave: wait for this CTA's hand-over, arrive on the wave's grid-wide counter, wait
         // (bounded) for all CTAs, convert this CTA's slice of the wave, arrive on the second counter
-        const int et = tid - 224;                      // 0..127 among the converter threads
+        const int et = tid - 224;                      // 0..95 among the converter threads
         const int n_routed = p.B * sh.k;
         uint32_t ep_phase = 0;                         // running parity of cv_bar
         uint64_t *ep_bar_p = &cv_bar;
@@ -530,47 +608,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 }
                 if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
                 s_flag = ok;
+                TCG(14 + w);
             }
             if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
             if (!s_flag) return false;
-            __threadfence();
+            __threadfence_block();                 // the counter was read with acquire by one thread of this barrier
             TCT(long long c3 = clock64(); te_sync += c3 - c2;)
-            // activations are stored flat exactly like act_offset(slot) + j: this CTA converts a
-            // contiguous slice of the wave's range
+            // pre holds a gate plane and an up plane, both indexed exactly like the activations
+            // (act_offset(slot) + row): this CTA converts a contiguous slice of the wave's range,
+            // four elements per thread and step
             const long long w_lo = w == 0 ? 0 : el_split, w_hi = (w == 0 && W == 2) ? el_split : n_el;
-            const long long lo_i = w_lo + (w_hi - w_lo) * blockIdx.x / gridDim.x;
-            const long long hi_i = w_lo + (w_hi - w_lo) * (blockIdx.x + 1) / gridDim.x;
-            const long long split = (long long)n_routed * sh.f;
-            for (long long i0 = lo_i + et; i0 < hi_i; i0 += 128 * 4) {
-                float gv[4], uv[4];
-                long long idx[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const long long i = i0 + (long long)r * 128;
-                    idx[r] = i;
-                    if (i < hi_i) {
-                        const int fg = i < split ? sh.f : sh.f_sh;
-                        const long long rel = i < split ? i : i - split;
-                        const long long j = rel % fg;
-                        const long long base = 2 * (i - j) + j;      // pre holds [gate f_g][up f_g] per slot
-                        gv[r] = __ldcg(&p.pre[base]);
-                        uv[r] = __ldcg(&p.pre[base + fg]);
-                    }
-                }
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (idx[r] < hi_i) {
-                        const float a = silu_mul(gv[r], uv[r]);
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-                        p.act_hi[idx[r]] = hi;
-                        p.act_lo[idx[r]] = __float2bfloat16_rn(a - __bfloat162float(hi));
-                    }
-                }
+            const long long n4 = (w_hi - w_lo) >> 2;
+            const long long lo4 = n4 * blockIdx.x / gridDim.x, hi4 = n4 * (blockIdx.x + 1) / gridDim.x;
+            for (long long q = lo4 + et; q < hi4; q += 96) {
+                const long long i = w_lo + 4 * q;
+                const float4 gv = __ldcg(reinterpret_cast<const float4 *>(p.pre + i));
+                const float4 uv = __ldcg(reinterpret_cast<const float4 *>(p.pre + n_el + i));
+                const float a0 = silu_mul(gv.x, uv.x), a1 = silu_mul(gv.y, uv.y), a2 = silu_mul(gv.z, uv.z),
+                            a3 = silu_mul(gv.w, uv.w);
+                const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
+                const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
+                const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
+                uint2 hv, lv;
+                hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+                lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+                *reinterpret_cast<uint2 *>(p.act_hi + i) = hv;
+                *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
             }
             __threadfence();
             fence_proxy_async();
             if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
-            if (et == 0) atomicAdd(&ws.sync[kTcReady - 4 + w], 1);
+            if (et == 0) { atomicAdd(&ws.sync[kTcReady - 4 + w], 1); TCG(23 + w); }
             TCT(te_conv += clock64() - c3;)
             return true;
         };
@@ -593,7 +661,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;                        // TMEM lane quarter this warp may read
         const int et = tid - 64;                       // 0..127 among the epilogue threads
-        unsigned ui = 0;
+        unsigned ui = 0, run = 0;
         uint32_t ep_phase = 0;
         const int n_routed = p.B * sh.k;
         bool alive = true;
@@ -610,6 +678,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             if (et == 0) {
                 __threadfence();                     // the CTA's reductions, ordered by the barrier above
                 mbar_arrive(&conv_go[w]);
+                TCG(12 + w);
             }
             return true;
         };
@@ -630,10 +699,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             for (; (int)ui < n_units && alive; ++ui) {
                 if (!service(seg_of_unit((int)ui))) { alive = false; break; }
                 const TcUnit t = unit_at((int)ui);
+                if (!t.last) continue;                 // the run's accumulator is read after its last unit
                 const StGroup &g = groups[t.a];
-                const int buf = ui & 1;
+                const int buf = run & 1;
                 TCT(long long c0 = clock64();)
-                if (!mbar_wait(&acc_full[buf], (ui >> 1) & 1u)) {
+                if (!mbar_wait(&acc_full[buf], (run >> 1) & 1u)) {
                     if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     alive = false;
                     break;
@@ -650,8 +720,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 if (t.phase == 1) {
                     const bool row_ok = row < g.f;
                     // slot of the expert's i-th token = g.off + i; walk its tokens in ascending order
-                    float *dst = p.pre + 2 * act_offset(g.off, n_routed, sh.f, sh.f_sh) + (size_t)t.mat * g.f + row;
-                    const size_t slot_stride = 2 * (size_t)g.f;
+                    float *dst = p.pre + (size_t)t.mat * n_el + act_offset(g.off, n_routed, sh.f, sh.f_sh) + row;
+                    const size_t slot_stride = (size_t)g.f;
                     for (int c = 0; c < t.n; c += 16) {
                         float v[16], v2[16];
                         tc_ld16(taddr + c, v);
@@ -693,6 +763,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                ++run;
                 TCT(te_red += clock64() - c1;)
             }
             if (alive && !service(4)) alive = false;
@@ -702,6 +773,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     // every path ends here (all waits above are bounded), so the TMEM is always returned
     tc_fence_before();
     __syncthreads();
+    TCT(if (tid == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[7] = clock64() - t_entry; unsigned long long g_exit; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_exit)); o[21] = (long long)g_entry; o[22] = (long long)g_exit; })
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)pl.tmem_cols)
                      : "memory");

@@ -33,7 +33,7 @@ struct s2moe_ctx {
     int n_sm = 0;
     __nv_bfloat16 *act_hi = nullptr, *act_lo = nullptr;
     size_t act_elems = 0;
-    float *pre = nullptr;                 // plan 3: fp32 pre-activations [slot][2][f]
+    float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
     int last_cuda = 0;
