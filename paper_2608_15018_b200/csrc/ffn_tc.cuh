@@ -42,7 +42,10 @@
 namespace s2moe {
 
 constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
-constexpr int kTcMaxStages = 12;
+#ifndef S2MOE_MAX_STAGES
+#define S2MOE_MAX_STAGES 10
+#endif
+constexpr int kTcMaxStages = S2MOE_MAX_STAGES;
 constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 KiB of weights
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
 constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
@@ -83,8 +86,9 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     const int G = sh.E + sh.n_sh;
     p.n_cta = n_sm;
     p.n1 = (B + 15) & ~15;
-    // phase-2 stages carry hi and lo tiles of up to n1 slots (a group never has more tokens than B)
-    p.stage_bytes = kTcWTile + 2 * p.n1 * 128;
+    // token area of a stage: phase 1 = n1 rows of 128 bytes; phase 2 = per 8 slots their hi rows
+    // (1 KiB) and right behind them their lo rows (a group never has more tokens than B)
+    p.stage_bytes = kTcWTile + 2048 * ((B + 7) / 8);
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
     p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
     // The ring is what keeps HBM busy (bytes in flight = stages x 16 KiB per SM, against a loaded
@@ -210,9 +214,9 @@ __device__ __forceinline__ void tc_ring_next(int &s, uint32_t &parity, int S)
     if (++s == S) { s = 0; parity ^= 1u; }
 }
 
-struct TcUnit {
+struct TcUnit {                        // plain ints: the single-thread roles read these on their critical path
     int phase, a, mat, rb, kt0, kt1;   // group slot, matrix (0 gate, 1 up, 2 down), row block, k-tile range
-    int n;                             // MMA N (tokens padded to 16)
+    int n;                             // MMA N: phase 1 tokens padded to 16; phase 2 16 per 8 slots (hi | lo)
     int seg;                           // 0 / 1: phase 1 of wave 0 / 1, 2 / 3: phase 2 of wave 0 / 1
     int first, last;                   // first / last unit of an accumulation run (see the kernel)
 };
@@ -242,7 +246,7 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
         t.mat = 2;
         t.kt0 = piece * kTcKT;
         t.kt1 = min((g.f + 63) / 64, t.kt0 + kTcKT);
-        t.n = (g.T + 15) & ~15;
+        t.n = 16 * ((g.T + 7) / 8);
     }
     return t;
 }
@@ -270,6 +274,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     const TcPlan &pl = p.plan;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     TCT(const long long t_entry = clock64(); unsigned long long g_entry; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_entry));)
+    // programmatic dependent launch: the routing kernel in front of this grid must have
+    // finished before its results are read; the next layer's routing kernel may be scheduled
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int n_active = ws.header[0], n_slots = ws.header[1];
     const int G = sh.E + sh.n_sh;
 
@@ -323,7 +331,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         s_ready[1] = 0;
     }
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
+        for (int s = 0; s < pl.stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 2);      // one commit from each MMA issuer
         }
@@ -339,7 +347,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        // TMEM: accumulators of two units
+        // TMEM: accumulators of two runs for each of the two issuers
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
                      "r"((uint32_t)pl.tmem_cols)
                      : "memory");
@@ -415,8 +423,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 uint8_t *op = ring + (size_t)s * pl.stage_bytes + kTcWTile;
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
-                // one copy per 16 slots: their hi tile (2 KiB) and, right behind it, their lo tile
-                for (int r = 0; r < tn; r += 16) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
+                // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
+                for (int r = 0; r < tn / 2; r += 8) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
             auto wait_ready = [&](int w) -> bool {
                 TCT(long long c0 = clock64();)
@@ -473,7 +481,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     }
                     TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
-                    const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 256u;
+                    const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 128u;
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
                     tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
                     if (t.phase == 1) {
@@ -533,9 +541,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     acc = 0;
                 }
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 4 * pl.n1 + half * 2 * pl.n1);
-                // phase 2: the hi and lo token tiles lie back to back, one MMA of N = 2n covers both;
-                // the epilogue adds the two halves
-                const uint32_t idesc = tc_idesc(t.phase == 1 ? t.n : 2 * t.n);
+                // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
+                // adds the two halves
+                const uint32_t idesc = tc_idesc(t.n);
                 for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
                     if (!mbar_wait(&full_bar[s], ring_par)) {
@@ -740,20 +748,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 } else {
                     const bool row_ok = row < sh.d;
                     for (int c = 0; c < t.n; c += 16) {
-                        float v[16], w[16];                       // columns: 16 hi, 16 lo, 16 hi, ...
-                        float v2[16], w2[16];
-                        tc_ld16(taddr + 2 * c, v);
-                        tc_ld16(taddr + 2 * c + 16, w);
-                        tc_ld16(taddr + other + 2 * c, v2);
-                        tc_ld16(taddr + other + 2 * c + 16, w2);
+                        float v[16], v2[16];                      // columns: 8 hi, 8 lo of slots c / 2 .. c / 2 + 7
+                        tc_ld16(taddr + c, v);
+                        tc_ld16(taddr + other + c, v2);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) { v[i] += v2[i]; w[i] += w2[i]; }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int ti = c + i;
+                        for (int i = 0; i < 8; ++i) {
+                            const int ti = (c >> 1) + i;
                             if (ti < g.T && row_ok) {
                                 const int slot = g.off + ti;
-                                atomicAdd(&p.y[(size_t)s_slot_token[slot] * sh.d + row], s_slot_w[slot] * (v[i] + w[i]));
+                                atomicAdd(&p.y[(size_t)s_slot_token[slot] * sh.d + row],
+                                          s_slot_w[slot] * ((v[i] + v2[i]) + (v[i + 8] + v2[i + 8])));
                             }
                         }
                     }
@@ -773,7 +777,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     // every path ends here (all waits above are bounded), so the TMEM is always returned
     tc_fence_before();
     __syncthreads();
-    TCT(if (tid == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[7] = clock64() - t_entry; unsigned long long g_exit; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_exit)); o[21] = (long long)g_entry; o[22] = (long long)g_exit; })
+    TCT(if (tid == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[7] = clock64() - t_entry; unsigned long long g_exit; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_exit)); o[21] = (long long)g_entry; o[22] = (long long)g_exit; unsigned smid_; asm volatile("mov.u32 %0, %smid;" : "=r"(smid_)); o[27] = smid_; o[19] = n_units; })
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)pl.tmem_cols)
                      : "memory");

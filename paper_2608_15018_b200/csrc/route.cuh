@@ -443,6 +443,11 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     extern __shared__ double s_dyn[];
     __shared__ int s_last;
     const int tid = threadIdx.x;
+    // Programmatic dependent launch: everything this kernel writes is read by the previous
+    // layer's kernels, so it waits for them first; the FFN kernel that follows may come up now
+    // and do its own set-up (both instructions do nothing in a plain launch).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef S2MOE_TIMING
     const long long t_start = clock64();
 #endif
