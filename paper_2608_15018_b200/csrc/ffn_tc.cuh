@@ -342,8 +342,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         mbar_init(&ep_bar, 4);
         mbar_init(&x_bar, 1);
         mbar_init(&cv_bar, 3);
-        mbar_init(&conv_go[0], 1);
-        mbar_init(&conv_go[1], 1);
+        mbar_init(&conv_go[0], 4);
+        mbar_init(&conv_go[1], 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -660,7 +660,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 __nanosleep(64);
             }
             if (!ok) { if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
-            if (et == 0) atomicAdd(&ws.sync[kTcReady - 8 + w], 1);
+            if (et == 0) {
+                __threadfence();                     // the CTA's reductions, observed through conv_go
+                atomicAdd(&ws.sync[kTcReady - 8 + w], 1);
+            }
             if (!wave_convert(w)) break;
         }
 #endif
@@ -681,10 +684,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
         const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
         int next_arrive = 0;
         auto wave_arrive = [&](int w) -> bool {
-            // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps
-            if (!tc_bar(&ep_bar, ep_phase, lane)) return false;
-            if (et == 0) {
-                __threadfence();                     // the CTA's reductions, ordered by the barrier above
+            // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps,
+            // whose first thread orders them (fence) before it arrives on the grid-wide counter, so
+            // that no epilogue thread stalls on a fence
+            __syncwarp();
+            if (lane == 0) {
                 mbar_arrive(&conv_go[w]);
                 TCG(12 + w);
             }

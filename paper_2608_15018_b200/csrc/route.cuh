@@ -26,6 +26,10 @@ __device__ __forceinline__ double warp_max(double v)
     return v;
 }
 
+// One copy of the double-precision exponential for the whole gating: the gating runs once, on
+// one block, with a cold instruction cache, so its cost follows the amount of distinct code.
+__device__ __noinline__ double exp_once(double x) { return exp(x); }
+
 // Monotone map from doubles (no NaN) to unsigned integers: a < b  <=>  dkey(a) < dkey(b), and
 // equal doubles (-0 included) have equal keys.  Keys of finite values are never 0.
 __device__ __forceinline__ unsigned long long dkey(double x)
@@ -46,156 +50,195 @@ __device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k)
     const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? (unsigned)k : 0u);
     return ((unsigned long long)mh << 32) | ml;
 }
+// lanes (as a ballot) that hold the largest key among the lanes with `has`; the common case
+// (one lane has the largest upper half) takes one warp reduction and one ballot
+__device__ __forceinline__ unsigned warp_max_holders(unsigned long long k, bool has)
+{
+    const unsigned hi = has ? (unsigned)(k >> 32) : 0u;
+    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+    bool hold = has && hi == mh;
+    unsigned hb = __ballot_sync(0xffffffffu, hold);
+    if (__popc(hb) > 1) {
+        const unsigned ml = __reduce_max_sync(0xffffffffu, hold ? (unsigned)k : 0u);
+        hold = hold && (unsigned)k == ml;
+        hb = __ballot_sync(0xffffffffu, hold);
+    }
+    return hb;
+}
+__device__ __forceinline__ unsigned long long shfl_key(unsigned long long k, int src)
+{
+    const unsigned lo = __shfl_sync(0xffffffffu, (unsigned)k, src);
+    const unsigned hi = __shfl_sync(0xffffffffu, (unsigned)(k >> 32), src);
+    return ((unsigned long long)hi << 32) | lo;
+}
+
 
 #ifdef S2MOE_TIMING
-__device__ long long g_gt_marks[8];
-#define GT_MARK(i) do { if (tid == 0) g_gt_marks[i] = clock64(); } while (0)
+__device__ long long g_gt_marks[16];
+#define GT_MARK(i) do { if (threadIdx.x == 0) g_gt_marks[i] = clock64(); } while (0)
 #else
 #define GT_MARK(i) do { } while (0)
 #endif
 
-// Per-token part of the gating, one warp per token: lane owns experts lane, lane + 32, ...
-// (J per lane, in registers).  lambda_b from the top-1 and (k+1)-th original logit, the k
-// experts of largest biased logit in the order (l' descending, l descending, id ascending),
-// softmax mixing weights.  Selection runs k (+ k + 1) rounds of a warp-wide maximum over
-// integer keys instead of ranking all E x E pairs.
+// Order statistics of one token's original logits, one warp per token (lane owns experts lane,
+// lane + 32, ...): lambda_b = alpha (l_(1) - l_(k+1)) by k + 1 rounds of a warp-wide maximum over
+// integer keys, and, for weight_mode 0, the softmax denominator over the original logits.
 template <int J>
-__device__ __forceinline__ void gate_tokens(const Shape &sh, int B, bool bias_on, const double *s_l,
-                                            const unsigned char *s_star, int *s_sel, float *s_pw,
-                                            unsigned long long *s_mask, int32_t *__restrict__ sel_idx,
-                                            float *__restrict__ sel_w, int tid, int nt)
+__device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on, const double *s_l, double *s_lam,
+                                           double *s_zmax, double *s_den, int lane)
 {
-    const unsigned full = 0xffffffffu;
-    const int warp = tid >> 5, lane = tid & 31, nw = nt >> 5, E = sh.E, k = sh.k;
-    for (int b = warp; b < B; b += nw) {
-        GT_MARK(0);
-        double l[J];
-        unsigned long long k1[J];
-        unsigned valid = 0, star = 0;
+    const int E = sh.E, k = sh.k;
+    GT_MARK(0);
+    unsigned long long k1[J];
+    unsigned valid = 0;
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            const int e = lane + 32 * j;
-            l[j] = 0.0;
-            k1[j] = 0ull;
-            if (e < E) {
-                l[j] = s_l[b * E + e] + 0.0;
-                k1[j] = dkey(l[j]);
-                valid |= 1u << j;
-                star |= (unsigned)s_star[e] << j;
-            }
-        }
-        GT_MARK(1);
-        // order statistics of the original logits: top-1 and (k+1)-th value (with multiplicity)
-        double lam = 0.0;
-        if (bias_on) {
-            unsigned alive = valid;
-            unsigned long long top1 = 0ull, m = 0ull;
-            for (int r = 0; r <= k; ++r) {
-                unsigned long long lm = 0ull;
-#pragma unroll
-                for (int j = 0; j < J; ++j)
-                    if (((alive >> j) & 1u) && k1[j] > lm) lm = k1[j];
-                m = warp_max_key(lm);
-                if (r == 0) top1 = m;
-                const unsigned hb = __ballot_sync(full, alive != 0u && lm == m);
-                if (lane == __ffs(hb) - 1) {            // drop one instance of the maximum
-                    bool done = false;
-#pragma unroll
-                    for (int j = 0; j < J; ++j)
-                        if (!done && ((alive >> j) & 1u) && k1[j] == m) { alive &= ~(1u << j); done = true; }
-                }
-            }
-            lam = sh.alpha * (dkey_value(top1) - dkey_value(m));
-        }
-        GT_MARK(2);
-        unsigned long long k2[J];
-#pragma unroll
-        for (int j = 0; j < J; ++j) k2[j] = ((star >> j) & 1u) ? dkey(l[j] + lam) : k1[j];
-        // biased top-k, one winner per round
-        unsigned alive = valid;
-        int my_sel = 0;
-        for (int r = 0; r < k; ++r) {
-            unsigned long long b2 = 0ull, b1 = 0ull;
-            int bj = -1;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                if ((alive >> j) & 1u) {
-                    const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
-                    if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
-                }
-            }
-            const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
-            const unsigned long long m2 = warp_max_key(b2);
-            bool hold = bj >= 0 && b2 == m2;
-            unsigned hb = __ballot_sync(full, hold);
-            if (__popc(hb) > 1) {                       // equal biased logits: larger original logit first
-                const unsigned long long m1 = warp_max_key(hold ? b1 : 0ull);
-                hold = hold && b1 == m1;
-                hb = __ballot_sync(full, hold);
-                if (__popc(hb) > 1) {                   // still equal: lower expert id first
-                    const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
-                    hold = hold && my_e == me;
-                    hb = __ballot_sync(full, hold);
-                }
-            }
-            const int wl = __ffs(hb) - 1;
-            const int we = (int)__shfl_sync(full, my_e, wl);
-            if (lane == wl) alive &= ~(1u << bj);
-            if (lane == r) my_sel = we;
-        }
-        GT_MARK(3);
-        // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
-        const double lamw = sh.weight_mode ? lam : 0.0;
-        double z[J];
-        unsigned long long zk = 0ull;
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-            z[j] = l[j] + (((star >> j) & 1u) ? lamw : 0.0);
-            if ((valid >> j) & 1u) { const unsigned long long q = dkey(z[j]); zk = q > zk ? q : zk; }
-        }
-        const double zmax = dkey_value(warp_max_key(zk));
-        double den = 0.0;
+    for (int j = 0; j < J; ++j) {
+        const int e = lane + 32 * j;
+        k1[j] = 0ull;
+        if (e < E) { k1[j] = dkey(s_l[b * E + e]); valid |= 1u << j; }
+    }
+    unsigned alive = valid;
+    unsigned long long top1 = 0ull, kth = 0ull;
+    const int rounds = bias_on ? k + 1 : 1;
+#pragma unroll 1
+    for (int r = 0; r < rounds; ++r) {
+        unsigned long long lm = 0ull;
+        int bj = 0;
 #pragma unroll
         for (int j = 0; j < J; ++j)
-            if ((valid >> j) & 1u) den += exp(z[j] - zmax);
-        den = warp_sum(den);
-        double p = 0.0;
-        if (lane < k) {
-            const double zs = s_l[b * E + my_sel] + (s_star[my_sel] ? lamw : 0.0);
-            p = exp(zs - zmax) / den;
-        }
-        if (sh.renorm) {
-            const double tot = warp_sum(p);
-            p /= tot;
-        }
-        if (lane < k) {
-            s_sel[b * k + lane] = my_sel;
-            s_pw[b * k + lane] = (float)p;
-            sel_idx[b * k + lane] = my_sel;
-            sel_w[b * k + lane] = (float)p;
-            atomicOr(&s_mask[my_sel], 1ull << b);
-        }
-        GT_MARK(4);
+            if (((alive >> j) & 1u) && k1[j] > lm) { lm = k1[j]; bj = j; }
+        const unsigned hb = warp_max_holders(lm, alive != 0u);
+        const int wl = __ffs(hb) - 1;
+        if (r == 0) top1 = shfl_key(lm, wl);
+        if (r == k) kth = shfl_key(lm, wl);
+        if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
     }
+    GT_MARK(1);
+    const double ztop = dkey_value(top1);
+    double den = 0.0;
+    if (!sh.weight_mode) {
+#pragma unroll 1
+        for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) - ztop);
+        den = warp_sum(den);
+    }
+    if (lane == 0) {
+        s_lam[b] = bias_on ? sh.alpha * (ztop - dkey_value(kth)) : 0.0;
+        s_zmax[b] = ztop;
+        s_den[b] = den;
+    }
+    GT_MARK(2);
 }
 
-// Gating of one batch by one thread block (any block size that is a multiple of 32).
+// Biased top-k of one token in the order (l' descending, l descending, id ascending), one
+// winner per round, and the mixing weights of the winners.
+template <int J>
+__device__ __forceinline__ void gate_select(const Shape &sh, int b, const double *s_l, const unsigned char *s_star,
+                                            const double *s_lam, const double *s_zmax, const double *s_den, int *s_sel,
+                                            float *s_pw, unsigned long long *s_mask, int32_t *__restrict__ sel_idx,
+                                            float *__restrict__ sel_w, int lane)
+{
+    const unsigned full = 0xffffffffu;
+    const int E = sh.E, k = sh.k;
+    GT_MARK(3);
+    const double lam = s_lam[b];
+    double l[J];
+    unsigned long long k1[J], k2[J];
+    unsigned valid = 0, star = 0;
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+        const int e = lane + 32 * j;
+        l[j] = 0.0;
+        k1[j] = 0ull;
+        k2[j] = 0ull;
+        if (e < E) {
+            l[j] = s_l[b * E + e] + 0.0;
+            k1[j] = dkey(l[j]);
+            const unsigned st = s_star[e];
+            star |= st << j;
+            k2[j] = st ? dkey(l[j] + lam) : k1[j];
+            valid |= 1u << j;
+        }
+    }
+    unsigned alive = valid;
+    GT_MARK(4);
+#pragma unroll 1
+    for (int r = 0; r < k; ++r) {
+        unsigned long long b2 = 0ull, b1 = 0ull;
+        int bj = -1;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            if ((alive >> j) & 1u) {
+                const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
+                if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
+            }
+        }
+        const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
+        unsigned hb = warp_max_holders(b2, bj >= 0);
+        if (__popc(hb) > 1) {                           // equal biased logits: larger original logit first
+            hb = warp_max_holders(b1, (hb >> lane) & 1u);
+            if (__popc(hb) > 1) {                       // still equal: lower expert id first
+                const bool hold = (hb >> lane) & 1u;
+                const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
+                hb = __ballot_sync(full, hold && my_e == me);
+            }
+        }
+        if (lane == __ffs(hb) - 1) {
+            alive &= ~(1u << bj);
+            s_sel[b * k + r] = (int)my_e;
+        }
+    }
+    __syncwarp();
+    GT_MARK(5);
+    // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
+    double zmax = s_zmax[b], den = s_den[b];
+    const double lamw = sh.weight_mode ? lam : 0.0;
+    if (sh.weight_mode) {
+        unsigned long long zk = 0ull;
+#pragma unroll
+        for (int j = 0; j < J; ++j)
+            if (((valid >> j) & 1u) && k2[j] > zk) zk = k2[j];
+        zmax = dkey_value(warp_max_key(zk));
+        den = 0.0;
+#pragma unroll 1
+        for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) + (s_star[e] ? lamw : 0.0) - zmax);
+        den = warp_sum(den);
+    }
+    double p = 0.0;
+    int my_sel = 0;
+    if (lane < k) {
+        my_sel = s_sel[b * k + lane];
+        const double zs = s_l[b * E + my_sel] + (s_star[my_sel] ? lamw : 0.0);
+        p = exp_once(zs - zmax) / den;
+    }
+    if (sh.renorm) {
+        const double tot = warp_sum(p);
+        p /= tot;
+    }
+    if (lane < k) {
+        s_pw[b * k + lane] = (float)p;
+        sel_idx[b * k + lane] = my_sel;
+        sel_w[b * k + lane] = (float)p;
+        atomicOr(&s_mask[my_sel], 1ull << b);
+    }
+    GT_MARK(6);
+}
+
+// Gating of one batch by one thread block of at least two warps.
 // s_l: shared memory for B*E doubles (the logits, copied from the workspace).
 __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
                                              int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
                                              int32_t *__restrict__ n_unique, double *s_l)
 {
     __shared__ unsigned long long s_gk[kMaxExperts];
-    __shared__ int s_rank[kMaxExperts];
     __shared__ unsigned char s_star[kMaxExperts];
-    __shared__ double s_w[kMaxTokens];
+    __shared__ double s_w[kMaxTokens], s_lam[kMaxTokens], s_zmax[kMaxTokens], s_den[kMaxTokens];
     __shared__ int s_sel[kMaxTokens * kMaxTopK];
     __shared__ float s_pw[kMaxTokens * kMaxTopK];
     __shared__ unsigned long long s_mask[kMaxExperts];
     __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_pos[kMaxExperts];
     __shared__ int s_U;
 
-    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
     const int E = sh.E, k = sh.k, cap = sh.cap;
     const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
 #ifdef S2MOE_TIMING
@@ -207,54 +250,67 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
 #endif
     GATE_MARK();
 
+#pragma unroll 1
     for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
+#pragma unroll 1
     for (int b = tid; b < B; b += nt) s_w[b] = conf ? (double)conf[b] : 1.0;
-    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; s_rank[e] = 0; }
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
     __syncthreads();
 
     GATE_MARK();
-    if (bias_on) {
+    // Two independent pieces run side by side on disjoint warps: the last cw warps pick the
+    // reuse-reward set E* (Eq. 4 aggregation, TopCap), the others take the per-token order
+    // statistics (lambda_b, softmax denominator).
+    const int cw = bias_on ? max(1, min(nw / 2, nw - B)) : 0, tw = nw - cw;
+    if (warp >= tw) {
+        const int ct = tid - tw * 32, cn = cw * 32;
         // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
-        for (int e = tid; e < E; e += nt) {
+#pragma unroll 1
+        for (int e = ct; e < E; e += cn) {
             double g = 0.0;
+#pragma unroll 1
             for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
             s_gk[e] = dkey(g);
         }
-        __syncthreads();
-        // TopCap by rank in the order (g descending, id ascending); P threads share an expert
-        int P = 1;
-        while (P < 8 && E * (P * 2) <= nt) P *= 2;
-        for (int i = tid; i < E * P; i += nt) {
-            const int e = i / P, part = i - e * P;
+        asm volatile("bar.sync 1, %0;" ::"r"(cn) : "memory");
+        // TopCap by rank in the order (g descending, id ascending)
+#pragma unroll 1
+        for (int e = ct; e < E; e += cn) {
             const unsigned long long ge = s_gk[e];
             int rank = 0;
-            for (int o = part; o < E; o += P) {
+#pragma unroll 4
+            for (int o = 0; o < E; ++o) {
                 const unsigned long long go = s_gk[o];
                 rank += (go > ge) | ((go == ge) & (o < e));
             }
-            if (rank) atomicAdd(&s_rank[e], rank);
+            s_star[e] = rank < cap;
         }
-        __syncthreads();
-        for (int e = tid; e < E; e += nt) s_star[e] = s_rank[e] < cap;
-        __syncthreads();
+    } else {
+#pragma unroll 1
+        for (int b = warp; b < B; b += tw) {
+            if (E <= 64) gate_stats<2>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
+            else if (E <= 128) gate_stats<4>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
+            else gate_stats<8>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
+        }
     }
+    __syncthreads();
 
     GATE_MARK();
-    if (E <= 64) gate_tokens<2>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
-    else if (E <= 128) gate_tokens<4>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
-    else gate_tokens<8>(sh, B, bias_on, s_l, s_star, s_sel, s_pw, s_mask, sel_idx, sel_w, tid, nt);
+#pragma unroll 1
+    for (int b = warp; b < B; b += nw) {
+        if (E <= 64) gate_select<2>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
+        else if (E <= 128) gate_select<4>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
+        else gate_select<8>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
+    }
     __syncthreads();
 
     GATE_MARK();
     // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts
-#ifdef S2MOE_TIMING
-#pragma unroll 1
-    for (int rep = 0; rep < 2; ++rep) {
-    if (rep == 1) GATE_MARK();
-#endif
     if (tid < 32) {
         const int C = (E + 31) >> 5, e0 = tid * C;
         int sum = 0, act = 0;
+#pragma unroll 1
         for (int i = 0; i < C; ++i) {
             const int e = e0 + i;
             if (e < E) {
@@ -271,6 +327,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             if (tid >= o) { xs += t; xa += u; }
         }
         int off = xs - sum, pos = xa - act;
+#pragma unroll 1
         for (int i = 0; i < C; ++i) {
             const int e = e0 + i;
             if (e < E) {
@@ -282,12 +339,10 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         }
         if (tid == 31) { s_off[E] = xs; s_U = xa; }
     }
-#ifdef S2MOE_TIMING
-    }
-#endif
     __syncthreads();
     GATE_MARK();
     const int U = s_U, n_routed = B * k;
+#pragma unroll 1
     for (int e = tid; e < E; e += nt) {
         ws.counts[e] = s_cnt[e];
         ws.offsets[e] = s_off[e];
@@ -295,6 +350,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     GATE_MARK();
     // bucket the (token, choice) pairs: tokens ascending inside an expert
+#pragma unroll 1
     for (int i = tid; i < n_routed; i += nt) {
         const int b = i / k;
         const int e = s_sel[i];
@@ -304,10 +360,11 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     GATE_MARK();
     // shared experts: every token, weight c_b
+#pragma unroll 1
     for (int i = tid; i < sh.n_sh * B; i += nt) {
         const int s = i / B, b = i - s * B;
         float c = 1.0f;
-        if (has_gate) c = (float)(1.0 / (1.0 + exp(-__ldcg(&ws.gate_logit[b]))));
+        if (has_gate) c = (float)(1.0 / (1.0 + exp_once(-__ldcg(&ws.gate_logit[b]))));
         ws.slot_token[n_routed + i] = b;
         ws.slot_w[n_routed + i] = c;
         if (b == 0) {
@@ -317,18 +374,23 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         }
     }
     GATE_MARK();
+#pragma unroll 1
     for (int e = tid; e < E; e += nt) ws.tokmask[e] = s_mask[e];
+#pragma unroll 1
     for (int s = tid; s < sh.n_sh; s += nt) ws.tokmask[E + s] = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
     if (sh.plan == 2) {
         // stage tables of the streaming kernel: per active group, its first phase-1 stage
         // (4 gate + 4 up rows each) and first phase-2 stage (8 down rows x one K-slice)
         __syncthreads();
+#pragma unroll 1
         for (int e = tid; e < E; e += nt)
             s_cnt[e] = s_cnt[e] > 0 ? st_nks(sh.f, s_cnt[e], sh.op_cap, sh.d) * (sh.d / 8) : 0;   // phase-2 stages
         __syncthreads();
+#pragma unroll 1
         for (int e = tid; e < E; e += nt) {
             if (s_mask[e]) {
                 int pre = 0;
+#pragma unroll 1
                 for (int o = 0; o < e; ++o) pre += s_cnt[o];
                 const int a = s_pos[e];
                 ws.upfx1[a] = a * (sh.f / 4);
@@ -340,6 +402,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         __syncthreads();
         if (tid == 0) {
             int t1 = U * (sh.f / 4), t2 = s_off[0];
+#pragma unroll 1
             for (int s = 0; s <= sh.n_sh; ++s) {
                 ws.upfx1[U + s] = t1;
                 ws.upfx2[U + s] = t2;
@@ -355,7 +418,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     GATE_MARK();
 #ifdef S2MOE_TIMING
-    if (tid == 0) for (int i = 0; i < 5; ++i) tm[20 + i] = g_gt_marks[i];
+    if (tid == 0) for (int i = 0; i < 8; ++i) tm[20 + i] = g_gt_marks[i];
 #endif
     if (tid == 0) {
         ws.offsets[E + sh.n_sh] = n_routed + sh.n_sh * B;
