@@ -253,6 +253,53 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
                         const void *hidden, const float *conf, int32_t *sel_idx, float *sel_w,
                         int32_t *n_unique, float *gate_out, void *cuda_stream);
 
+/*
+ * Routing-aware adaptive speculative expansion (Sec. 4.1): the step that chooses which draft
+ * candidates the verification layer will be run on.  Neither call uses a context, allocates
+ * or synchronises; both are asynchronous on the given stream.
+ *
+ * s2moe_expert_masks -- predicted expert sets E_i as bit masks ("Routing-aware Cost
+ * Estimation").  sel_idx: dev [n_tokens][top_k] expert ids (for example the sel_idx output of a
+ * draft pass: s2moe_verify_layer on a context created with the draft top-k and alpha = 0).
+ * masks: dev, word w of token t at masks[t * stride_words + w], bit (e % 64) of word (e / 64)
+ * for expert e; ceil(n_experts / 64) words are written per token, so that the masks of several
+ * layers can be interleaved by calling once per layer with an offset pointer.
+ * Errors: EINVAL (null pointer, n_experts or top_k out of range, stride too small), ECUDA.
+ */
+int s2moe_expert_masks(const int32_t *sel_idx, int32_t n_tokens, int32_t top_k, int32_t n_experts,
+                       uint64_t *masks, int32_t stride_words, void *cuda_stream);
+
+/*
+ * s2moe_adaptive_expand -- greedy admission by utility (Eq. 2, Eq. 3, "Adaptive Expansion").
+ *   p_i   = product of p_tok along the path to candidate i            (prefix confidence)
+ *   dC    = | E_i \ union of the admitted candidates' sets | * t_exp   (Eq. 2; the sets are given
+ *           per MoE layer and the new experts of all layers are added up)
+ *   U_i   = p_i * t_ar / (dC + c_draft[i])                            (Eq. 3; zero cost: +inf)
+ * A candidate is eligible once its parent is admitted (parent -1: always).  Every step admits
+ * the eligible candidate of largest utility (ties: lowest index) and stops when that utility is
+ * below 1.  All of it in float64, one rounding per operation.
+ *
+ *   n_cand    1 .. S2MOE_EXPAND_MAX_CAND; parents must precede their children
+ *   parent    dev [n_cand]   index of the parent candidate, or -1
+ *   p_tok     dev [n_cand]   token-level confidence of each candidate
+ *   masks     dev [n_cand][n_layers][ceil(n_experts / 64)]   predicted expert sets
+ *   c_draft   dev [n_cand]   draft expansion cost, or NULL for 0
+ *   t_ar      latency of one autoregressive step of the target model; t_exp latency of one
+ *             more expert in verification; both in the unit of c_draft
+ *   admitted  dev [n_cand]   out: 1 / 0
+ *   order     dev [n_cand]   out: admitted candidates in admission order, then -1
+ *   n_admitted dev scalar    out
+ *   union_out dev [n_layers][ceil(n_experts / 64)] or NULL   out: union of the admitted sets
+ * Errors: EINVAL (null pointer, bad sizes), ERANGE (n_cand or n_layers * words beyond the
+ * limits), ECUDA.
+ */
+#define S2MOE_EXPAND_MAX_CAND 256
+#define S2MOE_EXPAND_MAX_WORDS 512      /* n_layers * ceil(n_experts / 64) */
+int s2moe_adaptive_expand(int32_t n_cand, int32_t n_layers, int32_t n_experts, const int32_t *parent,
+                          const float *p_tok, const uint64_t *masks, const float *c_draft, float t_ar,
+                          float t_exp, int32_t *admitted, int32_t *order, int32_t *n_admitted,
+                          uint64_t *union_out, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

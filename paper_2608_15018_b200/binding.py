@@ -101,6 +101,11 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_profile_end.restype = ctypes.c_int
     lib.s2moe_kernel_class_name.argtypes = [i32]
     lib.s2moe_kernel_class_name.restype = ctypes.c_char_p
+    lib.s2moe_expert_masks.argtypes = [vp, i32, i32, i32, vp, i32, vp]
+    lib.s2moe_expert_masks.restype = ctypes.c_int
+    lib.s2moe_adaptive_expand.argtypes = [i32, i32, i32, vp, fp, vp, fp, ctypes.c_float, ctypes.c_float, vp, vp, vp,
+                                          vp, vp]
+    lib.s2moe_adaptive_expand.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -330,3 +335,42 @@ def route_noalloc(config: Config, hidden: torch.Tensor, router: torch.Tensor,
     if rc != OK:
         raise S2MoEError(rc, "s2moe_route_noalloc")
     return sel_idx, sel_w, n_unique, gate
+
+
+def expert_masks(sel_idx: torch.Tensor, n_experts: int, out: Optional[torch.Tensor] = None, layer: int = 0,
+                 stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Predicted expert sets as bit masks through ``s2moe_expert_masks``.  ``sel_idx`` is
+    [n_tokens][top_k] int32 on the device; the result is int64 [n_tokens][n_layers][words]
+    (bit e % 64 of word e / 64); with ``out`` given, layer ``layer`` of it is written."""
+    lib = load_library()
+    n, k = sel_idx.shape
+    words = (n_experts + 63) // 64
+    if out is None:
+        out = torch.zeros((n, 1, words), dtype=torch.int64, device=sel_idx.device)
+    n_layers = out.shape[1]
+    base = out.view(-1)[layer * words:]
+    rc = lib.s2moe_expert_masks(_dptr(sel_idx), n, k, n_experts, _dptr(base), n_layers * words, _stream_handle(stream))
+    if rc != OK:
+        raise S2MoEError(rc, "s2moe_expert_masks")
+    return out
+
+
+def adaptive_expand(parent: torch.Tensor, p_tok: torch.Tensor, masks: torch.Tensor, n_experts: int,
+                    c_draft: Optional[torch.Tensor], t_ar: float, t_exp: float,
+                    stream: Optional[torch.cuda.Stream] = None):
+    """Greedy routing-aware admission through ``s2moe_adaptive_expand``.  ``masks`` is int64
+    [n_cand][n_layers][words].  Returns (admitted, order, n_admitted, union) on the device."""
+    lib = load_library()
+    n, n_layers, words = masks.shape
+    dev = masks.device
+    admitted = torch.empty((n,), dtype=torch.int32, device=dev)
+    order = torch.empty((n,), dtype=torch.int32, device=dev)
+    n_adm = torch.empty((1,), dtype=torch.int32, device=dev)
+    union = torch.empty((n_layers, words), dtype=torch.int64, device=dev)
+    rc = lib.s2moe_adaptive_expand(n, n_layers, n_experts, _dptr(parent), _dptr(p_tok), _dptr(masks), _dptr(c_draft),
+                                   float(t_ar), float(t_exp), _dptr(admitted), _dptr(order), _dptr(n_adm),
+                                   _dptr(union), _stream_handle(stream))
+    if rc != OK:
+        raise S2MoEError(rc, "s2moe_adaptive_expand")
+    return admitted, order, n_adm, union
+

@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "ffn_simple.cuh"
 #include "ffn_stream.cuh"
+#include "expand.cuh"
 #include "ffn_tc.cuh"
 #include "route.cuh"
 
@@ -741,6 +742,38 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
         route_kernel<DT_BF16, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
                                                                           sel_idx, sel_w, n_unique, ZeroList{});
     if (gate_vec && gate_out) noalloc_gate_out_kernel<<<1, 64, 0, st>>>(ws.gate_logit, gate_out, n_tokens);
+    return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
+}
+
+// ---- routing-aware adaptive expansion (no context, no allocation) ----------------------
+
+int s2moe_expert_masks(const int32_t *sel_idx, int32_t n_tokens, int32_t top_k, int32_t n_experts, uint64_t *masks,
+                       int32_t stride_words, void *cuda_stream)
+{
+    if (n_tokens < 0 || top_k < 1 || top_k > S2MOE_MAX_TOP_K || n_experts < 1 || n_experts > S2MOE_MAX_EXPERTS)
+        return S2MOE_EINVAL;
+    const int words = (n_experts + 63) / 64;
+    if (stride_words < words) return S2MOE_EINVAL;
+    if (n_tokens == 0) return S2MOE_OK;
+    if (!sel_idx || !masks) return S2MOE_EINVAL;
+    expert_masks_kernel<<<(n_tokens + 127) / 128, 128, 0, (cudaStream_t)cuda_stream>>>(
+        sel_idx, n_tokens, top_k, words, reinterpret_cast<unsigned long long *>(masks), stride_words);
+    return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
+}
+
+int s2moe_adaptive_expand(int32_t n_cand, int32_t n_layers, int32_t n_experts, const int32_t *parent,
+                          const float *p_tok, const uint64_t *masks, const float *c_draft, float t_ar, float t_exp,
+                          int32_t *admitted, int32_t *order, int32_t *n_admitted, uint64_t *union_out,
+                          void *cuda_stream)
+{
+    if (n_cand < 1 || n_layers < 1 || n_experts < 1 || n_experts > S2MOE_MAX_EXPERTS) return S2MOE_EINVAL;
+    if (!parent || !p_tok || !masks || !admitted || !order || !n_admitted) return S2MOE_EINVAL;
+    const int lw = n_layers * ((n_experts + 63) / 64);
+    if (n_cand > kExpandMaxCand || lw > kExpandMaxWords) return S2MOE_ERANGE;
+    const int threads = ((n_cand + 31) / 32) * 32;
+    adaptive_expand_kernel<<<1, threads, 0, (cudaStream_t)cuda_stream>>>(
+        n_cand, lw, parent, p_tok, reinterpret_cast<const unsigned long long *>(masks), c_draft, t_ar, t_exp,
+        admitted, order, n_admitted, reinterpret_cast<unsigned long long *>(union_out));
     return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
 }
 

@@ -1,0 +1,114 @@
+"""GPU parity of the adaptive-expansion calls (Sec. 4.1) against the oracle: bit-exact sets,
+admission flags and admission order on seeded synthetic draft trees."""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import expansion as ox
+
+pytestmark = pytest.mark.gpu
+
+
+def _masks_tensor(masks, words, dev):
+    n, L = len(masks), len(masks[0])
+    a = np.zeros((n, L, words), dtype=np.uint64)
+    for i in range(n):
+        for l in range(L):
+            for w in range(words):
+                a[i, l, w] = (masks[i][l] >> (64 * w)) & 0xFFFFFFFFFFFFFFFF
+    return torch.from_numpy(a.view(np.int64)).to(dev)
+
+
+def _tree(rng, n, n_layers, n_experts, k, reuse):
+    """Draft tree in heap-like order; a child's predicted experts are its parent's with a few
+    replaced (neighbouring draft tokens share experts), as in the paper's workloads."""
+    parent = [-1 if i == 0 or rng.random() < 0.1 else rng.randrange(i) for i in range(n)]
+    p_tok = [float(np.float32(rng.uniform(0.3, 1.0))) for _ in range(n)]
+    sets = []
+    for i in range(n):
+        cand = []
+        for l in range(n_layers):
+            if parent[i] >= 0 and rng.random() < reuse:
+                base = set(sets[parent[i]][l])
+                for _ in range(rng.randint(0, 2)):
+                    base.discard(rng.choice(sorted(base)))
+                while len(base) < k:
+                    base.add(rng.randrange(n_experts))
+            else:
+                base = set(rng.sample(range(n_experts), k))
+            cand.append(sorted(base))
+        sets.append(cand)
+    return parent, p_tok, sets
+
+
+@pytest.mark.parametrize("n,n_layers,n_experts,k", [(1, 1, 8, 2), (16, 4, 64, 8), (64, 16, 64, 6), (48, 3, 128, 8),
+                                                  (256, 2, 256, 4), (33, 26, 64, 6)])
+def test_expand_matches_oracle(n, n_layers, n_experts, k):
+    from paper_2608_15018_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    rng = random.Random(1000 * n + n_layers)
+    words = (n_experts + 63) // 64
+    for trial in range(4):
+        parent, p_tok, sets = _tree(rng, n, n_layers, n_experts, k, reuse=0.7)
+        masks = [[sum(1 << e for e in layer) for layer in cand] for cand in sets]
+        c_draft = [float(np.float32(rng.uniform(0.0, 0.05))) for _ in range(n)]
+        t_ar = float(np.float32(1.0))
+        t_exp = float(np.float32(rng.choice([0.01, 0.03, 0.1]) / n_layers))
+        want_adm, want_order, want_union = ox.adaptive_expand(parent, p_tok, masks, c_draft, t_ar, t_exp)
+
+        # the sets go through the library's own mask builder, layer by layer
+        out = torch.zeros((n, n_layers, words), dtype=torch.int64, device=dev)
+        for l in range(n_layers):
+            sel = torch.tensor([sets[i][l] for i in range(n)], dtype=torch.int32, device=dev)
+            binding.expert_masks(sel, n_experts, out=out, layer=l)
+        torch.cuda.synchronize()
+        assert torch.equal(out.cpu(), _masks_tensor(masks, words, "cpu"))
+
+        adm, order, n_adm, union = binding.adaptive_expand(
+            torch.tensor(parent, dtype=torch.int32, device=dev), torch.tensor(p_tok, dtype=torch.float32, device=dev),
+            out, n_experts, torch.tensor(c_draft, dtype=torch.float32, device=dev), t_ar, t_exp)
+        torch.cuda.synchronize()
+        assert adm.cpu().tolist() == want_adm
+        assert n_adm.item() == len(want_order)
+        assert order.cpu().tolist() == want_order + [-1] * (n - len(want_order))
+        got_union = union.cpu().numpy().view(np.uint64)
+        for l in range(n_layers):
+            assert sum(int(got_union[l, w]) << (64 * w) for w in range(words)) == want_union[l]
+
+
+def test_expand_ties_and_degenerate_cases():
+    from paper_2608_15018_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    # identical siblings: equal utilities, the lowest index goes first; zero cost: utility +inf
+    parent = [-1, -1, -1, 0]
+    p_tok = [0.5, 0.5, 0.5, 1.0]
+    masks = [[0b11], [0b11], [0b11], [0b11]]
+    for c, t_exp in (([0.25] * 4, 0.125), ([0.0] * 4, 0.0)):
+        want = ox.adaptive_expand(parent, p_tok, masks, c, 1.0, t_exp)
+        adm, order, n_adm, _ = binding.adaptive_expand(
+            torch.tensor(parent, dtype=torch.int32, device=dev), torch.tensor(p_tok, dtype=torch.float32, device=dev),
+            _masks_tensor(masks, 1, dev), 8, torch.tensor(c, dtype=torch.float32, device=dev), 1.0, t_exp)
+        assert adm.cpu().tolist() == want[0]
+        assert order.cpu().tolist()[: n_adm.item()] == want[1]
+    # nothing reaches utility 1
+    adm, order, n_adm, union = binding.adaptive_expand(
+        torch.tensor([-1, 0], dtype=torch.int32, device=dev), torch.tensor([0.5, 0.5], dtype=torch.float32, device=dev),
+        _masks_tensor([[1], [2]], 1, dev), 8, None, 0.0, 0.25)
+    assert n_adm.item() == 0 and adm.cpu().tolist() == [0, 0] and order.cpu().tolist() == [-1, -1]
+    assert union.cpu().tolist() == [[0]]
+
+
+def test_expand_argument_errors():
+    from paper_2608_15018_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    big = torch.zeros((257, 1, 1), dtype=torch.int64, device=dev)
+    with pytest.raises(binding.S2MoEError):
+        binding.adaptive_expand(torch.zeros(257, dtype=torch.int32, device=dev),
+                                torch.ones(257, dtype=torch.float32, device=dev), big, 8, None, 1.0, 0.1)
+    with pytest.raises(binding.S2MoEError):
+        binding.expert_masks(torch.zeros((2, 2), dtype=torch.int32, device=dev), 1000)
