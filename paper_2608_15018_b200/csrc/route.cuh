@@ -97,21 +97,35 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
         k1[j] = 0ull;
         if (e < E) { k1[j] = dkey(s_l[b * E + e]); valid |= 1u << j; }
     }
-    unsigned alive = valid;
     unsigned long long top1 = 0ull, kth = 0ull;
     const int rounds = bias_on ? k + 1 : 1;
+    if constexpr (J == 2) {
+        // two elements per lane: the lane offers its larger one and, once that has won a round,
+        // the other (a key of 0 = nothing left); a round is one reduction and one ballot
+        unsigned long long cur = k1[0] > k1[1] ? k1[0] : k1[1], nxt = k1[0] > k1[1] ? k1[1] : k1[0];
 #pragma unroll 1
-    for (int r = 0; r < rounds; ++r) {
-        unsigned long long lm = 0ull;
-        int bj = 0;
+        for (int r = 0; r < rounds; ++r) {
+            const unsigned hb = warp_max_holders(cur, cur != 0ull);
+            const int wl = __ffs(hb) - 1;
+            if (r == 0) top1 = shfl_key(cur, wl);
+            if (r == k) kth = shfl_key(cur, wl);
+            if (lane == wl) { cur = nxt; nxt = 0ull; }       // drop one instance of the maximum
+        }
+    } else {
+        unsigned alive = valid;
+#pragma unroll 1
+        for (int r = 0; r < rounds; ++r) {
+            unsigned long long lm = 0ull;
+            int bj = 0;
 #pragma unroll
-        for (int j = 0; j < J; ++j)
-            if (((alive >> j) & 1u) && k1[j] > lm) { lm = k1[j]; bj = j; }
-        const unsigned hb = warp_max_holders(lm, alive != 0u);
-        const int wl = __ffs(hb) - 1;
-        if (r == 0) top1 = shfl_key(lm, wl);
-        if (r == k) kth = shfl_key(lm, wl);
-        if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
+            for (int j = 0; j < J; ++j)
+                if (((alive >> j) & 1u) && k1[j] > lm) { lm = k1[j]; bj = j; }
+            const unsigned hb = warp_max_holders(lm, alive != 0u);
+            const int wl = __ffs(hb) - 1;
+            if (r == 0) top1 = shfl_key(lm, wl);
+            if (r == k) kth = shfl_key(lm, wl);
+            if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
+        }
     }
     GT_MARK(1);
     const double ztop = dkey_value(top1);
@@ -159,32 +173,58 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
             valid |= 1u << j;
         }
     }
-    unsigned alive = valid;
     GT_MARK(4);
+    if constexpr (J == 2) {
+        // the lane offers its better element first (order: l' descending, l descending, id
+        // ascending; element 0 has the lower id), then the other one
+        const bool first0 = k2[0] > k2[1] || (k2[0] == k2[1] && k1[0] >= k1[1]);
+        unsigned long long c2 = first0 ? k2[0] : k2[1], c1 = first0 ? k1[0] : k1[1];
+        unsigned long long n2 = first0 ? k2[1] : k2[0], n1 = first0 ? k1[1] : k1[0];
+        unsigned ce = (unsigned)lane + (first0 ? 0u : 32u), ne = (unsigned)lane + (first0 ? 32u : 0u);
 #pragma unroll 1
-    for (int r = 0; r < k; ++r) {
-        unsigned long long b2 = 0ull, b1 = 0ull;
-        int bj = -1;
+        for (int r = 0; r < k; ++r) {
+            unsigned hb = warp_max_holders(c2, c2 != 0ull);
+            if (__popc(hb) > 1) {                       // equal biased logits: larger original logit first
+                hb = warp_max_holders(c1, (hb >> lane) & 1u);
+                if (__popc(hb) > 1) {                   // still equal: lower expert id first
+                    const bool hold = (hb >> lane) & 1u;
+                    const unsigned me = __reduce_min_sync(full, hold ? ce : 0xffffffffu);
+                    hb = __ballot_sync(full, hold && ce == me);
+                }
+            }
+            if (lane == __ffs(hb) - 1) {
+                s_sel[b * k + r] = (int)ce;
+                c2 = n2; c1 = n1; ce = ne;
+                n2 = 0ull;
+            }
+        }
+    } else {
+        unsigned alive = valid;
+#pragma unroll 1
+        for (int r = 0; r < k; ++r) {
+            unsigned long long b2 = 0ull, b1 = 0ull;
+            int bj = -1;
 #pragma unroll
-        for (int j = 0; j < J; ++j) {
-            if ((alive >> j) & 1u) {
-                const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
-                if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
+            for (int j = 0; j < J; ++j) {
+                if ((alive >> j) & 1u) {
+                    const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
+                    if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
+                }
             }
-        }
-        const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
-        unsigned hb = warp_max_holders(b2, bj >= 0);
-        if (__popc(hb) > 1) {                           // equal biased logits: larger original logit first
-            hb = warp_max_holders(b1, (hb >> lane) & 1u);
-            if (__popc(hb) > 1) {                       // still equal: lower expert id first
-                const bool hold = (hb >> lane) & 1u;
-                const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
-                hb = __ballot_sync(full, hold && my_e == me);
+            const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
+            unsigned hb = warp_max_holders(b2, bj >= 0);
+            if (__popc(hb) > 1) {                           // equal biased logits: larger original logit first
+                hb = warp_max_holders(b1, (hb >> lane) & 1u);
+                if (__popc(hb) > 1) {                       // still equal: lower expert id first
+                    const bool hold = (hb >> lane) & 1u;
+                    const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
+                    hb = __ballot_sync(full, hold && my_e == me);
+                }
             }
-        }
-        if (lane == __ffs(hb) - 1) {
-            alive &= ~(1u << bj);
-            s_sel[b * k + r] = (int)my_e;
+            if (lane == __ffs(hb) - 1) {
+                alive &= ~(1u << bj);
+                s_sel[b * k + r] = (int)my_e;
+            }
         }
     }
     __syncwarp();
@@ -218,7 +258,9 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
         s_pw[b * k + lane] = (float)p;
         sel_idx[b * k + lane] = my_sel;
         sel_w[b * k + lane] = (float)p;
-        atomicOr(&s_mask[my_sel], 1ull << b);
+        // the token's bit in the expert's 64-bit mask: a native 32-bit shared-memory atomic on the
+        // half that holds it (a 64-bit atomicOr would be a compare-and-swap loop)
+        atomicOr(reinterpret_cast<unsigned *>(&s_mask[my_sel]) + (b >> 5), 1u << (b & 31));
     }
     GT_MARK(6);
 }
@@ -545,7 +587,20 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
 #ifdef S2MOE_TIMING
     if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[15] = t_start; tm[14] = clock64(); }
 #endif
+#ifdef S2MOE_GATE_TWICE
+    {   // experiment: the same gating a second time, with whatever the first run left in the caches
+        const long long g0 = clock64();
+        gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+        __syncthreads();
+        const long long g1 = clock64();
+        gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+        __syncthreads();
+        const long long g2 = clock64();
+        if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[30] = g1 - g0; tm[31] = g2 - g1; }
+    }
+#else
     gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+#endif
 }
 
 }  // namespace s2moe

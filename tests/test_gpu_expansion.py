@@ -112,3 +112,52 @@ def test_expand_argument_errors():
                                 torch.ones(257, dtype=torch.float32, device=dev), big, 8, None, 1.0, 0.1)
     with pytest.raises(binding.S2MoEError):
         binding.expert_masks(torch.zeros((2, 2), dtype=torch.int32, device=dev), 1000)
+
+
+def test_draft_pass_then_expansion_then_verification():
+    """Expert-sparse draft pass (k_draft experts, no bias) -> predicted expert sets -> adaptive
+    expansion -> the verification layer on the admitted tokens only (Sec. 4.1 and Sec. 5.1
+    "Draft Experts"), every stage against the oracle."""
+    import oracle
+    from gpu_util import run_case
+    from oracle import parity
+    from paper_2608_15018_b200 import binding, workloads
+
+    dev = torch.device("cuda", 0)
+    wl = workloads.CONFIGS["cfg5"].with_(d_model=512, d_ff=352, d_ff_shared=352, n_layers=3)
+    B, k_draft = 16, 3
+    draft = wl.with_(top_k=k_draft, alpha=0.0)
+    words = (wl.n_experts + 63) // 64
+    masks = torch.zeros((B, wl.n_layers, words), dtype=torch.int64, device=dev)
+    want_masks = []
+    H = [workloads.hidden_states(wl, l, B, device=dev) for l in range(wl.n_layers)]
+    T = [workloads.layer_weights(wl, l, dev) for l in range(wl.n_layers)]
+    with binding.S2MoE(binding.Config.from_workload(draft, n_layers=wl.n_layers), T) as m:
+        for l in range(wl.n_layers):
+            o = m.verify_layer(l, H[l], None)
+            binding.expert_masks(o.sel_idx, wl.n_experts, out=masks, layer=l)
+            torch.cuda.synchronize()
+            ocfg, ow = parity.from_workload(draft, T[l])
+            logits = oracle.router_logits(ocfg, workloads.raw_numpy(H[l]), ow.router)
+            g = oracle.gating(ocfg, logits, None)
+            # the draft selection is plain top-k: sets must agree unless the k-th margin is a tie
+            assert (np.sort(o.sel_idx.cpu().numpy(), axis=1) == np.sort(g.sel, axis=1)).all() or g.m_tok.min() < 1e-6
+            want_masks.append(ox.expert_masks(o.sel_idx.cpu().tolist()))
+    want_masks = [[want_masks[l][b] for l in range(wl.n_layers)] for b in range(B)]
+    parent = [workloads.tree_parent(i) if i else -1 for i in range(B)]
+    gen = torch.Generator().manual_seed(7)
+    p_tok = (0.4 + 0.6 * torch.rand(B, generator=gen)).to(torch.float32)
+    t_ar, t_exp = 1.0, float(np.float32(0.05))
+    c_draft = torch.full((B,), float(np.float32(0.1)), dtype=torch.float32)
+    want_adm, want_order, _ = ox.adaptive_expand(parent, p_tok.tolist(), want_masks, c_draft.tolist(), t_ar, t_exp)
+    adm, order, n_adm, _ = binding.adaptive_expand(torch.tensor(parent, dtype=torch.int32, device=dev), p_tok.to(dev),
+                                                   masks, wl.n_experts, c_draft.to(dev), t_ar, t_exp)
+    torch.cuda.synchronize()
+    assert adm.cpu().tolist() == want_adm and order.cpu().tolist()[: n_adm.item()] == want_order
+    assert 0 < n_adm.item() < B, "the case should prune something and keep something"
+    # verification of the admitted tokens only, with their prefix confidences as gating weights
+    keep = [i for i in range(B) if want_adm[i]]
+    conf = torch.tensor([ox.prefix_confidence(parent, p_tok.tolist())[i] for i in keep], dtype=torch.float32)
+    for l in range(wl.n_layers):
+        rep, out = run_case(wl, layer=l, hidden=H[l][keep], conf=conf.to(dev))
+        assert rep.tokens_checked == len(keep)
