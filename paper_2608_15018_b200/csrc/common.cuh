@@ -59,6 +59,8 @@ struct Workspace {
     int32_t *upfx1;        // [n_active + 1] first phase-1 stage of each active group
     int32_t *upfx2;        // [n_active + 1] first phase-2 stage of each active group
     unsigned long long *tokmask;   // [E + n_sh] bit b set: token b is bucketed to the group
+    uint4 *gtab;           // [n_active][2] {group, tokens, first slot, 0}, {mask lo, mask hi, 0, 0}: the
+                           // active groups in their final form, or NULL when nobody reads it
 };
 
 __device__ __forceinline__ size_t act_offset(int slot, int n_routed_slots, int f, int f_sh)

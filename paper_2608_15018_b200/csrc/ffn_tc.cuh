@@ -281,7 +281,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     // finished before its results are read; the next layer's routing kernel may be scheduled
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int n_active = ws.header[0], n_slots = ws.header[1];
+    const int n_active = ws.header[0];
+    const int n_slots = p.B * sh.k + sh.n_sh * p.B;          // every token fills k routed slots
     const int G = sh.E + sh.n_sh;
 
     StGroup *groups = reinterpret_cast<StGroup *>(tc_smem);
@@ -296,19 +297,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     const int U = ws.header[2];
     const int u1r = tc_units1(sh.f, sh.d), u2r = tc_units2(sh.f, sh.d);
     const int u1s = sh.n_sh ? tc_units1(sh.f_sh, sh.d) : 0, u2s = sh.n_sh ? tc_units2(sh.f_sh, sh.d) : 0;
-    for (int a = tid; a < n_active; a += blockDim.x) {
-        StGroup gr;
-        gr.group = ws.active[a];
-        gr.T = ws.counts[gr.group];
-        gr.off = ws.offsets[gr.group];
-        gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
-        gr.mask = ws.tokmask[gr.group];
-        const int r = a < U ? a : U, s = a < U ? 0 : a - U;
-        gr.p1 = r * u1r + s * u1s;
-        gr.p2 = r * u2r + s * u2s;
-        gr.nks = 0;
-        gr.ksl = 0;
-        groups[a] = gr;
+    // one round of global loads: the header above, the group table in its final form and the
+    // slot arrays, whose sizes are known without the header
+    for (int a = tid; a < G; a += blockDim.x) {
+        const uint4 r0 = ws.gtab[2 * a], r1 = ws.gtab[2 * a + 1];
+        if (a < n_active) {
+            StGroup gr;
+            gr.group = (int)r0.x;
+            gr.T = (int)r0.y;
+            gr.off = (int)r0.z;
+            gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
+            gr.mask = (unsigned long long)r1.x | ((unsigned long long)r1.y << 32);
+            const int r = a < U ? a : U, s = a < U ? 0 : a - U;
+            gr.p1 = r * u1r + s * u1s;
+            gr.p2 = r * u2r + s * u2s;
+            gr.nks = 0;
+            gr.ksl = 0;
+            groups[a] = gr;
+        }
     }
     for (int i = tid; i < n_slots; i += blockDim.x) {
         s_slot_token[i] = ws.slot_token[i];

@@ -388,7 +388,13 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     for (int e = tid; e < E; e += nt) {
         ws.counts[e] = s_cnt[e];
         ws.offsets[e] = s_off[e];
-        if (s_cnt[e] > 0) ws.active[s_pos[e]] = e;
+        if (s_cnt[e] > 0) {
+            ws.active[s_pos[e]] = e;
+            if (ws.gtab) {
+                ws.gtab[2 * s_pos[e]] = make_uint4((unsigned)e, (unsigned)s_cnt[e], (unsigned)s_off[e], 0u);
+                ws.gtab[2 * s_pos[e] + 1] = make_uint4((unsigned)s_mask[e], (unsigned)(s_mask[e] >> 32), 0u, 0u);
+            }
+        }
     }
     GATE_MARK();
     // bucket the (token, choice) pairs: tokens ascending inside an expert
@@ -413,6 +419,11 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             ws.counts[E + s] = B;
             ws.offsets[E + s] = n_routed + s * B;
             ws.active[U + s] = E + s;
+            if (ws.gtab) {
+                const unsigned long long all = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
+                ws.gtab[2 * (U + s)] = make_uint4((unsigned)(E + s), (unsigned)B, (unsigned)(n_routed + s * B), 0u);
+                ws.gtab[2 * (U + s) + 1] = make_uint4((unsigned)all, (unsigned)(all >> 32), 0u, 0u);
+            }
         }
     }
     GATE_MARK();

@@ -407,6 +407,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_ahi = take(2 * act_floats), o_alo = take(2 * act_floats);
     const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
     const size_t o_tm = take(8 * (size_t)G);
+    const size_t o_gtab = take(32 * (size_t)(G + 1));
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
@@ -435,6 +436,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ws.act = (float *)(base + o_act); ws.sync = (int32_t *)(base + o_sync);
     ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
     ws.tokmask = (unsigned long long *)(base + o_tm);
+    ws.gtab = (uint4 *)(base + o_gtab);
     ctx->pre = (float *)(base + o_pre);
     // plan 3: tensor maps of the weights (one set per layer); without the driver entry point or
     // for other formats the plan is simply not offered
