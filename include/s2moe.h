@@ -113,10 +113,14 @@ typedef struct {
     int32_t weight_mode;   /* 0: mixing weights from l, 1: from l'                          */
     int32_t max_tokens;    /* 1..S2MOE_MAX_TOKENS: workspace bound for n_tokens             */
     int32_t n_layers;      /* >= 1                                                          */
-    int32_t kernel_plan;   /* 0: automatic (plan 2 where it applies, else plan 1);
+    int32_t kernel_plan;   /* 0: automatic (plan 3 where it applies, else 2, else 1);
                               1: plain CUDA-core kernels (every format and batch size);
                               2: streaming mma.sync kernel (bf16 weights and activations);
-                              3: streaming tcgen05 kernel (bf16 weights and activations)      */
+                              3: streaming tcgen05 kernel: bf16 activations with bf16 weights,
+                                 or with block-int4 weights when d_model, d_ff and
+                                 d_ff_shared are multiples of 256 (the int4 values are
+                                 dequantised to bf16, scale rounded to bf16 first, on their
+                                 way to the tensor core: up to 2^-8 relative per weight)      */
 } s2moe_config;
 
 /*

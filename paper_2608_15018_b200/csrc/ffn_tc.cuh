@@ -42,6 +42,10 @@
 namespace s2moe {
 
 constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
+constexpr int kTcQ4Threads = kTcThreads + 256; // block-int4 weights: eight more warps that dequantise
+constexpr int kTcQ4Packed = 128 * 32;          // bytes of one packed weight k-tile (128 rows x 64 nibbles)
+constexpr int kTcQ4Scales = 128 * 16;          // 8 binary16 scales per row: the 256 columns of the tile's unit
+constexpr int kTcMaxAStages = 6;               // stages of dequantised bf16 weight tiles
 #ifndef S2MOE_MAX_STAGES
 #define S2MOE_MAX_STAGES 10
 #endif
@@ -71,6 +75,11 @@ struct TcPlan {
     int tab_bytes;
     int x_bytes;       // > 0: the hidden states stay resident in shared memory (all k-tiles)
     int smem_bytes;
+    int q4;            // block-int4 weights: packed tiles in the ring, dequantised into a second ring
+    int a_stages;      // stages of that second ring
+    int tok_off;       // offset of the token tiles inside a stage
+    int kg;            // k-tiles per stage (1 for bf16 weights; 1, 2 or 4 for int4)
+    int tokb;          // bytes of the token tiles of one k-tile
 };
 
 struct TcArgs {
@@ -105,8 +114,31 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.tmem_cols = 32;
     while (p.tmem_cols < 8 * p.n1) p.tmem_cols <<= 1;   // 2 buffers x 2 issuers x up to 2 * n1 columns
     p.smem_bytes = p.tab_bytes + p.x_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align to 1024
+    p.tok_off = kTcWTile;
+    p.kg = 1;
+    p.tokb = 2048 * ((B + 7) / 8);
     p.feasible = p.stages >= 4 && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
                  sh.d % 64 == 0;
+    if (sh.weight_dtype == DT_Q4B32) {
+        // a stage holds the packed k-tile, its unit's scales and the token tiles; the TMA copy of
+        // the scales wants rows of a multiple of 16 bytes, i.e. contraction lengths of 256
+        // A packed k-tile is only 4 KiB, so a stage carries up to four of them (a whole unit): one
+        // TMA copy, one hand-over to the tensor core and one release per stage instead of four.
+        p.q4 = 1;
+        p.x_bytes = 0;
+        const int budget = kTcMaxSmem - p.tab_bytes - 1024;
+        for (p.kg = 4; p.kg >= 1; p.kg >>= 1) {
+            p.tok_off = p.kg * kTcQ4Packed + kTcQ4Scales;
+            p.stage_bytes = (p.tok_off + p.kg * p.tokb + 1023) & ~1023;
+            p.a_stages = p.kg == 4 ? 2 : (p.kg == 2 ? 3 : kTcMaxAStages);
+            p.stages = (budget - p.a_stages * p.kg * kTcWTile) / p.stage_bytes;
+            if (p.stages >= 3 || p.kg == 1) break;
+        }
+        if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
+        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + p.a_stages * p.kg * kTcWTile + 1024;
+        p.feasible = p.stages >= 3 && B <= kMaxTokens && sh.act_dtype == DT_BF16 && sh.d % 256 == 0 &&
+                     sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
+    }
     return p;
 }
 
@@ -257,15 +289,20 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
 // tensor maps: 0 gate, 1 up, 2 down, 3 sh_gate, 4 sh_up, 5 sh_down, 6 hidden, 7 activations of the
 // routed slots, 8 of the shared slots: 3-D {k, slot, hi|lo}, so that one copy of box {64, 16, 2}
 // lands the hi tile and, right behind it, the lo tile of 16 slots
+// block-int4 weights: 0..5 are the packed matrices (bytes) with a box of one k-tile, 9..14 their
+// scales (binary16), 15..20 and 21..26 the packed matrices again with boxes of two and four k-tiles
 struct TcMaps {
-    CUtensorMap m[9];
+    CUtensorMap m[27];
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
+template <bool Q4>
+__global__ void __launch_bounds__(Q4 ? kTcQ4Threads : kTcThreads, 1)
+ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
     __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
+    __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
@@ -292,6 +329,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     uint8_t *xres = tc_smem + pl.tab_bytes;
     xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
     uint8_t *ring = xres + pl.x_bytes;
+    uint8_t *aring = ring + (size_t)pl.stages * pl.stage_bytes;      // int4 only; 1024-byte aligned
 
     // group table; stage prefixes follow from the active list alone (routed groups first)
     const int U = ws.header[2];
@@ -342,11 +380,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
     if (tid == 0) {
         for (int s = 0; s < pl.stages; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 2);      // one commit from each MMA issuer
+            mbar_init(&empty_bar[s], Q4 ? 10 : 2);     // one commit from each MMA issuer (+ the eight dequantising warps)
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 2);
             mbar_init(&acc_empty[b], 4);
+        }
+        if (Q4) {
+            for (int t = 0; t < pl.a_stages; ++t) {
+                mbar_init(&a_full[t], 8);
+                mbar_init(&a_empty[t], 2);
+            }
         }
         mbar_init(&ep_bar, 4);
         mbar_init(&x_bar, 1);
@@ -429,11 +473,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
                 pend_tn[kTcMaxStages];
             TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0, tp_x = 0, tp_unit = 0; const long long tp0 = clock64();)
+            const int KG = Q4 ? pl.kg : 1;               // k-tiles per stage
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
-                uint8_t *op = ring + (size_t)s * pl.stage_bytes + kTcWTile;
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
-                // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
-                for (int r = 0; r < tn / 2; r += 8) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
+                for (int g = 0; g < KG; ++g) {
+                    uint8_t *op = ring + (size_t)s * pl.stage_bytes + pl.tok_off + g * pl.tokb;
+                    // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
+                    for (int r = 0; r < tn / 2; r += 8)
+                        tma_load_3d(op + r * 256, am, (kt + g) * 64, srow + r, 0, &full_bar[s]);
+                }
             };
             auto wait_ready = [&](int w) -> bool {
                 TCT(long long c0 = clock64();)
@@ -477,7 +525,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     }
                 }
                 TCT(tp_unit += clock64() - cu;)
-                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
+                for (int kt = t.kt0; kt < t.kt1 && alive; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
                     if (!ready && pend_n == S) {
                         if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
                         ready = true;
@@ -491,12 +539,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 128u;
-                    mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
-                    tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
+                    if (Q4) {
+                        // packed k-tiles (32 bytes of every row each) and the 8 scales per row of
+                        // the 256 columns they lie in (x in scales; kt0 is a multiple of 4)
+                        const int mi = (shared ? 3 : 0) + t.mat;
+                        const CUtensorMap *pm = &maps.m[KG == 1 ? mi : (KG == 2 ? 15 + mi : 21 + mi)];
+                        mbar_expect_tx(&full_bar[s], KG * kTcQ4Packed + kTcQ4Scales + KG * op_bytes);
+                        tma_load_2d_stream(stage, pm, kt * 32, row0, &full_bar[s], wpolicy);
+                        tma_load_2d(stage + KG * kTcQ4Packed, &maps.m[9 + mi], (kt & ~3) * 2, row0, &full_bar[s]);
+                    } else {
+                        mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
+                        tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
+                    }
                     if (t.phase == 1) {
-                        uint8_t *op = stage + kTcWTile;
                         if (!pl.x_bytes)
-                            for (int r = 0; r < t.n; r += 16) tma_load_2d(op + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
+                            for (int g = 0; g < KG; ++g) {
+                                uint8_t *op = stage + pl.tok_off + g * pl.tokb;
+                                for (int r = 0; r < t.n; r += 16)
+                                    tma_load_2d(op + r * 128, &maps.m[6], (kt + g) * 64, r, &full_bar[s]);
+                            }
                     } else if (ready) {
                         load_tokens2(s, kt, srow, shared, t.n);
                     } else {
@@ -524,6 +585,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             bool alive = true;
             int s = 0;
             uint32_t ring_par = 0;
+            int ta = 0;                                  // int4: slot and parity of the dequantised-tile ring
+            uint32_t a_par = 0;
             if (pl.x_bytes && half == 0) {
                 // all token tiles of the hidden states, once (this thread has nothing to issue before they land)
                 mbar_expect_tx(&x_bar, (uint32_t)pl.x_bytes);
@@ -553,9 +616,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                 // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
-                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
+                const int KG = Q4 ? pl.kg : 1;           // k-tiles per stage
+                for (int kt = t.kt0; kt < t.kt1; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
                     if (!mbar_wait(&full_bar[s], ring_par)) {
+                        atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                        alive = false;
+                        break;
+                    }
+                    if (Q4 && !mbar_wait(&a_full[ta], a_par)) {      // the k-tile as bf16, written by the dequantising warps
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
@@ -563,19 +632,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
                     TCT(long long c2 = clock64(); tm_full += c2 - c1;)
                     tc_fence_after();
                     const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
-                    const uint64_t ad = tc_smem_desc(stage);
-                    const uint64_t bd = (t.phase == 1 && pl.x_bytes) ? tc_smem_desc(xres + (size_t)kt * pl.n1 * 128)
-                                                                     : tc_smem_desc(stage + kTcWTile);
 #if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
+                    for (int g = 0; g < KG; ++g) {
+                        const uint64_t ad = tc_smem_desc(Q4 ? aring + ((size_t)ta * KG + g) * kTcWTile : stage);
+                        const uint64_t bd = (t.phase == 1 && pl.x_bytes) ? tc_smem_desc(xres + (size_t)kt * pl.n1 * 128)
+                                                                         : tc_smem_desc(stage + pl.tok_off + g * pl.tokb);
 #pragma unroll
-                    for (int k = 2 * half; k < 2 * half + 2; ++k) {   // K = 16 steps inside the 64-wide tile: +32 bytes each
-                        tc_mma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, acc);
-                        acc = 1;
+                        for (int k = 2 * half; k < 2 * half + 2; ++k) {   // K = 16 steps inside the 64-wide tile: +32 bytes each
+                            tc_mma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, acc);
+                            acc = 1;
+                        }
                     }
 #else
+                    const uint64_t ad = 0, bd = 0;
                     (void)ad; (void)bd; (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
 #endif
                     tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
+                    if (Q4) {
+                        tc_commit(&a_empty[ta]);
+                        tc_ring_next(ta, a_par, pl.a_stages);
+                    }
                     TCT(tm_mma += clock64() - c2;)
                 }
                 if (alive && t.last) {
@@ -585,6 +661,79 @@ __global__ void __launch_bounds__(kTcThreads, 1) ffn_tc_kernel(const __grid_cons
             }
             TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; })
         }
+    } else if (Q4 && warp >= 11) {
+        // ------------------------------------------------------------------ dequantising warps (int4)
+        // Every row of a packed k-tile (64 nibbles, stored q + 8) becomes 64 bf16 values q * scale
+        // in the 128-byte-swizzled layout the tensor core reads: per 32-bit word eight
+        // nibbles -> (128 + n) as bf16 by an OR into the mantissa, minus 136 (exact), times the
+        // block's scale rounded to bf16.  Scales that lie past the matrix read as 0 (TMA fill), so
+        // a ragged last tile contributes nothing.
+        // A stage holds KG k-tiles: per row 2 * KG chunks of 16 packed bytes (32 weights, one
+        // scale each).  Thread (r, h) of the 256 takes row r and chunks h * KG .. h * KG + KG - 1.
+        const int r = (tid - 352) & 127, h = (tid - 352) >> 7;
+        const int KG = pl.kg;
+        int s = 0, ta = 0;
+        uint32_t ring_par = 0, a_par = 1;
+        bool alive = true;
+        const __nv_bfloat162 minus136 = __floats2bfloat162_rn(-136.0f, -136.0f);
+        TCT(long long td_full = 0, td_aempty = 0, td_work = 0, td_fence = 0;)
+        for (int ui = 0; ui < n_units && alive; ++ui) {
+            const TcUnit t = unit_at(ui);
+            for (int kt = t.kt0; kt < t.kt1; kt += KG, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
+                TCT(const long long d0 = clock64();)
+                const bool ok_full = mbar_wait(&full_bar[s], ring_par);
+                TCT(const long long d1 = clock64(); td_full += d1 - d0;)
+                if (!ok_full || !mbar_wait(&a_empty[ta], a_par)) {
+                    if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                    alive = false;
+                    break;
+                }
+                TCT(const long long d2 = clock64(); td_aempty += d2 - d1;)
+                const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
+                const uint8_t *prow = stage + (size_t)r * (32 * KG);
+                const unsigned short *srow = reinterpret_cast<const unsigned short *>(stage + KG * kTcQ4Packed + r * 16) + (kt & 3) * 2;
+                uint8_t *atile = aring + (size_t)ta * KG * kTcWTile + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll 2
+                for (int qi = 0; qi < KG; ++qi) {
+                    const int q = h * KG + qi;                         // chunk of 32 weights inside the stage
+                    // the packed rows are swizzled over their own width by the TMA copy
+                    const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
+                    const uint4 pk = *reinterpret_cast<const uint4 *>(prow + ((q ^ sw) * 16));
+                    const float sf = __half2float(__ushort_as_half(srow[q]));
+                    const __nv_bfloat162 sc2 = __floats2bfloat162_rn(sf, sf);
+                    uint8_t *arow = atile + (size_t)(q >> 1) * kTcWTile;    // k-tile q / 2, its chunks 4 * (q % 2) ..
+                    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t m = 0x000F000Fu, one28 = 0x43004300u;       // bf16 128.0 twice
+                        const uint32_t x04 = (w[c] & m) | one28, x15 = ((w[c] >> 4) & m) | one28;
+                        const uint32_t x26 = ((w[c] >> 8) & m) | one28, x37 = ((w[c] >> 12) & m) | one28;
+                        uint32_t e[4] = {__byte_perm(x04, x15, 0x5410), __byte_perm(x26, x37, 0x5410),
+                                         __byte_perm(x04, x15, 0x7632), __byte_perm(x26, x37, 0x7632)};
+                        uint4 o;
+                        uint32_t *ov = reinterpret_cast<uint32_t *>(&o);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const __nv_bfloat162 v = __hmul2(__hadd2(*reinterpret_cast<const __nv_bfloat162 *>(&e[j]), minus136), sc2);
+                            ov[j] = *reinterpret_cast<const uint32_t *>(&v);
+                        }
+                        const int cc = 4 * (q & 1) + c;                 // 16-byte chunk of the bf16 row
+                        *reinterpret_cast<uint4 *>(arow + ((cc ^ (r & 7)) * 16)) = o;
+                    }
+                }
+                TCT(const long long d3 = clock64(); td_work += d3 - d2;)
+                // the tensor core reads these through the async proxy (shared memory only: the fence
+                // over all state spaces costs about a thousand cycles)
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&a_full[ta]);
+                    mbar_arrive(&empty_bar[s]);        // the packed tiles have been read
+                }
+                TCT(td_fence += clock64() - d3;)
+            }
+        }
+        TCT(if (tid == 352) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 12; o[0] = td_full; o[1] = td_aempty; o[2] = td_work; o[3] = td_fence; })
     } else if (warp == 10) {
         // ------------------------------------------------------------------ watcher
         // polls the waves' second counters (all CTAs have written their slice of the activations)

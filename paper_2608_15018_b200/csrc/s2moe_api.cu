@@ -110,8 +110,9 @@ int validate_config(const s2moe_config *c)
     if (c->max_tokens < 1 || c->max_tokens > S2MOE_MAX_TOKENS) return S2MOE_EINVAL;
     if (c->n_layers < 1) return S2MOE_EINVAL;
     if (c->kernel_plan < 0 || c->kernel_plan > 3) return S2MOE_EINVAL;
-    if (c->kernel_plan == 3 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
-    // the streaming plan covers bf16 weights with bf16 activations
+    // the tcgen05 plan covers bf16 activations with bf16 or block-int4 weights
+    if (c->kernel_plan == 3 && (c->weight_dtype == S2MOE_F32 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
+    // the mma.sync plan covers bf16 weights with bf16 activations
     if (c->kernel_plan == 2 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     return S2MOE_OK;
 }
@@ -260,6 +261,29 @@ bool make_map(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t
                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D tensor of `elem_bytes`-wide elements [rows][cols], box = box_cols x 128 rows (packed int4
+// weights as bytes, their scales as 16-bit words); out-of-range elements read as zero.  Byte boxes
+// of 32, 64 or 128 bytes are swizzled over their own width, so that threads which each read one
+// 16-byte chunk of consecutive rows do not meet in the same shared-memory banks.
+bool make_map_plain(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                    uint32_t box_cols, int elem_bytes)
+{
+    if (!ctx->encode_tiled || !base || rows == 0) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+    const cuuint32_t box[2] = {box_cols, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16,
+                                              2, const_cast<void *>(base), dims, strides, box, estr,
+                                              CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              elem_bytes != 1   ? CU_TENSOR_MAP_SWIZZLE_NONE
+                                              : box_cols == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                              : box_cols == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                                : CU_TENSOR_MAP_SWIZZLE_32B,
+                                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 3-D bf16 tensor {cols, rows, 2}: the hi array and, `plane_bytes` further, the lo array of the
 // activations; box = 64 columns x 8 rows x both planes
 bool make_map_hilo(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
@@ -330,8 +354,9 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
         a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
         LaunchScope scope(ctx, KC_TC, st);
-        cudaLaunchConfig_t lc = pdl_config(ctx, tp.n_cta, kTcThreads, tp.smem_bytes, st);
-        cudaLaunchKernelEx(&lc, ffn_tc_kernel, maps, a);
+        cudaLaunchConfig_t lc = pdl_config(ctx, tp.n_cta, tp.q4 ? kTcQ4Threads : kTcThreads, tp.smem_bytes, st);
+        if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true>, maps, a);
+        else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false>, maps, a);
     } else if (plan == 2) {
         StreamArgs a;
         a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
@@ -440,18 +465,56 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ctx->pre = (float *)(base + o_pre);
     // plan 3: tensor maps of the weights (one set per layer); without the driver entry point or
     // for other formats the plan is simply not offered
-    if (ctx->plan != 1 && ctx->plan != 2 && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16) {
+    if (ctx->plan != 1 && ctx->plan != 2 && (sh.weight_dtype == DT_BF16 || sh.weight_dtype == DT_Q4B32) &&
+        sh.act_dtype == DT_BF16) {
         cudaDriverEntryPointQueryResult qres;
         void *fn = nullptr;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess && fn) {
             ctx->encode_tiled = fn;
             ctx->tc_maps.resize(config->n_layers);
-            bool ok = cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
+            const bool q4 = sh.weight_dtype == DT_Q4B32;
+            bool ok = cudaFuncSetAttribute(ffn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(ffn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
+            // the int4 variant needs contraction lengths that are multiples of 256 (see tc_make_plan)
+            if (q4 && (sh.d % 256 || sh.f % 256 || (sh.n_sh && sh.f_sh % 256))) ok = false;
             for (int l = 0; l < config->n_layers && ok; ++l) {
                 const LayerPtrs &lp = ctx->layers[l];
                 TcMaps &m = ctx->tc_maps[l];
                 std::memset(&m, 0, sizeof(m));
+                if (q4) {
+                    const uint64_t Ef = (uint64_t)sh.E * sh.f, Ed = (uint64_t)sh.E * sh.d;
+                    ok = make_map_plain(ctx, &m.m[0], lp.w_gate, Ef, (uint64_t)sh.d / 2, 32, 1) &&
+                         make_map_plain(ctx, &m.m[1], lp.w_up, Ef, (uint64_t)sh.d / 2, 32, 1) &&
+                         make_map_plain(ctx, &m.m[2], lp.w_down, Ed, (uint64_t)sh.f / 2, 32, 1) &&
+                         make_map_plain(ctx, &m.m[9], lp.s_gate, Ef, (uint64_t)sh.d / 32, 8, 2) &&
+                         make_map_plain(ctx, &m.m[10], lp.s_up, Ef, (uint64_t)sh.d / 32, 8, 2) &&
+                         make_map_plain(ctx, &m.m[11], lp.s_down, Ed, (uint64_t)sh.f / 32, 8, 2);
+                    // the packed matrices again with boxes of two and of four k-tiles
+                    for (int j = 1; j <= 2 && ok; ++j) {
+                        const int base = 15 + 6 * (j - 1);
+                        const uint32_t bc = 32u << j;
+                        ok = make_map_plain(ctx, &m.m[base + 0], lp.w_gate, Ef, (uint64_t)sh.d / 2, bc, 1) &&
+                             make_map_plain(ctx, &m.m[base + 1], lp.w_up, Ef, (uint64_t)sh.d / 2, bc, 1) &&
+                             make_map_plain(ctx, &m.m[base + 2], lp.w_down, Ed, (uint64_t)sh.f / 2, bc, 1);
+                        if (ok && sh.n_sh) {
+                            const uint64_t Sf = (uint64_t)sh.n_sh * sh.f_sh, Sd = (uint64_t)sh.n_sh * sh.d;
+                            ok = make_map_plain(ctx, &m.m[base + 3], lp.sh_gate, Sf, (uint64_t)sh.d / 2, bc, 1) &&
+                                 make_map_plain(ctx, &m.m[base + 4], lp.sh_up, Sf, (uint64_t)sh.d / 2, bc, 1) &&
+                                 make_map_plain(ctx, &m.m[base + 5], lp.sh_down, Sd, (uint64_t)sh.f_sh / 2, bc, 1);
+                        }
+                    }
+                    if (ok && sh.n_sh) {
+                        const uint64_t Sf = (uint64_t)sh.n_sh * sh.f_sh, Sd = (uint64_t)sh.n_sh * sh.d;
+                        ok = make_map_plain(ctx, &m.m[3], lp.sh_gate, Sf, (uint64_t)sh.d / 2, 32, 1) &&
+                             make_map_plain(ctx, &m.m[4], lp.sh_up, Sf, (uint64_t)sh.d / 2, 32, 1) &&
+                             make_map_plain(ctx, &m.m[5], lp.sh_down, Sd, (uint64_t)sh.f_sh / 2, 32, 1) &&
+                             make_map_plain(ctx, &m.m[12], lp.sh_s_gate, Sf, (uint64_t)sh.d / 32, 8, 2) &&
+                             make_map_plain(ctx, &m.m[13], lp.sh_s_up, Sf, (uint64_t)sh.d / 32, 8, 2) &&
+                             make_map_plain(ctx, &m.m[14], lp.sh_s_down, Sd, (uint64_t)sh.f_sh / 32, 8, 2);
+                    }
+                    continue;
+                }
                 ok = make_map(ctx, &m.m[0], lp.w_gate, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
                      make_map(ctx, &m.m[1], lp.w_up, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
                      make_map(ctx, &m.m[2], lp.w_down, (uint64_t)sh.E * sh.d, (uint64_t)sh.f, 128);

@@ -9,8 +9,16 @@ TOL = {workloads.F32: 2e-3, workloads.BF16: 2e-3, workloads.Q4B32: 1e-2}
 
 
 def supports(wl, plan):
-    """Kernel plans 2 and 3 (streaming tensor-core kernels) cover bf16 weights with bf16 activations."""
-    return plan not in (2, 3) or (wl.weight_dtype == workloads.BF16 and wl.act_dtype == workloads.BF16)
+    """Kernel plan 2 (mma.sync) covers bf16 weights with bf16 activations; plan 3 (tcgen05) also
+    block-int4 weights whose contraction lengths are multiples of 256."""
+    if plan not in (2, 3):
+        return True
+    if wl.act_dtype != workloads.BF16:
+        return False
+    if wl.weight_dtype == workloads.BF16:
+        return True
+    q4_ok = wl.d_model % 256 == 0 and wl.d_ff % 256 == 0 and (wl.n_shared == 0 or wl.d_ff_shared % 256 == 0)
+    return plan == 3 and wl.weight_dtype == workloads.Q4B32 and q4_ok
 
 
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,

@@ -203,3 +203,23 @@ def test_reuse_aware_gating_lowers_unique_experts_on_average():
     u0 = m0.verify_stack(H, C).n_unique.float().mean().item()
     assert u1 <= u0
     m0.close(); m1.close()
+
+
+Q4_TC = CONFIGS["cfg4"].with_(d_model=1024, d_ff=1792)      # contraction lengths that are multiples of 256
+
+
+@pytest.mark.parametrize("B", [1, 2, 4, 8, 16, 32, 64])
+def test_q4_tensor_core_plan(B):
+    """Block-int4 weights on the tcgen05 kernel (packed tiles dequantised to bf16 in shared memory)."""
+    for layer in range(2):
+        rep, _ = run_case(Q4_TC, layer=layer, n_tokens=B, plan=3)
+        assert rep is not None and rep.plan == 3 and rep.tokens_checked == B
+
+
+def test_q4_tensor_core_plan_with_shared_experts_and_variants():
+    wl = CONFIGS["cfg3"].with_(d_model=512, d_ff=768, d_ff_shared=1280, weight_dtype=CONFIGS["cfg4"].weight_dtype)
+    rep, _ = run_case(wl, plan=3)
+    assert rep is not None and rep.plan == 3
+    rep, _ = run_case(Q4_TC.with_(renorm=0, weight_mode=1, alpha=1.0), plan=3, use_conf=False)
+    assert rep is not None and rep.plan == 3
+
