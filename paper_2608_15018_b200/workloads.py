@@ -75,6 +75,11 @@ CONFIGS: Dict[str, Workload] = {
     "cfg5": Workload("cfg5-dsv2lite-bf16", 2048, 1408, 64, 6, 26, 16, "tree", 0.3, 4,
                      n_shared=2, d_ff_shared=1408, cap=16),
 }
+# 128-expert shapes of Table 1 (cap 14 and 6 as listed there): token masks and expert sets span
+# two 64-bit words, the routing kernel holds four experts per lane.  Fewer layers than the models
+# have, so that a stack stays within tens of GB.
+CONFIGS["e128a"] = Workload("e128a-qwen3moe-like-bf16", 2048, 768, 128, 8, 12, 8, "chain", 0.5, 5, renorm=1, cap=14)
+CONFIGS["e128b"] = Workload("e128b-gptoss-like-bf16", 2880, 2880, 128, 4, 4, 8, "chain", 0.5, 6, renorm=1, cap=6)
 CFG4_BATCHES = (1, 2, 4, 8, 16, 32)
 CFG5_TREES = (1, 2, 4, 8, 16, 32, 64)
 CFG5_SIGMAS = (0.1, 0.2, 0.3, 0.5, 0.7, 1.0)

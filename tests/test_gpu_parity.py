@@ -223,3 +223,14 @@ def test_q4_tensor_core_plan_with_shared_experts_and_variants():
     rep, _ = run_case(Q4_TC.with_(renorm=0, weight_mode=1, alpha=1.0), plan=3, use_conf=False)
     assert rep is not None and rep.plan == 3
 
+
+@pytest.mark.parametrize("name", ["e128a", "e128b"])
+@pytest.mark.parametrize("plan", [1, 3])
+def test_128_expert_shapes(name, plan):
+    """The 128-expert families of Table 1 at reduced width: two-word expert sets, four experts per
+    lane in the gating, ragged row blocks (d_ff = 352 is not a multiple of 128)."""
+    wl = CONFIGS[name].with_(d_model=512, d_ff=352 if name == "e128b" else 256)
+    for B in (8, 33):
+        rep, _ = run_case(wl, n_tokens=B, plan=plan)
+        assert rep is not None and rep.tokens_checked == B
+
