@@ -708,8 +708,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         const uint32_t m = 0x000F000Fu, one28 = 0x43004300u;       // bf16 128.0 twice
                         const uint32_t x04 = (w[c] & m) | one28, x15 = ((w[c] >> 4) & m) | one28;
                         const uint32_t x26 = ((w[c] >> 8) & m) | one28, x37 = ((w[c] >> 12) & m) | one28;
-                        uint32_t e[4] = {__byte_perm(x04, x15, 0x5410), __byte_perm(x26, x37, 0x5410),
-                                         __byte_perm(x04, x15, 0x7632), __byte_perm(x26, x37, 0x7632)};
+                        // (n0, n4), (n1, n5), (n2, n6), (n3, n7): the token tiles carry the same
+                        // permutation of every 8 columns, so no instruction is spent on reordering
+                        uint32_t e[4] = {x04, x15, x26, x37};
                         uint4 o;
                         uint32_t *ov = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
@@ -795,11 +796,21 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
                 const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
                 const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
-                uint2 hv, lv;
-                hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
-                lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
-                *reinterpret_cast<uint2 *>(p.act_hi + i) = hv;
-                *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
+                if (Q4) {
+                    // columns i .. i + 3 of their group of 8 go to positions 0, 2, 4, 6 (first half of
+                    // the group) or 1, 3, 5, 7 (second half): the order the dequantised weights are in
+                    const long long g8 = i & ~7ll;
+                    const int odd = (int)((i >> 2) & 1);
+                    __nv_bfloat16 *ph = p.act_hi + g8 + odd, *pq = p.act_lo + g8 + odd;
+                    ph[0] = __low2bfloat16(h01); ph[2] = __high2bfloat16(h01); ph[4] = __low2bfloat16(h23); ph[6] = __high2bfloat16(h23);
+                    pq[0] = __low2bfloat16(l01); pq[2] = __high2bfloat16(l01); pq[4] = __low2bfloat16(l23); pq[6] = __high2bfloat16(l23);
+                } else {
+                    uint2 hv, lv;
+                    hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+                    lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+                    *reinterpret_cast<uint2 *>(p.act_hi + i) = hv;
+                    *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
+                }
             }
             __threadfence();
             fence_proxy_async();

@@ -504,6 +504,12 @@ constexpr int kRouteTok = 16;   // most tokens accumulated per pass
 struct ZeroList {
     void *ptr[3];
     unsigned long long n16[3];
+    // int4 tensor-core path: a copy of the bf16 hidden states whose columns are permuted inside
+    // every group of 8 (position p holds column [0,4,1,5,2,6,3,7][p]), the order in which the
+    // dequantising warps of the FFN kernel get the nibbles of a 32-bit word for free
+    const uint4 *perm_src;
+    uint4 *perm_dst;
+    unsigned long long perm_n16;
 };
 
 // One pass of a router row over NT tokens b0 .. b0 + NT - 1 (indices past B - 1 repeat token
@@ -573,6 +579,12 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
         for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.n16[z];
              i += (unsigned long long)gridDim.x * kRouteThreads)
             p[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.perm_n16;
+         i += (unsigned long long)gridDim.x * kRouteThreads) {
+        const uint4 v = zl.perm_src[i];             // halves h0..h7
+        zl.perm_dst[i] = make_uint4(__byte_perm(v.x, v.z, 0x5410), __byte_perm(v.x, v.z, 0x7632),
+                                    __byte_perm(v.y, v.w, 0x5410), __byte_perm(v.y, v.w, 0x7632));
     }
     const int row = blockIdx.x, d = sh.d;
     const size_t rb = RT == DT_F32 ? 4 : 2;

@@ -37,6 +37,7 @@ struct s2moe_ctx {
     size_t act_elems = 0;
     cudaLaunchAttribute pdl_attr{};
     bool use_pdl = true;                  // S2MOE_NO_PDL=1 in the environment turns it off
+    void *hperm = nullptr;                // int4 plan 3: column-permuted copy of the hidden states
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
@@ -338,6 +339,11 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         zl.n16[1] = used * 2 * sizeof(float) / 16;
         zl.ptr[2] = ctx->ws.sync + (kTcReady - 8);      // the hand-over counters of the two waves
         zl.n16[2] = 8 * sizeof(int32_t) / 16;
+        if (sh.weight_dtype == DT_Q4B32) {
+            zl.perm_src = (const uint4 *)hidden;
+            zl.perm_dst = (uint4 *)ctx->hperm;
+            zl.perm_n16 = (size_t)B * sh.d * 2 / 16;
+        }
     }
     launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
     if (plan == 3) {
@@ -345,7 +351,7 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         TcMaps maps = ctx->tc_maps[layer];
         const size_t n_routed = (size_t)B * sh.k;
         const uint64_t plane = (uint64_t)((const uint8_t *)ctx->act_lo - (const uint8_t *)ctx->act_hi);
-        bool ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
+        bool ok = make_map(ctx, &maps.m[6], tp.q4 ? ctx->hperm : hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
                   make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
         if (ok && sh.n_sh)
             ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
@@ -433,6 +439,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
     const size_t o_tm = take(8 * (size_t)G);
     const size_t o_gtab = take(32 * (size_t)(G + 1));
+    const size_t o_hperm = take(sh.weight_dtype == DT_Q4B32 ? 2 * (size_t)T * sh.d : 0);
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
@@ -462,6 +469,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
     ws.tokmask = (unsigned long long *)(base + o_tm);
     ws.gtab = (uint4 *)(base + o_gtab);
+    ctx->hperm = base + o_hperm;
     ctx->pre = (float *)(base + o_pre);
     // plan 3: tensor maps of the weights (one set per layer); without the driver entry point or
     // for other formats the plan is simply not offered
