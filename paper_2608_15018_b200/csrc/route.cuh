@@ -586,6 +586,10 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
         zl.perm_dst[i] = make_uint4(__byte_perm(v.x, v.z, 0x5410), __byte_perm(v.x, v.z, 0x7632),
                                     __byte_perm(v.y, v.w, 0x5410), __byte_perm(v.y, v.w, 0x7632));
     }
+    // blocks past the router's rows exist only to help with the clearing and the copy above (a
+    // layer with few experts and wide accumulators would otherwise clear megabytes with a few blocks)
+    const int n_rows = sh.E + (sh_scale ? 1 : 0);
+    if ((int)blockIdx.x >= n_rows) return;
     const int row = blockIdx.x, d = sh.d;
     const size_t rb = RT == DT_F32 ? 4 : 2;
     const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
@@ -601,7 +605,7 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     __syncthreads();
     if (tid == 0) {
         const unsigned t = atomicAdd(ws.ticket, 1u);
-        s_last = (t == gridDim.x - 1);
+        s_last = (t == (unsigned)n_rows - 1);
     }
     __syncthreads();
     if (!s_last) return;

@@ -175,9 +175,18 @@ template <int ACT, int RT>
 void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
                     int32_t *sel_idx, float *sel_w, int32_t *n_unique, const ZeroList &zl, cudaStream_t st)
 {
+    // one block per router row; more (up to one per SM) when there is a lot to clear or copy:
+    // 16 bytes per thread and pass, a handful of passes at most
     const int rows = sh.E + (lp.sh_scale ? 1 : 0);
+    const unsigned long long units = zl.n16[0] + zl.n16[1] + zl.n16[2] + zl.perm_n16;
+    int grid = rows;
+    if (units > (unsigned long long)rows * kRouteThreads * 4) {
+        const unsigned long long want = (units + kRouteThreads * 4 - 1) / (kRouteThreads * 4);
+        grid = (int)(want > (unsigned long long)ctx->n_sm ? (unsigned long long)ctx->n_sm : want);
+        if (grid < rows) grid = rows;
+    }
     LaunchScope scope(ctx, KC_ROUTER, st);
-    cudaLaunchConfig_t lc = pdl_config(ctx, rows, kRouteThreads, route_smem(B, sh.E), st);
+    cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st);
     cudaLaunchKernelEx(&lc, route_kernel<ACT, RT>, sh, B, ctx->ws, hidden, (const void *)lp.router,
                        (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
 }
