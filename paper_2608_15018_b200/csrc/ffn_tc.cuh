@@ -377,26 +377,26 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         s_ready[0] = 0;
         s_ready[1] = 0;
     }
-    if (tid == 0) {
-        for (int s = 0; s < pl.stages; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], Q4 ? 10 : 2);     // one commit from each MMA issuer (+ the eight dequantising warps)
+    if (warp == 2) {
+        // barrier set-up, spread over a warp so that it runs beside the table loads of the others
+        if (lane < pl.stages) {
+            mbar_init(&full_bar[lane], 1);
+            mbar_init(&empty_bar[lane], Q4 ? 10 : 2);   // one commit from each MMA issuer (+ the eight dequantising warps)
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 2);
-            mbar_init(&acc_empty[b], 4);
+        if (lane < 2) {
+            mbar_init(&acc_full[lane], 2);
+            mbar_init(&acc_empty[lane], 4);
+            mbar_init(&conv_go[lane], 4);
         }
-        if (Q4) {
-            for (int t = 0; t < pl.a_stages; ++t) {
-                mbar_init(&a_full[t], 8);
-                mbar_init(&a_empty[t], 2);
-            }
+        if (Q4 && lane < pl.a_stages) {
+            mbar_init(&a_full[lane], 8);
+            mbar_init(&a_empty[lane], 2);
         }
-        mbar_init(&ep_bar, 4);
-        mbar_init(&x_bar, 1);
-        mbar_init(&cv_bar, 3);
-        mbar_init(&conv_go[0], 4);
-        mbar_init(&conv_go[1], 4);
+        if (lane == 0) {
+            mbar_init(&ep_bar, 4);
+            mbar_init(&x_bar, 1);
+            mbar_init(&cv_bar, 3);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -425,10 +425,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         int rot = 0;
         auto share = [&](int begin, int n, int &start, int &cnt) {
             const int q = n / P, r = n - q * P;
-            const int c = ((int)blockIdx.x + P - rot) % P;
+            int c = (int)blockIdx.x - rot;               // (blockIdx.x - rot) mod P without a division:
+            if (c < 0) c += P;                           // the four calls would otherwise chain four of them
             cnt = q + (c < r ? 1 : 0);
             start = begin + c * q + min(c, r);
-            rot = (rot + r) % P;
+            rot += r;
+            if (rot >= P) rot -= P;
         };
         share(0, split1, my_start0, my_cnt0);
         share(split1, total1 - split1, my_start1, my_cnt1);
