@@ -11,6 +11,10 @@ by least squares and reports R^2 and the mean absolute percentage error, the two
 paper quotes for its own calibration.
 
     python -m paper_2608_15018_b200.calibrate [--workload cfg5] [--layers 26] [--json out.json]
+    python -m paper_2608_15018_b200.calibrate --workload cfg2 --top-k 2 --alpha 0     # draft pass
+
+With --top-k and --alpha 0 the same measurement gives the cost of the expert-sparse draft pass
+(Sec. 5.1, "Draft Experts"), the C^draft of the utility.
 
 Every layer has its own weights, so consecutive timed layers never re-read cached weights.
 """
@@ -77,9 +81,15 @@ def main(argv=None) -> int:
     ap.add_argument("--layers", type=int, default=0, help="layers of the stack (default: the workload's)")
     ap.add_argument("--batches", default="1,2,4,8,16,32,64")
     ap.add_argument("--sigmas", default="0.1,0.2,0.3,0.5,0.7,1.0")
+    ap.add_argument("--top-k", type=int, default=0, help="override top-k (e.g. the draft pass: fewer experts per token)")
+    ap.add_argument("--alpha", type=float, default=-1.0, help="override alpha (0 = plain top-k gating, as in the draft pass)")
     ap.add_argument("--json", default="")
     args = ap.parse_args(argv)
     wl = workloads.CONFIGS[args.workload]
+    if args.top_k:
+        wl = wl.with_(top_k=args.top_k, cap=max(args.top_k, min(wl.cap, wl.n_experts)))
+    if args.alpha >= 0.0:
+        wl = wl.with_(alpha=args.alpha)
     n_layers = args.layers or wl.n_layers
     batches = [int(x) for x in args.batches.split(",")]
     sigmas = [float(x) for x in args.sigmas.split(",")]
