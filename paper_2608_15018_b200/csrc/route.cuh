@@ -600,16 +600,16 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
         else if (left > 4) { route_pass<ACT, RT, 8>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 8; }
         else { route_pass<ACT, RT, 4>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 4; }
     }
-    // the block that arrives last sees every row (release by fence + ticket, acquire by fence)
-    __threadfence();
-    __syncthreads();
+    // the block that arrives last sees every row: the ticket is taken with release and acquire
+    // semantics by one thread, and the barriers on both sides of it (the one that ends the last
+    // pass, the one below) extend that to the block's other threads
     if (tid == 0) {
-        const unsigned t = atomicAdd(ws.ticket, 1u);
+        unsigned t;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(t) : "l"(ws.ticket) : "memory");
         s_last = (t == (unsigned)n_rows - 1);
     }
     __syncthreads();
     if (!s_last) return;
-    __threadfence();
     if (tid == 0) *ws.ticket = 0u;
 #ifdef S2MOE_TIMING
     if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[15] = t_start; tm[14] = clock64(); }
