@@ -243,6 +243,12 @@ __device__ __forceinline__ bool tc_bar(uint64_t *bar, uint32_t &phase, int lane)
     return ok;
 }
 
+// counter += 1 with release semantics at GPU scope (one instruction instead of fence + atomic)
+__device__ __forceinline__ void tc_red_release(int32_t *counter)
+{
+    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(counter) : "memory");
+}
+
 // next slot of the ring; the parity flips on wrap-around
 __device__ __forceinline__ void tc_ring_next(int &s, uint32_t &parity, int S)
 {
@@ -496,7 +502,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 TCT(tp_ready += clock64() - c0;)
                 if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); return false; }
                 __threadfence_block();
-                fence_proxy_async();
+                asm volatile("fence.proxy.async.global;" ::: "memory");
                 for (int i = 0; i < pend_n; ++i) load_tokens2(pend_stage[i], pend_kt[i], pend_row[i], pend_shared[i], pend_tn[i]);
                 pend_n = 0;
                 ready_w = w + 1;
@@ -814,10 +820,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
                 }
             }
-            __threadfence();
-            fence_proxy_async();
+            // the activations are read by TMA copies of other CTAs: proxy fence over global memory by
+            // every writer, then one release at GPU scope behind the barrier of the converter warps
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
-            if (et == 0) { atomicAdd(&ws.sync[kTcReady - 4 + w], 1); TCG(23 + w); }
+            if (et == 0) { tc_red_release(&ws.sync[kTcReady - 4 + w]); TCG(23 + w); }
             TCT(te_conv += clock64() - c3;)
             return true;
         };
@@ -831,10 +838,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 __nanosleep(64);
             }
             if (!ok) { if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
-            if (et == 0) {
-                __threadfence();                     // the CTA's reductions, observed through conv_go
-                atomicAdd(&ws.sync[kTcReady - 8 + w], 1);
-            }
+            if (et == 0) tc_red_release(&ws.sync[kTcReady - 8 + w]);   // orders the CTA's reductions, observed through conv_go
             if (!wave_convert(w)) break;
         }
 #endif
