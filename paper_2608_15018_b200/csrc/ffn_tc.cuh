@@ -19,10 +19,17 @@
 // consecutive k-pieces of a row block accumulate in TMEM and are reduced to memory once.
 //
 // Warp roles (352 threads): warp 0 = TMA producer; warps 1 and 6 = MMA issuers (warp 1 owns the
-// TMEM allocation); warps 2..5 = epilogue (TMEM -> registers -> red.add); warps 7..10 =
-// converters.  A ring of stages, each one weight k-tile (128 x 64 bf16 = 16 KiB) plus, in phase
-// 2, the matching token k-tiles; accumulators are double-buffered in TMEM.  tcgen05.mma:
-// M = 128 weight rows, N = tokens padded to 16, K = 16 per instruction, fp32 accumulate.
+// TMEM allocation); warps 2..5 = epilogue (TMEM -> registers -> red.add); warps 7..9 = converters;
+// warp 10 = watcher (polls the waves' second counters and publishes them in shared memory, so
+// that the producer never waits on global memory).  A ring of stages, each one weight k-tile
+// (128 x 64 bf16 = 16 KiB) plus the matching token k-tiles (phase 1: hidden states; phase 2: per
+// 8 slots their hi rows and, right behind, their lo rows); accumulators are double-buffered in
+// TMEM.  tcgen05.mma: M = 128 weight rows, N = 16 per 16 tokens (phase 1) or per 8 hi + lo slots
+// (phase 2), K = 16 per instruction, fp32 accumulate.
+//
+// Block-int4 weights (template parameter): the ring holds packed tiles, up to a whole unit per
+// stage, and eight more warps dequantise every stage into a second ring of bf16 tiles that the
+// MMA issuers read; see the dequantising branch below.
 #pragma once
 
 #include <cuda.h>
