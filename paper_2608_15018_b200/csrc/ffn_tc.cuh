@@ -27,9 +27,11 @@
 // TMEM.  tcgen05.mma: M = 128 weight rows, N = 16 per 16 tokens (phase 1) or per 8 hi + lo slots
 // (phase 2), K = 16 per instruction, fp32 accumulate.
 //
-// Block-int4 weights (template parameter): the ring holds packed tiles, up to a whole unit per
-// stage, and eight more warps dequantise every stage into a second ring of bf16 tiles that the
-// MMA issuers read; see the dequantising branch below.
+// Block-int4 weights (template parameter): the ring holds packed tiles and scales, up to a whole
+// unit per stage, and eight more warps dequantise every stage into a second ring of bf16 tiles that
+// the MMA issuers read (four of them where the accumulators fit); the token tiles of a stage are
+// fetched into a slot of that second ring, so a packed stage is free as soon as it has been read.
+// See the producer's int4 branch and the dequantising branch below.
 #pragma once
 
 #include <cuda.h>
@@ -49,7 +51,7 @@
 namespace s2moe {
 
 constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
-constexpr int kTcQ4Threads = kTcThreads + 256; // block-int4 weights: eight more warps that dequantise
+constexpr int kTcQ4Threads = kTcThreads + 256 + 64;   // block-int4 weights: eight more warps that dequantise, two more MMA issuers
 constexpr int kTcQ4Packed = 128 * 32;          // bytes of one packed weight k-tile (128 rows x 64 nibbles)
 constexpr int kTcQ4Scales = 128 * 16;          // 8 binary16 scales per row: the 256 columns of the tile's unit
 constexpr int kTcMaxAStages = 6;               // stages of dequantised bf16 weight tiles
@@ -79,6 +81,7 @@ struct TcPlan {
     int stage_bytes;   // weight tile + token tiles, multiple of 1024
     int n1;            // tokens padded to 16 (phase-1 N)
     int tmem_cols;     // power of two >= 32
+    int n_iss;         // MMA issuer warps (2, or 4 on the int4 path when the accumulators fit)
     int tab_bytes;
     int x_bytes;       // > 0: the hidden states stay resident in shared memory (all k-tiles)
     int smem_bytes;
@@ -118,6 +121,7 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     if ((kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes < kTcMaxStages) p.x_bytes = 0;
     p.stages = (kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes;
     if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
+    p.n_iss = 2;
     p.tmem_cols = 32;
     while (p.tmem_cols < 8 * p.n1) p.tmem_cols <<= 1;   // 2 buffers x 2 issuers x up to 2 * n1 columns
     p.smem_bytes = p.tab_bytes + p.x_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align to 1024
@@ -133,16 +137,26 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
         // TMA copy, one hand-over to the tensor core and one release per stage instead of four.
         p.q4 = 1;
         p.x_bytes = 0;
+        // the stage of an int4 unit is cheap to fetch, so the issue of its 16 MMAs is what has to
+        // keep up: four issuers where their accumulators fit into the 512 TMEM columns
+        if (16 * p.n1 <= 512) {
+            p.n_iss = 4;
+            while (p.tmem_cols < 16 * p.n1) p.tmem_cols <<= 1;
+        }
         const int budget = kTcMaxSmem - p.tab_bytes - 1024;
+        // The token tiles of a stage do not travel with its packed tiles: they are fetched into a
+        // slot that belongs to the ring of dequantised tiles, just before they are used, so that a
+        // stage is free again as soon as the dequantising warps have read it (its life decides
+        // how many bytes are in flight) and not only when the MMAs have completed.
         for (p.kg = 4; p.kg >= 1; p.kg >>= 1) {
             p.tok_off = p.kg * kTcQ4Packed + kTcQ4Scales;
-            p.stage_bytes = (p.tok_off + p.kg * p.tokb + 1023) & ~1023;
+            p.stage_bytes = (p.tok_off + 1023) & ~1023;
             p.a_stages = p.kg == 4 ? 2 : (p.kg == 2 ? 3 : kTcMaxAStages);
-            p.stages = (budget - p.a_stages * p.kg * kTcWTile) / p.stage_bytes;
+            p.stages = (budget - p.a_stages * p.kg * (kTcWTile + p.tokb)) / p.stage_bytes;
             if (p.stages >= 3 || p.kg == 1) break;
         }
         if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
-        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + p.a_stages * p.kg * kTcWTile + 1024;
+        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + p.a_stages * p.kg * (kTcWTile + p.tokb) + 1024;
         p.feasible = p.stages >= 3 && B <= kMaxTokens && sh.act_dtype == DT_BF16 && sh.d % 256 == 0 &&
                      sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
     }
@@ -187,6 +201,26 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, i
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, int x, int y, int z, int w, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
+// non-blocking test of a phase (a thread that serves two rings polls both)
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
@@ -204,6 +238,25 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
         "}\n" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// The same with the two descriptors given as their 32-bit halves: the shared-memory address sits in
+// the low 14 bits of the low word (in units of 16 bytes), so stepping from tile to tile is one
+// 32-bit add.  The issuing thread shares its scheduler with busy warps, and every instruction it
+// needs per MMA delays the MMA.
+__device__ __forceinline__ void tc_mma_bf16_parts(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                  uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, {%7, %7, %7, %7}, p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(0u)
         : "memory");
 }
 __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8])
@@ -233,6 +286,12 @@ __device__ __forceinline__ uint64_t tc_smem_desc(const void *p)
 {
     const uint64_t addr = (uint64_t)((smem_u32(p) >> 4) & 0x3FFFu);
     return addr | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// the same with 8-row groups `sbo` bytes apart
+__device__ __forceinline__ uint64_t tc_smem_desc_sbo(const void *p, uint32_t sbo)
+{
+    const uint64_t addr = (uint64_t)((smem_u32(p) >> 4) & 0x3FFFu);
+    return addr | (1ull << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 __device__ __forceinline__ uint32_t tc_idesc(int n)
 {
@@ -303,7 +362,10 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
 // routed slots, 8 of the shared slots: 3-D {k, slot, hi|lo}, so that one copy of box {64, 16, 2}
 // lands the hi tile and, right behind it, the lo tile of 16 slots
 // block-int4 weights: 0..5 are the packed matrices (bytes) with a box of one k-tile, 9..14 their
-// scales (binary16), 15..20 and 21..26 the packed matrices again with boxes of two and four k-tiles
+// scales (binary16), 15..20 and 21..26 the packed matrices again with boxes of two and four k-tiles;
+// 6 is the (column-permuted) hidden states as {k in tile, row, k-tile} with a box of all rows x kg
+// k-tiles, 7 and 8 the activations as {k in tile, slot, k-tile, hi|lo} with a box {64, 8, kg, 2}:
+// one copy per stage (per 8 slots) instead of one per k-tile
 struct TcMaps {
     CUtensorMap m[27];
 };
@@ -316,6 +378,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
     __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
     __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
+    __shared__ __align__(8) uint64_t tok_full[kTcMaxAStages];                          // int4: the token tiles used with them
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
@@ -325,6 +388,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
     const TcPlan &pl = p.plan;
+    const int NI = Q4 ? p.plan.n_iss : 2;          // MMA issuers: a compile-time 2 on the bf16 path
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     TCT(const long long t_entry = clock64(); unsigned long long g_entry; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_entry));)
     // programmatic dependent launch: the routing kernel in front of this grid must have
@@ -343,6 +407,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
     uint8_t *ring = xres + pl.x_bytes;
     uint8_t *aring = ring + (size_t)pl.stages * pl.stage_bytes;      // int4 only; 1024-byte aligned
+    uint8_t *tokring = aring + (size_t)pl.a_stages * pl.kg * kTcWTile;   // int4 only: token tiles, one slot per slot of aring
 
     // group table; stage prefixes follow from the active list alone (routed groups first)
     const int U = ws.header[2];
@@ -394,16 +459,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // barrier set-up, spread over a warp so that it runs beside the table loads of the others
         if (lane < pl.stages) {
             mbar_init(&full_bar[lane], 1);
-            mbar_init(&empty_bar[lane], Q4 ? 10 : 2);   // one commit from each MMA issuer (+ the eight dequantising warps)
+            mbar_init(&empty_bar[lane], Q4 ? 8 : NI);   // one commit from each MMA issuer; int4: the eight dequantising warps
         }
         if (lane < 2) {
-            mbar_init(&acc_full[lane], 2);
+            mbar_init(&acc_full[lane], NI);
             mbar_init(&acc_empty[lane], 4);
             mbar_init(&conv_go[lane], 4);
         }
         if (Q4 && lane < pl.a_stages) {
             mbar_init(&a_full[lane], 8);
-            mbar_init(&a_empty[lane], 2);
+            mbar_init(&a_empty[lane], NI);
+            mbar_init(&tok_full[lane], 1);
         }
         if (lane == 0) {
             mbar_init(&ep_bar, 4);
@@ -474,7 +540,87 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     if (warp == 0) {
         const uint64_t wpolicy = l2_evict_first_policy();
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (Q4 && lane == 0) {
+            // int4: two cursors over the same sequence of stages.  The packed tiles and scales go
+            // into the stage ring (a slot is free once the dequantising warps have read it); the
+            // token tiles go into the slot of the dequantised-tile ring they are used with (free
+            // once the MMAs that read it have completed), and in the second projection only when
+            // their wave's activations are written.  One thread serves both, so it polls.
+            const int KG = pl.kg;
+            const int n_routed = p.B * sh.k;
+            int pi = 0, ti = 0;                          // unit of each cursor
+            TcUnit pu = unit_at(0), tu = pu;
+            int pkt = pu.kt0, tkt = pu.kt0;
+            int s = 0, ta = 0;
+            uint32_t ring_par = 1, t_par = 1;
+            int ready_w = 0;
+            unsigned idle = 0;
+            bool alive = n_units > 0;
+            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
+            while (alive && (pi < n_units || ti < n_units)) {
+                bool progress = false;
+                if (pi < n_units && mbar_test(&empty_bar[s], ring_par)) {
+                    TCT(const long long c2 = clock64();)
+                    const StGroup &g = groups[pu.a];
+                    const bool shared = g.group >= sh.E;
+                    const int e = shared ? g.group - sh.E : g.group;
+                    const int row0 = e * (pu.mat == 2 ? sh.d : g.f) + pu.rb * 128;
+                    // packed k-tiles (32 bytes of every row each) and the 8 scales per row of the 256
+                    // columns they lie in (x in scales; kt0 is a multiple of 4)
+                    const int mi = (shared ? 3 : 0) + pu.mat;
+                    const CUtensorMap *pm = &maps.m[KG == 1 ? mi : (KG == 2 ? 15 + mi : 21 + mi)];
+                    uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
+                    mbar_expect_tx(&full_bar[s], KG * kTcQ4Packed + kTcQ4Scales);
+                    tma_load_2d_stream(stage, pm, pkt * 32, row0, &full_bar[s], wpolicy);
+                    tma_load_2d(stage + KG * kTcQ4Packed, &maps.m[9 + mi], (pkt & ~3) * 2, row0, &full_bar[s]);
+                    tc_ring_next(s, ring_par, S);
+                    pkt += KG;
+                    if (pkt >= pu.kt1 && ++pi < n_units) { pu = unit_at(pi); pkt = pu.kt0; }
+                    progress = true;
+                    TCT(tp_issue += clock64() - c2;)
+                }
+                if (ti < n_units) {
+                    const int wv = tu.a >= a_split ? 1 : 0;
+                    bool ready = tu.phase == 1 || wv < ready_w;
+                    if (!ready && s_ready[wv]) {
+                        // the activations of this wave are written: order them before the copies below
+                        __threadfence_block();
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        ready_w = wv + 1;
+                        ready = true;
+                    }
+                    if (ready && mbar_test(&a_empty[ta], t_par)) {
+                        TCT(const long long c2 = clock64();)
+                        uint8_t *op = tokring + (size_t)ta * KG * pl.tokb;
+                        if (tu.phase == 1) {
+                            // the hidden-state tiles of all KG k-tiles in one copy: [k-tile][tokb / 128 rows]
+                            mbar_expect_tx(&tok_full[ta], (uint32_t)(KG * pl.tokb));
+                            tma_load_3d(op, &maps.m[6], 0, 0, tkt, &tok_full[ta]);
+                        } else {
+                            // one copy per 8 slots for all KG k-tiles: [hi | lo][k-tile][8 rows]
+                            const StGroup &g = groups[tu.a];
+                            const bool shared = g.group >= sh.E;
+                            const int srow = shared ? g.off - n_routed : g.off;
+                            mbar_expect_tx(&tok_full[ta], (uint32_t)(KG * tu.n * 128));
+                            for (int r = 0; r < tu.n / 2; r += 8)
+                                tma_load_4d(op + r * 256 * KG, &maps.m[shared ? 8 : 7], 0, srow + r, tkt, 0, &tok_full[ta]);
+                        }
+                        tc_ring_next(ta, t_par, pl.a_stages);
+                        tkt += KG;
+                        if (tkt >= tu.kt1 && ++ti < n_units) { tu = unit_at(ti); tkt = tu.kt0; }
+                        progress = true;
+                        TCT(tp_ready += clock64() - c2;)
+                    }
+                }
+                if (progress) {
+                    idle = 0;
+                } else if (++idle > (kTcSpinLimit << 4)) {
+                    atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                    alive = false;
+                }
+            }
+            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry;)
+        } else if (lane == 0) {
             unsigned it = 0;
             bool alive = true;
 #if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
@@ -488,15 +634,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
                 pend_tn[kTcMaxStages];
             TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0, tp_x = 0, tp_unit = 0; const long long tp0 = clock64();)
-            const int KG = Q4 ? pl.kg : 1;               // k-tiles per stage
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
-                for (int g = 0; g < KG; ++g) {
-                    uint8_t *op = ring + (size_t)s * pl.stage_bytes + pl.tok_off + g * pl.tokb;
-                    // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
-                    for (int r = 0; r < tn / 2; r += 8)
-                        tma_load_3d(op + r * 256, am, (kt + g) * 64, srow + r, 0, &full_bar[s]);
-                }
+                uint8_t *op = ring + (size_t)s * pl.stage_bytes + pl.tok_off;
+                // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
+                for (int r = 0; r < tn / 2; r += 8) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
             auto wait_ready = [&](int w) -> bool {
                 TCT(long long c0 = clock64();)
@@ -540,7 +682,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     }
                 }
                 TCT(tp_unit += clock64() - cu;)
-                for (int kt = t.kt0; kt < t.kt1 && alive; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
+                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     if (!ready && pend_n == S) {
                         if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
                         ready = true;
@@ -554,25 +696,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 128u;
-                    if (Q4) {
-                        // packed k-tiles (32 bytes of every row each) and the 8 scales per row of
-                        // the 256 columns they lie in (x in scales; kt0 is a multiple of 4)
-                        const int mi = (shared ? 3 : 0) + t.mat;
-                        const CUtensorMap *pm = &maps.m[KG == 1 ? mi : (KG == 2 ? 15 + mi : 21 + mi)];
-                        mbar_expect_tx(&full_bar[s], KG * kTcQ4Packed + kTcQ4Scales + KG * op_bytes);
-                        tma_load_2d_stream(stage, pm, kt * 32, row0, &full_bar[s], wpolicy);
-                        tma_load_2d(stage + KG * kTcQ4Packed, &maps.m[9 + mi], (kt & ~3) * 2, row0, &full_bar[s]);
-                    } else {
-                        mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
-                        tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
-                    }
+                    mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
+                    tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
                     if (t.phase == 1) {
                         if (!pl.x_bytes)
-                            for (int g = 0; g < KG; ++g) {
-                                uint8_t *op = stage + pl.tok_off + g * pl.tokb;
-                                for (int r = 0; r < t.n; r += 16)
-                                    tma_load_2d(op + r * 128, &maps.m[6], (kt + g) * 64, r, &full_bar[s]);
-                            }
+                            for (int r = 0; r < t.n; r += 16)
+                                tma_load_2d(stage + pl.tok_off + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
                     } else if (ready) {
                         load_tokens2(s, kt, srow, shared, t.n);
                     } else {
@@ -585,16 +714,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 }
             }
             if (alive && pend_n > 0) wait_ready(pend_wave);
-            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry; o[5] = tp_x; o[6] = tp_unit;)
+            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry; (void)tp_x; (void)tp_unit;)
         }
-    } else if (warp == 1 || warp == 6) {
+    } else if (warp == 1 || warp == 6 || (Q4 && warp >= 19)) {
         // ------------------------------------------------------------------ MMA issuers
-        // Issuing one tcgen05.mma costs a thread on the order of 100 cycles whatever its shape, and
-        // with N = 16 every instruction covers only 4 KiB of weights, so two warps share the work:
-        // issuer h takes K-steps 2h and 2h + 1 of every k-tile and accumulates into its own TMEM
-        // columns; the epilogue adds the two partial accumulators.
-        const int half = warp == 1 ? 0 : 1;
-        if (lane == 0) {
+        // Issuing one tcgen05 instruction (an MMA or a commit) costs a thread on the order of 150
+        // cycles whatever its shape, and with N = 16 every MMA covers only 4 KiB of weights, so
+        // several warps share the work: with two issuers, issuer h takes K-steps 2h and 2h + 1 of
+        // every k-tile, with four (int4 path) K-step h; each accumulates into its own TMEM columns
+        // and the epilogue adds the partial accumulators.
+        const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - 17);
+        if (lane == 0 && half < NI) {
             unsigned it = 0, ui = 0, run = 0;
             uint32_t acc = 0;
             bool alive = true;
@@ -613,7 +743,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 alive = false;
             }
-            TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0; const long long tm0 = clock64();)
+            // descriptor halves (see tc_mma_bf16_parts); K-step k of a 64-wide tile lies 32 bytes further
+            const uint32_t ks = 4u / (uint32_t)NI, koff = 2u * ks * (uint32_t)half;
+            const uint32_t hi_std = (uint32_t)(tc_smem_desc(ring) >> 32);
+            const uint32_t hi_p2 = Q4 ? (uint32_t)(tc_smem_desc_sbo(ring, (uint32_t)pl.kg * 1024u) >> 32) : hi_std;
+            const uint32_t ring_lo = (uint32_t)tc_smem_desc(ring) + koff, xres_lo = (uint32_t)tc_smem_desc(xres) + koff;
+            const uint32_t aring_lo = (uint32_t)tc_smem_desc(aring) + koff, tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
+            TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0, tm_fence = 0, tm_mmas = 0; const long long tm0 = clock64();)
             for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
                 const int buf = run & 1;
@@ -627,45 +763,53 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     tc_fence_after();
                     acc = 0;
                 }
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 4 * pl.n1 + half * 2 * pl.n1);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * NI * pl.n1 + half * 2 * pl.n1);
                 // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
                 const int KG = Q4 ? pl.kg : 1;           // k-tiles per stage
                 for (int kt = t.kt0; kt < t.kt1; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
-                    if (!mbar_wait(&full_bar[s], ring_par)) {
-                        atomicExch(ws.status, ST_MBAR_TIMEOUT);
-                        alive = false;
-                        break;
-                    }
-                    if (Q4 && !mbar_wait(&a_full[ta], a_par)) {      // the k-tile as bf16, written by the dequantising warps
+                    // bf16: the stage; int4: the k-tiles as bf16, written by the dequantising warps, and their token tiles
+                    if (Q4 ? !(mbar_wait(&a_full[ta], a_par) && mbar_wait(&tok_full[ta], a_par)) : !mbar_wait(&full_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
                     }
                     TCT(long long c2 = clock64(); tm_full += c2 - c1;)
                     tc_fence_after();
-                    const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
+                    TCT(const long long c3 = clock64(); tm_fence += c3 - c2;)
 #if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
-                    for (int g = 0; g < KG; ++g) {
-                        const uint64_t ad = tc_smem_desc(Q4 ? aring + ((size_t)ta * KG + g) * kTcWTile : stage);
-                        const uint64_t bd = (t.phase == 1 && pl.x_bytes) ? tc_smem_desc(xres + (size_t)kt * pl.n1 * 128)
-                                                                         : tc_smem_desc(stage + pl.tok_off + g * pl.tokb);
-#pragma unroll
-                        for (int k = 2 * half; k < 2 * half + 2; ++k) {   // K = 16 steps inside the 64-wide tile: +32 bytes each
-                            tc_mma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, acc);
+                    if (Q4) {
+                        // dequantised k-tiles of slot ta (16 KiB apart) and their token tiles: phase 1
+                        // [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row groups KG KiB apart)
+                        uint32_t a_lo = aring_lo + (uint32_t)(ta * KG) * (kTcWTile >> 4);
+                        uint32_t b_lo = tok_lo + (uint32_t)(ta * KG) * ((uint32_t)pl.tokb >> 4);
+                        const uint32_t b_step = t.phase == 1 ? (uint32_t)pl.tokb >> 4 : 64u, b_hi = t.phase == 1 ? hi_std : hi_p2;
+                        for (int g = 0; g < KG; ++g, a_lo += kTcWTile >> 4, b_lo += b_step) {
+                            for (uint32_t k = 0; k < ks; ++k) {
+                                tc_mma_bf16_parts(d_tmem, a_lo + 2 * k, hi_std, b_lo + 2 * k, b_hi, idesc, acc);
+                                acc = 1;
+                            }
+                        }
+                    } else {
+                        const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
+                        const uint32_t b_lo = (t.phase == 1 && pl.x_bytes) ? xres_lo + (uint32_t)kt * ((uint32_t)pl.n1 * 8u)
+                                                                           : a_lo + ((uint32_t)pl.tok_off >> 4);
+                        for (uint32_t k = 0; k < ks; ++k) {       // K = 16 steps inside the 64-wide tile: +32 bytes each
+                            tc_mma_bf16_parts(d_tmem, a_lo + 2 * k, hi_std, b_lo + 2 * k, hi_std, idesc, acc);
                             acc = 1;
                         }
                     }
 #else
-                    const uint64_t ad = 0, bd = 0;
-                    (void)ad; (void)bd; (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
+                    (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
 #endif
-                    tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
+                    TCT(const long long c4 = clock64(); tm_mmas += c4 - c3;)
                     if (Q4) {
-                        tc_commit(&a_empty[ta]);
+                        tc_commit(&a_empty[ta]);       // frees the dequantised tiles and the token tiles
                         tc_ring_next(ta, a_par, pl.a_stages);
+                    } else {
+                        tc_commit(&empty_bar[s]);      // frees the stage when these MMAs have read it
                     }
                     TCT(tm_mma += clock64() - c2;)
                 }
@@ -674,7 +818,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     ++run;
                 }
             }
-            TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; })
+            TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; o[-3] = tm_fence; o[-2] = tm_mmas;   /* slots 5, 6 */ })
         }
     } else if (Q4 && warp >= 11) {
         // ------------------------------------------------------------------ dequantising warps (int4)
@@ -909,8 +1053,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 #endif
                 {
                 const int row = t.rb * 128 + q * 32 + lane;           // row of the matrix inside the expert
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 4 * pl.n1);
-                const uint32_t other = (uint32_t)(2 * pl.n1);      // the second issuer's partial accumulator
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * NI * pl.n1);
+                const uint32_t other = (uint32_t)(2 * pl.n1);      // the next issuer's partial accumulator
                 if (t.phase == 1) {
                     const bool row_ok = row < g.f;
                     // slot of the expert's i-th token = g.off + i; walk its tokens in ascending order
@@ -919,9 +1063,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     for (int c = 0; c < t.n; c += 16) {
                         float v[16], v2[16];
                         tc_ld16(taddr + c, v);
-                        tc_ld16(taddr + other + c, v2);
+                        for (int h = 1; h < NI; ++h) {
+                            tc_ld16(taddr + h * other + c, v2);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] += v2[i];
+                            for (int i = 0; i < 16; ++i) v[i] += v2[i];
+                        }
                         const unsigned m16 = (unsigned)((g.mask >> c) & 0xffffull);
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
@@ -936,14 +1082,18 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     for (int c = 0; c < t.n; c += 16) {
                         float v[16], v2[16];                      // columns: 8 hi, 8 lo of slots c / 2 .. c / 2 + 7
                         tc_ld16(taddr + c, v);
-                        tc_ld16(taddr + other + c, v2);
+                        for (int h = 1; h < NI; ++h) {
+                            tc_ld16(taddr + h * other + c, v2);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] += v2[i];
+                        }
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const int ti = (c >> 1) + i;
                             if (ti < g.T && row_ok) {
                                 const int slot = g.off + ti;
                                 atomicAdd(&p.y[(size_t)s_slot_token[slot] * sh.d + row],
-                                          s_slot_w[slot] * ((v[i] + v2[i]) + (v[i + 8] + v2[i + 8])));
+                                          s_slot_w[slot] * (v[i] + v[i + 8]));
                             }
                         }
                     }

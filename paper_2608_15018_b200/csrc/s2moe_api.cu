@@ -310,6 +310,38 @@ bool make_map_hilo(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uin
                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// int4 path: the hidden states as {64 columns, rows, k-tiles of 64 columns}, box = 64 x box_rows x kg:
+// the token tiles of kg consecutive k-tiles in one copy, each tile box_rows x 128 bytes
+bool make_map_ktiles(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                     uint32_t box_rows, uint32_t kg)
+{
+    if (!ctx->encode_tiled || !base || rows == 0 || cols % 64) return false;
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {cols * 2, 128};
+    const cuuint32_t box[3] = {64, box_rows, kg};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// int4 path: the activations as {64 columns, rows, k-tiles, hi / lo}, box = 64 x 8 x kg x 2: per copy
+// the hi rows of 8 slots for kg k-tiles and, behind them, their lo rows
+bool make_map_hilo_ktiles(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
+                          uint64_t plane_bytes, uint32_t kg)
+{
+    if (!ctx->encode_tiled || !base || rows == 0 || cols % 64) return false;
+    const cuuint64_t dims[4] = {64, rows, cols / 64, 2};
+    const cuuint64_t strides[3] = {cols * 2, 128, plane_bytes};
+    const cuuint32_t box[4] = {64, 8, kg, 2};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The plan a batch of B tokens runs with: the streaming kernel when it is allowed and its
 // shared-memory layout fits, else the CUDA-core kernels; 0 when plan 2 was demanded and does not fit.
 int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
@@ -360,10 +392,19 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         TcMaps maps = ctx->tc_maps[layer];
         const size_t n_routed = (size_t)B * sh.k;
         const uint64_t plane = (uint64_t)((const uint8_t *)ctx->act_lo - (const uint8_t *)ctx->act_hi);
-        bool ok = make_map(ctx, &maps.m[6], tp.q4 ? ctx->hperm : hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
-                  make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
-        if (ok && sh.n_sh)
-            ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
+        bool ok;
+        if (tp.q4) {
+            ok = make_map_ktiles(ctx, &maps.m[6], ctx->hperm, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp.tokb / 128, (uint32_t)tp.kg) &&
+                 make_map_hilo_ktiles(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane, (uint32_t)tp.kg);
+            if (ok && sh.n_sh)
+                ok = make_map_hilo_ktiles(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B,
+                                          (uint64_t)sh.f_sh, plane, (uint32_t)tp.kg);
+        } else {
+            ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
+                 make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
+            if (ok && sh.n_sh)
+                ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
+        }
         if (!ok) return S2MOE_ECUDA;
         TcArgs a;
         a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
