@@ -55,6 +55,9 @@ constexpr int kTcQ4Threads = kTcThreads + 256 + 64;   // block-int4 weights: eig
 constexpr int kTcQ4Packed = 128 * 32;          // bytes of one packed weight k-tile (128 rows x 64 nibbles)
 constexpr int kTcQ4Scales = 128 * 16;          // 8 binary16 scales per row: the 256 columns of the tile's unit
 constexpr int kTcMaxAStages = 6;               // stages of dequantised bf16 weight tiles
+constexpr int kTcQ4KG = 4;                     // int4: k-tiles per stage (a whole unit)
+static_assert(kTcQ4KG == 4, "the int4 path takes a stage to be a whole unit of four k-tiles");
+constexpr int kTcQ4ACol = 256;                 // int4: TMEM columns 256.. hold the dequantised tiles (32 per k-tile), 0..255 the accumulators
 #ifndef S2MOE_MAX_STAGES
 #define S2MOE_MAX_STAGES 10
 #endif
@@ -131,32 +134,30 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.feasible = p.stages >= 4 && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
                  sh.d % 64 == 0;
     if (sh.weight_dtype == DT_Q4B32) {
-        // a stage holds the packed k-tile, its unit's scales and the token tiles; the TMA copy of
-        // the scales wants rows of a multiple of 16 bytes, i.e. contraction lengths of 256
-        // A packed k-tile is only 4 KiB, so a stage carries up to four of them (a whole unit): one
+        // a stage holds the packed k-tiles and their unit's scales; the TMA copy of the scales
+        // wants rows of a multiple of 16 bytes, i.e. contraction lengths of 256.
+        // A packed k-tile is only 4 KiB, so a stage carries four of them (a whole unit): one
         // TMA copy, one hand-over to the tensor core and one release per stage instead of four.
         p.q4 = 1;
         p.x_bytes = 0;
-        // the stage of an int4 unit is cheap to fetch, so the issue of its 16 MMAs is what has to
-        // keep up: four issuers where their accumulators fit into the 512 TMEM columns
-        if (16 * p.n1 <= 512) {
-            p.n_iss = 4;
-            while (p.tmem_cols < 16 * p.n1) p.tmem_cols <<= 1;
-        }
         const int budget = kTcMaxSmem - p.tab_bytes - 1024;
+        // The dequantised tiles live in tensor memory (A operand of the MMAs): columns 256..511 hold
+        // two slots of a whole unit (4 k-tiles x 32 columns of bf16 pairs), columns 0..255 the
+        // accumulators: 2 buffers x issuers x 2 * n1 columns.  Issuing is what has to keep up with
+        // a stage that is cheap to fetch, so as many issuers as the accumulators leave room for.
+        p.n_iss = 16 * p.n1 <= kTcQ4ACol ? 4 : (8 * p.n1 <= kTcQ4ACol ? 2 : 1);
+        p.tmem_cols = 512;
         // The token tiles of a stage do not travel with its packed tiles: they are fetched into a
         // slot that belongs to the ring of dequantised tiles, just before they are used, so that a
         // stage is free again as soon as the dequantising warps have read it (its life decides
         // how many bytes are in flight) and not only when the MMAs have completed.
-        for (p.kg = 4; p.kg >= 1; p.kg >>= 1) {
-            p.tok_off = p.kg * kTcQ4Packed + kTcQ4Scales;
-            p.stage_bytes = (p.tok_off + 1023) & ~1023;
-            p.a_stages = p.kg == 4 ? 2 : (p.kg == 2 ? 3 : kTcMaxAStages);
-            p.stages = (budget - p.a_stages * p.kg * (kTcWTile + p.tokb)) / p.stage_bytes;
-            if (p.stages >= 3 || p.kg == 1) break;
-        }
+        p.kg = kTcQ4KG;
+        p.tok_off = p.kg * kTcQ4Packed + kTcQ4Scales;
+        p.stage_bytes = (p.tok_off + 1023) & ~1023;
+        p.a_stages = 2;
+        p.stages = (budget - p.a_stages * p.kg * p.tokb) / p.stage_bytes;
         if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
-        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + p.a_stages * p.kg * (kTcWTile + p.tokb) + 1024;
+        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + p.a_stages * p.kg * p.tokb + 1024;
         p.feasible = p.stages >= 3 && B <= kMaxTokens && sh.act_dtype == DT_BF16 && sh.d % 256 == 0 &&
                      sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
     }
@@ -257,6 +258,30 @@ __device__ __forceinline__ void tc_mma_bf16_parts(uint32_t d_tmem, uint32_t a_lo
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, {%7, %7, %7, %7}, p;\n\t"
         "}\n" ::"r"(d_tmem),
         "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// A operand in tensor memory (row i of the 128 x 16 tile in lane i, two bf16 per 32-bit column)
+__device__ __forceinline__ void tc_mma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                                   uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, {%6, %6, %6, %6}, p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
 __device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8])
@@ -406,8 +431,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     uint8_t *xres = tc_smem + pl.tab_bytes;
     xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
     uint8_t *ring = xres + pl.x_bytes;
-    uint8_t *aring = ring + (size_t)pl.stages * pl.stage_bytes;      // int4 only; 1024-byte aligned
-    uint8_t *tokring = aring + (size_t)pl.a_stages * pl.kg * kTcWTile;   // int4 only: token tiles, one slot per slot of aring
+    uint8_t *tokring = ring + (size_t)pl.stages * pl.stage_bytes;    // int4 only: token tiles, one slot per slot of dequantised tiles
 
     // group table; stage prefixes follow from the active list alone (routed groups first)
     const int U = ws.header[2];
@@ -546,7 +570,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             // token tiles go into the slot of the dequantised-tile ring they are used with (free
             // once the MMAs that read it have completed), and in the second projection only when
             // their wave's activations are written.  One thread serves both, so it polls.
-            const int KG = pl.kg;
+            constexpr int KG = kTcQ4KG;
             const int n_routed = p.B * sh.k;
             int pi = 0, ti = 0;                          // unit of each cursor
             TcUnit pu = unit_at(0), tu = pu;
@@ -723,7 +747,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // several warps share the work: with two issuers, issuer h takes K-steps 2h and 2h + 1 of
         // every k-tile, with four (int4 path) K-step h; each accumulates into its own TMEM columns
         // and the epilogue adds the partial accumulators.
-        const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - 17);
+        const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - 17);     // with one issuer (int4, many tokens): warp 1
         if (lane == 0 && half < NI) {
             unsigned it = 0, ui = 0, run = 0;
             uint32_t acc = 0;
@@ -746,9 +770,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             // descriptor halves (see tc_mma_bf16_parts); K-step k of a 64-wide tile lies 32 bytes further
             const uint32_t ks = 4u / (uint32_t)NI, koff = 2u * ks * (uint32_t)half;
             const uint32_t hi_std = (uint32_t)(tc_smem_desc(ring) >> 32);
-            const uint32_t hi_p2 = Q4 ? (uint32_t)(tc_smem_desc_sbo(ring, (uint32_t)pl.kg * 1024u) >> 32) : hi_std;
+            const uint32_t hi_p2 = Q4 ? (uint32_t)(tc_smem_desc_sbo(ring, (uint32_t)kTcQ4KG * 1024u) >> 32) : hi_std;
             const uint32_t ring_lo = (uint32_t)tc_smem_desc(ring) + koff, xres_lo = (uint32_t)tc_smem_desc(xres) + koff;
-            const uint32_t aring_lo = (uint32_t)tc_smem_desc(aring) + koff, tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
+            const uint32_t tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
+            const uint32_t a_tmem0 = tmem_base + (uint32_t)kTcQ4ACol + 4u * koff;     // 8 columns per K-step
             TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0, tm_fence = 0, tm_mmas = 0; const long long tm0 = clock64();)
             for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
@@ -767,7 +792,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
-                const int KG = Q4 ? pl.kg : 1;           // k-tiles per stage
+                constexpr int KG = Q4 ? kTcQ4KG : 1;     // k-tiles per stage
                 for (int kt = t.kt0; kt < t.kt1; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
                     // bf16: the stage; int4: the k-tiles as bf16, written by the dequantising warps, and their token tiles
@@ -781,14 +806,15 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     TCT(const long long c3 = clock64(); tm_fence += c3 - c2;)
 #if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
                     if (Q4) {
-                        // dequantised k-tiles of slot ta (16 KiB apart) and their token tiles: phase 1
-                        // [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row groups KG KiB apart)
-                        uint32_t a_lo = aring_lo + (uint32_t)(ta * KG) * (kTcWTile >> 4);
+                        // dequantised k-tiles of slot ta (tensor memory, 32 columns each) and their token
+                        // tiles: phase 1 [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row
+                        // groups KG KiB apart)
+                        uint32_t a_tm = a_tmem0 + (uint32_t)(ta * KG) * 32u;
                         uint32_t b_lo = tok_lo + (uint32_t)(ta * KG) * ((uint32_t)pl.tokb >> 4);
                         const uint32_t b_step = t.phase == 1 ? (uint32_t)pl.tokb >> 4 : 64u, b_hi = t.phase == 1 ? hi_std : hi_p2;
-                        for (int g = 0; g < KG; ++g, a_lo += kTcWTile >> 4, b_lo += b_step) {
+                        for (int g = 0; g < KG; ++g, a_tm += 32u, b_lo += b_step) {
                             for (uint32_t k = 0; k < ks; ++k) {
-                                tc_mma_bf16_parts(d_tmem, a_lo + 2 * k, hi_std, b_lo + 2 * k, b_hi, idesc, acc);
+                                tc_mma_bf16_tmem_a(d_tmem, a_tm + 8 * k, b_lo + 2 * k, b_hi, idesc, acc);
                                 acc = 1;
                             }
                         }
@@ -822,23 +848,27 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         }
     } else if (Q4 && warp >= 11) {
         // ------------------------------------------------------------------ dequantising warps (int4)
-        // Every row of a packed k-tile (64 nibbles, stored q + 8) becomes 64 bf16 values q * scale
-        // in the 128-byte-swizzled layout the tensor core reads: per 32-bit word eight
-        // nibbles -> (128 + n) as bf16 by an OR into the mantissa, minus 136 (exact), times the
-        // block's scale rounded to bf16.  Scales that lie past the matrix read as 0 (TMA fill), so
-        // a ragged last tile contributes nothing.
+        // Every row of a packed k-tile (64 nibbles, stored q + 8) becomes 64 bf16 values q * scale,
+        // written to tensor memory as the A operand of the MMAs (row = lane, two values per 32-bit
+        // column): per 32-bit word eight nibbles -> (128 + n) as bf16 by an OR into the mantissa,
+        // minus 136 (exact), times the block's scale rounded to bf16.  Scales that lie past the
+        // matrix read as 0 (TMA fill), so a ragged last tile contributes nothing.
         // A stage holds KG k-tiles: per row 2 * KG chunks of 16 packed bytes (32 weights, one
-        // scale each).  Thread (r, h) of the 256 takes row r and chunks h * KG .. h * KG + KG - 1.
-        const int r = (tid - 352) & 127, h = (tid - 352) >> 7;
-        const int KG = pl.kg;
+        // scale each).  A warp reaches the 32 lanes of its quarter (warp index mod 4) only, so
+        // thread (r, h) takes row r = 32 * (warp mod 4) + lane and chunks h * KG .. h * KG + KG - 1,
+        // h = 0 for the first four warps, 1 for the others.
+        const int r = 32 * (warp & 3) + lane, h = (warp - 11) >> 2;
+        constexpr int KG = kTcQ4KG;
         int s = 0, ta = 0;
         uint32_t ring_par = 0, a_par = 1;
         bool alive = true;
         const __nv_bfloat162 minus136 = __floats2bfloat162_rn(-136.0f, -136.0f);
+        const uint32_t a_lane = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)kTcQ4ACol;
         TCT(long long td_full = 0, td_aempty = 0, td_work = 0, td_fence = 0;)
-        for (int ui = 0; ui < n_units && alive; ++ui) {
-            const TcUnit t = unit_at(ui);
-            for (int kt = t.kt0; kt < t.kt1; kt += KG, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
+        // contraction lengths are multiples of 256 here, so every unit is exactly one stage and
+        // nothing of it has to be decoded
+        {
+            for (int ui = 0; ui < n_units && alive; ++ui, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
                 TCT(const long long d0 = clock64();)
                 const bool ok_full = mbar_wait(&full_bar[s], ring_par);
                 TCT(const long long d1 = clock64(); td_full += d1 - d0;)
@@ -847,21 +877,24 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     alive = false;
                     break;
                 }
+                tc_fence_after();                  // the MMAs that read this slot have completed
                 TCT(const long long d2 = clock64(); td_aempty += d2 - d1;)
                 const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                 const uint8_t *prow = stage + (size_t)r * (32 * KG);
-                const unsigned short *srow = reinterpret_cast<const unsigned short *>(stage + KG * kTcQ4Packed + r * 16) + (kt & 3) * 2;
-                uint8_t *atile = aring + (size_t)ta * KG * kTcWTile + (r >> 3) * 1024 + (r & 7) * 128;
-#pragma unroll 2
+                // this thread's four scales (binary16) in one load
+                const uint2 sc4 = *reinterpret_cast<const uint2 *>(stage + KG * kTcQ4Packed + r * 16 + h * 8);
+                const uint32_t a_slot = a_lane + (uint32_t)(ta * KG) * 32u;
+#pragma unroll
                 for (int qi = 0; qi < KG; ++qi) {
                     const int q = h * KG + qi;                         // chunk of 32 weights inside the stage
                     // the packed rows are swizzled over their own width by the TMA copy
                     const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
                     const uint4 pk = *reinterpret_cast<const uint4 *>(prow + ((q ^ sw) * 16));
-                    const float sf = __half2float(__ushort_as_half(srow[q]));
+                    const uint32_t sbits = (qi < 2 ? sc4.x : sc4.y) >> (16 * (qi & 1));
+                    const float sf = __half2float(__ushort_as_half((unsigned short)(sbits & 0xffffu)));
                     const __nv_bfloat162 sc2 = __floats2bfloat162_rn(sf, sf);
-                    uint8_t *arow = atile + (size_t)(q >> 1) * kTcWTile;    // k-tile q / 2, its chunks 4 * (q % 2) ..
                     const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+                    uint32_t o[16];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         const uint32_t m = 0x000F000Fu, one28 = 0x43004300u;       // bf16 128.0 twice
@@ -870,21 +903,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         // (n0, n4), (n1, n5), (n2, n6), (n3, n7): the token tiles carry the same
                         // permutation of every 8 columns, so no instruction is spent on reordering
                         uint32_t e[4] = {x04, x15, x26, x37};
-                        uint4 o;
-                        uint32_t *ov = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const __nv_bfloat162 v = __hmul2(__hadd2(*reinterpret_cast<const __nv_bfloat162 *>(&e[j]), minus136), sc2);
-                            ov[j] = *reinterpret_cast<const uint32_t *>(&v);
+                            o[4 * c + j] = *reinterpret_cast<const uint32_t *>(&v);
                         }
-                        const int cc = 4 * (q & 1) + c;                 // 16-byte chunk of the bf16 row
-                        *reinterpret_cast<uint4 *>(arow + ((cc ^ (r & 7)) * 16)) = o;
                     }
+                    tc_st16(a_slot + (uint32_t)q * 16u, o);          // k-tile q / 2, its columns 16 * (q % 2) ..
                 }
                 TCT(const long long d3 = clock64(); td_work += d3 - d2;)
-                // the tensor core reads these through the async proxy (shared memory only: the fence
-                // over all state spaces costs about a thousand cycles)
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(&a_full[ta]);
@@ -893,7 +922,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 TCT(td_fence += clock64() - d3;)
             }
         }
-        TCT(if (tid == 352) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 12; o[0] = td_full; o[1] = td_aempty; o[2] = td_work; o[3] = td_fence; })
+        TCT(if (warp == 11 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 12; o[0] = td_full; o[1] = td_aempty; o[2] = td_work; o[3] = td_fence; })
     } else if (warp == 10) {
         // ------------------------------------------------------------------ watcher
         // polls the waves' second counters (all CTAs have written their slice of the activations)
