@@ -51,7 +51,11 @@
 namespace s2moe {
 
 constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
-constexpr int kTcQ4Threads = kTcThreads + 256 + 64;   // block-int4 weights: eight more warps that dequantise, two more MMA issuers
+// block-int4 weights: warps that dequantise (8 or 16: 4 or 2 chunks of a row per thread).  The path is
+// bound by the instructions it issues, and 16 warps spend more of them on waiting and signalling
+// than they gain in latency hiding (measured: 156 us against 145 us per layer of the Mixtral shape).
+constexpr int kTcQ4DeqWarps = 8;
+constexpr int kTcQ4Threads = kTcThreads + 32 * kTcQ4DeqWarps + 64;   // ... and two more MMA issuers behind them
 constexpr int kTcQ4Packed = 128 * 32;          // bytes of one packed weight k-tile (128 rows x 64 nibbles)
 constexpr int kTcQ4Scales = 128 * 16;          // 8 binary16 scales per row: the 256 columns of the tile's unit
 constexpr int kTcMaxAStages = 6;               // stages of dequantised bf16 weight tiles
@@ -208,6 +212,11 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, i
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
+}
+// (x & mask) | bits in one logic instruction
+__device__ __forceinline__ void tc_nibble_pair(uint32_t &out, uint32_t x, uint32_t mask, uint32_t bits)
+{
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(out) : "r"(x), "r"(mask), "r"(bits));
 }
 // non-blocking test of a phase (a thread that serves two rings polls both)
 __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
@@ -383,6 +392,13 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
     return t;
 }
 
+// first | last << 1 | (phase == 2) << 2 | n << 8: the single-thread roles share their schedulers with
+// busy warps, so every instruction they do not need per unit counts
+__device__ __forceinline__ uint32_t tc_unit_meta(const TcUnit &t)
+{
+    return (uint32_t)t.first | ((uint32_t)t.last << 1) | ((t.phase == 2 ? 1u : 0u) << 2) | ((uint32_t)t.n << 8);
+}
+
 // tensor maps: 0 gate, 1 up, 2 down, 3 sh_gate, 4 sh_up, 5 sh_down, 6 hidden, 7 activations of the
 // routed slots, 8 of the shared slots: 3-D {k, slot, hi|lo}, so that one copy of box {64, 16, 2}
 // lands the hi tile and, right behind it, the lo tile of 16 slots
@@ -403,10 +419,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
     __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
     __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
-    __shared__ __align__(8) uint64_t tok_full[kTcMaxAStages];                          // int4: the token tiles used with them
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
+    __shared__ uint32_t s_umeta[kTcMaxUnits];      // what an MMA issuer needs of a unit, in one word (tc_unit_meta)
     __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
     __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
 
@@ -483,7 +499,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // barrier set-up, spread over a warp so that it runs beside the table loads of the others
         if (lane < pl.stages) {
             mbar_init(&full_bar[lane], 1);
-            mbar_init(&empty_bar[lane], Q4 ? 8 : NI);   // one commit from each MMA issuer; int4: the eight dequantising warps
+            mbar_init(&empty_bar[lane], Q4 ? kTcQ4DeqWarps : NI);   // one commit from each MMA issuer; int4: the dequantising warps
         }
         if (lane < 2) {
             mbar_init(&acc_full[lane], NI);
@@ -491,9 +507,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             mbar_init(&conv_go[lane], 4);
         }
         if (Q4 && lane < pl.a_stages) {
-            mbar_init(&a_full[lane], 8);
+            mbar_init(&a_full[lane], kTcQ4DeqWarps + 1);   // the dequantising warps and the producer's arrival with the token bytes
             mbar_init(&a_empty[lane], NI);
-            mbar_init(&tok_full[lane], 1);
         }
         if (lane == 0) {
             mbar_init(&ep_bar, 4);
@@ -555,9 +570,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     };
     // decoded once by all threads: the single-thread roles below then read a unit from shared
     // memory instead of dividing
-    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x) s_units[i] = unit_make(i);
+    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x) {
+        const TcUnit t = unit_make(i);
+        s_units[i] = t;
+        s_umeta[i] = tc_unit_meta(t);
+    }
     __syncthreads();
     auto unit_at = [&](int i) -> TcUnit { return i < kTcMaxUnits ? s_units[i] : unit_make(i); };
+    auto umeta_at = [&](int i) -> uint32_t { return i < kTcMaxUnits ? s_umeta[i] : tc_unit_meta(unit_make(i)); };
     auto seg_of_unit = [&](int i) -> int { return i < n_units ? unit_at(i).seg : 4; };
 
     TCT(const long long t_roles = clock64();)
@@ -568,8 +588,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             // int4: two cursors over the same sequence of stages.  The packed tiles and scales go
             // into the stage ring (a slot is free once the dequantising warps have read it); the
             // token tiles go into the slot of the dequantised-tile ring they are used with (free
-            // once the MMAs that read it have completed), and in the second projection only when
-            // their wave's activations are written.  One thread serves both, so it polls.
+            // once the MMAs that read it have completed; their bytes are counted by the barrier
+            // the dequantising warps arrive on, so that an MMA issuer waits once), and in the
+            // second projection only when their wave's activations are written.  One thread
+            // serves both, so it polls.
             constexpr int KG = kTcQ4KG;
             const int n_routed = p.B * sh.k;
             int pi = 0, ti = 0;                          // unit of each cursor
@@ -618,16 +640,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         uint8_t *op = tokring + (size_t)ta * KG * pl.tokb;
                         if (tu.phase == 1) {
                             // the hidden-state tiles of all KG k-tiles in one copy: [k-tile][tokb / 128 rows]
-                            mbar_expect_tx(&tok_full[ta], (uint32_t)(KG * pl.tokb));
-                            tma_load_3d(op, &maps.m[6], 0, 0, tkt, &tok_full[ta]);
+                            mbar_expect_tx(&a_full[ta], (uint32_t)(KG * pl.tokb));
+                            tma_load_3d(op, &maps.m[6], 0, 0, tkt, &a_full[ta]);
                         } else {
                             // one copy per 8 slots for all KG k-tiles: [hi | lo][k-tile][8 rows]
                             const StGroup &g = groups[tu.a];
                             const bool shared = g.group >= sh.E;
                             const int srow = shared ? g.off - n_routed : g.off;
-                            mbar_expect_tx(&tok_full[ta], (uint32_t)(KG * tu.n * 128));
+                            mbar_expect_tx(&a_full[ta], (uint32_t)(KG * tu.n * 128));
                             for (int r = 0; r < tu.n / 2; r += 8)
-                                tma_load_4d(op + r * 256 * KG, &maps.m[shared ? 8 : 7], 0, srow + r, tkt, 0, &tok_full[ta]);
+                                tma_load_4d(op + r * 256 * KG, &maps.m[shared ? 8 : 7], 0, srow + r, tkt, 0, &a_full[ta]);
                         }
                         tc_ring_next(ta, t_par, pl.a_stages);
                         tkt += KG;
@@ -638,9 +660,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 }
                 if (progress) {
                     idle = 0;
-                } else if (++idle > (kTcSpinLimit << 4)) {
-                    atomicExch(ws.status, ST_MBAR_TIMEOUT);
-                    alive = false;
+                } else {
+                    // nothing to issue: leave the scheduler to the dequantising warps for a while
+                    __nanosleep(100);
+                    if (++idle > kTcSpinLimit) {
+                        atomicExch(ws.status, ST_MBAR_TIMEOUT);
+                        alive = false;
+                    }
                 }
             }
             TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry;)
@@ -740,14 +766,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             if (alive && pend_n > 0) wait_ready(pend_wave);
             TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry; (void)tp_x; (void)tp_unit;)
         }
-    } else if (warp == 1 || warp == 6 || (Q4 && warp >= 19)) {
+    } else if (warp == 1 || warp == 6 || (Q4 && warp >= 11 + kTcQ4DeqWarps)) {
         // ------------------------------------------------------------------ MMA issuers
         // Issuing one tcgen05 instruction (an MMA or a commit) costs a thread on the order of 150
         // cycles whatever its shape, and with N = 16 every MMA covers only 4 KiB of weights, so
         // several warps share the work: with two issuers, issuer h takes K-steps 2h and 2h + 1 of
         // every k-tile, with four (int4 path) K-step h; each accumulates into its own TMEM columns
         // and the epilogue adds the partial accumulators.
-        const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - 17);     // with one issuer (int4, many tokens): warp 1
+        const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - (9 + kTcQ4DeqWarps));     // with one issuer (int4, many tokens): warp 1
         if (lane == 0 && half < NI) {
             unsigned it = 0, ui = 0, run = 0;
             uint32_t acc = 0;
@@ -775,6 +801,52 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const uint32_t tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
             const uint32_t a_tmem0 = tmem_base + (uint32_t)kTcQ4ACol + 4u * koff;     // 8 columns per K-step
             TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0, tm_fence = 0, tm_mmas = 0; const long long tm0 = clock64();)
+            if (Q4) {
+                // int4: a unit is one stage; everything this thread needs of it is one word
+                uint32_t d_tmem = tmem_base + (uint32_t)(half * 2 * pl.n1), buf = 0, run_par = 1;
+                const uint32_t tok_slot = (uint32_t)kTcQ4KG * ((uint32_t)pl.tokb >> 4), tok_step1 = (uint32_t)pl.tokb >> 4;
+                for (; (int)ui < n_units; ++ui) {
+                    const uint32_t um = umeta_at((int)ui);
+                    if (um & 1u) {
+                        TCT(long long c0 = clock64();)
+                        if (!mbar_wait(&acc_empty[buf], run_par)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
+                        TCT(tm_acc += clock64() - c0;)
+                        acc = 0;
+                    }
+                    TCT(long long c1 = clock64();)
+                    // the unit as bf16 in tensor memory, written by the dequantising warps, and its token tiles
+                    if (!mbar_wait(&a_full[ta], a_par)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
+                    TCT(long long c2 = clock64(); tm_full += c2 - c1;)
+                    tc_fence_after();
+#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
+                    {
+                        // dequantised k-tiles of slot ta (32 columns each) and their token tiles: phase 1
+                        // [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row groups KG KiB apart)
+                        const uint32_t idesc = tc_idesc((int)(um >> 8));
+                        const bool p2 = (um & 4u) != 0;
+                        uint32_t a_tm = a_tmem0 + (uint32_t)ta * (kTcQ4KG * 32u);
+                        uint32_t b_lo = tok_lo + (uint32_t)ta * tok_slot;
+                        const uint32_t b_step = p2 ? 64u : tok_step1, b_hi = p2 ? hi_p2 : hi_std;
+#pragma unroll
+                        for (int g = 0; g < kTcQ4KG; ++g, a_tm += 32u, b_lo += b_step) {
+                            for (uint32_t k = 0; k < ks; ++k) {
+                                tc_mma_bf16_tmem_a(d_tmem, a_tm + 8 * k, b_lo + 2 * k, b_hi, idesc, acc);
+                                acc = 1;
+                            }
+                        }
+                    }
+#endif
+                    tc_commit(&a_empty[ta]);           // frees the dequantised tiles and the token tiles
+                    tc_ring_next(ta, a_par, pl.a_stages);
+                    if (um & 2u) {
+                        tc_commit(&acc_full[buf]);
+                        buf ^= 1u;
+                        if (buf == 0) run_par ^= 1u;
+                        d_tmem = tmem_base + (uint32_t)(buf * 2 * NI * pl.n1 + half * 2 * pl.n1);
+                    }
+                    TCT(tm_mma += clock64() - c2;)
+                }
+            } else
             for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
                 const int buf = run & 1;
@@ -792,11 +864,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
-                constexpr int KG = Q4 ? kTcQ4KG : 1;     // k-tiles per stage
-                for (int kt = t.kt0; kt < t.kt1; kt += KG, ++it, tc_ring_next(s, ring_par, S)) {
+                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     TCT(long long c1 = clock64();)
-                    // bf16: the stage; int4: the k-tiles as bf16, written by the dequantising warps, and their token tiles
-                    if (Q4 ? !(mbar_wait(&a_full[ta], a_par) && mbar_wait(&tok_full[ta], a_par)) : !mbar_wait(&full_bar[s], ring_par)) {
+                    if (!mbar_wait(&full_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
@@ -805,20 +875,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     tc_fence_after();
                     TCT(const long long c3 = clock64(); tm_fence += c3 - c2;)
 #if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
-                    if (Q4) {
-                        // dequantised k-tiles of slot ta (tensor memory, 32 columns each) and their token
-                        // tiles: phase 1 [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row
-                        // groups KG KiB apart)
-                        uint32_t a_tm = a_tmem0 + (uint32_t)(ta * KG) * 32u;
-                        uint32_t b_lo = tok_lo + (uint32_t)(ta * KG) * ((uint32_t)pl.tokb >> 4);
-                        const uint32_t b_step = t.phase == 1 ? (uint32_t)pl.tokb >> 4 : 64u, b_hi = t.phase == 1 ? hi_std : hi_p2;
-                        for (int g = 0; g < KG; ++g, a_tm += 32u, b_lo += b_step) {
-                            for (uint32_t k = 0; k < ks; ++k) {
-                                tc_mma_bf16_tmem_a(d_tmem, a_tm + 8 * k, b_lo + 2 * k, b_hi, idesc, acc);
-                                acc = 1;
-                            }
-                        }
-                    } else {
+                    {
                         const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
                         const uint32_t b_lo = (t.phase == 1 && pl.x_bytes) ? xres_lo + (uint32_t)kt * ((uint32_t)pl.n1 * 8u)
                                                                            : a_lo + ((uint32_t)pl.tok_off >> 4);
@@ -831,12 +888,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
 #endif
                     TCT(const long long c4 = clock64(); tm_mmas += c4 - c3;)
-                    if (Q4) {
-                        tc_commit(&a_empty[ta]);       // frees the dequantised tiles and the token tiles
-                        tc_ring_next(ta, a_par, pl.a_stages);
-                    } else {
-                        tc_commit(&empty_bar[s]);      // frees the stage when these MMAs have read it
-                    }
+                    tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
                     TCT(tm_mma += clock64() - c2;)
                 }
                 if (alive && t.last) {
@@ -859,6 +911,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // h = 0 for the first four warps, 1 for the others.
         const int r = 32 * (warp & 3) + lane, h = (warp - 11) >> 2;
         constexpr int KG = kTcQ4KG;
+        constexpr int CP = 2 * KG / (kTcQ4DeqWarps / 4);      // chunks of its row per thread
         int s = 0, ta = 0;
         uint32_t ring_par = 0, a_par = 1;
         bool alive = true;
@@ -881,16 +934,21 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 TCT(const long long d2 = clock64(); td_aempty += d2 - d1;)
                 const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                 const uint8_t *prow = stage + (size_t)r * (32 * KG);
-                // this thread's four scales (binary16) in one load
-                const uint2 sc4 = *reinterpret_cast<const uint2 *>(stage + KG * kTcQ4Packed + r * 16 + h * 8);
+                uint32_t sc[2];                    // this thread's CP scales (binary16) in one load
+                if (CP == 4) {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(stage + KG * kTcQ4Packed + r * 16 + h * 8);
+                    sc[0] = v.x; sc[1] = v.y;
+                } else {
+                    sc[0] = *reinterpret_cast<const uint32_t *>(stage + KG * kTcQ4Packed + r * 16 + h * 4); sc[1] = 0;
+                }
                 const uint32_t a_slot = a_lane + (uint32_t)(ta * KG) * 32u;
 #pragma unroll
-                for (int qi = 0; qi < KG; ++qi) {
-                    const int q = h * KG + qi;                         // chunk of 32 weights inside the stage
+                for (int qi = 0; qi < CP; ++qi) {
+                    const int q = h * CP + qi;                         // chunk of 32 weights inside the stage
                     // the packed rows are swizzled over their own width by the TMA copy
                     const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
                     const uint4 pk = *reinterpret_cast<const uint4 *>(prow + ((q ^ sw) * 16));
-                    const uint32_t sbits = (qi < 2 ? sc4.x : sc4.y) >> (16 * (qi & 1));
+                    const uint32_t sbits = sc[qi >> 1] >> (16 * (qi & 1));
                     const float sf = __half2float(__ushort_as_half((unsigned short)(sbits & 0xffffu)));
                     const __nv_bfloat162 sc2 = __floats2bfloat162_rn(sf, sf);
                     const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
@@ -898,11 +956,15 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         const uint32_t m = 0x000F000Fu, one28 = 0x43004300u;       // bf16 128.0 twice
-                        const uint32_t x04 = (w[c] & m) | one28, x15 = ((w[c] >> 4) & m) | one28;
-                        const uint32_t x26 = ((w[c] >> 8) & m) | one28, x37 = ((w[c] >> 12) & m) | one28;
                         // (n0, n4), (n1, n5), (n2, n6), (n3, n7): the token tiles carry the same
-                        // permutation of every 8 columns, so no instruction is spent on reordering
-                        uint32_t e[4] = {x04, x15, x26, x37};
+                        // permutation of every 8 columns, so no instruction is spent on reordering.
+                        // Seven instructions per word, written out: from the C expression the
+                        // compiler makes eleven.
+                        uint32_t e[4];
+                        tc_nibble_pair(e[0], w[c], m, one28);
+                        tc_nibble_pair(e[1], w[c] >> 4, m, one28);
+                        tc_nibble_pair(e[2], w[c] >> 8, m, one28);
+                        tc_nibble_pair(e[3], w[c] >> 12, m, one28);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const __nv_bfloat162 v = __hmul2(__hadd2(*reinterpret_cast<const __nv_bfloat162 *>(&e[j]), minus136), sc2);
