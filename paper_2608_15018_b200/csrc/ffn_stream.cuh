@@ -31,7 +31,7 @@ constexpr int kStConsumerWarps = 7;   // + 1 producer warp = 256 threads, so a t
 constexpr int kStThreads = (kStConsumerWarps + 1) * 32;
 constexpr int kStMaxStages = 8;
 constexpr int kStMaxGroups = kMaxExperts + kMaxShared;
-constexpr unsigned kStSpinLimit = 1u << 22;   // bounded waits (a poll takes some tens of ns)
+constexpr unsigned kStSpinLimit = 1u << 20;   // bounded waits: a poll takes between some tens of ns and kMbarSuspendNs, so about a second at most
 constexpr int kStMaxSmem = 232448 - 2048;     // dynamic shared memory the kernel may use
 
 // Per-call plan, computed on the host (st_make_plan) and passed by value.
@@ -154,15 +154,18 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// upper bound in nanoseconds of the time a thread may stay suspended in one try_wait (it wakes when
+// the phase completes): a waiting thread then costs its scheduler next to no issue slots
+constexpr uint32_t kMbarSuspendNs = 1000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kMbarSuspendNs)
         : "memory");
     return ok != 0;
 }
