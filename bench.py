@@ -30,9 +30,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 # DRAM bytes (read + write) per algorithmic byte, from the ncu captures summarised under profiles/
-# (ffn_tc_kernel_cfg2_2layers.md, ffn_stream_kernel_cfg2_2layers.md); traffic grows with the
+# (ffn_tc_kernel_cfg2_2layers.md, ffn_tc_kernel_int4_cfg4_2layers.md, ffn_stream_kernel_cfg2_2layers.md); traffic grows with the
 # number of distinct experts exactly as the algorithmic bytes do.
-TRAFFIC_RATIO = {"ffn_tc_kernel": 1.03, "ffn_stream_kernel": 1.005}
+TRAFFIC_RATIO = {"ffn_tc_kernel": 1.03, "ffn_tc_kernel/int4": 1.02, "ffn_stream_kernel": 1.005}
 
 
 def parse_args():
@@ -305,9 +305,10 @@ def run_own(args, wl, B, sigma):
             share = {"ffn_gateup_simple": 2.0 / 3.0, "ffn_down_simple": 1.0 / 3.0}.get(dom, 1.0)
             bytes_per_launch = share * step_bytes / L / max(launches_per_layer, 1e-9)
             achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
+            ratio = TRAFFIC_RATIO.get(dom + "/int4" if wl.weight_dtype == workloads.Q4B32 else dom, TRAFFIC_RATIO.get(dom))
             roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                    "traffic": TRAFFIC_RATIO[dom] * bytes_per_launch if dom in TRAFFIC_RATIO else None,
+                    "traffic": ratio * bytes_per_launch if ratio else None,
                     "traffic_source": "ncu capture of a 2-layer case, scaled by algorithmic bytes",
                     "bytes_per_launch": bytes_per_launch, "us_per_launch": per_launch_ms * 1e3}
         line = {
