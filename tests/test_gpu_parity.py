@@ -210,7 +210,7 @@ Q4_TC = CONFIGS["cfg4"].with_(d_model=1024, d_ff=1792)      # contraction length
 
 @pytest.mark.parametrize("B", [1, 2, 4, 8, 16, 32, 64])
 def test_q4_tensor_core_plan(B):
-    """Block-int4 weights on the tcgen05 kernel (packed tiles dequantised to bf16 in shared memory)."""
+    """Block-int4 weights on the tcgen05 kernel (packed tiles dequantised to bf16 into tensor memory)."""
     for layer in range(2):
         rep, _ = run_case(Q4_TC, layer=layer, n_tokens=B, plan=3)
         assert rep is not None and rep.plan == 3 and rep.tokens_checked == B
