@@ -68,7 +68,8 @@ typedef enum { S2MOE_F32 = 0, S2MOE_BF16 = 1, S2MOE_Q4B32 = 2 } s2moe_dtype;
 typedef enum {
     S2MOE_OK = 0,
     S2MOE_EINVAL = -1,    /* bad config, shape, null pointer or alignment            */
-    S2MOE_ERANGE = -2,    /* n_tokens > max_tokens, layer index out of range         */
+    S2MOE_ERANGE = -2,    /* n_tokens > max_tokens, layer index out of range, more
+                             active experts than an offloaded context has slots     */
     S2MOE_ENOMEM = -3,    /* workspace allocation failed                             */
     S2MOE_ECUDA = -4,     /* a CUDA call failed; see s2moe_last_cuda_error           */
     S2MOE_ETIMEOUT = -5   /* a bounded device-side wait gave up (device status != 0) */
@@ -170,6 +171,64 @@ int s2moe_verify_stack_host(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden
 
 /* Free the workspace.  NULL is allowed.  The caller's buffers are untouched. */
 int s2moe_destroy(s2moe_ctx *ctx);
+
+/*
+ * Expert-level offloading with hot experts kept resident (Sec. 5, "Edge memory constraints and
+ * expert-level offloading": non-expert and shared parameters stay in device memory, individual
+ * experts are fetched on demand, frequently activated experts are kept resident from an offline
+ * profile).
+ *
+ * A context created by s2moe_create_offloaded keeps, per layer, a pool of n_slots device slots for
+ * routed experts.  In its `layers`, w_gate, w_up, w_down and s_gate, s_up, s_down are HOST
+ * pointers (page-locked memory recommended; same layouts as above, all n_experts experts);
+ * router, the shared experts and sh_scale are dev pointers as usual.  The host arrays must stay
+ * valid and unchanged for the life of the context.  pinned: host [n_layers][n_pinned] expert
+ * ids that own slots 0..n_pinned-1 of their layer for good and are copied at create; NULL with
+ * n_pinned == 0.  Replacement policy: see s2moe_cache_access.
+ *
+ * s2moe_verify_layer / _stack / _stack_host then work as before with two differences: between
+ * the routing kernel and the expert kernel of a layer the call waits for the stream, reads the
+ * active experts back and copies the missing ones into their slots (so the calls block and must
+ * not be captured into a CUDA graph), and a step that activates more distinct experts than can
+ * be resident at once fails with S2MOE_ERANGE.  Results are identical to those of a resident
+ * context.  Needs the tcgen05 kernel (kernel_plan 0 or 3; bf16 activations; bf16 weights, or
+ * block-int4 weights with d_model, d_ff, d_ff_shared multiples of 256) for every batch size up
+ * to max_tokens: EINVAL otherwise.  Other errors: EINVAL (null, n_slots outside 1..n_experts,
+ * n_pinned > n_slots, bad or repeated pinned id), ENOMEM, ECUDA.
+ */
+typedef struct {
+    int32_t n_slots;        /* device slots per layer for routed experts               */
+    int32_t n_pinned;       /* experts per layer that are never evicted (0..n_slots)    */
+    const int32_t *pinned;  /* host [n_layers][n_pinned], or NULL                       */
+} s2moe_residency;
+
+int s2moe_create_offloaded(const s2moe_config *config, const s2moe_layer_weights *layers,
+                           const s2moe_residency *residency, s2moe_ctx **out);
+
+/* Totals over all layers since create: experts found resident, experts fetched, bytes copied
+ * from host memory.  Any pointer may be NULL.  EINVAL when ctx is not offloaded. */
+int s2moe_residency_stats(const s2moe_ctx *ctx, int64_t *hits, int64_t *misses, int64_t *bytes_fetched);
+
+/* uses_out: host [n_experts], steps of `layer` that activated each expert since create: the
+ * profile from which a hot set is chosen.  EINVAL, ERANGE (layer). */
+int s2moe_residency_uses(const s2moe_ctx *ctx, int32_t layer, int64_t *uses_out);
+
+/*
+ * The replacement policy of one layer as a host-only object (no CUDA call): what an offloaded
+ * context runs internally.  pinned experts own slots 0..n_pinned-1.  One access names n distinct
+ * experts that must be resident together; slots_out[i] is the slot of experts[i], missed_out[i]
+ * is 1 when it had to be fetched.  A missing expert takes the free slot of lowest index, else
+ * the unpinned slot used least recently that is not wanted by this access (ties: lowest slot);
+ * misses are served in the order given.  s2moe_cache_access returns ERANGE and changes nothing
+ * when the experts cannot all be resident, an id is out of range or repeated.
+ * All arrays host.
+ */
+typedef struct s2moe_cache s2moe_cache;
+int s2moe_cache_create(int32_t n_experts, int32_t n_slots, const int32_t *pinned, int32_t n_pinned,
+                       s2moe_cache **out);
+int s2moe_cache_access(s2moe_cache *cache, const int32_t *experts, int32_t n, int32_t *slots_out,
+                       int32_t *missed_out);
+int s2moe_cache_destroy(s2moe_cache *cache);
 
 /* Static description of a status code. */
 const char *s2moe_strerror(int status);

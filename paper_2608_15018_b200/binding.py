@@ -8,7 +8,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
-from typing import Dict, List, Optional, Sequence
+from typing import Dict, List, Optional, Sequence, Tuple
 
 import torch
 
@@ -25,13 +25,20 @@ EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_ve
            "s2moe_destroy", "s2moe_strerror", "s2moe_last_device_status", "s2moe_last_cuda_error",
            "s2moe_kernel_launches", "s2moe_unique_expert_bytes", "s2moe_debug_read",
            "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan",
-           "s2moe_route_noalloc")
+           "s2moe_route_noalloc", "s2moe_expert_masks", "s2moe_adaptive_expand", "s2moe_create_offloaded",
+           "s2moe_residency_stats", "s2moe_residency_uses", "s2moe_cache_create", "s2moe_cache_access",
+           "s2moe_cache_destroy")
+OFFLOADED_FIELDS = ("w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down")   # host tensors of an offloaded context
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_EXPERTS = 64, 128
 KERNEL_CLASSES = 6
 
 
 class LayerWeightsC(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_FIELDS]
+
+
+class ResidencyC(ctypes.Structure):
+    _fields_ = [("n_slots", ctypes.c_int32), ("n_pinned", ctypes.c_int32), ("pinned", ctypes.c_void_p)]
 
 
 class ConfigC(ctypes.Structure):
@@ -106,6 +113,20 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_adaptive_expand.argtypes = [i32, i32, i32, vp, fp, vp, fp, ctypes.c_float, ctypes.c_float, vp, vp, vp,
                                           vp, vp]
     lib.s2moe_adaptive_expand.restype = ctypes.c_int
+    lib.s2moe_create_offloaded.argtypes = [ctypes.POINTER(ConfigC), ctypes.POINTER(LayerWeightsC),
+                                           ctypes.POINTER(ResidencyC), ctypes.POINTER(vp)]
+    lib.s2moe_create_offloaded.restype = ctypes.c_int
+    lib.s2moe_residency_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                                          ctypes.POINTER(ctypes.c_int64)]
+    lib.s2moe_residency_stats.restype = ctypes.c_int
+    lib.s2moe_residency_uses.argtypes = [vp, i32, vp]
+    lib.s2moe_residency_uses.restype = ctypes.c_int
+    lib.s2moe_cache_create.argtypes = [i32, i32, vp, i32, ctypes.POINTER(vp)]
+    lib.s2moe_cache_create.restype = ctypes.c_int
+    lib.s2moe_cache_access.argtypes = [vp, vp, i32, vp, vp]
+    lib.s2moe_cache_access.restype = ctypes.c_int
+    lib.s2moe_cache_destroy.argtypes = [vp]
+    lib.s2moe_cache_destroy.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -171,7 +192,11 @@ class LayerOutput:
 class S2MoE:
     """A context of the library: ``n_layers`` MoE layers whose weights stay resident."""
 
-    def __init__(self, config: Config, layers: Sequence[Dict[str, torch.Tensor]]):
+    def __init__(self, config: Config, layers: Sequence[Dict[str, torch.Tensor]], n_slots: int = 0,
+                 pinned: Optional[Sequence[Sequence[int]]] = None):
+        """``n_slots`` > 0 makes an offloaded context: the routed experts' weights (OFFLOADED_FIELDS
+        of every layer dict) are host tensors, ``n_slots`` of them at a time are resident per
+        layer, ``pinned[layer]`` lists the experts that are never evicted."""
         self._lib = load_library()
         self._h = ctypes.c_void_p(None)
         self.config = config
@@ -181,13 +206,43 @@ class S2MoE:
         arr = (LayerWeightsC * config.n_layers)()
         for i, lw in enumerate(layers):
             for name in WEIGHT_FIELDS:
-                setattr(arr[i], name, _dptr(lw.get(name)))
+                t = lw.get(name)
+                if n_slots > 0 and name in OFFLOADED_FIELDS:
+                    if t is not None and t.is_cuda:
+                        raise ValueError(f"offloaded context: {name} must be a host tensor")
+                    setattr(arr[i], name, None if t is None else t.data_ptr())
+                else:
+                    setattr(arr[i], name, _dptr(t))
         cfg = config.c()
-        rc = self._lib.s2moe_create(ctypes.byref(cfg), arr, ctypes.byref(self._h))
+        self.offloaded = n_slots > 0
+        if self.offloaded:
+            n_pinned = len(pinned[0]) if pinned else 0
+            flat = [int(e) for row in (pinned or []) for e in row]
+            if pinned and (len(pinned) != config.n_layers or len(flat) != n_pinned * config.n_layers):
+                raise ValueError("pinned: one list of equal length per layer")
+            self._pinned = (ctypes.c_int32 * max(1, len(flat)))(*flat)
+            res = ResidencyC(int(n_slots), n_pinned, ctypes.cast(self._pinned, ctypes.c_void_p) if flat else None)
+            rc = self._lib.s2moe_create_offloaded(ctypes.byref(cfg), arr, ctypes.byref(res), ctypes.byref(self._h))
+        else:
+            rc = self._lib.s2moe_create(ctypes.byref(cfg), arr, ctypes.byref(self._h))
         if rc != OK:
             self._h = ctypes.c_void_p(None)
-            raise S2MoEError(rc, "s2moe_create")
-        self.device = next(iter(layers[0].values())).device
+            raise S2MoEError(rc, "s2moe_create_offloaded" if self.offloaded else "s2moe_create")
+        self.device = layers[0]["router"].device
+
+    def residency_stats(self) -> Tuple[int, int, int]:
+        """(hits, misses, bytes fetched from host memory) since create, over all layers."""
+        h, m, b = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+        self._check(self._lib.s2moe_residency_stats(self._h, ctypes.byref(h), ctypes.byref(m), ctypes.byref(b)),
+                    "s2moe_residency_stats")
+        return h.value, m.value, b.value
+
+    def residency_uses(self, layer: int) -> List[int]:
+        """Per expert of ``layer``: the steps that activated it (the profile a hot set is chosen from)."""
+        out = (ctypes.c_int64 * self.config.n_experts)()
+        self._check(self._lib.s2moe_residency_uses(self._h, int(layer), ctypes.cast(out, ctypes.c_void_p)),
+                    "s2moe_residency_uses")
+        return list(out)
 
     # -- lifetime
     def close(self) -> None:
@@ -374,3 +429,39 @@ def adaptive_expand(parent: torch.Tensor, p_tok: torch.Tensor, masks: torch.Tens
         raise S2MoEError(rc, "s2moe_adaptive_expand")
     return admitted, order, n_adm, union
 
+
+
+class ExpertCache:
+    """The replacement policy of one layer of an offloaded context, host only (``s2moe_cache_*``)."""
+
+    def __init__(self, n_experts: int, n_slots: int, pinned: Sequence[int] = ()):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p(None)
+        arr = (ctypes.c_int32 * max(1, len(pinned)))(*[int(e) for e in pinned])
+        rc = self._lib.s2moe_cache_create(int(n_experts), int(n_slots), ctypes.cast(arr, ctypes.c_void_p) if pinned else None,
+                                          len(pinned), ctypes.byref(self._h))
+        if rc != OK:
+            self._h = ctypes.c_void_p(None)
+            raise S2MoEError(rc, "s2moe_cache_create")
+
+    def access(self, experts: Sequence[int]) -> Tuple[List[int], List[int]]:
+        """Slots of ``experts`` (distinct ids) and which of them had to be fetched."""
+        n = len(experts)
+        ex = (ctypes.c_int32 * max(1, n))(*[int(e) for e in experts])
+        sl, ms = (ctypes.c_int32 * max(1, n))(), (ctypes.c_int32 * max(1, n))()
+        rc = self._lib.s2moe_cache_access(self._h, ctypes.cast(ex, ctypes.c_void_p), n, ctypes.cast(sl, ctypes.c_void_p),
+                                          ctypes.cast(ms, ctypes.c_void_p))
+        if rc != OK:
+            raise S2MoEError(rc, "s2moe_cache_access")
+        return list(sl)[:n], list(ms)[:n]
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.s2moe_cache_destroy(self._h)
+            self._h = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

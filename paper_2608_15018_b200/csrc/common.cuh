@@ -61,6 +61,8 @@ struct Workspace {
     unsigned long long *tokmask;   // [E + n_sh] bit b set: token b is bucketed to the group
     uint4 *gtab;           // [n_active][2] {group, tokens, first slot, 0}, {mask lo, mask hi, 0, 0}: the
                            // active groups in their final form, or NULL when nobody reads it
+    const int32_t *slot_of;  // [E] device slot that holds each routed expert's weights (expert offloading), or
+                             // NULL: every expert is resident at its own index
 };
 
 __device__ __forceinline__ size_t act_offset(int slot, int n_routed_slots, int f, int f_sh)

@@ -468,6 +468,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             gr.p1 = r * u1r + s * u1s;
             gr.p2 = r * u2r + s * u2s;
             gr.nks = 0;
+            gr.slot = (ws.slot_of && gr.group < sh.E) ? __ldg(&ws.slot_of[gr.group]) : gr.group;
+            gr.pad_ = 0;
             gr.ksl = 0;
             groups[a] = gr;
         }
@@ -609,7 +611,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     TCT(const long long c2 = clock64();)
                     const StGroup &g = groups[pu.a];
                     const bool shared = g.group >= sh.E;
-                    const int e = shared ? g.group - sh.E : g.group;
+                    const int e = shared ? g.group - sh.E : g.slot;
                     const int row0 = e * (pu.mat == 2 ? sh.d : g.f) + pu.rb * 128;
                     // packed k-tiles (32 bytes of every row each) and the 8 scales per row of the 256
                     // columns they lie in (x in scales; kt0 is a multiple of 4)
@@ -716,7 +718,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const TcUnit t = unit_at(i);
                 const StGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
-                const int e = shared ? g.group - sh.E : g.group;
+                const int e = shared ? g.group - sh.E : g.slot;
                 const CUtensorMap *wmap = &maps.m[(shared ? 3 : 0) + t.mat];
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;

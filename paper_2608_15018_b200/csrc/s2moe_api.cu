@@ -17,6 +17,8 @@
 #include "ffn_tc.cuh"
 #include "route.cuh"
 
+#include "expert_cache.h"
+
 using namespace s2moe;
 
 struct s2moe_ctx {
@@ -49,6 +51,23 @@ struct s2moe_ctx {
     std::vector<cudaEvent_t> prof_ev;   // 2 per record
     std::vector<int> prof_cls;
     size_t prof_cap = 0;
+    // expert offloading (s2moe_create_offloaded): the routed experts' weights live in host memory,
+    // n_w_experts = n_slots of them at a time in a device pool that the weight pointers of
+    // `layers` point into
+    bool offload = false;
+    int n_w_experts = 0;                  // experts the device weight tensors hold (n_experts, or n_slots)
+    std::vector<ExpertCache> caches;      // per layer
+    std::vector<LayerPtrs> host_w;        // per layer: host pointers of the routed experts
+    void *pool = nullptr;
+    int32_t *h_route = nullptr;           // pinned: {n_active, n_slots, U, B} and the active list
+    int32_t *h_slot_of = nullptr;         // pinned [E]
+    int32_t *d_slot_of = nullptr;         // device [E]
+    size_t mat_bytes[6] = {0, 0, 0, 0, 0, 0};   // one expert's bytes in w_gate, w_up, w_down, s_gate, s_up, s_down
+    int64_t fetched_bytes = 0;
+};
+
+struct s2moe_cache {
+    ExpertCache c;
 };
 
 enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_TC = 5, KC_COUNT = 6 };
@@ -360,6 +379,44 @@ int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
     return want == 2 ? 0 : 1;
 }
 
+// Expert offloading, between the routing kernel and the FFN kernel of a layer: read the list of
+// active experts back, let the layer's cache name a slot for each, copy the missing ones from
+// host memory into their slots and hand the expert-to-slot table to the FFN kernel.  Host and
+// stream meet here (the host has to see the routing result), so an offloaded layer is not
+// captured into a graph.
+int fetch_experts(s2moe_ctx *ctx, int layer, cudaStream_t st)
+{
+    const Shape &sh = ctx->shape;
+    const int G = sh.E + sh.n_sh;
+    CU(ctx, cudaMemcpyAsync(ctx->h_route, ctx->ws.header, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaMemcpyAsync(ctx->h_route + 8, ctx->ws.active, (size_t)G * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU(ctx, cudaStreamSynchronize(st));
+    const int U = ctx->h_route[2];
+    if (U < 0 || U > sh.E) return S2MOE_ECUDA;
+    ExpertCache &cache = ctx->caches[(size_t)layer];
+    std::vector<int32_t> slots((size_t)U), missed((size_t)U);
+    if (!cache.access(ctx->h_route + 8, U, slots.data(), missed.data())) return S2MOE_ERANGE;
+    const LayerPtrs &hw = ctx->host_w[(size_t)layer], &dw = ctx->layers[(size_t)layer];
+    const void *src[6] = {hw.w_gate, hw.w_up, hw.w_down, hw.s_gate, hw.s_up, hw.s_down};
+    const void *dst[6] = {dw.w_gate, dw.w_up, dw.w_down, dw.s_gate, dw.s_up, dw.s_down};
+    for (int i = 0; i < U; ++i) {
+        if (!missed[(size_t)i]) continue;
+        const size_t e = (size_t)ctx->h_route[8 + i], sl = (size_t)slots[(size_t)i];
+        for (int m = 0; m < 6; ++m) {
+            const size_t nb = ctx->mat_bytes[m];
+            if (!nb) continue;
+            CU(ctx, cudaMemcpyAsync((uint8_t *)const_cast<void *>(dst[m]) + nb * sl, (const uint8_t *)src[m] + nb * e, nb,
+                                    cudaMemcpyHostToDevice, st));
+            ctx->fetched_bytes += (int64_t)nb;
+        }
+    }
+    for (int e = 0; e < sh.E; ++e) ctx->h_slot_of[e] = cache.slot_of[(size_t)e] < 0 ? 0 : cache.slot_of[(size_t)e];
+    CU(ctx, cudaMemcpyAsync(ctx->d_slot_of, ctx->h_slot_of, (size_t)sh.E * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    // h_slot_of is reused by the next call: the copy must have left the host buffer
+    CU(ctx, cudaStreamSynchronize(st));
+    return S2MOE_OK;
+}
+
 int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float *conf, float *out,
                int32_t *sel_idx, float *sel_w, int32_t *n_unique, cudaStream_t st)
 {
@@ -387,6 +444,10 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         }
     }
     launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
+    if (ctx->offload) {
+        const int rc = fetch_experts(ctx, layer, st);
+        if (rc != S2MOE_OK) return rc;
+    }
     if (plan == 3) {
         const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
         TcMaps maps = ctx->tc_maps[layer];
@@ -443,7 +504,21 @@ int check_call(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden, float *out,
 
 extern "C" {
 
+namespace {
+int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, int n_w_experts, s2moe_ctx **out);
+}
+
 int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, s2moe_ctx **out)
+{
+    if (out) *out = nullptr;
+    if (!config || !layers || !out) return S2MOE_EINVAL;
+    return create_impl(config, layers, config->n_experts, out);
+}
+
+namespace {
+// n_w_experts: how many experts the routed-expert weight tensors of `layers` hold (all of them,
+// or the slots of the device pool of an offloaded context)
+int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, int n_w_experts, s2moe_ctx **out)
 {
     if (out) *out = nullptr;
     if (!config || !layers || !out) return S2MOE_EINVAL;
@@ -456,6 +531,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     s2moe_ctx *ctx = new (std::nothrow) s2moe_ctx();
     if (!ctx) return S2MOE_ENOMEM;
     ctx->cfg = *config;
+    ctx->n_w_experts = n_w_experts;
     Shape &sh = ctx->shape;
     sh.d = config->d_model; sh.f = config->d_ff; sh.E = config->n_experts; sh.k = config->top_k;
     sh.n_sh = config->n_shared; sh.f_sh = config->n_shared ? config->d_ff_shared : 0;
@@ -541,7 +617,7 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
                 TcMaps &m = ctx->tc_maps[l];
                 std::memset(&m, 0, sizeof(m));
                 if (q4) {
-                    const uint64_t Ef = (uint64_t)sh.E * sh.f, Ed = (uint64_t)sh.E * sh.d;
+                    const uint64_t Ef = (uint64_t)n_w_experts * sh.f, Ed = (uint64_t)n_w_experts * sh.d;
                     ok = make_map_plain(ctx, &m.m[0], lp.w_gate, Ef, (uint64_t)sh.d / 2, 32, 1) &&
                          make_map_plain(ctx, &m.m[1], lp.w_up, Ef, (uint64_t)sh.d / 2, 32, 1) &&
                          make_map_plain(ctx, &m.m[2], lp.w_down, Ed, (uint64_t)sh.f / 2, 32, 1) &&
@@ -573,9 +649,9 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
                     }
                     continue;
                 }
-                ok = make_map(ctx, &m.m[0], lp.w_gate, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
-                     make_map(ctx, &m.m[1], lp.w_up, (uint64_t)sh.E * sh.f, (uint64_t)sh.d, 128) &&
-                     make_map(ctx, &m.m[2], lp.w_down, (uint64_t)sh.E * sh.d, (uint64_t)sh.f, 128);
+                ok = make_map(ctx, &m.m[0], lp.w_gate, (uint64_t)n_w_experts * sh.f, (uint64_t)sh.d, 128) &&
+                     make_map(ctx, &m.m[1], lp.w_up, (uint64_t)n_w_experts * sh.f, (uint64_t)sh.d, 128) &&
+                     make_map(ctx, &m.m[2], lp.w_down, (uint64_t)n_w_experts * sh.d, (uint64_t)sh.f, 128);
                 if (ok && sh.n_sh)
                     ok = make_map(ctx, &m.m[3], lp.sh_gate, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
                          make_map(ctx, &m.m[4], lp.sh_up, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
@@ -589,6 +665,129 @@ int s2moe_create(const s2moe_config *config, const s2moe_layer_weights *layers, 
     ctx->st_out = (float *)(base + o_sto); ctx->st_sel = (int32_t *)(base + o_sts);
     ctx->st_selw = (float *)(base + o_stw); ctx->st_nu = (int32_t *)(base + o_stn);
     *out = ctx;
+    return S2MOE_OK;
+}
+}  // namespace
+
+int s2moe_create_offloaded(const s2moe_config *config, const s2moe_layer_weights *layers, const s2moe_residency *res,
+                           s2moe_ctx **out)
+{
+    if (out) *out = nullptr;
+    if (!config || !layers || !res || !out) return S2MOE_EINVAL;
+    int rc = validate_config(config);
+    if (rc != S2MOE_OK) return rc;
+    const int E = config->n_experts, L = config->n_layers;
+    if (res->n_slots < 1 || res->n_slots > E || res->n_pinned < 0 || res->n_pinned > res->n_slots) return S2MOE_EINVAL;
+    if (res->n_pinned > 0 && !res->pinned) return S2MOE_EINVAL;
+    // the expert-to-slot indirection lives in the tcgen05 kernel
+    if (config->kernel_plan != 0 && config->kernel_plan != 3) return S2MOE_EINVAL;
+    if (config->act_dtype != S2MOE_BF16 || (config->weight_dtype != S2MOE_BF16 && config->weight_dtype != S2MOE_Q4B32))
+        return S2MOE_EINVAL;
+    for (int l = 0; l < L; ++l) {
+        rc = validate_layer(config, &layers[l]);     // non-null and 16-byte aligned holds for host pointers too
+        if (rc != S2MOE_OK) return rc;
+    }
+    const bool q4 = config->weight_dtype == S2MOE_Q4B32;
+    const size_t d = (size_t)config->d_model, f = (size_t)config->d_ff;
+    size_t mb[6] = {0, 0, 0, 0, 0, 0};
+    mb[0] = mb[1] = mb[2] = q4 ? f * d / 2 : f * d * 2;
+    if (q4) mb[3] = mb[4] = mb[5] = f * (d / 32) * 2;
+    size_t per_layer = 0;
+    for (int i = 0; i < 6; ++i) per_layer += align_up(mb[i] * (size_t)res->n_slots, 256);
+    void *pool = nullptr;
+    cudaError_t e = cudaMalloc(&pool, per_layer * (size_t)L);
+    if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? S2MOE_ENOMEM : S2MOE_ECUDA;
+    std::vector<s2moe_layer_weights> dev((size_t)L);
+    for (int l = 0; l < L; ++l) {
+        dev[(size_t)l] = layers[l];
+        uint8_t *p = (uint8_t *)pool + per_layer * (size_t)l;
+        const void **dst[6] = {&dev[(size_t)l].w_gate, &dev[(size_t)l].w_up, &dev[(size_t)l].w_down,
+                               &dev[(size_t)l].s_gate, &dev[(size_t)l].s_up, &dev[(size_t)l].s_down};
+        for (int i = 0; i < 6; ++i) {
+            if (mb[i]) *dst[i] = p;
+            p += align_up(mb[i] * (size_t)res->n_slots, 256);
+        }
+    }
+    s2moe_config cfg3 = *config;
+    cfg3.kernel_plan = 3;
+    s2moe_ctx *ctx = nullptr;
+    rc = create_impl(&cfg3, dev.data(), res->n_slots, &ctx);
+    if (rc != S2MOE_OK) { cudaFree(pool); return rc; }
+    ctx->pool = pool;
+    ctx->offload = true;
+    for (int i = 0; i < 6; ++i) ctx->mat_bytes[i] = mb[i];
+    ctx->host_w.resize((size_t)L);
+    std::memcpy(ctx->host_w.data(), layers, sizeof(LayerPtrs) * (size_t)L);
+    // every batch size up to max_tokens must run on the tcgen05 kernel
+    bool ok = !ctx->tc_maps.empty();
+    for (int B = 1; B <= config->max_tokens && ok; ++B) ok = plan_for(ctx, B, nullptr) == 3;
+    ctx->caches.resize((size_t)L);
+    for (int l = 0; l < L && ok; ++l)
+        ok = ctx->caches[(size_t)l].init(E, res->n_slots, res->n_pinned ? res->pinned + (size_t)l * res->n_pinned : nullptr,
+                                         res->n_pinned);
+    if (!ok) { s2moe_destroy(ctx); return S2MOE_EINVAL; }
+    e = cudaMallocHost((void **)&ctx->h_route, sizeof(int32_t) * (size_t)(8 + E + config->n_shared));
+    if (e == cudaSuccess) e = cudaMallocHost((void **)&ctx->h_slot_of, sizeof(int32_t) * (size_t)E);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->d_slot_of, sizeof(int32_t) * (size_t)E);
+    // the pinned experts go to their slots now
+    for (int l = 0; l < L && e == cudaSuccess; ++l) {
+        const LayerPtrs &hw = ctx->host_w[(size_t)l], &dw = ctx->layers[(size_t)l];
+        const void *src[6] = {hw.w_gate, hw.w_up, hw.w_down, hw.s_gate, hw.s_up, hw.s_down};
+        const void *dstp[6] = {dw.w_gate, dw.w_up, dw.w_down, dw.s_gate, dw.s_up, dw.s_down};
+        for (int i = 0; i < res->n_pinned && e == cudaSuccess; ++i) {
+            const size_t ex = (size_t)res->pinned[(size_t)l * res->n_pinned + i];
+            for (int m = 0; m < 6 && e == cudaSuccess; ++m)
+                if (mb[m])
+                    e = cudaMemcpy((uint8_t *)const_cast<void *>(dstp[m]) + mb[m] * (size_t)i,
+                                   (const uint8_t *)src[m] + mb[m] * ex, mb[m], cudaMemcpyHostToDevice);
+        }
+    }
+    if (e != cudaSuccess) { s2moe_destroy(ctx); return e == cudaErrorMemoryAllocation ? S2MOE_ENOMEM : S2MOE_ECUDA; }
+    ctx->ws.slot_of = ctx->d_slot_of;
+    *out = ctx;
+    return S2MOE_OK;
+}
+
+int s2moe_residency_stats(const s2moe_ctx *ctx, int64_t *hits, int64_t *misses, int64_t *bytes_fetched)
+{
+    if (!ctx || !ctx->offload) return S2MOE_EINVAL;
+    int64_t h = 0, m = 0;
+    for (const ExpertCache &c : ctx->caches) { h += c.hits; m += c.misses; }
+    if (hits) *hits = h;
+    if (misses) *misses = m;
+    if (bytes_fetched) *bytes_fetched = ctx->fetched_bytes;
+    return S2MOE_OK;
+}
+
+int s2moe_residency_uses(const s2moe_ctx *ctx, int32_t layer, int64_t *uses_out)
+{
+    if (!ctx || !ctx->offload || !uses_out) return S2MOE_EINVAL;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return S2MOE_ERANGE;
+    const ExpertCache &c = ctx->caches[(size_t)layer];
+    for (int e = 0; e < c.n_experts; ++e) uses_out[e] = c.uses[(size_t)e];
+    return S2MOE_OK;
+}
+
+int s2moe_cache_create(int32_t n_experts, int32_t n_slots, const int32_t *pinned, int32_t n_pinned, s2moe_cache **out)
+{
+    if (out) *out = nullptr;
+    if (!out) return S2MOE_EINVAL;
+    s2moe_cache *c = new (std::nothrow) s2moe_cache();
+    if (!c) return S2MOE_ENOMEM;
+    if (!c->c.init(n_experts, n_slots, pinned, n_pinned)) { delete c; return S2MOE_EINVAL; }
+    *out = c;
+    return S2MOE_OK;
+}
+
+int s2moe_cache_access(s2moe_cache *cache, const int32_t *experts, int32_t n, int32_t *slots_out, int32_t *missed_out)
+{
+    if (!cache || (n > 0 && (!experts || !slots_out || !missed_out))) return S2MOE_EINVAL;
+    return cache->c.access(experts, n, slots_out, missed_out) ? S2MOE_OK : S2MOE_ERANGE;
+}
+
+int s2moe_cache_destroy(s2moe_cache *cache)
+{
+    delete cache;
     return S2MOE_OK;
 }
 
@@ -649,6 +848,10 @@ int s2moe_destroy(s2moe_ctx *ctx)
     if (!ctx) return S2MOE_OK;
     cudaError_t e = cudaSuccess;
     if (ctx->slab) e = cudaFree(ctx->slab);
+    if (ctx->pool) cudaFree(ctx->pool);
+    if (ctx->d_slot_of) cudaFree(ctx->d_slot_of);
+    if (ctx->h_route) cudaFreeHost(ctx->h_route);
+    if (ctx->h_slot_of) cudaFreeHost(ctx->h_slot_of);
     for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
     delete ctx;
     return e == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
@@ -659,7 +862,7 @@ const char *s2moe_strerror(int status)
     switch (status) {
         case S2MOE_OK: return "ok";
         case S2MOE_EINVAL: return "invalid argument (config, shape, null pointer or alignment)";
-        case S2MOE_ERANGE: return "n_tokens or layer out of range";
+        case S2MOE_ERANGE: return "n_tokens or layer out of range, or more active experts than resident slots";
         case S2MOE_ENOMEM: return "out of device memory";
         case S2MOE_ECUDA: return "CUDA call failed";
         case S2MOE_ETIMEOUT: return "a bounded device-side wait gave up";

@@ -55,3 +55,12 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
         parity.check_bucketing(lists, sel, w, wl.n_experts, wl.n_shared)
     rep.plan = used
     return rep, o
+
+
+def check_outputs(wl, T, H, conf, o):
+    """One layer's outputs `o` for hidden states H (confidences conf) against the float64 oracle run
+    on the weights T (a layer dict with every tensor's values; device or host)."""
+    ocfg, ow = parity.from_workload(wl, T)
+    return parity.check_layer(ocfg, ow, workloads.raw_numpy(H), None if conf is None else conf.cpu().numpy(),
+                              o.out.cpu().numpy(), o.sel_idx.cpu().numpy(), o.sel_w.cpu().numpy(),
+                              int(o.n_unique.item()), TOL[wl.weight_dtype])
