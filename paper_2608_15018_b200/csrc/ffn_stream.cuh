@@ -53,7 +53,6 @@ struct StGroup {      // one active group, in shared memory
     int group, T, off, f;      // group id, tokens, first slot, inner dim
     int p1, p2;                // first phase-1 / phase-2 stage of the group
     int nks, ksl;              // K-slices of a phase-2 row and their length
-    int slot, pad_;            // tcgen05 kernel: where the expert's weights lie (= group unless experts are offloaded)
 };
 
 struct StageDesc {

@@ -460,6 +460,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         if (a < n_active) {
             StGroup gr;
             gr.group = (int)r0.x;
+            // offloaded experts: from here on the group id of a routed expert is the device slot its
+            // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
+            if (ws.slot_of && gr.group < sh.E) gr.group = __ldg(&ws.slot_of[gr.group]);
             gr.T = (int)r0.y;
             gr.off = (int)r0.z;
             gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
@@ -468,8 +471,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             gr.p1 = r * u1r + s * u1s;
             gr.p2 = r * u2r + s * u2s;
             gr.nks = 0;
-            gr.slot = (ws.slot_of && gr.group < sh.E) ? __ldg(&ws.slot_of[gr.group]) : gr.group;
-            gr.pad_ = 0;
             gr.ksl = 0;
             groups[a] = gr;
         }
@@ -611,7 +612,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     TCT(const long long c2 = clock64();)
                     const StGroup &g = groups[pu.a];
                     const bool shared = g.group >= sh.E;
-                    const int e = shared ? g.group - sh.E : g.slot;
+                    const int e = shared ? g.group - sh.E : g.group;
                     const int row0 = e * (pu.mat == 2 ? sh.d : g.f) + pu.rb * 128;
                     // packed k-tiles (32 bytes of every row each) and the 8 scales per row of the 256
                     // columns they lie in (x in scales; kt0 is a multiple of 4)
@@ -718,7 +719,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const TcUnit t = unit_at(i);
                 const StGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
-                const int e = shared ? g.group - sh.E : g.slot;
+                const int e = shared ? g.group - sh.E : g.group;
                 const CUtensorMap *wmap = &maps.m[(shared ? 3 : 0) + t.mat];
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
