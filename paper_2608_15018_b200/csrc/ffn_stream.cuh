@@ -213,7 +213,8 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ int upper_group1(const StGroup *g, int n, int u)
+template <typename G>
+__device__ __forceinline__ int upper_group1(const G *g, int n, int u)
 {
     int lo = 0, hi = n;   // largest a with g[a].p1 <= u
     while (hi - lo > 1) {
@@ -222,7 +223,8 @@ __device__ __forceinline__ int upper_group1(const StGroup *g, int n, int u)
     }
     return lo;
 }
-__device__ __forceinline__ int upper_group2(const StGroup *g, int n, int u)
+template <typename G>
+__device__ __forceinline__ int upper_group2(const G *g, int n, int u)
 {
     int lo = 0, hi = n;
     while (hi - lo > 1) {

@@ -81,6 +81,15 @@ constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once 
 constexpr int kTcSplitNum = S2MOE_SPLIT_NUM, kTcSplitDen = S2MOE_SPLIT_DEN;
 constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 8 + w], [kTcReady - 4 + w]: the two counters of wave w
 
+// one active group in shared memory: 32 bytes, so that an entry is two aligned 16-byte reads
+// (wider entries were measured: 48 bytes cost 0.7 us per layer)
+struct TcGroup {
+    unsigned long long mask;   // tokens of the batch bucketed to this group
+    int group, T, off, f;      // group id (offloaded experts: device slot), tokens, first slot, inner dim
+    int p1, p2;                // first phase-1 / phase-2 unit of the group
+};
+static_assert(sizeof(TcGroup) == 32, "layout");
+
 struct TcPlan {
     int feasible;
     int n_cta;
@@ -119,7 +128,7 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     // (1 KiB) and right behind them their lo rows (a group never has more tokens than B)
     p.stage_bytes = kTcWTile + 2048 * ((B + 7) / 8);
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
-    p.tab_bytes = ((int)sizeof(StGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
+    p.tab_bytes = ((int)sizeof(TcGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
     // The ring is what keeps HBM busy (bytes in flight = stages x 16 KiB per SM, against a loaded
     // latency of 2-3 us), so shared memory goes to stages first: the hidden-state tiles stay
     // resident only if the ring reaches its maximum depth anyway, otherwise every stage fetches
@@ -362,13 +371,13 @@ struct TcUnit {                        // plain ints: the single-thread roles re
     int first, last;                   // first / last unit of an accumulation run (see the kernel)
 };
 
-__device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active, int total1, int u, int d, int n1)
+__device__ __forceinline__ TcUnit tc_decode(const TcGroup *groups, int n_active, int total1, int u, int d, int n1)
 {
     TcUnit t;
     if (u < total1) {
         t.phase = 1;
         t.a = upper_group1(groups, n_active, u);
-        const StGroup &g = groups[t.a];
+        const TcGroup &g = groups[t.a];
         const int local = u - g.p1, kp = tc_kpieces(d), rbs = (g.f + 127) / 128;
         const int piece = local % kp, rest = local / kp;
         t.rb = rest % rbs;
@@ -380,7 +389,7 @@ __device__ __forceinline__ TcUnit tc_decode(const StGroup *groups, int n_active,
         t.phase = 2;
         const int v = u - total1;
         t.a = upper_group2(groups, n_active, v);
-        const StGroup &g = groups[t.a];
+        const TcGroup &g = groups[t.a];
         const int local = v - g.p2, kp = tc_kpieces(g.f);
         const int piece = local % kp;
         t.rb = local / kp;
@@ -440,9 +449,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     const int n_slots = p.B * sh.k + sh.n_sh * p.B;          // every token fills k routed slots
     const int G = sh.E + sh.n_sh;
 
-    StGroup *groups = reinterpret_cast<StGroup *>(tc_smem);
-    const int tab_rest = pl.tab_bytes - (int)sizeof(StGroup) * (G + 1);
-    int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(StGroup) * (G + 1));
+    TcGroup *groups = reinterpret_cast<TcGroup *>(tc_smem);
+    const int tab_rest = pl.tab_bytes - (int)sizeof(TcGroup) * (G + 1);
+    int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(TcGroup) * (G + 1));
     float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
     uint8_t *xres = tc_smem + pl.tab_bytes;
     xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
@@ -458,7 +467,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     for (int a = tid; a < G; a += blockDim.x) {
         const uint4 r0 = ws.gtab[2 * a], r1 = ws.gtab[2 * a + 1];
         if (a < n_active) {
-            StGroup gr;
+            TcGroup gr;
             gr.group = (int)r0.x;
             // offloaded experts: from here on the group id of a routed expert is the device slot its
             // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
@@ -470,8 +479,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const int r = a < U ? a : U, s = a < U ? 0 : a - U;
             gr.p1 = r * u1r + s * u1s;
             gr.p2 = r * u2r + s * u2s;
-            gr.nks = 0;
-            gr.ksl = 0;
             groups[a] = gr;
         }
     }
@@ -610,7 +617,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 bool progress = false;
                 if (pi < n_units && mbar_test(&empty_bar[s], ring_par)) {
                     TCT(const long long c2 = clock64();)
-                    const StGroup &g = groups[pu.a];
+                    const TcGroup &g = groups[pu.a];
                     const bool shared = g.group >= sh.E;
                     const int e = shared ? g.group - sh.E : g.group;
                     const int row0 = e * (pu.mat == 2 ? sh.d : g.f) + pu.rb * 128;
@@ -647,7 +654,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                             tma_load_3d(op, &maps.m[6], 0, 0, tkt, &a_full[ta]);
                         } else {
                             // one copy per 8 slots for all KG k-tiles: [hi | lo][k-tile][8 rows]
-                            const StGroup &g = groups[tu.a];
+                            const TcGroup &g = groups[tu.a];
                             const bool shared = g.group >= sh.E;
                             const int srow = shared ? g.off - n_routed : g.off;
                             mbar_expect_tx(&a_full[ta], (uint32_t)(KG * tu.n * 128));
@@ -717,7 +724,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             for (int i = 0; i < n_units && alive; ++i) {
                 TCT(const long long cu = clock64();)
                 const TcUnit t = unit_at(i);
-                const StGroup &g = groups[t.a];
+                const TcGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
                 const int e = shared ? g.group - sh.E : g.group;
                 const CUtensorMap *wmap = &maps.m[(shared ? 3 : 0) + t.mat];
@@ -1132,7 +1139,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 if (!service(seg_of_unit((int)ui))) { alive = false; break; }
                 const TcUnit t = unit_at((int)ui);
                 if (!t.last) continue;                 // the run's accumulator is read after its last unit
-                const StGroup &g = groups[t.a];
+                const TcGroup &g = groups[t.a];
                 const int buf = run & 1;
                 TCT(long long c0 = clock64();)
                 if (!mbar_wait(&acc_full[buf], (run >> 1) & 1u)) {
