@@ -2,7 +2,7 @@
 //
 //   route_kernel : l_{b,e} = h_b . W_r[e] (and the shared-expert gate logit) in float64, so
 //                  that the discrete choices below do not depend on the summation order;
-//                  the last block to finish then runs gating_block:
+//                  block 0 then runs gating_block once every row has arrived:
 //   gating_block : Eq. 4 aggregation, TopCap, lambda_b, biased top-k, mixing weights,
 //                  union / unique count, token->expert bucketing, stage tables.
 #pragma once
