@@ -749,8 +749,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const int wv = t.a >= a_split ? 1 : 0;
                 bool ready = t.phase == 1 || wv < ready_w;
                 if (!ready) {
-                    // tiles still pending belong to an earlier wave only if that wave is not ready either
-                    if (pend_n > 0 && wv > ready_w) { if (!wait_ready(ready_w)) { alive = false; break; } }
+                    // the pending tiles all belong to one wave (pend_wave); if that is an earlier wave than
+                    // this unit's, it has to become ready before tiles of this wave may be pending.  (A CTA
+                    // without second-projection units of wave 0 reaches here with ready_w still 0 and
+                    // tiles of wave 1 pending: those must wait for wave 1, not for wave 0.)
+                    if (pend_n > 0 && wv > pend_wave) { if (!wait_ready(pend_wave)) { alive = false; break; } }
                     if (s_ready[wv]) {
                         alive = wait_ready(wv);
                         ready = alive;
