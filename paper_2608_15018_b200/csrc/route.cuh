@@ -267,6 +267,7 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
 
 // Gating of one batch by one thread block of at least two warps.
 // s_l: shared memory for B*E doubles (the logits, copied from the workspace).
+template <int JE>
 __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
                                              int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
                                              int32_t *__restrict__ n_unique, double *s_l)
@@ -331,9 +332,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     } else {
 #pragma unroll 1
         for (int b = warp; b < B; b += tw) {
-            if (E <= 64) gate_stats<2>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
-            else if (E <= 128) gate_stats<4>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
-            else gate_stats<8>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
+            gate_stats<JE>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
         }
     }
     __syncthreads();
@@ -341,9 +340,7 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     GATE_MARK();
 #pragma unroll 1
     for (int b = warp; b < B; b += nw) {
-        if (E <= 64) gate_select<2>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
-        else if (E <= 128) gate_select<4>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
-        else gate_select<8>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
+        gate_select<JE>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
     }
     __syncthreads();
 
@@ -556,7 +553,9 @@ __device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const
 // shared-expert gate vector) against all B tokens in float64; the block that finishes last
 // (atomic ticket, nobody waits) then runs the gating for the whole batch.
 // Dynamic shared memory: max(B * E, 16 * kRouteTok) doubles.
-template <int ACT, int RT>
+// JE: experts per lane in the gating (2, 4 or 8 for up to 64, 128, 256 experts): a kernel of its own
+// for each, so that the gating code of a launch is one straight piece
+template <int ACT, int RT, int JE>
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
              const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
@@ -631,16 +630,16 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
 #ifdef S2MOE_GATE_TWICE
     {   // experiment: the same gating a second time, with whatever the first run left in the caches
         const long long g0 = clock64();
-        gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+        gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
         __syncthreads();
         const long long g1 = clock64();
-        gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+        gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
         __syncthreads();
         const long long g2 = clock64();
         if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[30] = g1 - g0; tm[31] = g2 - g1; }
     }
 #else
-    gating_block(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+    gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
 #endif
 }
 

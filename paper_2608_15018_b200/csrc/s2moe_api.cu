@@ -206,8 +206,15 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
     }
     LaunchScope scope(ctx, KC_ROUTER, st);
     cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st);
-    cudaLaunchKernelEx(&lc, route_kernel<ACT, RT>, sh, B, ctx->ws, hidden, (const void *)lp.router,
-                       (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+    if (sh.E <= 64)
+        cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+    else if (sh.E <= 128)
+        cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 4>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+    else
+        cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 8>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
 }
 
 void launch_route(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
@@ -220,13 +227,22 @@ void launch_route(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, c
     else launch_route_t<DT_BF16, DT_BF16>(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
 }
 
+template <int ACT, int RT>
+cudaError_t prepare_route_t(int bytes)
+{
+    cudaError_t e = cudaFuncSetAttribute(route_kernel<ACT, RT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<ACT, RT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<ACT, RT, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
+}
+
 cudaError_t prepare_route()
 {
     const int bytes = (int)(sizeof(double) * kMaxTokens * kMaxExperts);
-    cudaError_t e = cudaFuncSetAttribute(route_kernel<DT_F32, DT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_F32, DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_BF16, DT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<DT_BF16, DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaError_t e = prepare_route_t<DT_F32, DT_F32>(bytes);
+    if (e == cudaSuccess) e = prepare_route_t<DT_F32, DT_BF16>(bytes);
+    if (e == cudaSuccess) e = prepare_route_t<DT_BF16, DT_F32>(bytes);
+    if (e == cudaSuccess) e = prepare_route_t<DT_BF16, DT_BF16>(bytes);
     return e;
 }
 
@@ -1055,18 +1071,21 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
     const int rows = sh.E + (gate_vec ? 1 : 0);
     const size_t smem = route_smem(n_tokens, sh.E);
     const bool af = sh.act_dtype == DT_F32, rf = sh.router_dtype == DT_F32;
-    if (af && rf)
-        route_kernel<DT_F32, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                        sel_idx, sel_w, n_unique, ZeroList{});
-    else if (af)
-        route_kernel<DT_F32, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                         sel_idx, sel_w, n_unique, ZeroList{});
-    else if (rf)
-        route_kernel<DT_BF16, DT_F32><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                         sel_idx, sel_w, n_unique, ZeroList{});
-    else
-        route_kernel<DT_BF16, DT_BF16><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf,
-                                                                          sel_idx, sel_w, n_unique, ZeroList{});
+    // (the no-allocation entry covers up to 128 experts: two or four per lane in the gating)
+#define S2MOE_ROUTE_NA(A, R)                                                                                         \
+    do {                                                                                                             \
+        if (sh.E <= 64)                                                                                              \
+            route_kernel<A, R, 2><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf, \
+                                                                     sel_idx, sel_w, n_unique, ZeroList{});          \
+        else                                                                                                         \
+            route_kernel<A, R, 4><<<rows, kRouteThreads, smem, st>>>(sh, n_tokens, ws, hidden, router, gate_vec, conf, \
+                                                                     sel_idx, sel_w, n_unique, ZeroList{});          \
+    } while (0)
+    if (af && rf) S2MOE_ROUTE_NA(DT_F32, DT_F32);
+    else if (af) S2MOE_ROUTE_NA(DT_F32, DT_BF16);
+    else if (rf) S2MOE_ROUTE_NA(DT_BF16, DT_F32);
+    else S2MOE_ROUTE_NA(DT_BF16, DT_BF16);
+#undef S2MOE_ROUTE_NA
     if (gate_vec && gate_out) noalloc_gate_out_kernel<<<1, 64, 0, st>>>(ws.gate_logit, gate_out, n_tokens);
     return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
 }
