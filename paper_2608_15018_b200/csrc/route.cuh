@@ -507,15 +507,18 @@ struct ZeroList {
     const uint4 *perm_src;
     uint4 *perm_dst;
     unsigned long long perm_n16;
+    // logit pass: the tokens of a batch are split into this many groups, each with its own set of
+    // row blocks (0 and 1: every row block takes all tokens)
+    int groups;
 };
 
 // One pass of a router row over NT tokens b0 .. b0 + NT - 1 (indices past B - 1 repeat token
 // B - 1, so that every load is unconditional and issued before the first use).
 template <int ACT, int RT, int NT>
-__device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const Workspace &ws, const uint8_t *wrow,
+__device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const Workspace &ws, int row, const uint8_t *wrow,
                                            const void *__restrict__ hidden, double *s_part)
 {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, d = sh.d, row = blockIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, d = sh.d;
     const size_t ab = ACT == DT_F32 ? 4 : 2;
     double acc[NT];
 #pragma unroll
@@ -549,9 +552,9 @@ __device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const
     __syncthreads();
 }
 
-// Router logits and gating in one launch.  Block r computes row r of the router (row E is the
-// shared-expert gate vector) against all B tokens in float64; the block that finishes last
-// (atomic ticket, nobody waits) then runs the gating for the whole batch.
+// Router logits and gating in one launch.  A block computes one row of the router (row E is the
+// shared-expert gate vector) against one group of the batch's tokens in float64; block 0 then
+// runs the gating for the whole batch once every block has arrived (atomic ticket).
 // Dynamic shared memory: max(B * E, 16 * kRouteTok) doubles.
 // JE: experts per lane in the gating (2, 4 or 8 for up to 64, 128, 256 experts): a kernel of its own
 // for each, so that the gating code of a launch is one straight piece
@@ -587,17 +590,23 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     }
     // blocks past the router's rows exist only to help with the clearing and the copy above (a
     // layer with few experts and wide accumulators would otherwise clear megabytes with a few blocks)
+    // A row block takes one router row and one group of tokens: a larger batch is split over
+    // several sets of row blocks (as many as fit on the SMs beside each other), because a block
+    // takes 16 tokens per pass and its passes run one after the other (B = 64: 22 us in one set).
     const int n_rows = sh.E + (sh_scale ? 1 : 0);
-    if ((int)blockIdx.x >= n_rows) return;
-    const int row = blockIdx.x, d = sh.d;
+    const int n_grp = zl.groups > 1 ? zl.groups : 1, n_arrive = n_rows * n_grp;
+    if ((int)blockIdx.x >= n_arrive) return;
+    const int row = (int)blockIdx.x % n_rows, grp = (int)blockIdx.x / n_rows, d = sh.d;
+    const int tg = 8 * ((B + 8 * n_grp - 1) / (8 * n_grp));            // tokens per group, a multiple of 8
+    const int b_lo = min(B, grp * tg), b_hi = min(B, b_lo + tg);
     const size_t rb = RT == DT_F32 ? 4 : 2;
     const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
                                      : reinterpret_cast<const uint8_t *>(sh_scale);
-    for (int b0 = 0; b0 < B;) {
-        const int left = B - b0;
-        if (left > 8) { route_pass<ACT, RT, 16>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 16; }
-        else if (left > 4) { route_pass<ACT, RT, 8>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 8; }
-        else { route_pass<ACT, RT, 4>(sh, B, b0, ws, wrow, hidden, s_dyn); b0 += 4; }
+    for (int b0 = b_lo; b0 < b_hi;) {
+        const int left = b_hi - b0;
+        if (left > 8) { route_pass<ACT, RT, 16>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 16; }
+        else if (left > 4) { route_pass<ACT, RT, 8>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 8; }
+        else { route_pass<ACT, RT, 4>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 4; }
     }
     // Block 0 runs the gating once every row has arrived (its SM tends to be the same from layer
     // to layer, so part of the gating code is still in its instruction cache: measured 0.6 % of
@@ -609,12 +618,12 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
         unsigned t;
         asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(t) : "l"(ws.ticket) : "memory");
         int ok = blockIdx.x == 0 ? 1 : 0;
-        if (blockIdx.x == 0 && t != (unsigned)n_rows - 1) {
+        if (blockIdx.x == 0 && t != (unsigned)n_arrive - 1) {
             ok = 0;
             for (unsigned i = 0; i < (1u << 22); ++i) {
                 unsigned v;
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ws.ticket) : "memory");
-                if (v >= (unsigned)n_rows) { ok = 1; break; }
+                if (v >= (unsigned)n_arrive) { ok = 1; break; }
                 __nanosleep(20);
             }
             if (!ok) atomicExch(ws.status, ST_TICKET_TIMEOUT);

@@ -198,23 +198,31 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
     // 16 bytes per thread and pass, a handful of passes at most
     const int rows = sh.E + (lp.sh_scale ? 1 : 0);
     const unsigned long long units = zl.n16[0] + zl.n16[1] + zl.n16[2] + zl.perm_n16;
-    int grid = rows;
+    // batches of more than 8 tokens: their tokens in groups of at least 8, each group with its own
+    // set of row blocks, as many sets as run beside each other (a block per SM)
+    ZeroList zg = zl;
+    zg.groups = 1;
+    if (B > 8) {
+        const int fit = ctx->n_sm / rows, want = (B + 7) / 8;
+        zg.groups = fit < 1 ? 1 : (want < fit ? want : fit);
+    }
+    int grid = rows * zg.groups;
     if (units > (unsigned long long)rows * kRouteThreads * 4) {
         const unsigned long long want = (units + kRouteThreads * 4 - 1) / (kRouteThreads * 4);
         grid = (int)(want > (unsigned long long)ctx->n_sm ? (unsigned long long)ctx->n_sm : want);
-        if (grid < rows) grid = rows;
+        if (grid < rows * zg.groups) grid = rows * zg.groups;
     }
     LaunchScope scope(ctx, KC_ROUTER, st);
     cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st);
     if (sh.E <= 64)
         cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
-                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
     else if (sh.E <= 128)
         cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 4>, sh, B, ctx->ws, hidden, (const void *)lp.router,
-                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
     else
         cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 8>, sh, B, ctx->ws, hidden, (const void *)lp.router,
-                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+                           (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
 }
 
 void launch_route(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B, const void *hidden, const float *conf,
