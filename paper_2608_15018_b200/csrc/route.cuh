@@ -597,7 +597,7 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     const int n_grp = zl.groups > 1 ? zl.groups : 1, n_arrive = n_rows * n_grp;
     if ((int)blockIdx.x >= n_arrive) return;
     const int row = (int)blockIdx.x % n_rows, grp = (int)blockIdx.x / n_rows, d = sh.d;
-    const int tg = 8 * ((B + 8 * n_grp - 1) / (8 * n_grp));            // tokens per group, a multiple of 8
+    const int tg = 4 * ((B + 4 * n_grp - 1) / (4 * n_grp));            // tokens per group, a multiple of 4
     const int b_lo = min(B, grp * tg), b_hi = min(B, b_lo + tg);
     const size_t rb = RT == DT_F32 ? 4 : 2;
     const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb

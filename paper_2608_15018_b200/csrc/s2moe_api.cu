@@ -198,12 +198,13 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
     // 16 bytes per thread and pass, a handful of passes at most
     const int rows = sh.E + (lp.sh_scale ? 1 : 0);
     const unsigned long long units = zl.n16[0] + zl.n16[1] + zl.n16[2] + zl.perm_n16;
-    // batches of more than 8 tokens: their tokens in groups of at least 8, each group with its own
-    // set of row blocks, as many sets as run beside each other (a block per SM)
+    // batches of more than 4 tokens: their tokens in groups of at least 4, each group with its own
+    // set of row blocks, as many sets as run beside each other (a block per SM); measured at 64
+    // experts: 1.1 % of a layer at B = 8, 4.5 % at B = 16
     ZeroList zg = zl;
     zg.groups = 1;
-    if (B > 8) {
-        const int fit = ctx->n_sm / rows, want = (B + 7) / 8;
+    if (B > 4) {
+        const int fit = ctx->n_sm / rows, want = (B + 3) / 4;
         zg.groups = fit < 1 ? 1 : (want < fit ? want : fit);
     }
     int grid = rows * zg.groups;
