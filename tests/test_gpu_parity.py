@@ -160,6 +160,36 @@ def test_stack_host_and_graph_agree_with_single_calls(plan):
     m.close()
 
 
+@pytest.mark.parametrize("L", [1, 2, 5])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_stack_host_layer_counts_and_repeated_calls(L, pinned):
+    """The host-buffer call copies results back in pieces while later layers run: every layer
+    count takes another split, and a second call with other inputs must not see the first's."""
+    wl = SMALL["cfg2"]
+    B = wl.n_tokens
+    m, T = _ctx(wl, L, 3)
+    dev = torch.device("cuda", 0)
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    for rep in range(2):
+        w = wl.with_(seed=wl.seed + 77 * rep)
+        H = torch.stack([workloads.hidden_states(w, l, device=dev) for l in range(L)])
+        C = torch.stack([workloads.confidences(w, l, device=dev) for l in range(L)])
+        single = [m.verify_layer(l, H[l], C[l]) for l in range(L)]
+        torch.cuda.synchronize()
+        ref_out = torch.stack([s.out for s in single]).cpu()
+        ref_sel = torch.stack([s.sel_idx for s in single]).cpu()
+        ref_w = torch.stack([s.sel_w for s in single]).cpu()
+        ref_u = torch.cat([s.n_unique for s in single]).cpu()
+        hh, hc = pin(H.cpu()), pin(C.cpu())
+        ho, hs = pin(torch.full_like(ref_out, float("nan"))), pin(torch.full_like(ref_sel, -1))
+        hw, hu = pin(torch.full_like(ref_w, float("nan"))), pin(torch.full_like(ref_u, -1))
+        m.verify_stack_host(hh, hc, ho, hs, hw, hu)
+        assert torch.equal(hs, ref_sel) and torch.equal(hu, ref_u) and torch.equal(hw, ref_w)
+        assert (ho - ref_out).abs().max().item() <= 1e-5 * ref_out.abs().max().item()
+    assert m.device_status() == 0
+    m.close()
+
+
 def test_argument_errors_on_device():
     wl = SMALL["cfg1"]
     m, T = _ctx(wl, 1, max_tokens=8)
