@@ -163,9 +163,10 @@ int s2moe_verify_stack(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden, con
  * s2moe_verify_stack with HOST input and output buffers of the same shapes: copies
  * hidden (and conf, if not NULL) to staging memory the context owns, runs the stack,
  * copies out, sel_idx, sel_w and n_unique back and returns when all of it is complete.
- * The copies overlap the kernels: the inputs of the layers after the first and the results
+ * The copies overlap the kernels: the inputs of the layers after the first and the outputs
  * of all layers but the last travel on two streams the context owns, ordered against
- * cuda_stream by events.  The host buffers must not be touched until the call returns;
+ * cuda_stream by events; sel_idx, sel_w and n_unique of all layers arrive in one copy in
+ * page-locked memory of the context and are copied from there by the calling thread.  The host buffers must not be touched until the call returns;
  * page-locked host memory is needed for the overlap (pageable memory works, serialised).
  */
 int s2moe_verify_stack_host(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden_host,

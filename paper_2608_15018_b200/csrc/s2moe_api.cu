@@ -66,7 +66,8 @@ struct s2moe_ctx {
     int64_t fetched_bytes = 0;
     // host-buffer entry point: streams and events of its copies, made at the first call
     cudaStream_t cs_in = nullptr, cs_out = nullptr;
-    cudaEvent_t ev_copy[3] = {nullptr, nullptr, nullptr};
+    cudaEvent_t ev_copy[4] = {nullptr, nullptr, nullptr, nullptr};
+    uint8_t *h_small = nullptr;           // page-locked landing place of the indices, weights and counts
 };
 
 struct s2moe_cache {
@@ -858,54 +859,70 @@ int s2moe_verify_stack_host(s2moe_ctx *ctx, int32_t n_tokens, const void *hidden
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const Shape &sh = ctx->shape;
     const size_t ab = sh.act_dtype == DT_F32 ? 4 : 2, L = (size_t)ctx->cfg.n_layers, B = (size_t)n_tokens;
-    // The copies run beside the kernels: the first layer's inputs go ahead on the caller's stream and
-    // the other layers' follow on a stream of their own; the results of the layers up to the middle
-    // of the stack, and of those up to the last but one, leave on a third stream while the later
-    // layers run, so that only the last layer's results are copied after the last kernel.
+    // The copies run beside the kernels.  In: the first layer's inputs go ahead on the caller's
+    // stream, the other layers' follow on a stream of their own once the first layer is launched.
+    // Out: the outputs of the layers up to the middle of the stack, and of those up to the last but
+    // one, leave on a third stream while the later layers run; after the last kernel the last
+    // layer's outputs and, in one copy into page-locked memory of the context, the indices, weights
+    // and counts of all layers travel on two streams at once.
     if (!ctx->cs_in) CU(ctx, cudaStreamCreateWithFlags(&ctx->cs_in, cudaStreamNonBlocking));
     if (!ctx->cs_out) CU(ctx, cudaStreamCreateWithFlags(&ctx->cs_out, cudaStreamNonBlocking));
     for (cudaEvent_t &ev : ctx->ev_copy)
         if (!ev) CU(ctx, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    // st_sel, st_selw and st_nu lie one after the other in the workspace, sized for max_tokens: this
+    // call packs its indices, weights and counts at the front of that region
+    const size_t region = (size_t)((const uint8_t *)(ctx->st_nu + L) - (const uint8_t *)ctx->st_sel);
+    if (!ctx->h_small) CU(ctx, cudaHostAlloc((void **)&ctx->h_small, region, cudaHostAllocDefault));
+    const size_t nsel = L * B * sh.k * 4, small_bytes = 2 * nsel + L * 4;
+    uint8_t *const d_small = (uint8_t *)ctx->st_sel;
+    int32_t *const d_sel = (int32_t *)d_small, *const d_nu = (int32_t *)(d_small + 2 * nsel);
+    float *const d_selw = (float *)(d_small + nsel);
     const size_t hb = B * sh.d * ab;
     const int nl = (int)L;
     CU(ctx, cudaMemcpyAsync(ctx->st_hidden, hidden_host, hb, cudaMemcpyHostToDevice, st));
     if (conf_host) CU(ctx, cudaMemcpyAsync(ctx->st_conf, conf_host, L * B * 4, cudaMemcpyHostToDevice, st));
-    if (nl > 1) {
-        CU(ctx, cudaMemcpyAsync((uint8_t *)ctx->st_hidden + hb, (const uint8_t *)hidden_host + hb, (L - 1) * hb,
-                                cudaMemcpyHostToDevice, ctx->cs_in));
-        CU(ctx, cudaEventRecord(ctx->ev_copy[0], ctx->cs_in));
-    }
-    auto copy_back = [&](int lo, int hi, cudaStream_t cs) -> int {     // layers lo .. hi - 1
-        const size_t o = (size_t)lo * B, n = (size_t)(hi - lo) * B;
-        CU(ctx, cudaMemcpyAsync(out_host + o * sh.d, ctx->st_out + o * sh.d, n * sh.d * 4, cudaMemcpyDeviceToHost, cs));
-        CU(ctx, cudaMemcpyAsync(sel_idx_host + o * sh.k, ctx->st_sel + o * sh.k, n * sh.k * 4, cudaMemcpyDeviceToHost, cs));
-        CU(ctx, cudaMemcpyAsync(sel_w_host + o * sh.k, ctx->st_selw + o * sh.k, n * sh.k * 4, cudaMemcpyDeviceToHost, cs));
-        CU(ctx, cudaMemcpyAsync(n_unique_host + lo, ctx->st_nu + lo, (size_t)(hi - lo) * 4, cudaMemcpyDeviceToHost, cs));
+    auto copy_out = [&](int lo, int hi, cudaStream_t cs) -> int {      // outputs of layers lo .. hi - 1
+        const size_t o = (size_t)lo * B * sh.d, n = (size_t)(hi - lo) * B * sh.d;
+        CU(ctx, cudaMemcpyAsync(out_host + o, ctx->st_out + o, n * 4, cudaMemcpyDeviceToHost, cs));
         return S2MOE_OK;
     };
     const int cut1 = nl >= 4 ? nl / 2 : 0, cut2 = nl >= 2 ? nl - 1 : 0;   // layers copied early: [0, cut1), [cut1, cut2)
     int done = 0, rc = S2MOE_OK;
     for (int l = 0; l < nl && rc == S2MOE_OK; ++l) {
-        if (l == 1) CU(ctx, cudaStreamWaitEvent(st, ctx->ev_copy[0], 0));
+        if (l == 1) {
+            CU(ctx, cudaMemcpyAsync((uint8_t *)ctx->st_hidden + hb, (const uint8_t *)hidden_host + hb, (L - 1) * hb,
+                                    cudaMemcpyHostToDevice, ctx->cs_in));
+            CU(ctx, cudaEventRecord(ctx->ev_copy[0], ctx->cs_in));
+            CU(ctx, cudaStreamWaitEvent(st, ctx->ev_copy[0], 0));
+        }
         rc = verify_one(ctx, l, n_tokens, (const uint8_t *)ctx->st_hidden + (size_t)l * hb,
                         conf_host ? ctx->st_conf + (size_t)l * B : nullptr, ctx->st_out + (size_t)l * B * sh.d,
-                        ctx->st_sel + (size_t)l * B * sh.k, ctx->st_selw + (size_t)l * B * sh.k, ctx->st_nu + l, st);
+                        d_sel + (size_t)l * B * sh.k, d_selw + (size_t)l * B * sh.k, d_nu + l, st);
         if (rc == S2MOE_OK && (l + 1 == cut1 || l + 1 == cut2) && l + 1 > done) {
             cudaEvent_t ev = ctx->ev_copy[l + 1 == cut1 ? 1 : 2];
             CU(ctx, cudaEventRecord(ev, st));
             CU(ctx, cudaStreamWaitEvent(ctx->cs_out, ev, 0));
-            rc = copy_back(done, l + 1, ctx->cs_out);
+            rc = copy_out(done, l + 1, ctx->cs_out);
             done = l + 1;
         }
     }
-    if (rc == S2MOE_OK) rc = copy_back(done, nl, st);
-    // both streams are drained whatever happened, so that no copy of this call outlives it
+    if (rc == S2MOE_OK) {
+        CU(ctx, cudaEventRecord(ctx->ev_copy[3], st));
+        CU(ctx, cudaStreamWaitEvent(ctx->cs_out, ctx->ev_copy[3], 0));
+        CU(ctx, cudaMemcpyAsync(ctx->h_small, d_small, small_bytes, cudaMemcpyDeviceToHost, ctx->cs_out));
+        rc = copy_out(done, nl, st);
+    }
+    // all streams are drained whatever happened, so that no copy of this call outlives it
     const cudaError_t e1 = cudaStreamSynchronize(st), e2 = cudaStreamSynchronize(ctx->cs_out),
                       e3 = cudaStreamSynchronize(ctx->cs_in);
     if (rc != S2MOE_OK) return rc;
     CU(ctx, e1);
     CU(ctx, e2);
     CU(ctx, e3);
+    const uint8_t *hs = ctx->h_small;
+    memcpy(sel_idx_host, hs, nsel);
+    memcpy(sel_w_host, hs + nsel, nsel);
+    memcpy(n_unique_host, hs + 2 * nsel, L * 4);
     return S2MOE_OK;
 }
 
@@ -920,6 +937,7 @@ int s2moe_destroy(s2moe_ctx *ctx)
     if (ctx->h_slot_of) cudaFreeHost(ctx->h_slot_of);
     for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
     for (cudaEvent_t ev : ctx->ev_copy) if (ev) cudaEventDestroy(ev);
+    if (ctx->h_small) cudaFreeHost(ctx->h_small);
     if (ctx->cs_in) cudaStreamDestroy(ctx->cs_in);
     if (ctx->cs_out) cudaStreamDestroy(ctx->cs_out);
     delete ctx;
