@@ -637,15 +637,17 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[15] = t_start; tm[14] = clock64(); }
 #endif
 #ifdef S2MOE_GATE_TWICE
-    {   // experiment: the same gating a second time, with whatever the first run left in the caches
-        const long long g0 = clock64();
-        gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
-        __syncthreads();
-        const long long g1 = clock64();
-        gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
-        __syncthreads();
-        const long long g2 = clock64();
-        if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[30] = g1 - g0; tm[31] = g2 - g1; }
+    {   // experiment: the same gating code (one copy, in a loop) a second time, with whatever the
+        // first run left in the caches
+        long long g[3];
+        g[0] = clock64();
+#pragma unroll 1
+        for (int rep = 0; rep < 2; ++rep) {
+            gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+            __syncthreads();
+            g[rep + 1] = clock64();
+        }
+        if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[30] = g[1] - g[0]; tm[31] = g[2] - g[1]; }
     }
 #else
     gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
