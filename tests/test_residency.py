@@ -152,6 +152,39 @@ def test_offloaded_context_matches_oracle_and_resident_context(weights):
 
 
 @pytest.mark.gpu
+def test_offloaded_context_through_the_host_buffer_stack_call():
+    """The stack call with host buffers overlaps its copies with the layers; an offloaded context
+    meets the host between the two kernels of every layer on top of that: same results as resident."""
+    from paper_2608_15018_b200 import workloads
+    from paper_2608_15018_b200.workloads import CONFIGS
+
+    wl = CONFIGS["cfg2"].with_(d_model=512, d_ff=512, n_experts=16, top_k=2, cap=4, n_layers=5)
+    dev = torch.device("cuda", 0)
+    L, B = wl.n_layers, 4
+    layers = [workloads.layer_weights(wl, l, dev) for l in range(L)]
+    cfg = binding.Config.from_workload(wl, n_layers=L, kernel_plan=3)
+    with binding.S2MoE(cfg, layers) as res, binding.S2MoE(cfg, _offloaded_layers(layers), n_slots=10) as off:
+        for step in range(3):
+            w = wl.with_(seed=wl.seed + 31 * step)
+            H = torch.stack([workloads.hidden_states(w, l, B, 0.5, dev) for l in range(L)])
+            C = torch.stack([workloads.confidences(w, l, B, dev) for l in range(L)])
+            want = res.verify_stack(H, C)
+            torch.cuda.synchronize()
+            hh, hc = H.cpu().pin_memory(), C.cpu().pin_memory()
+            ho = torch.full_like(want.out.cpu(), float("nan")).pin_memory()
+            hs = torch.full_like(want.sel_idx.cpu(), -1).pin_memory()
+            hw = torch.full_like(want.sel_w.cpu(), float("nan")).pin_memory()
+            hu = torch.full_like(want.n_unique.cpu(), -1).pin_memory()
+            off.verify_stack_host(hh, hc, ho, hs, hw, hu)
+            assert torch.equal(hs, want.sel_idx.cpu()) and torch.equal(hu, want.n_unique.cpu())
+            assert torch.equal(hw, want.sel_w.cpu())
+            assert torch.allclose(ho, want.out.cpu(), rtol=1e-5, atol=1e-6)
+        hits, misses, _ = off.residency_stats()
+        assert misses > 0 and hits + misses > 0
+        assert off.device_status() == 0
+
+
+@pytest.mark.gpu
 def test_offloaded_context_errors():
     from paper_2608_15018_b200 import workloads
     from paper_2608_15018_b200.workloads import CONFIGS
