@@ -72,11 +72,13 @@ constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the res
 constexpr unsigned kTcSpinLimit = 1u << 22;
 constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
 // Share of the experts in wave 0.  A little more than half: the second projection of wave 0 is
-// what hides the hand-over of wave 1 (measured at the OLMoE-like shape: 9/16 and 5/8 beat 1/2
-// and 11/16).
+// what hides the hand-over of wave 1.  Measured again with the kernel as it stands, 16 layers of
+// the OLMoE-like shape: 0.7757 ms per step at 1/2, 0.7746 at 9/16, 0.7791 at 5/8, 0.7767 at 11/16,
+// 0.7830 at 3/4; 9/16 also takes 1 to 3 % off the shapes with shared experts and costs 0.7 % at
+// 64 tokens.
 #ifndef S2MOE_SPLIT_NUM
-#define S2MOE_SPLIT_NUM 5
-#define S2MOE_SPLIT_DEN 8
+#define S2MOE_SPLIT_NUM 9
+#define S2MOE_SPLIT_DEN 16
 #endif
 constexpr int kTcSplitNum = S2MOE_SPLIT_NUM, kTcSplitDen = S2MOE_SPLIT_DEN;
 constexpr int kTcReady = 512;                  // ws.sync[kTcReady - 8 + w], [kTcReady - 4 + w]: the two counters of wave w
