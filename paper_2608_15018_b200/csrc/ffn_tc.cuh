@@ -1025,7 +1025,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 bool ok = false;
                 for (unsigned i = 0; i < (1u << 21); ++i) {
                     if (ld_acquire(&ws.sync[kTcReady - 4 + w]) >= (int)gridDim.x) { ok = true; break; }
-                    __nanosleep(100);
+                    __nanosleep(32);
                 }
                 if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); break; }
                 __threadfence_block();
@@ -1051,7 +1051,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 bool ok = false;
                 for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
                     if (ld_acquire(&ws.sync[kTcReady - 8 + w]) >= (int)gridDim.x) { ok = true; break; }
-                    __nanosleep(40);
+                    __nanosleep(16);
                 }
                 if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
                 s_flag = ok;
@@ -1107,7 +1107,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             bool ok = false;
             for (unsigned i = 0; i < (1u << 22); ++i) {
                 if (mbar_try_wait(&conv_go[w], 0)) { ok = true; break; }
-                __nanosleep(64);
+                __nanosleep(24);
             }
             if (!ok) { if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
             if (et == 0) tc_red_release(&ws.sync[kTcReady - 8 + w]);   // orders the CTA's reductions, observed through conv_go
