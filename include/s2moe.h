@@ -312,6 +312,10 @@ int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
  * words that must start at zero, the rest keeps the previous call's contents, and two
  * calls that overlap on the GPU (different streams, no ordering between them) race.
  * Errors: EINVAL (null pointer, bad config, misaligned hidden or router), ERANGE, ECUDA.
+ * The one bounded wait of the routing kernel reports through a status word inside the
+ * scratch array, which every call clears: if that wait ever gives up, sel_idx, sel_w and
+ * n_unique of that call stay unwritten although the call returned OK.  A caller that wants
+ * to know reads the word with s2moe_route_noalloc_status before its next call.
  */
 #define S2MOE_NOALLOC_MAX_TOKENS 64
 #define S2MOE_NOALLOC_MAX_EXPERTS 128
@@ -319,6 +323,14 @@ int s2moe_debug_read(s2moe_ctx *ctx, int32_t what, void *host_out, size_t bytes)
 int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *router, const void *gate_vec,
                         const void *hidden, const float *conf, int32_t *sel_idx, float *sel_w,
                         int32_t *n_unique, float *gate_out, void *cuda_stream);
+
+/*
+ * Device status of the last s2moe_route_noalloc call on the current device (no counterpart in
+ * the paper).  Synchronises the device, copies the status word out of the scratch array (no
+ * allocation) and returns OK with *host_out = 0, or ETIMEOUT with the device code when the
+ * routing kernel's bounded wait gave up.  Before the first call on a device: OK and 0.
+ */
+int s2moe_route_noalloc_status(int32_t *host_out);
 
 /*
  * Routing-aware adaptive speculative expansion (Sec. 4.1): the step that chooses which draft
@@ -346,7 +358,10 @@ int s2moe_expert_masks(const int32_t *sel_idx, int32_t n_tokens, int32_t top_k, 
  * the eligible candidate of largest utility (ties: lowest index) and stops when that utility is
  * below 1.  All of it in float64, one rounding per operation.
  *
- *   n_cand    1 .. S2MOE_EXPAND_MAX_CAND; parents must precede their children
+ *   n_cand    1 .. S2MOE_EXPAND_MAX_CAND; parents must precede their children: a candidate
+ *             whose parent index is not below its own is never admitted (nor is anything
+ *             below it) and the call reports n_admitted = -1; the other outputs then hold
+ *             the result for the well-formed rest
  *   parent    dev [n_cand]   index of the parent candidate, or -1
  *   p_tok     dev [n_cand]   token-level confidence of each candidate
  *   masks     dev [n_cand][n_layers][ceil(n_experts / 64)]   predicted expert sets
@@ -355,7 +370,7 @@ int s2moe_expert_masks(const int32_t *sel_idx, int32_t n_tokens, int32_t top_k, 
  *             more expert in verification; both in the unit of c_draft
  *   admitted  dev [n_cand]   out: 1 / 0
  *   order     dev [n_cand]   out: admitted candidates in admission order, then -1
- *   n_admitted dev scalar    out
+ *   n_admitted dev scalar    out: number of admitted candidates, or -1 (malformed parent[])
  *   union_out dev [n_layers][ceil(n_experts / 64)] or NULL   out: union of the admitted sets
  * Errors: EINVAL (null pointer, bad sizes), ERANGE (n_cand or n_layers * words beyond the
  * limits), ECUDA.

@@ -3,16 +3,19 @@
 TEST INFRASTRUCTURE.  Takes arrays only, so it imports nothing from the CUDA path.
 
 Rules applied
-  * selected experts are compared per token as sets and the unique-expert count
-    exactly.  A differing token is tolerated only as a router tie: the oracle's
+  * selected experts are compared per token exactly and in selection order (biased
+    logit descending, original logit descending, id ascending), and the unique-expert
+    count exactly.  A differing token is tolerated only as a router tie: the oracle's
     margin at that decision (k-th minus (k+1)-th biased logit of the token, or the
-    cap-th minus (cap+1)-th aggregated importance) must be below ``tie_eps``; the
-    oracle is then re-evaluated with the other side's choice forced, and the tie is
-    reported.
+    cap-th minus (cap+1)-th aggregated importance; for a difference in order alone, the
+    gap between the two swapped biased logits) must be below ``tie_eps``; the oracle is
+    then re-evaluated with the other side's choice forced, and the tie is reported.
   * mixing weights are matched by expert id, absolute tolerance ``w_tol``.
   * outputs: per token, max |y - y_ref| / max |y_ref| <= ``y_tol`` (per-token
     infinity-norm relative error; element-wise relative error is meaningless at the
-    zero crossings of y).
+    zero crossings of y); and, so that an error confined to small elements cannot
+    hide under the largest one, the per-token RMS error relative to the RMS of y_ref
+    must stay below ``y_tol / 4``.
 """
 from __future__ import annotations
 
@@ -21,7 +24,7 @@ from typing import List, Optional, Sequence
 
 import numpy as np
 
-from . import Config, Weights, layer as oracle_layer
+from . import Config, Weights, gating as oracle_gating, layer as oracle_layer
 
 
 @dataclass
@@ -32,6 +35,7 @@ class ParityReport:
     n_unique: int = 0
     ties: List[str] = field(default_factory=list)
     tokens_checked: int = 0
+    order_checked: int = 0      # tokens whose selection ORDER was compared exactly
 
 
 def check_layer(cfg: Config, w: Weights, hidden_raw: np.ndarray, conf: Optional[np.ndarray],
@@ -48,6 +52,24 @@ def check_layer(cfg: Config, w: Weights, hidden_raw: np.ndarray, conf: Optional[
     got_sel = np.asarray(got_sel).reshape(B, k)
     got_w = np.asarray(got_w, dtype=np.float64).reshape(B, k)
     mism = [b for b in range(B) if set(got_sel[b].tolist()) != set(ref.sel[b].tolist())]
+    # same set, other order: allowed only between experts whose biased logits differ by less
+    # than the tie threshold in the oracle
+    gate = None
+    for b in range(B):
+        if b in mism:
+            continue
+        if got_sel[b].tolist() == ref.sel[b].tolist():
+            rep.order_checked += 1
+            continue
+        if gate is None:
+            gate = oracle_gating(cfg, ref.logits, conf64)
+        l2 = gate.l2[b]
+        for j in range(k):
+            a, c = int(got_sel[b, j]), int(ref.sel[b, j])
+            if a != c and abs(l2[a] - l2[c]) >= tie_eps:
+                raise AssertionError(f"token {b}: selection order {got_sel[b].tolist()} != oracle "
+                                     f"{ref.sel[b].tolist()} (biased logits {l2[a]:.9g}, {l2[c]:.9g}: not a tie)")
+        rep.ties.append(f"token {b}: order of near-equal biased logits")
     if mism:
         wsum = float(conf64.sum()) if conf64 is not None else float(B)
         cap_tie = ref.m_cap < tie_eps * max(1.0, wsum)
@@ -85,6 +107,7 @@ def check_layer(cfg: Config, w: Weights, hidden_raw: np.ndarray, conf: Optional[
         rep.max_rel_err = float(max(errs)) if errs else 0.0
         rep.tokens_checked = len(toks)
         assert rep.max_rel_err <= y_tol, f"output relative error {rep.max_rel_err:.3e} > {y_tol}"
+        assert rep.rms_rel_err <= y_tol / 4, f"output RMS relative error {rep.rms_rel_err:.3e} > {y_tol / 4}"
     return rep
 
 

@@ -25,7 +25,7 @@ EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_ve
            "s2moe_destroy", "s2moe_strerror", "s2moe_last_device_status", "s2moe_last_cuda_error",
            "s2moe_kernel_launches", "s2moe_unique_expert_bytes", "s2moe_debug_read",
            "s2moe_profile_begin", "s2moe_profile_end", "s2moe_kernel_class_name", "s2moe_kernel_plan",
-           "s2moe_route_noalloc", "s2moe_expert_masks", "s2moe_adaptive_expand", "s2moe_create_offloaded",
+           "s2moe_route_noalloc", "s2moe_route_noalloc_status", "s2moe_expert_masks", "s2moe_adaptive_expand", "s2moe_create_offloaded",
            "s2moe_residency_stats", "s2moe_residency_uses", "s2moe_cache_create", "s2moe_cache_access",
            "s2moe_cache_destroy")
 OFFLOADED_FIELDS = ("w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down")   # host tensors of an offloaded context
@@ -102,6 +102,8 @@ def load_library(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.s2moe_debug_read.restype = ctypes.c_int
     lib.s2moe_route_noalloc.argtypes = [ctypes.POINTER(ConfigC), i32, vp, vp, vp, fp, vp, fp, vp, fp, vp]
     lib.s2moe_route_noalloc.restype = ctypes.c_int
+    lib.s2moe_route_noalloc_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+    lib.s2moe_route_noalloc_status.restype = ctypes.c_int
     lib.s2moe_profile_begin.argtypes = [vp, i32]
     lib.s2moe_profile_begin.restype = ctypes.c_int
     lib.s2moe_profile_end.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
@@ -390,6 +392,16 @@ def route_noalloc(config: Config, hidden: torch.Tensor, router: torch.Tensor,
     if rc != OK:
         raise S2MoEError(rc, "s2moe_route_noalloc")
     return sel_idx, sel_w, n_unique, gate
+
+
+def route_noalloc_status() -> int:
+    """Device status word of the last ``route_noalloc`` call on the current device (0: no bounded
+    wait gave up).  Synchronises the device."""
+    out = ctypes.c_int32(0)
+    rc = load_library().s2moe_route_noalloc_status(ctypes.byref(out))
+    if rc not in (OK, ETIMEOUT):
+        raise S2MoEError(rc, "s2moe_route_noalloc_status")
+    return int(out.value)
 
 
 def expert_masks(sel_idx: torch.Tensor, n_experts: int, out: Optional[torch.Tensor] = None, layer: int = 0,

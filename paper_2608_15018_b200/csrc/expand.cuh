@@ -40,28 +40,35 @@ adaptive_expand_kernel(int n, int lw, const int32_t *__restrict__ parent, const 
     __shared__ unsigned long long s_union[kExpandMaxWords];
     __shared__ double s_wu[kExpandMaxCand / 32];
     __shared__ int s_wi[kExpandMaxCand / 32];
-    __shared__ int s_best, s_count;
+    __shared__ int s_best, s_count, s_bad;
 
     const int i = threadIdx.x, lane = i & 31, warp = i >> 5, nw = blockDim.x >> 5;
     if (i < n) s_adm[i] = 0;
     for (int w = i; w < lw; w += blockDim.x) s_union[w] = 0ull;
     if (i == 0) {
-        // prefix confidence p_i = p_parent * p_{i,j}; parents precede their children
+        // prefix confidence p_i = p_parent * p_{i,j}; parents precede their children.  A parent
+        // index that does not (>= the candidate's own) is not followed: the candidate gets
+        // confidence 0, is never eligible (nor are its descendants) and the call reports it
+        int bad = 0;
         for (int c = 0; c < n; ++c) {
             const int a = parent[c];
+            if (a >= c) { s_p[c] = 0.0; bad = 1; continue; }
             s_p[c] = a < 0 ? (double)p_tok[c] : __dmul_rn(s_p[a], (double)p_tok[c]);
         }
         s_count = 0;
+        s_bad = bad;
     }
     __syncthreads();
-    const int par = i < n ? parent[i] : -1;
+    const int par_in = i < n ? parent[i] : -1;
+    const bool malformed = i < n && par_in >= i;
+    const int par = malformed ? -1 : par_in;
     const double cd = (i < n && c_draft) ? (double)c_draft[i] : 0.0;
     const double benefit = i < n ? __dmul_rn(s_p[i], (double)t_ar) : 0.0;
     const double neg_inf = -__longlong_as_double(0x7ff0000000000000ll), pos_inf = -neg_inf;
 
     for (int step = 0; step < n; ++step) {
         double u = neg_inf;
-        if (i < n && !s_adm[i] && (par < 0 || s_adm[par])) {
+        if (i < n && !malformed && !s_adm[i] && (par < 0 || s_adm[par])) {
             int fresh = 0;                                         // Eq. 2: | E_i \ union |, all layers
             for (int w = 0; w < lw; ++w) fresh += __popcll(masks[(size_t)i * lw + w] & ~s_union[w]);
             const double cost = __dadd_rn(__dmul_rn((double)fresh, (double)t_exp), cd);
@@ -101,7 +108,7 @@ adaptive_expand_kernel(int n, int lw, const int32_t *__restrict__ parent, const 
         admitted[i] = s_adm[i];
         if (i >= s_count) order[i] = -1;
     }
-    if (i == 0) *n_admitted = s_count;
+    if (i == 0) *n_admitted = s_bad ? -1 : s_count;      // -1: parent[] was malformed
     if (union_out)
         for (int w = i; w < lw; w += blockDim.x) union_out[w] = s_union[w];
 }

@@ -90,6 +90,18 @@ struct ExpertCache {
         }
         return true;
     }
+
+    // Undo the residency of an expert whose weights did not arrive in its slot (a failed copy):
+    // the slot is free again and the expert counts as not resident.  Pinned slots are left alone.
+    void evict(int e)
+    {
+        if (e < 0 || e >= n_experts) return;
+        const int s = slot_of[(size_t)e];
+        if (s < n_pinned) return;            // not resident (-1) or pinned
+        slot_of[(size_t)e] = -1;
+        owner[(size_t)s] = -1;
+        last_use[(size_t)s] = 0;
+    }
 };
 
 }  // namespace s2moe

@@ -705,24 +705,12 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
         // waiter saw complete, so two warps must never poll the same slot for different uses.
         const int mt_all = (st_pad8(p.B) + 15) >> 4;
         bool x_ready = false;
-#ifdef S2MOE_TIMING
-        long long t_wait = 0, t_p1 = 0, t_p2 = 0, t_opw = 0, n_st = 0;
-        const long long t_begin = clock64();
-#endif
         for (int n = warp; n < n_mine && warp < S; n += S) {
             const int slot = warp;
-#ifdef S2MOE_TIMING
-            const long long tw0 = clock64();
-#endif
             if (!mbar_wait(&full_bar[slot], ((uint32_t)(n / S)) & 1u)) {
                 if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                 break;
             }
-#ifdef S2MOE_TIMING
-            const long long tw1 = clock64();
-            t_wait += tw1 - tw0;
-            ++n_st;
-#endif
             const StageDesc d = desc[slot];
             const StGroup &gr = groups[d.gslot];
             const uint8_t *wreg = ring + (size_t)slot * pl.slot_bytes;
@@ -740,13 +728,7 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
                 }
             } else {
                 // generation g of the operand completes phase g - 1 of its barrier
-#ifdef S2MOE_TIMING
-                const long long to0 = clock64();
-#endif
                 ok = mbar_wait(&op_bar, (uint32_t)(d.op_gen - 1) & 1u);
-#ifdef S2MOE_TIMING
-                t_opw += clock64() - to0;
-#endif
                 if (ok) {
                     const int mt = (st_pad8(gr.T) + 15) >> 4;
                     if (mt == 1) consume_phase2<1>(p, gr, d, wreg, oreg, s_slot_token, s_slot_w, lane);
@@ -761,16 +743,7 @@ __global__ void __launch_bounds__(kStThreads, 1) ffn_stream_kernel(StreamArgs p)
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[slot]);
-#ifdef S2MOE_TIMING
-            if (d.phase == 1) t_p1 += clock64() - tw1; else t_p2 += clock64() - tw1;
-#endif
         }
-#ifdef S2MOE_TIMING
-        if (lane == 0 && warp < S) {
-            long long *o = reinterpret_cast<long long *>(ws.act) + ((size_t)blockIdx.x * 8 + warp) * 8;
-            o[0] = t_wait; o[1] = t_p1; o[2] = t_p2; o[3] = n_st; o[4] = clock64() - t_begin; o[5] = t_opw;
-        }
-#endif
     }
 }
 

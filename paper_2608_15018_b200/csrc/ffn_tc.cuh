@@ -39,15 +39,6 @@
 #include "common.cuh"
 #include "ffn_stream.cuh"
 
-// cycle-counter statements, compiled only with -DS2MOE_TIMING
-#ifdef S2MOE_TIMING
-#define TCT(...) __VA_ARGS__
-#define TCG(slot) do { unsigned long long g_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_)); (reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32)[slot] = (long long)g_; } while (0)
-#else
-#define TCT(...)
-#define TCG(slot) do { } while (0)
-#endif
-
 namespace s2moe {
 
 constexpr int kTcThreads = 352;                // warps: producer, MMA issuer 0, 4 epilogue, MMA issuer 1, 4 converters
@@ -442,7 +433,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     const TcPlan &pl = p.plan;
     const int NI = Q4 ? p.plan.n_iss : 2;          // MMA issuers: a compile-time 2 on the bf16 path
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    TCT(const long long t_entry = clock64(); unsigned long long g_entry; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_entry));)
+
     // programmatic dependent launch: the routing kernel in front of this grid must have
     // finished before its results are read; the next layer's routing kernel may be scheduled
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -607,7 +598,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     auto umeta_at = [&](int i) -> uint32_t { return i < kTcMaxUnits ? s_umeta[i] : tc_unit_meta(unit_make(i)); };
     auto seg_of_unit = [&](int i) -> int { return i < n_units ? unit_at(i).seg : 4; };
 
-    TCT(const long long t_roles = clock64();)
     if (warp == 0) {
         const uint64_t wpolicy = l2_evict_first_policy();
         // ------------------------------------------------------------------ TMA producer
@@ -629,11 +619,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             int ready_w = 0;
             unsigned idle = 0;
             bool alive = n_units > 0;
-            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0; const long long tp0 = clock64();)
+
             while (alive && (pi < n_units || ti < n_units)) {
                 bool progress = false;
                 if (pi < n_units && mbar_test(&empty_bar[s], ring_par)) {
-                    TCT(const long long c2 = clock64();)
+
                     const TcGroup &g = groups[pu.a];
                     const bool shared = g.group >= sh.E;
                     const int e = shared ? g.group - sh.E : g.group;
@@ -650,7 +640,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     pkt += KG;
                     if (pkt >= pu.kt1 && ++pi < n_units) { pu = unit_at(pi); pkt = pu.kt0; }
                     progress = true;
-                    TCT(tp_issue += clock64() - c2;)
+
                 }
                 if (ti < n_units) {
                     const int wv = tu.a >= a_split ? 1 : 0;
@@ -663,7 +653,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         ready = true;
                     }
                     if (ready && mbar_test(&a_empty[ta], t_par)) {
-                        TCT(const long long c2 = clock64();)
+
                         uint8_t *op = tokring + (size_t)ta * KG * pl.tokb;
                         if (tu.phase == 1) {
                             // the hidden-state tiles of all KG k-tiles in one copy: [k-tile][tokb / 128 rows]
@@ -682,7 +672,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         tkt += KG;
                         if (tkt >= tu.kt1 && ++ti < n_units) { tu = unit_at(ti); tkt = tu.kt0; }
                         progress = true;
-                        TCT(tp_ready += clock64() - c2;)
+
                     }
                 }
                 if (progress) {
@@ -696,21 +686,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     }
                 }
             }
-            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry;)
+
         } else if (lane == 0) {
             unsigned it = 0;
             bool alive = true;
-#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
-            int ready_w = 2;                     // waves whose activations are known to be written
-#else
             int ready_w = 0;
-#endif
             // phase-2 stages whose weight tile is in flight but whose token tiles wait for the
             // activations (second grid-wide counter)
             int pend_wave = 0;
             int pend_n = 0, pend_stage[kTcMaxStages], pend_kt[kTcMaxStages], pend_row[kTcMaxStages], pend_shared[kTcMaxStages],
                 pend_tn[kTcMaxStages];
-            TCT(long long tp_empty = 0, tp_ready = 0, tp_issue = 0, tp_x = 0, tp_unit = 0; const long long tp0 = clock64();)
+
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
                 uint8_t *op = ring + (size_t)s * pl.stage_bytes + pl.tok_off;
@@ -718,14 +704,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 for (int r = 0; r < tn / 2; r += 8) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
             auto wait_ready = [&](int w) -> bool {
-                TCT(long long c0 = clock64();)
-                TCG(30 + w);
+
                 bool ok = false;
                 for (unsigned i = 0; i < kTcSpinLimit; ++i) {
                     if (s_ready[w]) { ok = true; break; }
                     __nanosleep(32);
                 }
-                TCT(tp_ready += clock64() - c0;)
+
                 if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); return false; }
                 __threadfence_block();
                 asm volatile("fence.proxy.async.global;" ::: "memory");
@@ -737,9 +722,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const int n_routed = p.B * sh.k;
             int s = 0;                                   // ring slot of the next k-tile
             uint32_t ring_par = 1;                       // parity to wait for on its empty barrier
-            TCT(tp_x = clock64() - tp0;)
+
             for (int i = 0; i < n_units && alive; ++i) {
-                TCT(const long long cu = clock64();)
+
                 const TcUnit t = unit_at(i);
                 const TcGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
@@ -761,19 +746,19 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         ready = alive;
                     }
                 }
-                TCT(tp_unit += clock64() - cu;)
+
                 for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
                     if (!ready && pend_n == S) {
                         if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
                         ready = true;
                     }
-                    TCT(long long c1 = clock64();)
+
                     if (!mbar_wait(&empty_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
                     }
-                    TCT(long long c2 = clock64(); tp_empty += c2 - c1;)
+
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                     const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 128u;
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
@@ -790,11 +775,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         pend_wave = wv;
                         ++pend_n;
                     }
-                    TCT(tp_issue += clock64() - c2;)
+
                 }
             }
             if (alive && pend_n > 0) wait_ready(pend_wave);
-            TCT(long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[0] = tp_empty; o[1] = tp_ready; o[2] = tp_issue; o[3] = clock64() - tp0; o[4] = t_roles - t_entry; (void)tp_x; (void)tp_unit;)
+
         }
     } else if (warp == 1 || warp == 6 || (Q4 && warp >= 11 + kTcQ4DeqWarps)) {
         // ------------------------------------------------------------------ MMA issuers
@@ -830,7 +815,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const uint32_t ring_lo = (uint32_t)tc_smem_desc(ring) + koff, xres_lo = (uint32_t)tc_smem_desc(xres) + koff;
             const uint32_t tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
             const uint32_t a_tmem0 = tmem_base + (uint32_t)kTcQ4ACol + 4u * koff;     // 8 columns per K-step
-            TCT(long long tm_acc = 0, tm_full = 0, tm_mma = 0, tm_fence = 0, tm_mmas = 0; const long long tm0 = clock64();)
+
             if (Q4) {
                 // int4: a unit is one stage; everything this thread needs of it is one word
                 uint32_t d_tmem = tmem_base + (uint32_t)(half * 2 * pl.n1), buf = 0, run_par = 1;
@@ -838,17 +823,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 for (; (int)ui < n_units; ++ui) {
                     const uint32_t um = umeta_at((int)ui);
                     if (um & 1u) {
-                        TCT(long long c0 = clock64();)
+
                         if (!mbar_wait(&acc_empty[buf], run_par)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
-                        TCT(tm_acc += clock64() - c0;)
+
                         acc = 0;
                     }
-                    TCT(long long c1 = clock64();)
+
                     // the unit as bf16 in tensor memory, written by the dequantising warps, and its token tiles
                     if (!mbar_wait(&a_full[ta], a_par)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); break; }
-                    TCT(long long c2 = clock64(); tm_full += c2 - c1;)
+
                     tc_fence_after();
-#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
                     {
                         // dequantised k-tiles of slot ta (32 columns each) and their token tiles: phase 1
                         // [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row groups KG KiB apart)
@@ -865,7 +849,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                             }
                         }
                     }
-#endif
                     tc_commit(&a_empty[ta]);           // frees the dequantised tiles and the token tiles
                     tc_ring_next(ta, a_par, pl.a_stages);
                     if (um & 2u) {
@@ -874,19 +857,19 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         if (buf == 0) run_par ^= 1u;
                         d_tmem = tmem_base + (uint32_t)(buf * 2 * NI * pl.n1 + half * 2 * pl.n1);
                     }
-                    TCT(tm_mma += clock64() - c2;)
+
                 }
             } else
             for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
                 const int buf = run & 1;
                 if (t.first) {
-                    TCT(long long c0 = clock64();)
+
                     if (!mbar_wait(&acc_empty[buf], ((run >> 1) & 1u) ^ 1u)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         break;
                     }
-                    TCT(tm_acc += clock64() - c0;)
+
                     tc_fence_after();
                     acc = 0;
                 }
@@ -895,16 +878,15 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
                 for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
-                    TCT(long long c1 = clock64();)
+
                     if (!mbar_wait(&full_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         alive = false;
                         break;
                     }
-                    TCT(long long c2 = clock64(); tm_full += c2 - c1;)
+
                     tc_fence_after();
-                    TCT(const long long c3 = clock64(); tm_fence += c3 - c2;)
-#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 1)
+
                     {
                         const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
                         const uint32_t b_lo = (t.phase == 1 && pl.x_bytes) ? xres_lo + (uint32_t)kt * ((uint32_t)pl.n1 * 8u)
@@ -914,19 +896,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                             acc = 1;
                         }
                     }
-#else
-                    (void)idesc; (void)acc; (void)d_tmem;   // speed experiment: no MMAs
-#endif
-                    TCT(const long long c4 = clock64(); tm_mmas += c4 - c3;)
+
                     tc_commit(&empty_bar[s]);          // frees the stage when these MMAs have read it
-                    TCT(tm_mma += clock64() - c2;)
+
                 }
                 if (alive && t.last) {
                     tc_commit(&acc_full[buf]);
                     ++run;
                 }
             }
-            TCT(if (half == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 8; o[0] = tm_acc; o[1] = tm_full; o[2] = tm_mma; o[3] = clock64() - tm0; o[-3] = tm_fence; o[-2] = tm_mmas;   /* slots 5, 6 */ })
+
         }
     } else if (Q4 && warp >= 11) {
         // ------------------------------------------------------------------ dequantising warps (int4)
@@ -947,21 +926,21 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         bool alive = true;
         const __nv_bfloat162 minus136 = __floats2bfloat162_rn(-136.0f, -136.0f);
         const uint32_t a_lane = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)kTcQ4ACol;
-        TCT(long long td_full = 0, td_aempty = 0, td_work = 0, td_fence = 0;)
+
         // contraction lengths are multiples of 256 here, so every unit is exactly one stage and
         // nothing of it has to be decoded
         {
             for (int ui = 0; ui < n_units && alive; ++ui, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
-                TCT(const long long d0 = clock64();)
+
                 const bool ok_full = mbar_wait(&full_bar[s], ring_par);
-                TCT(const long long d1 = clock64(); td_full += d1 - d0;)
+
                 if (!ok_full || !mbar_wait(&a_empty[ta], a_par)) {
                     if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     alive = false;
                     break;
                 }
                 tc_fence_after();                  // the MMAs that read this slot have completed
-                TCT(const long long d2 = clock64(); td_aempty += d2 - d1;)
+
                 const uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
                 const uint8_t *prow = stage + (size_t)r * (32 * KG);
                 uint32_t sc[2];                    // this thread's CP scales (binary16) in one load
@@ -1003,7 +982,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     }
                     tc_st16(a_slot + (uint32_t)q * 16u, o);          // k-tile q / 2, its columns 16 * (q % 2) ..
                 }
-                TCT(const long long d3 = clock64(); td_work += d3 - d2;)
+
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
@@ -1011,15 +990,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     mbar_arrive(&a_full[ta]);
                     mbar_arrive(&empty_bar[s]);        // the packed tiles have been read
                 }
-                TCT(td_fence += clock64() - d3;)
+
             }
         }
-        TCT(if (warp == 11 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 12; o[0] = td_full; o[1] = td_aempty; o[2] = td_work; o[3] = td_fence; })
+
     } else if (warp == 10) {
         // ------------------------------------------------------------------ watcher
         // polls the waves' second counters (all CTAs have written their slice of the activations)
         // and publishes them in shared memory, so that the producer never waits on global memory
-#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 4)
         if (lane == 0) {
             for (int w = 0; w < W; ++w) {
                 bool ok = false;
@@ -1030,10 +1008,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 if (!ok) { atomicExch(ws.status, ST_DEP_TIMEOUT); break; }
                 __threadfence_block();
                 s_ready[w] = 1;
-                TCG(25 + w);
+
             }
         }
-#endif
     } else if (warp >= 7) {
         // ------------------------------------------------------------------ converter warps
         // per wave: wait for this CTA's hand-over, arrive on the wave's grid-wide counter, wait
@@ -1044,9 +1021,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         uint64_t *ep_bar_p = &cv_bar;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
         const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
-        TCT(long long te_sync = 0, te_conv = 0;)
+
         auto wave_convert = [&](int w) -> bool {
-            TCT(long long c2 = clock64();)
+
             if (et == 0) {
                 bool ok = false;
                 for (unsigned i = 0; i < (kTcSpinLimit >> 2); ++i) {
@@ -1055,12 +1032,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 }
                 if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
                 s_flag = ok;
-                TCG(14 + w);
+
             }
             if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
             if (!s_flag) return false;
             __threadfence_block();                 // the counter was read with acquire by one thread of this barrier
-            TCT(long long c3 = clock64(); te_sync += c3 - c2;)
+
             // pre holds a gate plane and an up plane, both indexed exactly like the activations
             // (act_offset(slot) + row): this CTA converts a contiguous slice of the wave's range,
             // four elements per thread and step
@@ -1096,12 +1073,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             // every writer, then one release at GPU scope behind the barrier of the converter warps
             asm volatile("fence.proxy.async.global;" ::: "memory");
             if (!tc_bar(ep_bar_p, ep_phase, lane)) return false;
-            if (et == 0) { tc_red_release(&ws.sync[kTcReady - 4 + w]); TCG(23 + w); }
-            TCT(te_conv += clock64() - c3;)
+            if (et == 0) { tc_red_release(&ws.sync[kTcReady - 4 + w]);  }
+
             return true;
         };
 
-#if !defined(S2MOE_ABLATE) || !(S2MOE_ABLATE & 4)
         for (int w = 0; w < W; ++w) {
             // the hand-over may come late in the kernel: a long but bounded wait
             bool ok = false;
@@ -1113,8 +1089,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             if (et == 0) tc_red_release(&ws.sync[kTcReady - 8 + w]);   // orders the CTA's reductions, observed through conv_go
             if (!wave_convert(w)) break;
         }
-#endif
-        TCT(if (et == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 28; o[0] = te_sync; o[1] = te_conv; })
+
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;                        // TMEM lane quarter this warp may read
@@ -1123,7 +1098,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         uint32_t ep_phase = 0;
         const int n_routed = p.B * sh.k;
         bool alive = true;
-        TCT(long long te_wait = 0, te_red = 0, te_sync = 0, te_conv = 0; const long long te0 = clock64();)
+
         // ---- hand-over between the projections, per wave (see the header comment)
         const int n_routed_el = n_routed;   // (alias used below)
         (void)n_routed_el;
@@ -1137,7 +1112,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(&conv_go[w]);
-                TCG(12 + w);
+
             }
             return true;
         };
@@ -1151,9 +1126,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             }
             return true;
         };
-#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 4)
-        next_arrive = W;
-#endif
         {
             for (; (int)ui < n_units && alive; ++ui) {
                 if (!service(seg_of_unit((int)ui))) { alive = false; break; }
@@ -1161,17 +1133,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 if (!t.last) continue;                 // the run's accumulator is read after its last unit
                 const TcGroup &g = groups[t.a];
                 const int buf = run & 1;
-                TCT(long long c0 = clock64();)
+
                 if (!mbar_wait(&acc_full[buf], (run >> 1) & 1u)) {
                     if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     alive = false;
                     break;
                 }
-                TCT(long long c1 = clock64(); te_wait += c1 - c0;)
+
                 tc_fence_after();
-#if defined(S2MOE_ABLATE) && (S2MOE_ABLATE & 2)
-                if (false)
-#endif
                 {
                 const int row = t.rb * 128 + q * 32 + lane;           // row of the matrix inside the expert
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * NI * pl.n1);
@@ -1225,16 +1194,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 ++run;
-                TCT(te_red += clock64() - c1;)
+
             }
             if (alive && !service(4)) alive = false;
         }
-        TCT(if (warp == 2 && lane == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32 + 16; o[0] = te_wait; o[1] = te_red; o[2] = te_sync; o[3] = te_conv; o[4] = clock64() - te0; })
+
     }
     // every path ends here (all waits above are bounded), so the TMEM is always returned
     tc_fence_before();
     __syncthreads();
-    TCT(if (tid == 0) { long long *o = reinterpret_cast<long long *>(ws.act) + (size_t)blockIdx.x * 32; o[7] = clock64() - t_entry; unsigned long long g_exit; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g_exit)); o[21] = (long long)g_entry; o[22] = (long long)g_exit; unsigned smid_; asm volatile("mov.u32 %0, %smid;" : "=r"(smid_)); o[27] = smid_; o[19] = n_units; })
+
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)pl.tmem_cols)
                      : "memory");

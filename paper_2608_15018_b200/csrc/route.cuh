@@ -73,13 +73,6 @@ __device__ __forceinline__ unsigned long long shfl_key(unsigned long long k, int
 }
 
 
-#ifdef S2MOE_TIMING
-__device__ long long g_gt_marks[16];
-#define GT_MARK(i) do { if (threadIdx.x == 0) g_gt_marks[i] = clock64(); } while (0)
-#else
-#define GT_MARK(i) do { } while (0)
-#endif
-
 // Order statistics of one token's original logits, one warp per token (lane owns experts lane,
 // lane + 32, ...): lambda_b = alpha (l_(1) - l_(k+1)) by k + 1 rounds of a warp-wide maximum over
 // integer keys, and, for weight_mode 0, the softmax denominator over the original logits.
@@ -88,7 +81,6 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
                                            double *s_zmax, double *s_den, int lane)
 {
     const int E = sh.E, k = sh.k;
-    GT_MARK(0);
     unsigned long long k1[J];
     unsigned valid = 0;
 #pragma unroll
@@ -127,7 +119,6 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
             if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
         }
     }
-    GT_MARK(1);
     const double ztop = dkey_value(top1);
     double den = 0.0;
     if (!sh.weight_mode) {
@@ -140,7 +131,6 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
         s_zmax[b] = ztop;
         s_den[b] = den;
     }
-    GT_MARK(2);
 }
 
 // Biased top-k of one token in the order (l' descending, l descending, id ascending), one
@@ -153,7 +143,6 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
 {
     const unsigned full = 0xffffffffu;
     const int E = sh.E, k = sh.k;
-    GT_MARK(3);
     const double lam = s_lam[b];
     double l[J];
     unsigned long long k1[J], k2[J];
@@ -173,7 +162,6 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
             valid |= 1u << j;
         }
     }
-    GT_MARK(4);
     if constexpr (J == 2) {
         // the lane offers its better element first (order: l' descending, l descending, id
         // ascending; element 0 has the lower id), then the other one
@@ -228,7 +216,6 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
         }
     }
     __syncwarp();
-    GT_MARK(5);
     // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
     double zmax = s_zmax[b], den = s_den[b];
     const double lamw = sh.weight_mode ? lam : 0.0;
@@ -262,7 +249,6 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
         // half that holds it (a 64-bit atomicOr would be a compare-and-swap loop)
         atomicOr(reinterpret_cast<unsigned *>(&s_mask[my_sel]) + (b >> 5), 1u << (b & 31));
     }
-    GT_MARK(6);
 }
 
 // Gating of one batch by one thread block of at least two warps.
@@ -284,14 +270,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
     const int E = sh.E, k = sh.k, cap = sh.cap;
     const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
-#ifdef S2MOE_TIMING
-    long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64;
-    int tmi = 0;
-#define GATE_MARK() do { __syncthreads(); if (tid == 0) tm[tmi] = clock64(); ++tmi; } while (0)
-#else
-#define GATE_MARK() do { } while (0)
-#endif
-    GATE_MARK();
 
 #pragma unroll 1
     for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
@@ -301,7 +279,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
     __syncthreads();
 
-    GATE_MARK();
     // Two independent pieces run side by side on disjoint warps: the last cw warps pick the
     // reuse-reward set E* (Eq. 4 aggregation, TopCap), the others take the per-token order
     // statistics (lambda_b, softmax denominator).
@@ -337,14 +314,12 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
     __syncthreads();
 
-    GATE_MARK();
 #pragma unroll 1
     for (int b = warp; b < B; b += nw) {
         gate_select<JE>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
     }
     __syncthreads();
 
-    GATE_MARK();
     // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts
     if (tid < 32) {
         const int C = (E + 31) >> 5, e0 = tid * C;
@@ -379,7 +354,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         if (tid == 31) { s_off[E] = xs; s_U = xa; }
     }
     __syncthreads();
-    GATE_MARK();
     const int U = s_U, n_routed = B * k;
 #pragma unroll 1
     for (int e = tid; e < E; e += nt) {
@@ -393,7 +367,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             }
         }
     }
-    GATE_MARK();
     // bucket the (token, choice) pairs: tokens ascending inside an expert
 #pragma unroll 1
     for (int i = tid; i < n_routed; i += nt) {
@@ -403,7 +376,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         ws.slot_token[pos] = b;
         ws.slot_w[pos] = s_pw[i];
     }
-    GATE_MARK();
     // shared experts: every token, weight c_b
 #pragma unroll 1
     for (int i = tid; i < sh.n_sh * B; i += nt) {
@@ -423,7 +395,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             }
         }
     }
-    GATE_MARK();
 #pragma unroll 1
     for (int e = tid; e < E; e += nt) ws.tokmask[e] = s_mask[e];
 #pragma unroll 1
@@ -466,10 +437,6 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             ws.header[5] = t2;
         }
     }
-    GATE_MARK();
-#ifdef S2MOE_TIMING
-    if (tid == 0) for (int i = 0; i < 8; ++i) tm[20 + i] = g_gt_marks[i];
-#endif
     if (tid == 0) {
         ws.offsets[E + sh.n_sh] = n_routed + sh.n_sh * B;
         ws.header[0] = U + sh.n_sh;
@@ -572,9 +539,6 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     // and do its own set-up (both instructions do nothing in a plain launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-#ifdef S2MOE_TIMING
-    const long long t_start = clock64();
-#endif
 #pragma unroll
     for (int z = 0; z < 3; ++z) {
         uint4 *p = reinterpret_cast<uint4 *>(zl.ptr[z]);
@@ -611,19 +575,38 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     // Block 0 runs the gating once every row has arrived (its SM tends to be the same from layer
     // to layer, so part of the gating code is still in its instruction cache: measured 0.6 % of
     // a layer against letting the last block to arrive do it).  Every block takes a ticket with
-    // release and acquire semantics by one thread; block 0 then polls the counter, bounded, and
-    // the barriers on both sides extend the ordering to the block's other threads.  The other
-    // blocks wait for nothing, so block 0 cannot starve them.
+    // release and acquire semantics by one thread.  The block that takes the last ticket puts the
+    // counter back to zero (nobody else touches it before the next launch) and publishes, in the
+    // word behind the counter, the token that block 0 wrote two words further in front of its own ticket;
+    // block 0 polls, bounded, for exactly that token.  So a wait that ran out leaves nothing
+    // behind: the late blocks still reset the counter, and what they publish afterwards is the
+    // token of a launch that is over, which no later launch waits for.  The barriers on both
+    // sides extend the ordering to the block's other threads; the other blocks wait for nothing.
     if (tid == 0) {
+        unsigned token = 0u;
+        if (blockIdx.x == 0) {
+            // differs from launch to launch (a wrapped nanosecond timer; never 0)
+            unsigned long long gt;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+            token = (unsigned)gt | 1u;
+            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 2), "r"(token) : "memory");
+        }
         unsigned t;
         asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(t) : "l"(ws.ticket) : "memory");
-        int ok = blockIdx.x == 0 ? 1 : 0;
-        if (blockIdx.x == 0 && t != (unsigned)n_arrive - 1) {
-            ok = 0;
+        const bool last = t == (unsigned)n_arrive - 1;
+        if (last) {
+            unsigned tk;
+            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(tk) : "l"(ws.ticket + 2) : "memory");
+            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket), "r"(0u) : "memory");
+            if (blockIdx.x != 0)
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 1), "r"(tk) : "memory");
+        }
+        int ok = (blockIdx.x == 0 && last) ? 1 : 0;
+        if (blockIdx.x == 0 && !last) {
             for (unsigned i = 0; i < (1u << 22); ++i) {
                 unsigned v;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ws.ticket) : "memory");
-                if (v >= (unsigned)n_arrive) { ok = 1; break; }
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ws.ticket + 1) : "memory");
+                if (v == token) { ok = 1; break; }
                 __nanosleep(20);
             }
             if (!ok) atomicExch(ws.status, ST_TICKET_TIMEOUT);
@@ -632,26 +615,7 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     }
     __syncthreads();
     if (!s_last) return;
-    if (tid == 0) *ws.ticket = 0u;
-#ifdef S2MOE_TIMING
-    if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[15] = t_start; tm[14] = clock64(); }
-#endif
-#ifdef S2MOE_GATE_TWICE
-    {   // experiment: the same gating code (one copy, in a loop) a second time, with whatever the
-        // first run left in the caches
-        long long g[3];
-        g[0] = clock64();
-#pragma unroll 1
-        for (int rep = 0; rep < 2; ++rep) {
-            gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
-            __syncthreads();
-            g[rep + 1] = clock64();
-        }
-        if (tid == 0) { long long *tm = reinterpret_cast<long long *>(ws.act) + 148 * 64; tm[30] = g[1] - g[0]; tm[31] = g[2] - g[1]; }
-    }
-#else
     gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
-#endif
 }
 
 }  // namespace s2moe

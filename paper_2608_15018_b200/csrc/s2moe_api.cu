@@ -428,14 +428,22 @@ int fetch_experts(s2moe_ctx *ctx, int layer, cudaStream_t st)
     const LayerPtrs &hw = ctx->host_w[(size_t)layer], &dw = ctx->layers[(size_t)layer];
     const void *src[6] = {hw.w_gate, hw.w_up, hw.w_down, hw.s_gate, hw.s_up, hw.s_down};
     const void *dst[6] = {dw.w_gate, dw.w_up, dw.w_down, dw.s_gate, dw.s_up, dw.s_down};
+    // the cache already counts the missing experts as resident: if a copy cannot be issued, every
+    // expert whose copies are not all on the stream is taken out again, so that a later call
+    // fetches it instead of reading a slot that holds another expert's weights
     for (int i = 0; i < U; ++i) {
         if (!missed[(size_t)i]) continue;
         const size_t e = (size_t)ctx->h_route[8 + i], sl = (size_t)slots[(size_t)i];
         for (int m = 0; m < 6; ++m) {
             const size_t nb = ctx->mat_bytes[m];
             if (!nb) continue;
-            CU(ctx, cudaMemcpyAsync((uint8_t *)const_cast<void *>(dst[m]) + nb * sl, (const uint8_t *)src[m] + nb * e, nb,
-                                    cudaMemcpyHostToDevice, st));
+            const cudaError_t ce = cudaMemcpyAsync((uint8_t *)const_cast<void *>(dst[m]) + nb * sl,
+                                                   (const uint8_t *)src[m] + nb * e, nb, cudaMemcpyHostToDevice, st);
+            if (ce != cudaSuccess) {
+                for (int j = i; j < U; ++j)
+                    if (missed[(size_t)j]) cache.evict(ctx->h_route[8 + j]);
+                return cuda_fail(ctx, ce);
+            }
             ctx->fetched_bytes += (int64_t)nb;
         }
     }
@@ -963,7 +971,10 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out)
     CU(ctx, cudaDeviceSynchronize());
     CU(ctx, cudaMemcpy(host_out, ctx->ws.status, 4, cudaMemcpyDeviceToHost));
     if (*host_out != 0) {
+        // the device is idle here: put the status word and the routing kernel's arrival words back,
+        // so that the next call starts clean whatever the abandoned wait left behind
         CU(ctx, cudaMemset(ctx->ws.status, 0, 4));
+        CU(ctx, cudaMemset(ctx->ws.ticket, 0, 16));
         return S2MOE_ETIMEOUT;
     }
     return S2MOE_OK;
@@ -1107,6 +1118,10 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return S2MOE_ECUDA;
         if (prepare_route() != cudaSuccess) return S2MOE_ECUDA;
+        // load the small kernel's module now as well, so that no later call (one made under a
+        // stream capture, say) is the first to touch it
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, noalloc_gate_out_kernel) != cudaSuccess) return S2MOE_ECUDA;
         g_noalloc_ptr[dev] = p;
     }
     uint8_t *base = (uint8_t *)g_noalloc_ptr[dev];
@@ -1159,6 +1174,26 @@ int s2moe_route_noalloc(const s2moe_config *cfg, int32_t n_tokens, const void *r
 #undef S2MOE_ROUTE_NA
     if (gate_vec && gate_out) noalloc_gate_out_kernel<<<1, 64, 0, st>>>(ws.gate_logit, gate_out, n_tokens);
     return cudaGetLastError() == cudaSuccess ? S2MOE_OK : S2MOE_ECUDA;
+}
+
+int s2moe_route_noalloc_status(int32_t *host_out)
+{
+    if (!host_out) return S2MOE_EINVAL;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoallocMaxDevices) return S2MOE_ECUDA;
+    *host_out = 0;
+    if (!g_noalloc_ptr[dev]) return S2MOE_OK;            // never called on this device: nothing to report
+    if (cudaDeviceSynchronize() != cudaSuccess) return S2MOE_ECUDA;
+    // the status word sits behind the logits, the gate logits and the arrival words (see the carving above)
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    take(sizeof(double) * S2MOE_NOALLOC_MAX_TOKENS * S2MOE_NOALLOC_MAX_EXPERTS);
+    take(sizeof(double) * S2MOE_NOALLOC_MAX_TOKENS);
+    take(256);
+    const size_t o_status = take(256);
+    if (cudaMemcpy(host_out, (const uint8_t *)g_noalloc_ptr[dev] + o_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return S2MOE_ECUDA;
+    return *host_out != 0 ? S2MOE_ETIMEOUT : S2MOE_OK;
 }
 
 // ---- routing-aware adaptive expansion (no context, no allocation) ----------------------

@@ -22,10 +22,13 @@ def supports(wl, plan):
 
 
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
-             hidden=None, conf=None, check_lists=True):
-    """Returns (report, outputs), or (None, None) when the demanded plan does not cover the case
-    (format not covered, or the batch does not fit the streaming kernel's shared memory)."""
+             hidden=None, conf=None, check_lists=True, optional=False):
+    """Runs one layer through the C ABI and compares it with the oracle; returns (report, outputs).
+    A demanded plan that does not cover the case (format not covered, or the batch does not fit
+    the streaming kernel's shared memory) is an error, unless the caller says ``optional=True``
+    and handles the returned (None, None) itself (by skipping or by counting)."""
     if not supports(wl, plan):
+        assert optional, f"kernel plan {plan} does not cover this case (use supports() and skip)"
         return None, None
     dev = torch.device("cuda", 0)
     T = workloads.layer_weights(wl, layer, dev)
@@ -36,6 +39,7 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
     with binding.S2MoE(cfg, [T]) as m:
         used = m.kernel_plan(H.shape[0])
         if plan in (2, 3) and used != plan:
+            assert optional, f"kernel plan {plan} was demanded, the library chose {used}"
             return None, None
         assert used in (1, 2, 3) and (plan == 0 or used == plan)
         o = m.verify_layer(0, H, conf)

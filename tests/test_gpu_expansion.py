@@ -102,6 +102,28 @@ def test_expand_ties_and_degenerate_cases():
     assert union.cpu().tolist() == [[0]]
 
 
+def test_expand_reports_a_malformed_parent_array():
+    """A parent index that is not below the candidate's own is not followed: that candidate and its
+    descendants are never admitted, the call reports n_admitted = -1, and the well-formed rest is
+    decided as if the malformed candidates were not there."""
+    from paper_2608_15018_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    #          0   1   2     3 (self)  4 (forward)  5 (child of 3)  6 (beyond n)
+    parent = [-1,  0,  0,    3,        5,           3,              40]
+    p_tok = [0.9] * 7
+    masks = [[1 << i] for i in range(7)]
+    adm, order, n_adm, union = binding.adaptive_expand(
+        torch.tensor(parent, dtype=torch.int32, device=dev), torch.tensor(p_tok, dtype=torch.float32, device=dev),
+        _masks_tensor(masks, 1, dev), 8, None, 1.0, 0.125)
+    torch.cuda.synchronize()
+    want_adm, want_order, want_union = ox.adaptive_expand(parent[:3], p_tok[:3], masks[:3], [0.0] * 3, 1.0, 0.125)
+    assert n_adm.item() == -1
+    assert adm.cpu().tolist() == want_adm + [0, 0, 0, 0]
+    assert order.cpu().tolist()[: len(want_order)] == want_order
+    assert int(union.cpu().numpy().view(np.uint64)[0, 0]) == want_union[0]
+
+
 def test_expand_argument_errors():
     from paper_2608_15018_b200 import binding
 

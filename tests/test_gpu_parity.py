@@ -42,8 +42,9 @@ def test_small_configs(name, plan):
 @pytest.mark.parametrize("renorm,mode,alpha", [(0, 0, 0.5), (1, 0, 0.25), (0, 1, 1.0), (1, 1, 0.5), (0, 0, 0.0)])
 def test_gating_variants(plan, renorm, mode, alpha):
     wl = SMALL["cfg2"].with_(renorm=renorm, weight_mode=mode, alpha=alpha)
-    run_case(wl, plan=plan)
-    run_case(wl, plan=plan, use_conf=False)
+    for use_conf in (True, False):
+        rep, _ = run_case(wl, plan=plan, use_conf=use_conf)
+        assert rep.plan == plan and rep.tokens_checked == wl.n_tokens
 
 
 @pytest.mark.parametrize("plan", PLANS)
@@ -57,38 +58,60 @@ def test_cfg4_batch_sweep(plan, B):
 @pytest.mark.parametrize("plan", PLANS)
 @pytest.mark.parametrize("B,sigma", [(1, 0.3), (2, 1.0), (7, 0.5), (16, 0.1), (33, 0.7), (64, 1.0), (64, 0.1)])
 def test_cfg5_tree_sweep(plan, B, sigma):
-    rep, o = run_case(SMALL["cfg5"], n_tokens=B, sigma=sigma, plan=plan)
+    rep, o = run_case(SMALL["cfg5"], n_tokens=B, sigma=sigma, plan=plan, optional=plan == 2)
     if rep is None:
         pytest.skip("batch too large for the streaming kernel's shared memory")
+    assert rep.plan == plan and rep.tokens_checked == B
     assert SMALL["cfg5"].top_k <= rep.n_unique <= 64
 
 
 @pytest.mark.parametrize("plan", PLANS)
 def test_degenerate_cases(plan):
     base = SMALL["cfg5"]
-    run_case(base.with_(top_k=4, cap=64), plan=plan)                      # cap = E: bias off
-    run_case(base.with_(n_experts=8, top_k=8, cap=8), plan=plan)          # k = E: dense sum
-    run_case(base.with_(n_experts=256, top_k=16, cap=40), n_tokens=64, plan=plan)   # limits
-    run_case(base.with_(n_shared=0, d_ff_shared=0), plan=plan)
+    ran = []
+
+    def case(wl, big=False, **kw):
+        # the streaming plan does not hold 64 tokens in shared memory: those two cases may be
+        # declined by it, every other case must run on the demanded plan
+        rep, _ = run_case(wl, plan=plan, optional=plan == 2 and (big or wl.n_experts == 8), **kw)
+        if rep is not None:
+            assert rep.plan == plan and rep.tokens_checked > 0
+            ran.append(rep)
+        return rep
+
+    case(base.with_(top_k=4, cap=64))                                    # cap = E: bias off
+    case(base.with_(n_experts=8, top_k=8, cap=8))                        # k = E: dense sum
+    case(base.with_(n_experts=256, top_k=16, cap=40), big=True, n_tokens=64)   # limits
+    case(base.with_(n_shared=0, d_ff_shared=0))
     # identical tokens: U = k, reuse ratio 1/B
     H = workloads.hidden_states(base, 0, 1, device="cuda").repeat(8, 1)
-    rep, _ = run_case(base, hidden=H, plan=plan)
+    rep = case(base, hidden=H)
     assert rep.n_unique == base.top_k
     # all-zero confidences: E* falls back to the lowest ids
-    run_case(base, conf=torch.zeros(16, device="cuda"), plan=plan)
+    case(base, conf=torch.zeros(16, device="cuda"))
     # uncorrelated tokens reach (almost) every expert
     Hr = torch.randn(64, base.d_model, device="cuda", generator=torch.Generator("cuda").manual_seed(5)).to(torch.bfloat16)
-    rep, _ = run_case(base, hidden=Hr, plan=plan)
+    rep = case(base, big=True, hidden=Hr)
     assert rep is None or rep.n_unique > 48
+    assert len(ran) >= (4 if plan == 2 else 7)
 
 
 @pytest.mark.parametrize("plan", PLANS)
 def test_mixed_storage_formats(plan):
-    run_case(SMALL["cfg2"].with_(act_dtype=F32, router_dtype=F32), plan=plan)
-    run_case(SMALL["cfg4"].with_(act_dtype=F32), plan=plan)
-    run_case(SMALL["cfg3"].with_(weight_dtype=Q4B32, d_ff_shared=704), plan=plan)
-    if plan == 1:
-        run_case(SMALL["cfg2"].with_(weight_dtype=F32), plan=plan)
+    cases = [SMALL["cfg2"].with_(act_dtype=F32, router_dtype=F32),          # fp32 activations and router
+             SMALL["cfg4"].with_(act_dtype=F32),
+             SMALL["cfg3"].with_(weight_dtype=Q4B32, d_ff_shared=704),      # int4 with a gated shared expert
+             SMALL["cfg3"].with_(weight_dtype=Q4B32, d_ff=256, d_ff_shared=768),
+             SMALL["cfg2"].with_(weight_dtype=F32),
+             SMALL["cfg2"].with_(router_dtype=F32)]                         # fp32 router, bf16 everything else
+    ran = 0
+    for wl in cases:
+        if not supports(wl, plan):
+            continue                      # counted below: every plan must cover its share
+        rep, _ = run_case(wl, plan=plan)
+        assert rep.plan == plan and rep.tokens_checked == wl.n_tokens
+        ran += 1
+    assert ran >= {1: 6, 2: 1, 3: 2}[plan]
 
 
 @pytest.mark.parametrize("name,tokens", [("cfg2", [0, 7]), ("cfg3", [0, 15]), ("cfg4", [3]), ("cfg5", [9])])
@@ -97,8 +120,22 @@ def test_full_size_layer_sampled_tokens(name, tokens):
     wl = CONFIGS[name]
     rep, _ = run_case(wl, layer=1, plan=0, tok_list=tokens)
     assert rep.tokens_checked == len(tokens)
-    if wl.weight_dtype == BF16:
-        assert rep.plan in (2, 3)     # a streaming plan, as the benchmark times
+    assert rep.plan == 3              # the tcgen05 plan, as the benchmark times
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name,B,sigma,tokens", [("cfg4", 1, None, [0]), ("cfg4", 2, None, [0, 1]),
+                                                 ("cfg4", 16, None, [5, 15]), ("cfg4", 32, None, [0, 31]),
+                                                 ("cfg5", 1, 0.3, [0]), ("cfg5", 32, 0.5, [7, 31]),
+                                                 ("cfg5", 64, 1.0, [17, 63]), ("cfg5", 64, 0.1, [0, 40]),
+                                                 ("cfg3", 64, None, [33])])
+def test_full_size_sweep_points(name, B, sigma, tokens):
+    """The ends of the batch sweeps at full width, in the launch configuration the benchmark
+    times: ring depth, resident hidden states and the number of MMA issuers follow from the
+    width and the batch size together, so the reduced-width sweeps do not reach these."""
+    wl = CONFIGS[name]
+    rep, _ = run_case(wl, layer=1, n_tokens=B, sigma=sigma, plan=0, tok_list=tokens)
+    assert rep.tokens_checked == len(tokens) and rep.plan == 3
     torch.cuda.empty_cache()
 
 

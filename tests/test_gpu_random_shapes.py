@@ -33,7 +33,7 @@ def test_random_shapes_on_the_tensor_core_plan(seed):
     ran = 0
     for trial in range(25):
         wl, B, use_conf = _case(rng, trial)
-        rep, _ = run_case(wl, n_tokens=B, plan=3, use_conf=use_conf)
+        rep, _ = run_case(wl, n_tokens=B, plan=3, use_conf=use_conf, optional=True)
         if rep is not None:
             assert rep.plan == 3 and rep.tokens_checked == B
             ran += 1

@@ -187,6 +187,33 @@ def test_alpha_one_tie_keeps_original_top1():
     assert r.sel[0].tolist() == [0]
 
 
+def test_full_tie_goes_to_lower_id_in_selection_order():
+    """Third key of the per-token order: equal biased AND equal original logits -> lower expert id
+    first, inside the selected set and at its boundary (the selection is returned in that order)."""
+    # bias off: three equal logits, k = 2 -> experts 0 and 1, in that order (2 loses the tie)
+    r = oracle.gating(gate_cfg(4, 2, 4, 0.0), np.array([[1.0, 1.0, 1.0, 0.0]]), None)
+    assert r.sel[0].tolist() == [0, 1]
+    assert r.m_tok[0] == 0.0
+    r = oracle.gating(gate_cfg(4, 3, 4, 0.0), np.array([[0.0, 2.0, 2.0, 2.0]]), None)
+    assert r.sel[0].tolist() == [1, 2, 3]
+    # biased: token 1 (all the confidence) makes E* = {1, 3}; token 0 has l = (5, 2, 4, 2, 0),
+    # k = 2: lam = 0.5 * (5 - 2) = 1.5 (the third largest is 2), l' = (5, 3.5, 4, 3.5, 0).
+    # Now make the two members of E* tie with expert 2 on l' only -> original logit decides:
+    L = np.array([[5.0, 2.5, 4.0, 2.5, 0.0], [0.0, 9.0, 0.0, 9.0, 0.0]])
+    cfg = gate_cfg(5, 3, 2, 0.5)
+    r = oracle.gating(cfg, L, np.array([0.0, 1.0]))
+    assert np.nonzero(r.estar)[0].tolist() == [1, 3]
+    # token 0: top-1 5, (k+1)-th = 4th largest = 2.5 -> lam = 1.25, l' = (5, 3.75, 4, 3.75, 0):
+    # order 0, 2, then experts 1 and 3 tie on l' (3.75) and on l (2.5): id 1 first, 3 is left out
+    assert r.lam[0] == 1.25
+    assert r.sel[0].tolist() == [0, 2, 1]
+    assert r.m_tok[0] == 0.0
+    # and with k = 4 both are taken, lower id first
+    r = oracle.gating(gate_cfg(5, 4, 2, 0.5), L, np.array([0.0, 1.0]))
+    # (k+1)-th = 5th largest = 0 -> lam = 2.5, l' = (5, 5, 4, 5, 0): l' ties of 0, 1, 3 -> l: 0 first, then 1, 3 by id
+    assert r.sel[0].tolist() == [0, 1, 3, 2]
+
+
 # ------------------------------------------------- gating: special cases and invariants
 
 @pytest.mark.parametrize("renorm", [0, 1])
@@ -348,6 +375,26 @@ def test_q4b32_codec_bounds():
     assert p2[0, 0].item() == (15 | (1 << 4)) and p2[0, 15].item() == (8 | (11 << 4))
     dec = oracle.decode_row(Q4B32, p2.numpy(), wl.raw_numpy(s2), 0, 32)
     assert dec[0] == 7.0 and dec[1] == -7.0 and dec[31] == 3.0 and dec[2] == 0.0
+
+
+def test_q4b32_scale_decoding_subnormal():
+    """Binary16 scales below the normal range are m * 2^-24: checked against the bit patterns'
+    textbook values and against numpy's own binary16 decoding.  (Infinite and NaN scales cannot
+    be read back through a dot product with unit vectors, and the quantiser never writes them:
+    that branch of the decoder stays unpinned.)"""
+    packed = np.full((1, 16 * 4), 0x99, dtype=np.uint8)         # every nibble 9 -> q = +1
+    bits = np.array([[0x0001, 0x03ff, 0x8001, 0x0400]], dtype=np.uint16)
+    dec = oracle.decode_row(Q4B32, packed, bits, 0, 32 * 4)
+    assert dec[0] == 2.0 ** -24 and dec[31] == 2.0 ** -24       # smallest subnormal
+    assert dec[32] == 1023 * 2.0 ** -24                         # largest subnormal
+    assert dec[64] == -(2.0 ** -24)                             # sign of a subnormal
+    assert dec[96] == 2.0 ** -14                                # smallest normal
+    ref = bits.view(np.float16).astype(np.float64)[0]
+    for b in range(4):
+        assert dec[32 * b] == ref[b]
+    # q = nibble - 8: nibble 1 -> -7 times a subnormal scale stays exact
+    packed[0, 0] = 0x11
+    assert oracle.decode_row(Q4B32, packed, bits, 0, 32 * 4)[0] == -7 * 2.0 ** -24
 
 
 def test_bf16_f32_decode_rows():
