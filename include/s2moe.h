@@ -119,9 +119,12 @@ typedef struct {
                               2: streaming mma.sync kernel (bf16 weights and activations);
                               3: streaming tcgen05 kernel: bf16 activations with bf16 weights,
                                  or with block-int4 weights when d_model, d_ff and
-                                 d_ff_shared are multiples of 256 (the int4 values are
-                                 dequantised to bf16, scale rounded to bf16 first, on their
-                                 way to the tensor core: up to 2^-8 relative per weight)      */
+                                 d_ff_shared are multiples of 256 (the int4 values reach the
+                                 tensor core as binary16 q * scale, rounded once: up to
+                                 2^-12 relative per weight; block scales below 2^-17 lose
+                                 precision in binary16's subnormal range; the hidden states
+                                 are converted to binary16 for this kernel, so they must
+                                 stay below 65504 in magnitude)                               */
 } s2moe_config;
 
 /*

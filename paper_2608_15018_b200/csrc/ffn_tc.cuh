@@ -334,6 +334,12 @@ __device__ __forceinline__ uint32_t tc_idesc(int n)
     // D = F32, A = B = BF16, both K-major, N = n, M = 128
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
 }
+__device__ __forceinline__ uint32_t tc_idesc_f16(int n)
+{
+    // the same with A = B = binary16 (int4 path: the dequantised weights and, because the two
+    // operands of an instruction must have one format, the token tiles as well)
+    return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
 
 // Barrier among the four epilogue warps on an mbarrier (count 4), so that the wait is bounded.
 __device__ __forceinline__ bool tc_bar(uint64_t *bar, uint32_t &phase, int lane)
@@ -836,7 +842,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     {
                         // dequantised k-tiles of slot ta (32 columns each) and their token tiles: phase 1
                         // [k-tile][rows], phase 2 [8 slots][hi | lo][k-tile][8 rows] (8-row groups KG KiB apart)
-                        const uint32_t idesc = tc_idesc((int)(um >> 8));
+                        const uint32_t idesc = tc_idesc_f16((int)(um >> 8));
                         const bool p2 = (um & 4u) != 0;
                         uint32_t a_tm = a_tmem0 + (uint32_t)ta * (kTcQ4KG * 32u);
                         uint32_t b_lo = tok_lo + (uint32_t)ta * tok_slot;
@@ -909,10 +915,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         }
     } else if (Q4 && warp >= 11) {
         // ------------------------------------------------------------------ dequantising warps (int4)
-        // Every row of a packed k-tile (64 nibbles, stored q + 8) becomes 64 bf16 values q * scale,
-        // written to tensor memory as the A operand of the MMAs (row = lane, two values per 32-bit
-        // column): per 32-bit word eight nibbles -> (128 + n) as bf16 by an OR into the mantissa,
-        // minus 136 (exact), times the block's scale rounded to bf16.  Scales that lie past the
+        // Every row of a packed k-tile (64 nibbles, stored q + 8) becomes 64 binary16 values
+        // q * scale, written to tensor memory as the A operand of the MMAs (row = lane, two values
+        // per 32-bit column): per 32-bit word eight nibbles -> 1024 + n or 1024 + 16 n as binary16
+        // by an OR into the mantissa, then n - 8 (exact), times the block's scale (binary16 as
+        // stored, so the product is the only rounding: 2^-12 relative).  Scales that lie past the
         // matrix read as 0 (TMA fill), so a ragged last tile contributes nothing.
         // A stage holds KG k-tiles: per row 2 * KG chunks of 16 packed bytes (32 weights, one
         // scale each).  A warp reaches the 32 lanes of its quarter (warp index mod 4) only, so
@@ -924,7 +931,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         int s = 0, ta = 0;
         uint32_t ring_par = 0, a_par = 1;
         bool alive = true;
-        const __nv_bfloat162 minus136 = __floats2bfloat162_rn(-136.0f, -136.0f);
+        const __half2 minus1032 = __floats2half2_rn(-1032.0f, -1032.0f), sixteenth = __floats2half2_rn(0.0625f, 0.0625f),
+                      minus72 = __floats2half2_rn(-72.0f, -72.0f);
         const uint32_t a_lane = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)kTcQ4ACol;
 
         // contraction lengths are multiples of 256 here, so every unit is exactly one stage and
@@ -957,26 +965,32 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     // the packed rows are swizzled over their own width by the TMA copy
                     const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
                     const uint4 pk = *reinterpret_cast<const uint4 *>(prow + ((q ^ sw) * 16));
-                    const uint32_t sbits = sc[qi >> 1] >> (16 * (qi & 1));
-                    const float sf = __half2float(__ushort_as_half((unsigned short)(sbits & 0xffffu)));
-                    const __nv_bfloat162 sc2 = __floats2bfloat162_rn(sf, sf);
+                    // the block's scale is binary16 already: both halves of a register
+                    const uint32_t sc2u = __byte_perm(sc[qi >> 1], 0u, (qi & 1) ? 0x3232u : 0x1010u);
+                    const __half2 sc2 = *reinterpret_cast<const __half2 *>(&sc2u);
                     const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
                     uint32_t o[16];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const uint32_t m = 0x000F000Fu, one28 = 0x43004300u;       // bf16 128.0 twice
+                        // A nibble n OR-ed into the mantissa of binary16 1024 is 1024 + n exactly; one
+                        // that sits four bits higher gives 1024 + 16 n, which one fused multiply-add
+                        // (x / 16 - 72) turns into the same n - 8 without a shift.  So a 32-bit word
+                        // costs one shift and four logic instructions, and the pairs come out as
                         // (n0, n4), (n1, n5), (n2, n6), (n3, n7): the token tiles carry the same
                         // permutation of every 8 columns, so no instruction is spent on reordering.
-                        // Seven instructions per word, written out: from the C expression the
-                        // compiler makes eleven.
+                        // n - 8 is exact; the product with the scale rounds once (2^-12 relative).
+                        const uint32_t mlo = 0x000F000Fu, mhi = 0x00F000F0u, k1024 = 0x64006400u;
+                        const uint32_t w8 = w[c] >> 8;
                         uint32_t e[4];
-                        tc_nibble_pair(e[0], w[c], m, one28);
-                        tc_nibble_pair(e[1], w[c] >> 4, m, one28);
-                        tc_nibble_pair(e[2], w[c] >> 8, m, one28);
-                        tc_nibble_pair(e[3], w[c] >> 12, m, one28);
+                        tc_nibble_pair(e[0], w[c], mlo, k1024);
+                        tc_nibble_pair(e[1], w[c], mhi, k1024);
+                        tc_nibble_pair(e[2], w8, mlo, k1024);
+                        tc_nibble_pair(e[3], w8, mhi, k1024);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const __nv_bfloat162 v = __hmul2(__hadd2(*reinterpret_cast<const __nv_bfloat162 *>(&e[j]), minus136), sc2);
+                            const __half2 x = *reinterpret_cast<const __half2 *>(&e[j]);
+                            const __half2 qv = (j & 1) ? __hfma2(x, sixteenth, minus72) : __hadd2(x, minus1032);
+                            const __half2 v = __hmul2(qv, sc2);
                             o[4 * c + j] = *reinterpret_cast<const uint32_t *>(&v);
                         }
                     }
@@ -1050,18 +1064,22 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const float4 uv = __ldcg(reinterpret_cast<const float4 *>(p.pre + n_el + i));
                 const float a0 = silu_mul(gv.x, uv.x), a1 = silu_mul(gv.y, uv.y), a2 = silu_mul(gv.z, uv.z),
                             a3 = silu_mul(gv.w, uv.w);
-                const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
-                const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
-                const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
                 if (Q4) {
-                    // columns i .. i + 3 of their group of 8 go to positions 0, 2, 4, 6 (first half of
-                    // the group) or 1, 3, 5, 7 (second half): the order the dequantised weights are in
+                    // binary16 hi + lo parts (the int4 path's operand format).  Columns i .. i + 3 of
+                    // their group of 8 go to positions 0, 2, 4, 6 (first half of the group) or
+                    // 1, 3, 5, 7 (second half): the order the dequantised weights are in
+                    const __half2 h01 = __floats2half2_rn(a0, a1), h23 = __floats2half2_rn(a2, a3);
+                    const __half2 l01 = __floats2half2_rn(a0 - __low2float(h01), a1 - __high2float(h01));
+                    const __half2 l23 = __floats2half2_rn(a2 - __low2float(h23), a3 - __high2float(h23));
                     const long long g8 = i & ~7ll;
                     const int odd = (int)((i >> 2) & 1);
-                    __nv_bfloat16 *ph = p.act_hi + g8 + odd, *pq = p.act_lo + g8 + odd;
-                    ph[0] = __low2bfloat16(h01); ph[2] = __high2bfloat16(h01); ph[4] = __low2bfloat16(h23); ph[6] = __high2bfloat16(h23);
-                    pq[0] = __low2bfloat16(l01); pq[2] = __high2bfloat16(l01); pq[4] = __low2bfloat16(l23); pq[6] = __high2bfloat16(l23);
+                    __half *ph = reinterpret_cast<__half *>(p.act_hi) + g8 + odd, *pq = reinterpret_cast<__half *>(p.act_lo) + g8 + odd;
+                    ph[0] = __low2half(h01); ph[2] = __high2half(h01); ph[4] = __low2half(h23); ph[6] = __high2half(h23);
+                    pq[0] = __low2half(l01); pq[2] = __high2half(l01); pq[4] = __low2half(l23); pq[6] = __high2half(l23);
                 } else {
+                    const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
+                    const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
+                    const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
                     uint2 hv, lv;
                     hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
                     lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);

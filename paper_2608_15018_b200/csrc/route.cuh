@@ -465,12 +465,19 @@ constexpr int kRouteTok = 16;   // most tokens accumulated per pass
 
 // Buffers that the layer's later kernels accumulate into and that must start at zero; the
 // routing blocks clear them (16-byte units) so that no separate fill precedes the layer.
+// two bf16 values -> two binary16 values (round to nearest; exact for magnitudes in [2^-14, 65504])
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t u)
+{
+    const __half2 h = __floats2half2_rn(bf16_lo(u), bf16_hi(u));
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
 struct ZeroList {
     void *ptr[3];
     unsigned long long n16[3];
-    // int4 tensor-core path: a copy of the bf16 hidden states whose columns are permuted inside
-    // every group of 8 (position p holds column [0,4,1,5,2,6,3,7][p]), the order in which the
-    // dequantising warps of the FFN kernel get the nibbles of a 32-bit word for free
+    // int4 tensor-core path: a binary16 copy of the bf16 hidden states whose columns are permuted
+    // inside every group of 8 (position p holds column [0,4,1,5,2,6,3,7][p]), the order in which
+    // the dequantising warps of the FFN kernel get the nibbles of a 32-bit word for free
     const uint4 *perm_src;
     uint4 *perm_dst;
     unsigned long long perm_n16;
@@ -548,9 +555,9 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     }
     for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.perm_n16;
          i += (unsigned long long)gridDim.x * kRouteThreads) {
-        const uint4 v = zl.perm_src[i];             // halves h0..h7
-        zl.perm_dst[i] = make_uint4(__byte_perm(v.x, v.z, 0x5410), __byte_perm(v.x, v.z, 0x7632),
-                                    __byte_perm(v.y, v.w, 0x5410), __byte_perm(v.y, v.w, 0x7632));
+        const uint4 v = zl.perm_src[i];             // halves h0..h7 (bf16)
+        zl.perm_dst[i] = make_uint4(bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x7632)),
+                                    bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x7632)));
     }
     // blocks past the router's rows exist only to help with the clearing and the copy above (a
     // layer with few experts and wide accumulators would otherwise clear megabytes with a few blocks)
