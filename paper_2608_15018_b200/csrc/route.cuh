@@ -4,366 +4,35 @@
 //                  that the discrete choices below do not depend on the summation order;
 //                  block 0 then runs gating_block once every row has arrived:
 //   gating_block : Eq. 4 aggregation, TopCap, lambda_b, biased top-k, mixing weights,
-//                  union / unique count, token->expert bucketing, stage tables.
+//                  union / unique count (gating.cuh), token->expert bucketing, stage tables.
 #pragma once
 
 #include "common.cuh"
 #include "ffn_stream.cuh"
+#include "gating.cuh"
 
 namespace s2moe {
 
 
-__device__ __forceinline__ double warp_sum(double v)
+// What the expert kernels read of a finished gating (see gating_group for gm): the bucketing
+// arrays in the workspace, tokens ascending inside an expert, the shared experts' groups behind
+// the routed ones, and the stage tables of the streaming kernel.
+__device__ __forceinline__ void gating_writeout(const Shape &sh, int B, const Workspace &ws, const GateMem &gm, int has_gate,
+                                                int32_t *__restrict__ n_unique, const GateGroup gg)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-__device__ __forceinline__ double warp_max(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-
-// One copy of the double-precision exponential for the whole gating: the gating runs once, on
-// one block, with a cold instruction cache, so its cost follows the amount of distinct code.
-__device__ __noinline__ double exp_once(double x) { return exp(x); }
-
-// Monotone map from doubles (no NaN) to unsigned integers: a < b  <=>  dkey(a) < dkey(b), and
-// equal doubles (-0 included) have equal keys.  Keys of finite values are never 0.
-__device__ __forceinline__ unsigned long long dkey(double x)
-{
-    const long long b = __double_as_longlong(x + 0.0);
-    return (unsigned long long)(b ^ ((b >> 63) | (long long)0x8000000000000000ull));
-}
-__device__ __forceinline__ double dkey_value(unsigned long long k)
-{
-    const long long b = (long long)k;
-    return __longlong_as_double(b < 0 ? (b ^ (long long)0x8000000000000000ull) : ~b);
-}
-// maximum of a 64-bit key over the warp: two 32-bit warp reductions
-__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long k)
-{
-    const unsigned hi = (unsigned)(k >> 32);
-    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
-    const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? (unsigned)k : 0u);
-    return ((unsigned long long)mh << 32) | ml;
-}
-// lanes (as a ballot) that hold the largest key among the lanes with `has`; the common case
-// (one lane has the largest upper half) takes one warp reduction and one ballot
-__device__ __forceinline__ unsigned warp_max_holders(unsigned long long k, bool has)
-{
-    const unsigned hi = has ? (unsigned)(k >> 32) : 0u;
-    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
-    bool hold = has && hi == mh;
-    unsigned hb = __ballot_sync(0xffffffffu, hold);
-    if (__popc(hb) > 1) {
-        const unsigned ml = __reduce_max_sync(0xffffffffu, hold ? (unsigned)k : 0u);
-        hold = hold && (unsigned)k == ml;
-        hb = __ballot_sync(0xffffffffu, hold);
-    }
-    return hb;
-}
-__device__ __forceinline__ unsigned long long shfl_key(unsigned long long k, int src)
-{
-    const unsigned lo = __shfl_sync(0xffffffffu, (unsigned)k, src);
-    const unsigned hi = __shfl_sync(0xffffffffu, (unsigned)(k >> 32), src);
-    return ((unsigned long long)hi << 32) | lo;
-}
-
-
-// Order statistics of one token's original logits, one warp per token (lane owns experts lane,
-// lane + 32, ...): lambda_b = alpha (l_(1) - l_(k+1)) by k + 1 rounds of a warp-wide maximum over
-// integer keys, and, for weight_mode 0, the softmax denominator over the original logits.
-template <int J>
-__device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on, const double *s_l, double *s_lam,
-                                           double *s_zmax, double *s_den, int lane)
-{
+    const int tid = gg.t, nt = gg.n;
     const int E = sh.E, k = sh.k;
-    unsigned long long k1[J];
-    unsigned valid = 0;
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-        const int e = lane + 32 * j;
-        k1[j] = 0ull;
-        if (e < E) { k1[j] = dkey(s_l[b * E + e]); valid |= 1u << j; }
-    }
-    unsigned long long top1 = 0ull, kth = 0ull;
-    const int rounds = bias_on ? k + 1 : 1;
-    if constexpr (J == 2) {
-        // two elements per lane: the lane offers its larger one and, once that has won a round,
-        // the other (a key of 0 = nothing left); a round is one reduction and one ballot
-        unsigned long long cur = k1[0] > k1[1] ? k1[0] : k1[1], nxt = k1[0] > k1[1] ? k1[1] : k1[0];
-#pragma unroll 1
-        for (int r = 0; r < rounds; ++r) {
-            const unsigned hb = warp_max_holders(cur, cur != 0ull);
-            const int wl = __ffs(hb) - 1;
-            if (r == 0) top1 = shfl_key(cur, wl);
-            if (r == k) kth = shfl_key(cur, wl);
-            if (lane == wl) { cur = nxt; nxt = 0ull; }       // drop one instance of the maximum
-        }
-    } else {
-        unsigned alive = valid;
-#pragma unroll 1
-        for (int r = 0; r < rounds; ++r) {
-            unsigned long long lm = 0ull;
-            int bj = 0;
-#pragma unroll
-            for (int j = 0; j < J; ++j)
-                if (((alive >> j) & 1u) && k1[j] > lm) { lm = k1[j]; bj = j; }
-            const unsigned hb = warp_max_holders(lm, alive != 0u);
-            const int wl = __ffs(hb) - 1;
-            if (r == 0) top1 = shfl_key(lm, wl);
-            if (r == k) kth = shfl_key(lm, wl);
-            if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
-        }
-    }
-    const double ztop = dkey_value(top1);
-    double den = 0.0;
-    if (!sh.weight_mode) {
-#pragma unroll 1
-        for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) - ztop);
-        den = warp_sum(den);
-    }
-    if (lane == 0) {
-        s_lam[b] = bias_on ? sh.alpha * (ztop - dkey_value(kth)) : 0.0;
-        s_zmax[b] = ztop;
-        s_den[b] = den;
-    }
-}
-
-// Biased top-k of one token in the order (l' descending, l descending, id ascending), one
-// winner per round, and the mixing weights of the winners.
-template <int J>
-__device__ __forceinline__ void gate_select(const Shape &sh, int b, const double *s_l, const unsigned char *s_star,
-                                            const double *s_lam, const double *s_zmax, const double *s_den, int *s_sel,
-                                            float *s_pw, unsigned long long *s_mask, int32_t *__restrict__ sel_idx,
-                                            float *__restrict__ sel_w, int lane)
-{
-    const unsigned full = 0xffffffffu;
-    const int E = sh.E, k = sh.k;
-    const double lam = s_lam[b];
-    double l[J];
-    unsigned long long k1[J], k2[J];
-    unsigned valid = 0, star = 0;
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-        const int e = lane + 32 * j;
-        l[j] = 0.0;
-        k1[j] = 0ull;
-        k2[j] = 0ull;
-        if (e < E) {
-            l[j] = s_l[b * E + e] + 0.0;
-            k1[j] = dkey(l[j]);
-            const unsigned st = s_star[e];
-            star |= st << j;
-            k2[j] = st ? dkey(l[j] + lam) : k1[j];
-            valid |= 1u << j;
-        }
-    }
-    if constexpr (J == 2) {
-        // the lane offers its better element first (order: l' descending, l descending, id
-        // ascending; element 0 has the lower id), then the other one
-        const bool first0 = k2[0] > k2[1] || (k2[0] == k2[1] && k1[0] >= k1[1]);
-        unsigned long long c2 = first0 ? k2[0] : k2[1], c1 = first0 ? k1[0] : k1[1];
-        unsigned long long n2 = first0 ? k2[1] : k2[0], n1 = first0 ? k1[1] : k1[0];
-        unsigned ce = (unsigned)lane + (first0 ? 0u : 32u), ne = (unsigned)lane + (first0 ? 32u : 0u);
-#pragma unroll 1
-        for (int r = 0; r < k; ++r) {
-            unsigned hb = warp_max_holders(c2, c2 != 0ull);
-            if (__popc(hb) > 1) {                       // equal biased logits: larger original logit first
-                hb = warp_max_holders(c1, (hb >> lane) & 1u);
-                if (__popc(hb) > 1) {                   // still equal: lower expert id first
-                    const bool hold = (hb >> lane) & 1u;
-                    const unsigned me = __reduce_min_sync(full, hold ? ce : 0xffffffffu);
-                    hb = __ballot_sync(full, hold && ce == me);
-                }
-            }
-            if (lane == __ffs(hb) - 1) {
-                s_sel[b * k + r] = (int)ce;
-                c2 = n2; c1 = n1; ce = ne;
-                n2 = 0ull;
-            }
-        }
-    } else {
-        unsigned alive = valid;
-#pragma unroll 1
-        for (int r = 0; r < k; ++r) {
-            unsigned long long b2 = 0ull, b1 = 0ull;
-            int bj = -1;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                if ((alive >> j) & 1u) {
-                    const bool better = k2[j] > b2 || (k2[j] == b2 && k1[j] > b1);
-                    if (bj < 0 || better) { b2 = k2[j]; b1 = k1[j]; bj = j; }
-                }
-            }
-            const unsigned my_e = (unsigned)(lane + 32 * (bj < 0 ? 0 : bj));
-            unsigned hb = warp_max_holders(b2, bj >= 0);
-            if (__popc(hb) > 1) {                           // equal biased logits: larger original logit first
-                hb = warp_max_holders(b1, (hb >> lane) & 1u);
-                if (__popc(hb) > 1) {                       // still equal: lower expert id first
-                    const bool hold = (hb >> lane) & 1u;
-                    const unsigned me = __reduce_min_sync(full, hold ? my_e : 0xffffffffu);
-                    hb = __ballot_sync(full, hold && my_e == me);
-                }
-            }
-            if (lane == __ffs(hb) - 1) {
-                alive &= ~(1u << bj);
-                s_sel[b * k + r] = (int)my_e;
-            }
-        }
-    }
-    __syncwarp();
-    // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
-    double zmax = s_zmax[b], den = s_den[b];
-    const double lamw = sh.weight_mode ? lam : 0.0;
-    if (sh.weight_mode) {
-        unsigned long long zk = 0ull;
-#pragma unroll
-        for (int j = 0; j < J; ++j)
-            if (((valid >> j) & 1u) && k2[j] > zk) zk = k2[j];
-        zmax = dkey_value(warp_max_key(zk));
-        den = 0.0;
-#pragma unroll 1
-        for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) + (s_star[e] ? lamw : 0.0) - zmax);
-        den = warp_sum(den);
-    }
-    double p = 0.0;
-    int my_sel = 0;
-    if (lane < k) {
-        my_sel = s_sel[b * k + lane];
-        const double zs = s_l[b * E + my_sel] + (s_star[my_sel] ? lamw : 0.0);
-        p = exp_once(zs - zmax) / den;
-    }
-    if (sh.renorm) {
-        const double tot = warp_sum(p);
-        p /= tot;
-    }
-    if (lane < k) {
-        s_pw[b * k + lane] = (float)p;
-        sel_idx[b * k + lane] = my_sel;
-        sel_w[b * k + lane] = (float)p;
-        // the token's bit in the expert's 64-bit mask: a native 32-bit shared-memory atomic on the
-        // half that holds it (a 64-bit atomicOr would be a compare-and-swap loop)
-        atomicOr(reinterpret_cast<unsigned *>(&s_mask[my_sel]) + (b >> 5), 1u << (b & 31));
-    }
-}
-
-// Gating of one batch by one thread block of at least two warps.
-// s_l: shared memory for B*E doubles (the logits, copied from the workspace).
-template <int JE>
-__device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
-                                             int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
-                                             int32_t *__restrict__ n_unique, double *s_l)
-{
-    __shared__ unsigned long long s_gk[kMaxExperts];
-    __shared__ unsigned char s_star[kMaxExperts];
-    __shared__ double s_w[kMaxTokens], s_lam[kMaxTokens], s_zmax[kMaxTokens], s_den[kMaxTokens];
-    __shared__ int s_sel[kMaxTokens * kMaxTopK];
-    __shared__ float s_pw[kMaxTokens * kMaxTopK];
-    __shared__ unsigned long long s_mask[kMaxExperts];
-    __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_pos[kMaxExperts];
-    __shared__ int s_U;
-
-    const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
-    const int E = sh.E, k = sh.k, cap = sh.cap;
-    const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
-
-#pragma unroll 1
-    for (int i = tid; i < B * E; i += nt) s_l[i] = __ldcg(&ws.logits[i]);
-#pragma unroll 1
-    for (int b = tid; b < B; b += nt) s_w[b] = conf ? (double)conf[b] : 1.0;
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) { s_star[e] = 0; s_mask[e] = 0ull; }
-    __syncthreads();
-
-    // Two independent pieces run side by side on disjoint warps: the last cw warps pick the
-    // reuse-reward set E* (Eq. 4 aggregation, TopCap), the others take the per-token order
-    // statistics (lambda_b, softmax denominator).
-    const int cw = bias_on ? max(1, min(nw / 2, nw - B)) : 0, tw = nw - cw;
-    if (warp >= tw) {
-        const int ct = tid - tw * 32, cn = cw * 32;
-        // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
-#pragma unroll 1
-        for (int e = ct; e < E; e += cn) {
-            double g = 0.0;
-#pragma unroll 1
-            for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
-            s_gk[e] = dkey(g);
-        }
-        asm volatile("bar.sync 1, %0;" ::"r"(cn) : "memory");
-        // TopCap by rank in the order (g descending, id ascending)
-#pragma unroll 1
-        for (int e = ct; e < E; e += cn) {
-            const unsigned long long ge = s_gk[e];
-            int rank = 0;
-#pragma unroll 4
-            for (int o = 0; o < E; ++o) {
-                const unsigned long long go = s_gk[o];
-                rank += (go > ge) | ((go == ge) & (o < e));
-            }
-            s_star[e] = rank < cap;
-        }
-    } else {
-#pragma unroll 1
-        for (int b = warp; b < B; b += tw) {
-            gate_stats<JE>(sh, b, bias_on, s_l, s_lam, s_zmax, s_den, lane);
-        }
-    }
-    __syncthreads();
-
-#pragma unroll 1
-    for (int b = warp; b < B; b += nw) {
-        gate_select<JE>(sh, b, s_l, s_star, s_lam, s_zmax, s_den, s_sel, s_pw, s_mask, sel_idx, sel_w, lane);
-    }
-    __syncthreads();
-
-    // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts
-    if (tid < 32) {
-        const int C = (E + 31) >> 5, e0 = tid * C;
-        int sum = 0, act = 0;
-#pragma unroll 1
-        for (int i = 0; i < C; ++i) {
-            const int e = e0 + i;
-            if (e < E) {
-                const int c = __popcll(s_mask[e]);
-                s_cnt[e] = c;
-                sum += c;
-                act += c > 0;
-            }
-        }
-        int xs = sum, xa = act;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, xs, o), u = __shfl_up_sync(0xffffffffu, xa, o);
-            if (tid >= o) { xs += t; xa += u; }
-        }
-        int off = xs - sum, pos = xa - act;
-#pragma unroll 1
-        for (int i = 0; i < C; ++i) {
-            const int e = e0 + i;
-            if (e < E) {
-                s_off[e] = off;
-                s_pos[e] = pos;
-                off += s_cnt[e];
-                pos += s_cnt[e] > 0;
-            }
-        }
-        if (tid == 31) { s_off[E] = xs; s_U = xa; }
-    }
-    __syncthreads();
-    const int U = s_U, n_routed = B * k;
+    const int U = *gm.U, n_routed = B * k;
 #pragma unroll 1
     for (int e = tid; e < E; e += nt) {
-        ws.counts[e] = s_cnt[e];
-        ws.offsets[e] = s_off[e];
-        if (s_cnt[e] > 0) {
-            ws.active[s_pos[e]] = e;
+        ws.counts[e] = gm.cnt[e];
+        ws.offsets[e] = gm.off[e];
+        ws.tokmask[e] = gm.mask[e];
+        if (gm.cnt[e] > 0) {
+            ws.active[gm.pos[e]] = e;
             if (ws.gtab) {
-                ws.gtab[2 * s_pos[e]] = make_uint4((unsigned)e, (unsigned)s_cnt[e], (unsigned)s_off[e], 0u);
-                ws.gtab[2 * s_pos[e] + 1] = make_uint4((unsigned)s_mask[e], (unsigned)(s_mask[e] >> 32), 0u, 0u);
+                ws.gtab[2 * gm.pos[e]] = make_uint4((unsigned)e, (unsigned)gm.cnt[e], (unsigned)gm.off[e], 0u);
+                ws.gtab[2 * gm.pos[e] + 1] = make_uint4((unsigned)gm.mask[e], (unsigned)(gm.mask[e] >> 32), 0u, 0u);
             }
         }
     }
@@ -371,12 +40,13 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
 #pragma unroll 1
     for (int i = tid; i < n_routed; i += nt) {
         const int b = i / k;
-        const int e = s_sel[i];
-        const int pos = s_off[e] + __popcll(s_mask[e] & ((1ull << b) - 1ull));
+        const int e = gm.sel[i];
+        const int pos = gm.off[e] + __popcll(gm.mask[e] & ((1ull << b) - 1ull));
         ws.slot_token[pos] = b;
-        ws.slot_w[pos] = s_pw[i];
+        ws.slot_w[pos] = gm.pw[i];
     }
     // shared experts: every token, weight c_b
+    const unsigned long long all = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
 #pragma unroll 1
     for (int i = tid; i < sh.n_sh * B; i += nt) {
         const int s = i / B, b = i - s * B;
@@ -388,41 +58,37 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             ws.counts[E + s] = B;
             ws.offsets[E + s] = n_routed + s * B;
             ws.active[U + s] = E + s;
+            ws.tokmask[E + s] = all;
             if (ws.gtab) {
-                const unsigned long long all = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
                 ws.gtab[2 * (U + s)] = make_uint4((unsigned)(E + s), (unsigned)B, (unsigned)(n_routed + s * B), 0u);
                 ws.gtab[2 * (U + s) + 1] = make_uint4((unsigned)all, (unsigned)(all >> 32), 0u, 0u);
             }
         }
     }
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) ws.tokmask[e] = s_mask[e];
-#pragma unroll 1
-    for (int s = tid; s < sh.n_sh; s += nt) ws.tokmask[E + s] = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
     if (sh.plan == 2) {
         // stage tables of the streaming kernel: per active group, its first phase-1 stage
         // (4 gate + 4 up rows each) and first phase-2 stage (8 down rows x one K-slice)
-        __syncthreads();
+        gate_sync(gg);
 #pragma unroll 1
         for (int e = tid; e < E; e += nt)
-            s_cnt[e] = s_cnt[e] > 0 ? st_nks(sh.f, s_cnt[e], sh.op_cap, sh.d) * (sh.d / 8) : 0;   // phase-2 stages
-        __syncthreads();
+            gm.cnt[e] = gm.cnt[e] > 0 ? st_nks(sh.f, gm.cnt[e], sh.op_cap, sh.d) * (sh.d / 8) : 0;   // phase-2 stages
+        gate_sync(gg);
 #pragma unroll 1
         for (int e = tid; e < E; e += nt) {
-            if (s_mask[e]) {
+            if (gm.mask[e]) {
                 int pre = 0;
 #pragma unroll 1
-                for (int o = 0; o < e; ++o) pre += s_cnt[o];
-                const int a = s_pos[e];
+                for (int o = 0; o < e; ++o) pre += gm.cnt[o];
+                const int a = gm.pos[e];
                 ws.upfx1[a] = a * (sh.f / 4);
                 ws.upfx2[a] = pre;
                 ws.sync[a] = 0;
-                if (a == U - 1) s_off[0] = pre + s_cnt[e];   // all routed phase-2 stages
+                if (a == U - 1) gm.off[0] = pre + gm.cnt[e];   // all routed phase-2 stages
             }
         }
-        __syncthreads();
+        gate_sync(gg);
         if (tid == 0) {
-            int t1 = U * (sh.f / 4), t2 = s_off[0];
+            int t1 = U * (sh.f / 4), t2 = gm.off[0];
 #pragma unroll 1
             for (int s = 0; s <= sh.n_sh; ++s) {
                 ws.upfx1[U + s] = t1;
@@ -445,6 +111,34 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
         ws.header[3] = B;
         *n_unique = U;
     }
+}
+
+// Gating of one batch by a whole thread block (kRouteThreads threads) on the logits in the workspace.
+// s_l: shared memory for B * E + B doubles (the logits and the confidences are staged there).
+template <int JE>
+__device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
+                                             int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
+                                             int32_t *__restrict__ n_unique, double *s_l)
+{
+    __shared__ unsigned long long s_mask[kMaxExperts], s_gk[kMaxExperts];
+    __shared__ double s_lam[kMaxTokens], s_zmax[kMaxTokens], s_den[kMaxTokens];
+    __shared__ int s_sel[kMaxTokens * kMaxTopK];
+    __shared__ float s_pw[kMaxTokens * kMaxTopK];
+    __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_pos[kMaxExperts];
+    __shared__ int s_U;
+    __shared__ unsigned char s_star[kMaxExperts];
+    GateMem gm;
+    gm.mask = s_mask; gm.gk = s_gk; gm.lam = s_lam; gm.zmax = s_zmax; gm.den = s_den; gm.sel = s_sel; gm.pw = s_pw;
+    gm.cnt = s_cnt; gm.off = s_off; gm.pos = s_pos; gm.U = &s_U; gm.star = s_star;
+    const GateGroup gg{(int)threadIdx.x, (int)blockDim.x, 0};
+    double *s_w = s_l + B * sh.E;
+#pragma unroll 1
+    for (int i = gg.t; i < B * sh.E; i += gg.n) s_l[i] = __ldcg(&ws.logits[i]);
+#pragma unroll 1
+    for (int b = gg.t; b < B; b += gg.n) s_w[b] = conf ? (double)conf[b] : 1.0;
+    // (gating_group's first barrier orders these writes before the first read)
+    gating_group<JE>(sh, B, s_l, s_w, gg, gm, sel_idx, sel_w);
+    gating_writeout(sh, B, ws, gm, has_gate, n_unique, gg);
 }
 
 // 4 consecutive elements of a plain (f32 / bf16) row starting at column c (c % 4 == 0)
@@ -529,7 +223,7 @@ __device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const
 // Router logits and gating in one launch.  A block computes one row of the router (row E is the
 // shared-expert gate vector) against one group of the batch's tokens in float64; block 0 then
 // runs the gating for the whole batch once every block has arrived (atomic ticket).
-// Dynamic shared memory: max(B * E, 16 * kRouteTok) doubles.
+// Dynamic shared memory: max(B * E + B, 16 * kRouteTok) doubles.
 // JE: experts per lane in the gating (2, 4 or 8 for up to 64, 128, 256 experts): a kernel of its own
 // for each, so that the gating code of a launch is one straight piece
 template <int ACT, int RT, int JE>
@@ -592,10 +286,8 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     if (tid == 0) {
         unsigned token = 0u;
         if (blockIdx.x == 0) {
-            // differs from launch to launch (a wrapped nanosecond timer; never 0)
-            unsigned long long gt;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-            token = (unsigned)gt | 1u;
+            // differs from launch to launch (the SM's cycle counter; never 0)
+            token = (unsigned)clock() | 1u;
             asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 2), "r"(token) : "memory");
         }
         unsigned t;

@@ -190,7 +190,7 @@ cudaLaunchConfig_t pdl_config(s2moe_ctx *ctx, int grid, int block, size_t smem, 
 
 size_t route_smem(int B, int E)
 {
-    const size_t a = (size_t)B * E, b = (size_t)(kRouteThreads / 32) * kRouteTok;
+    const size_t a = (size_t)B * E + (size_t)B, b = (size_t)(kRouteThreads / 32) * kRouteTok;
     return sizeof(double) * (a > b ? a : b);
 }
 
@@ -251,7 +251,7 @@ cudaError_t prepare_route_t(int bytes)
 
 cudaError_t prepare_route()
 {
-    const int bytes = (int)(sizeof(double) * kMaxTokens * kMaxExperts);
+    const int bytes = (int)route_smem(kMaxTokens, kMaxExperts);
     cudaError_t e = prepare_route_t<DT_F32, DT_F32>(bytes);
     if (e == cudaSuccess) e = prepare_route_t<DT_F32, DT_BF16>(bytes);
     if (e == cudaSuccess) e = prepare_route_t<DT_BF16, DT_F32>(bytes);
