@@ -124,7 +124,14 @@ typedef struct {
                                  2^-12 relative per weight; block scales below 2^-17 lose
                                  precision in binary16's subnormal range; the hidden states
                                  are converted to binary16 for this kernel, so they must
-                                 stay below 65504 in magnitude)                               */
+                                 stay below 65504 in magnitude);
+                              4: plan 3's kernel as the whole layer in ONE launch: its CTAs
+                                 share the router's logit pass, meet once, every CTA runs the
+                                 gating for itself, and the shared experts and the expert of
+                                 every token's largest logit stream while it does (same
+                                 formats as plan 3; not for offloaded contexts; needs room
+                                 for n_tokens * n_experts float64 logits in shared memory).
+                                 On demand only: measured slower than plan 3's two launches  */
 } s2moe_config;
 
 /*
@@ -247,7 +254,7 @@ int s2moe_last_device_status(s2moe_ctx *ctx, int32_t *host_out);
 /* The last cudaError_t a call on this context saw (0 = cudaSuccess). */
 int s2moe_last_cuda_error(const s2moe_ctx *ctx);
 
-/* The kernel plan a batch of n_tokens runs with (1, 2 or 3; see s2moe_config.kernel_plan).
+/* The kernel plan a batch of n_tokens runs with (1, 2, 3 or 4; see s2moe_config.kernel_plan).
  * 0: NULL context, n_tokens out of range, or plan 2 / 3 was demanded and this batch size
  * does not fit its shared-memory layout (s2moe_verify_layer then returns EINVAL). */
 int s2moe_kernel_plan(const s2moe_ctx *ctx, int32_t n_tokens);

@@ -90,11 +90,13 @@ struct GateMem {
     float *pw;                  // [B * k] their mixing weights
     int *cnt, *off, *pos;       // [E] tokens per expert, [E + 1] first slot, [E] index in the active list
     int *U;                     // [1] distinct selected experts
+    unsigned *star32;           // [8] E* as bit words (bit i of word j: expert i + 32 j)
+    unsigned *topk;             // [B][J] every token's first k experts by original logit, same bit layout (bias on only)
     unsigned char *star;        // [E] member of E*
 };
 __host__ __device__ __forceinline__ size_t gate_mem_bytes(int E, int B, int k)
 {
-    return 16 * (size_t)E + 24 * (size_t)B + 8 * (size_t)B * k + 4 * (size_t)(3 * E + 1) + 4 +
+    return 16 * (size_t)E + 24 * (size_t)B + 8 * (size_t)B * k + 4 * (size_t)(3 * E + 1) + 4 + 32 + 4 * (size_t)B * 8 +
            (((size_t)E + 15) & ~(size_t)15) + 16;
 }
 __device__ __forceinline__ GateMem gate_mem_carve(void *base, int E, int B, int k)
@@ -112,17 +114,23 @@ __device__ __forceinline__ GateMem gate_mem_carve(void *base, int E, int B, int 
     m.off = reinterpret_cast<int *>(p); p += 4 * (size_t)(E + 1);
     m.pos = reinterpret_cast<int *>(p); p += 4 * (size_t)E;
     m.U = reinterpret_cast<int *>(p); p += 4;
+    m.star32 = reinterpret_cast<unsigned *>(p); p += 32;
+    m.topk = reinterpret_cast<unsigned *>(p); p += 4 * (size_t)B * 8;
     m.star = p;
     return m;
 }
 
 // Order statistics of one token's original logits, one warp per token (lane owns experts lane,
 // lane + 32, ...): lambda_b = alpha (l_(1) - l_(k+1)) by k + 1 rounds of a warp-wide maximum over
-// integer keys, and, for weight_mode 0, the softmax denominator over the original logits.
+// integer keys, winners in the exact order (logit descending, id ascending); the token's first k
+// experts in that order as bit words (word j, bit i: expert i + 32 j; s_topk, or NULL); and, for
+// weight_mode 0 and unless the caller leaves it to gate_select (with_den false), the softmax
+// denominator over the original logits.
 template <int J>
 __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on, const double *s_l, double *s_lam,
-                                           double *s_zmax, double *s_den, int lane)
+                                           double *s_zmax, double *s_den, unsigned *s_topk, bool with_den, int lane)
 {
+    const unsigned full = 0xffffffffu;
     const int E = sh.E, k = sh.k;
     unsigned long long k1[J];
     unsigned valid = 0;
@@ -134,17 +142,28 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
     }
     unsigned long long top1 = 0ull, kth = 0ull;
     const int rounds = bias_on ? k + 1 : 1;
+    unsigned won = 0;                                    // bit j: element j of this lane is among the first k
     if constexpr (J == 2) {
-        // two elements per lane: the lane offers its larger one and, once that has won a round,
-        // the other (a key of 0 = nothing left); a round is one reduction and one ballot
-        unsigned long long cur = k1[0] > k1[1] ? k1[0] : k1[1], nxt = k1[0] > k1[1] ? k1[1] : k1[0];
+        // two elements per lane: the lane offers its first one in the order and, once that has won a
+        // round, the other (a key of 0 = nothing left); a round is one reduction and one ballot
+        const bool first0 = k1[0] >= k1[1];
+        unsigned long long cur = first0 ? k1[0] : k1[1], nxt = first0 ? k1[1] : k1[0];
+        unsigned cj = first0 ? 0u : 1u;
 #pragma unroll 1
         for (int r = 0; r < rounds; ++r) {
-            const unsigned hb = warp_max_holders(cur, cur != 0ull);
+            unsigned hb = warp_max_holders(cur, cur != 0ull);
+            if (__popc(hb) > 1) {                        // equal logits: lower expert id first
+                const bool hold = (hb >> lane) & 1u;
+                const unsigned me = __reduce_min_sync(full, hold ? (unsigned)lane + 32u * cj : 0xffffffffu);
+                hb = __ballot_sync(full, hold && (unsigned)lane + 32u * cj == me);
+            }
             const int wl = __ffs(hb) - 1;
             if (r == 0) top1 = shfl_key(cur, wl);
             if (r == k) kth = shfl_key(cur, wl);
-            if (lane == wl) { cur = nxt; nxt = 0ull; }       // drop one instance of the maximum
+            if (lane == wl) {                            // drop the winner
+                if (r < k) won |= 1u << cj;
+                cur = nxt; nxt = 0ull; cj ^= 1u;
+            }
         }
     } else {
         unsigned alive = valid;
@@ -155,16 +174,31 @@ __device__ __forceinline__ void gate_stats(const Shape &sh, int b, bool bias_on,
 #pragma unroll
             for (int j = 0; j < J; ++j)
                 if (((alive >> j) & 1u) && k1[j] > lm) { lm = k1[j]; bj = j; }
-            const unsigned hb = warp_max_holders(lm, alive != 0u);
+            unsigned hb = warp_max_holders(lm, alive != 0u);
+            if (__popc(hb) > 1) {                        // equal logits: lower expert id first
+                const bool hold = (hb >> lane) & 1u;
+                const unsigned me = __reduce_min_sync(full, hold ? (unsigned)(lane + 32 * bj) : 0xffffffffu);
+                hb = __ballot_sync(full, hold && (unsigned)(lane + 32 * bj) == me);
+            }
             const int wl = __ffs(hb) - 1;
             if (r == 0) top1 = shfl_key(lm, wl);
             if (r == k) kth = shfl_key(lm, wl);
-            if (lane == wl) alive &= ~(1u << bj);            // drop one instance of the maximum
+            if (lane == wl) {                            // drop the winner
+                if (r < k) won |= 1u << bj;
+                alive &= ~(1u << bj);
+            }
+        }
+    }
+    if (s_topk) {
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const unsigned word = __ballot_sync(full, (won >> j) & 1u);
+            if (lane == 0) s_topk[b * J + j] = word;
         }
     }
     const double ztop = dkey_value(top1);
     double den = 0.0;
-    if (!sh.weight_mode) {
+    if (!sh.weight_mode && with_den) {
 #pragma unroll 1
         for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) - ztop);
         den = warp_sum(den);
@@ -182,7 +216,7 @@ template <int J>
 __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double *s_l, const unsigned char *s_star,
                                             const double *s_lam, const double *s_zmax, const double *s_den, int *s_sel,
                                             float *s_pw, unsigned long long *s_mask, int32_t *__restrict__ sel_idx,
-                                            float *__restrict__ sel_w, int lane)
+                                            float *__restrict__ sel_w, bool have_den, int lane)
 {
     const unsigned full = 0xffffffffu;
     const int E = sh.E, k = sh.k;
@@ -262,6 +296,12 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
     // mixing weights: softmax over all experts of l (weight_mode 0) or l' (weight_mode 1)
     double zmax = s_zmax[b], den = s_den[b];
     const double lamw = sh.weight_mode ? lam : 0.0;
+    if (!sh.weight_mode && !have_den) {
+        den = 0.0;
+#pragma unroll 1
+        for (int e = lane; e < E; e += 32) den += exp_once((s_l[b * E + e] + 0.0) - zmax);
+        den = warp_sum(den);
+    }
     if (sh.weight_mode) {
         unsigned long long zk = 0ull;
 #pragma unroll
@@ -298,65 +338,89 @@ __device__ __forceinline__ void gate_select(const Shape &sh, int b, const double
 
 // Steps O2..O5 for B tokens on `s_l` [B][E] (logits) and `s_w` [B] (confidences), both in SHARED
 // memory and visible to the group (every row is read several times and E* needs all of them, so a
-// caller stages them once: one memory round trip for the whole gating), by the warps of `gg`.
-// On return (the group is synchronised) gm holds: sel / pw in selection order, the per-expert
-// token masks and counts, the exclusive scan `off`, the index `pos` of every active expert in the
-// ascending list of active experts, and U.  sel_idx / sel_w (global, or NULL) receive the
-// selection and the weights.  J: experts per lane (2, 4, 8 for up to 64, 128, 256 experts).
+// caller stages them once: one memory round trip for the whole gating), by the warps of `gg`, in
+// two parts.  After gating_part1 (the group is synchronised) gm holds E* (star, star32), lambda_b and
+// every token's first k experts by original logit (topk: with the bias on these are the experts
+// that the token keeps whenever they are in E*, see the fused kernel); after gating_part2 sel / pw
+// in selection order, the per-expert token masks and counts, the exclusive scan `off`, the index
+// `pos` of every active expert in the ascending list of active experts, and U.  sel_idx / sel_w
+// (global, or NULL) receive the selection and the weights.  den_early: the softmax denominators are
+// taken in part 1 (beside the search for E*), else in part 2.
+// J: experts per lane (2, 4, 8 for up to 64, 128, 256 experts).
+// E* by cn threads (thread ct of them; a multiple of 32) that meet on hardware barrier `bar`:
+// Eq. 4 aggregation, TopCap by rank.  gm.star and gm.star32 must have been cleared.
+__device__ __forceinline__ void gating_estar(const Shape &sh, int B, const double *__restrict__ s_l,
+                                             const double *__restrict__ s_w, const GateMem &gm, int ct, int cn, int bar)
+{
+    const int E = sh.E, cap = sh.cap;
+    // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
+#pragma unroll 1
+    for (int e = ct; e < E; e += cn) {
+        double g = 0.0;
+#pragma unroll 1
+        for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
+        gm.gk[e] = dkey(g);
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(cn) : "memory");
+    // TopCap by rank in the order (g descending, id ascending)
+#pragma unroll 1
+    for (int e = ct; e < E; e += cn) {
+        const unsigned long long ge = gm.gk[e];
+        int rank = 0;
+#pragma unroll 4
+        for (int o = 0; o < E; ++o) {
+            const unsigned long long go = gm.gk[o];
+            rank += (go > ge) | ((go == ge) & (o < e));
+        }
+        gm.star[e] = rank < cap;
+        if (rank < cap) atomicOr(&gm.star32[e >> 5], 1u << (e & 31));
+    }
+}
+
 template <int J>
-__device__ __forceinline__ void gating_group(const Shape &sh, int B, const double *__restrict__ s_l,
-                                             const double *__restrict__ s_w, const GateGroup gg, const GateMem gm,
-                                             int32_t *__restrict__ sel_idx, float *__restrict__ sel_w)
+__device__ __forceinline__ void gating_part1(const Shape &sh, int B, const double *__restrict__ s_l,
+                                             const double *__restrict__ s_w, const GateGroup gg, const GateMem gm, bool den_early,
+                                             bool star_done = false, bool want_topk = false)
 {
     const int tid = gg.t, nt = gg.n, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
     const int E = sh.E, k = sh.k, cap = sh.cap;
     const bool bias_on = sh.alpha > 0.0 && cap < E && k < E;
 #pragma unroll 1
-    for (int e = tid; e < E; e += nt) { gm.star[e] = 0; gm.mask[e] = 0ull; }
+    for (int e = tid; e < E; e += nt) {
+        if (!star_done) gm.star[e] = 0;
+        gm.mask[e] = 0ull;
+    }
+    if (tid < 8 && !star_done) gm.star32[tid] = 0u;
     gate_sync(gg);
 
-    // E* (Eq. 4 aggregation, TopCap by rank) on cw warps, the per-token order statistics
-    // (lambda_b, softmax denominator) on the others.  With two or more warps to spare beside the
-    // first pass of tokens the two run side by side; else the first cw warps find E* first and
-    // then take tokens like everybody else.
+    // E* on cw warps (unless the caller has it already), the per-token order statistics (lambda_b,
+    // softmax denominator) on the others.  With two or more warps to spare beside the first pass
+    // of tokens the two run side by side; else the first cw warps find E* first and then take
+    // tokens like everybody else.
     const int spare = nw - (B < nw ? B : nw);
-    const bool side = spare >= 2;
-    const int cw = !bias_on ? 0 : (side ? (spare < nw / 2 ? spare : nw / 2) : (nw < 2 ? nw : 2));
+    const bool side = spare >= 2 && !star_done;
+    const int cw = (!bias_on || star_done) ? 0 : (side ? (spare < nw / 2 ? spare : nw / 2) : (nw < 2 ? nw : 2));
     const int c0 = side ? nw - cw : 0;                 // first of the cw warps
-    if (warp >= c0 && warp < c0 + cw) {
-        const int ct = tid - c0 * 32, cn = cw * 32;
-        // Eq. 4: g_e = sum_b w_b l_{b,e}, tokens in ascending order
-#pragma unroll 1
-        for (int e = ct; e < E; e += cn) {
-            double g = 0.0;
-#pragma unroll 1
-            for (int b = 0; b < B; ++b) g = fma(s_w[b], s_l[b * E + e], g);
-            gm.gk[e] = dkey(g);
-        }
-        asm volatile("bar.sync %0, %1;" ::"r"(gg.bar + 1), "r"(cn) : "memory");
-        // TopCap by rank in the order (g descending, id ascending)
-#pragma unroll 1
-        for (int e = ct; e < E; e += cn) {
-            const unsigned long long ge = gm.gk[e];
-            int rank = 0;
-#pragma unroll 4
-            for (int o = 0; o < E; ++o) {
-                const unsigned long long go = gm.gk[o];
-                rank += (go > ge) | ((go == ge) & (o < e));
-            }
-            gm.star[e] = rank < cap;
-        }
-    }
+    if (warp >= c0 && warp < c0 + cw) gating_estar(sh, B, s_l, s_w, gm, tid - c0 * 32, cw * 32, gg.bar + 1);
     if (!side || warp < c0) {
         const int tw = side ? c0 : nw;
 #pragma unroll 1
-        for (int b = warp; b < B; b += tw) gate_stats<J>(sh, b, bias_on, s_l, gm.lam, gm.zmax, gm.den, lane);
+        for (int b = warp; b < B; b += tw)
+            gate_stats<J>(sh, b, bias_on, s_l, gm.lam, gm.zmax, gm.den, (bias_on && want_topk) ? gm.topk : nullptr, den_early, lane);
     }
     gate_sync(gg);
+}
 
+template <int J>
+__device__ __forceinline__ void gating_part2(const Shape &sh, int B, const double *__restrict__ s_l, const GateGroup gg,
+                                             const GateMem gm, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
+                                             bool den_early)
+{
+    const int tid = gg.t, nt = gg.n, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
+    const int E = sh.E;
 #pragma unroll 1
     for (int b = warp; b < B; b += nw)
-        gate_select<J>(sh, b, s_l, gm.star, gm.lam, gm.zmax, gm.den, gm.sel, gm.pw, gm.mask, sel_idx, sel_w, lane);
+        gate_select<J>(sh, b, s_l, gm.star, gm.lam, gm.zmax, gm.den, gm.sel, gm.pw, gm.mask, sel_idx, sel_w, den_early, lane);
     gate_sync(gg);
 
     // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts

@@ -126,10 +126,12 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     __shared__ float s_pw[kMaxTokens * kMaxTopK];
     __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_pos[kMaxExperts];
     __shared__ int s_U;
+    __shared__ unsigned s_star32[8];
     __shared__ unsigned char s_star[kMaxExperts];
     GateMem gm;
     gm.mask = s_mask; gm.gk = s_gk; gm.lam = s_lam; gm.zmax = s_zmax; gm.den = s_den; gm.sel = s_sel; gm.pw = s_pw;
-    gm.cnt = s_cnt; gm.off = s_off; gm.pos = s_pos; gm.U = &s_U; gm.star = s_star;
+    gm.cnt = s_cnt; gm.off = s_off; gm.pos = s_pos; gm.U = &s_U; gm.star = s_star; gm.star32 = s_star32;
+    gm.topk = reinterpret_cast<unsigned *>(s_sel);      // (the selection overwrites it: nobody reads it here)
     const GateGroup gg{(int)threadIdx.x, (int)blockDim.x, 0};
     double *s_w = s_l + B * sh.E;
 #pragma unroll 1
@@ -137,7 +139,8 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
 #pragma unroll 1
     for (int b = gg.t; b < B; b += gg.n) s_w[b] = conf ? (double)conf[b] : 1.0;
     // (gating_group's first barrier orders these writes before the first read)
-    gating_group<JE>(sh, B, s_l, s_w, gg, gm, sel_idx, sel_w);
+    gating_part1<JE>(sh, B, s_l, s_w, gg, gm, true);
+    gating_part2<JE>(sh, B, s_l, gg, gm, sel_idx, sel_w, true);
     gating_writeout(sh, B, ws, gm, has_gate, n_unique, gg);
 }
 
@@ -240,6 +243,10 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     // and do its own set-up (both instructions do nothing in a plain launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // (block 0: where the arrival counter stood when the launch before had ended; see below)
+    unsigned ticket_base = 0u;
+    if (blockIdx.x == 0 && tid == 0)
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(ticket_base) : "l"(ws.ticket + 1) : "memory");
 #pragma unroll
     for (int z = 0; z < 3; ++z) {
         uint4 *p = reinterpret_cast<uint4 *>(zl.ptr[z]);
@@ -275,38 +282,31 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     }
     // Block 0 runs the gating once every row has arrived (its SM tends to be the same from layer
     // to layer, so part of the gating code is still in its instruction cache: measured 0.6 % of
-    // a layer against letting the last block to arrive do it).  Every block takes a ticket with
-    // release and acquire semantics by one thread.  The block that takes the last ticket puts the
-    // counter back to zero (nobody else touches it before the next launch) and publishes, in the
-    // word behind the counter, the token that block 0 wrote two words further in front of its own ticket;
-    // block 0 polls, bounded, for exactly that token.  So a wait that ran out leaves nothing
-    // behind: the late blocks still reset the counter, and what they publish afterwards is the
-    // token of a launch that is over, which no later launch waits for.  The barriers on both
-    // sides extend the ordering to the block's other threads; the other blocks wait for nothing.
+    // a layer against letting the last block to arrive do it).  Every block adds one arrival, with
+    // release and acquire semantics by one thread, to a counter that is never reset; block 0
+    // polls it, bounded, for the value it has when all blocks of THIS launch have arrived: the
+    // value it will end on was left in the word behind the counter by the launch before (launches of
+    // a context follow each other in stream order), and block 0 leaves the next one there, whether
+    // its wait succeeded or not, since the late blocks still arrive.  So a wait that ran out poisons
+    // nothing, and the waiting path is one atomic and one polled load, as short as it can be.  The
+    // barriers on both sides extend the ordering to the block's other threads; the other blocks
+    // wait for nothing.
     if (tid == 0) {
-        unsigned token = 0u;
+        unsigned target = 0u;
         if (blockIdx.x == 0) {
-            // differs from launch to launch (the SM's cycle counter; never 0)
-            token = (unsigned)clock() | 1u;
-            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 2), "r"(token) : "memory");
+            target = ticket_base + (unsigned)n_arrive;
+            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 1), "r"(target) : "memory");
         }
         unsigned t;
         asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(t) : "l"(ws.ticket) : "memory");
-        const bool last = t == (unsigned)n_arrive - 1;
-        if (last) {
-            unsigned tk;
-            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(tk) : "l"(ws.ticket + 2) : "memory");
-            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket), "r"(0u) : "memory");
-            if (blockIdx.x != 0)
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ws.ticket + 1), "r"(tk) : "memory");
-        }
-        int ok = (blockIdx.x == 0 && last) ? 1 : 0;
-        if (blockIdx.x == 0 && !last) {
-            for (unsigned i = 0; i < (1u << 22); ++i) {
+        int ok = 0;
+        if (blockIdx.x == 0) {
+            ok = (int)(t + 1u - target) >= 0 ? 1 : 0;
+            for (unsigned i = 0; i < (1u << 22) && !ok; ++i) {
                 unsigned v;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ws.ticket + 1) : "memory");
-                if (v == token) { ok = 1; break; }
-                __nanosleep(20);
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ws.ticket) : "memory");
+                if ((int)(v - target) >= 0) ok = 1;
+                else __nanosleep(20);
             }
             if (!ok) atomicExch(ws.status, ST_TICKET_TIMEOUT);
         }

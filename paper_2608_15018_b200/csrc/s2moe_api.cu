@@ -40,6 +40,7 @@ struct s2moe_ctx {
     cudaLaunchAttribute pdl_attr{};
     bool use_pdl = true;                  // S2MOE_NO_PDL=1 in the environment turns it off
     void *hperm = nullptr;                // int4 plan 3: column-permuted copy of the hidden states
+    double *lpart = nullptr;              // fused layer kernel: partial router logits [piece][token][row]
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
@@ -74,7 +75,7 @@ struct s2moe_cache {
     ExpertCache c;
 };
 
-enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_TC = 5, KC_COUNT = 6 };
+enum KernelClass { KC_ROUTER = 0, KC_GATING = 1, KC_GATEUP = 2, KC_DOWN = 3, KC_STREAM = 4, KC_TC = 5, KC_LAYER = 6, KC_COUNT = 7 };
 
 namespace {
 
@@ -133,9 +134,9 @@ int validate_config(const s2moe_config *c)
     if (c->weight_mode != 0 && c->weight_mode != 1) return S2MOE_EINVAL;
     if (c->max_tokens < 1 || c->max_tokens > S2MOE_MAX_TOKENS) return S2MOE_EINVAL;
     if (c->n_layers < 1) return S2MOE_EINVAL;
-    if (c->kernel_plan < 0 || c->kernel_plan > 3) return S2MOE_EINVAL;
+    if (c->kernel_plan < 0 || c->kernel_plan > 4) return S2MOE_EINVAL;
     // the tcgen05 plan covers bf16 activations with bf16 or block-int4 weights
-    if (c->kernel_plan == 3 && (c->weight_dtype == S2MOE_F32 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
+    if (c->kernel_plan >= 3 && (c->weight_dtype == S2MOE_F32 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     // the mma.sync plan covers bf16 weights with bf16 activations
     if (c->kernel_plan == 2 && (c->weight_dtype != S2MOE_BF16 || c->act_dtype != S2MOE_BF16)) return S2MOE_EINVAL;
     return S2MOE_OK;
@@ -397,6 +398,15 @@ int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
     const Shape &s0 = ctx->shape;
     const int want = ctx->cfg.kernel_plan;
     if (want == 1) return 1;
+    if (want == 4) {
+        // the whole layer in one launch, on demand only: measured slower than routing kernel + expert
+        // kernel on every workload here (the gating runs two to three times longer inside the busy
+        // CTAs than on a block of its own, and delays the first hand-over between the projections).
+        // An offloaded context meets the host between routing and the experts: two launches.
+        if (ctx->offload || ctx->tc_maps.empty()) return 0;
+        const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B, true);
+        return tp.feasible ? 4 : 0;
+    }
     if (want == 0 || want == 3) {
         const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
         if (tp.feasible && !ctx->tc_maps.empty()) return 3;
@@ -468,7 +478,7 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     ZeroList zl{};
     zl.ptr[0] = out;
     zl.n16[0] = (size_t)B * sh.d * sizeof(float) / 16;
-    if (plan == 3) {
+    if (plan == 3 || plan == 4) {
         const size_t used = (size_t)B * sh.k * sh.f + (size_t)sh.n_sh * B * sh.f_sh;
         zl.ptr[1] = ctx->pre;
         zl.n16[1] = used * 2 * sizeof(float) / 16;
@@ -480,13 +490,13 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
             zl.perm_n16 = (size_t)B * sh.d * 2 / 16;
         }
     }
-    launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
+    if (plan != 4) launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
     if (ctx->offload) {
         const int rc = fetch_experts(ctx, layer, st);
         if (rc != S2MOE_OK) return rc;
     }
-    if (plan == 3) {
-        const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
+    if (plan == 3 || plan == 4) {
+        const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B, plan == 4);
         TcMaps maps = ctx->tc_maps[layer];
         const size_t n_routed = (size_t)B * sh.k;
         const uint64_t plane = (uint64_t)((const uint8_t *)ctx->act_lo - (const uint8_t *)ctx->act_hi);
@@ -507,10 +517,27 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         TcArgs a;
         a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
         a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
-        LaunchScope scope(ctx, KC_TC, st);
+        a.rt = TcRoute{};
+        if (plan == 4) {
+            a.sh.plan = 3;
+            a.rt.hidden = hidden; a.rt.router = lp.router; a.rt.sh_scale = lp.sh_scale; a.rt.conf = conf;
+            a.rt.sel_idx = sel_idx; a.rt.sel_w = sel_w; a.rt.n_unique = n_unique;
+            a.rt.lpart = ctx->lpart;
+            a.rt.gbar = reinterpret_cast<unsigned long long *>(ctx->ws.ticket + 4);
+            a.rt.zl = zl;
+            // the expert of a token's largest logit stays in its top-k under any bias of alpha <= 1
+            const bool bias_on = sh.alpha > 0.0 && sh.cap < sh.E && sh.k < sh.E;
+            a.rt.early = (!bias_on || sh.alpha <= 1.0) ? 1 : 0;
+        }
+        LaunchScope scope(ctx, plan == 4 ? KC_LAYER : KC_TC, st);
         cudaLaunchConfig_t lc = pdl_config(ctx, tp.n_cta, tp.q4 ? kTcQ4Threads : kTcThreads, tp.smem_bytes, st);
-        if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true>, maps, a);
-        else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false>, maps, a);
+        if (plan == 4) {
+            if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true, true>, maps, a);
+            else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false, true>, maps, a);
+        } else {
+            if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true, false>, maps, a);
+            else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false, false>, maps, a);
+        }
     } else if (plan == 2) {
         StreamArgs a;
         a.sh = sh; a.lp = lp; a.ws = ctx->ws; a.plan = pl; a.hidden = hidden; a.y = out;
@@ -603,6 +630,7 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     const size_t o_tm = take(8 * (size_t)G);
     const size_t o_gtab = take(32 * (size_t)(G + 1));
     const size_t o_hperm = take(sh.weight_dtype == DT_Q4B32 ? 2 * (size_t)T * sh.d : 0);
+    const size_t o_lpart = take(sizeof(double) * 8 * (size_t)T * (E + 1));
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
     const size_t o_sto = take(4 * (size_t)L * T * sh.d), o_sts = take(4 * (size_t)L * T * sh.k);
     const size_t o_stw = take(4 * (size_t)L * T * sh.k), o_stn = take(4 * (size_t)L);
@@ -633,6 +661,7 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     ws.tokmask = (unsigned long long *)(base + o_tm);
     ws.gtab = (uint4 *)(base + o_gtab);
     ctx->hperm = base + o_hperm;
+    ctx->lpart = (double *)(base + o_lpart);
     ctx->pre = (float *)(base + o_pre);
     // plan 3: tensor maps of the weights (one set per layer); without the driver entry point or
     // for other formats the plan is simply not offered
@@ -645,8 +674,10 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
             ctx->encode_tiled = fn;
             ctx->tc_maps.resize(config->n_layers);
             const bool q4 = sh.weight_dtype == DT_Q4B32;
-            bool ok = cudaFuncSetAttribute(ffn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
-                      cudaFuncSetAttribute(ffn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
+            bool ok = cudaFuncSetAttribute(ffn_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(ffn_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(ffn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(ffn_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
             // the int4 variant needs contraction lengths that are multiples of 256 (see tc_make_plan)
             if (q4 && (sh.d % 256 || sh.f % 256 || (sh.n_sh && sh.f_sh % 256))) ok = false;
             for (int l = 0; l < config->n_layers && ok; ++l) {
@@ -1043,6 +1074,7 @@ const char *s2moe_kernel_class_name(int32_t cls)
         case KC_DOWN: return "ffn_down_simple";
         case KC_STREAM: return "ffn_stream_kernel";
         case KC_TC: return "ffn_tc_kernel";
+        case KC_LAYER: return "ffn_tc_kernel/fused";
         default: return nullptr;
     }
 }

@@ -9,16 +9,17 @@ TOL = {workloads.F32: 2e-3, workloads.BF16: 2e-3, workloads.Q4B32: 1e-2}
 
 
 def supports(wl, plan):
-    """Kernel plan 2 (mma.sync) covers bf16 weights with bf16 activations; plan 3 (tcgen05) also
-    block-int4 weights whose contraction lengths are multiples of 256."""
-    if plan not in (2, 3):
+    """Kernel plan 2 (mma.sync) covers bf16 weights with bf16 activations; plans 3 and 4 (tcgen05;
+    4 is the whole layer in one launch) also block-int4 weights whose contraction lengths are
+    multiples of 256."""
+    if plan not in (2, 3, 4):
         return True
     if wl.act_dtype != workloads.BF16:
         return False
     if wl.weight_dtype == workloads.BF16:
         return True
     q4_ok = wl.d_model % 256 == 0 and wl.d_ff % 256 == 0 and (wl.n_shared == 0 or wl.d_ff_shared % 256 == 0)
-    return plan == 3 and wl.weight_dtype == workloads.Q4B32 and q4_ok
+    return plan in (3, 4) and wl.weight_dtype == workloads.Q4B32 and q4_ok
 
 
 def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_list=None,
@@ -38,10 +39,10 @@ def run_case(wl, layer=0, n_tokens=None, sigma=None, use_conf=True, plan=0, tok_
     cfg = binding.Config.from_workload(wl, n_layers=1, kernel_plan=plan)
     with binding.S2MoE(cfg, [T]) as m:
         used = m.kernel_plan(H.shape[0])
-        if plan in (2, 3) and used != plan:
+        if plan in (2, 3, 4) and used != plan:
             assert optional, f"kernel plan {plan} was demanded, the library chose {used}"
             return None, None
-        assert used in (1, 2, 3) and (plan == 0 or used == plan)
+        assert used in (1, 2, 3, 4) and (plan == 0 or used == plan)
         o = m.verify_layer(0, H, conf)
         torch.cuda.synchronize()
         status = m.device_status()

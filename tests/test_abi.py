@@ -43,7 +43,7 @@ def test_create_rejects_bad_configs_before_touching_the_device():
            dict(top_k=9), dict(cap=1), dict(cap=9), dict(alpha=-1.0), dict(max_tokens=65),
            dict(max_tokens=0), dict(n_layers=0), dict(weight_dtype=3), dict(act_dtype=2),
            dict(router_dtype=2), dict(renorm=2), dict(weight_mode=2), dict(n_shared=5),
-           dict(n_shared=1, d_ff_shared=40), dict(kernel_plan=4), dict(top_k=17, n_experts=32, cap=20)]
+           dict(n_shared=1, d_ff_shared=40), dict(kernel_plan=5), dict(top_k=17, n_experts=32, cap=20)]
     w = (binding.LayerWeightsC * 1)()
     for change in bad:
         cfg = binding.Config(**{**good, **change}).c()

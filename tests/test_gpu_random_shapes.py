@@ -1,4 +1,4 @@
-"""Seeded random shapes through the tcgen05 kernel (bf16 and block-int4 weights) against the
+"""Seeded random shapes through the tcgen05 kernels (two launches per layer, and the fused one) (bf16 and block-int4 weights) against the
 oracle: expert counts from 1 to 256, ragged widths, shared experts with and without the sigmoid
 gate, every batch size class, all gating variants."""
 import random
@@ -27,14 +27,15 @@ def _case(rng, trial):
     return wl, rng.choice([1, 2, 3, 7, 8, 9, 16, 31, 33, 64]), rng.random() < 0.7
 
 
+@pytest.mark.parametrize("plan", [3, 4])
 @pytest.mark.parametrize("seed", [11, 12])
-def test_random_shapes_on_the_tensor_core_plan(seed):
+def test_random_shapes_on_the_tensor_core_plan(seed, plan):
     rng = random.Random(seed)
     ran = 0
     for trial in range(25):
         wl, B, use_conf = _case(rng, trial)
-        rep, _ = run_case(wl, n_tokens=B, plan=3, use_conf=use_conf, optional=True)
+        rep, _ = run_case(wl, n_tokens=B, plan=plan, use_conf=use_conf, optional=True)
         if rep is not None:
-            assert rep.plan == 3 and rep.tokens_checked == B
+            assert rep.plan == plan and rep.tokens_checked == B
             ran += 1
     assert ran >= 20
