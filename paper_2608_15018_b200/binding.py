@@ -30,7 +30,7 @@ EXPORTS = ("s2moe_create", "s2moe_verify_layer", "s2moe_verify_stack", "s2moe_ve
            "s2moe_cache_destroy")
 OFFLOADED_FIELDS = ("w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down")   # host tensors of an offloaded context
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_EXPERTS = 64, 128
-KERNEL_CLASSES = 6
+KERNEL_CLASSES = 7
 
 
 class LayerWeightsC(ctypes.Structure):

@@ -42,15 +42,34 @@ def fit_line(u: np.ndarray, t: np.ndarray):
     return float(t0), float(t_exp), r2, mape
 
 
-def measure(wl, n_layers: int, batches, sigmas, repeats: int = 3):
-    """Per-layer (B, sigma, layer, U, microseconds): median over `repeats` timed passes."""
+class _Borrowed:
+    """A context that the caller owns, used where ``with`` expects one."""
+
+    def __init__(self, m):
+        self.m = m
+
+    def __enter__(self):
+        return self.m
+
+    def __exit__(self, *exc):
+        return False
+
+
+def measure(wl, n_layers: int, batches, sigmas, repeats: int = 3, model=None):
+    """Per-layer (B, sigma, layer, U, microseconds): median over `repeats` timed passes.  ``model``:
+    a context for ``wl`` with ``n_layers`` layers that the caller has built already (its weights stay
+    where they are), else one is built here."""
     dev = torch.device("cuda", torch.cuda.current_device())
     wl = wl.with_(n_layers=n_layers)
-    weights = [workloads.layer_weights(wl, l, dev) for l in range(n_layers)]
-    cfg = binding.Config.from_workload(wl, n_layers=n_layers)
     stream = torch.cuda.Stream()
     rows = []
-    with binding.S2MoE(cfg, weights) as m, torch.cuda.stream(stream):
+    if model is None:
+        weights = [workloads.layer_weights(wl, l, dev) for l in range(n_layers)]
+        cfg = binding.Config.from_workload(wl, n_layers=n_layers)
+        holder = binding.S2MoE(cfg, weights)
+    else:
+        holder = _Borrowed(model)
+    with holder as m, torch.cuda.stream(stream):
         for B in batches:
             for sigma in sigmas:
                 H = [workloads.hidden_states(wl, l, B, sigma, dev) for l in range(n_layers)]

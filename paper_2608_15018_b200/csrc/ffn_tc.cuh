@@ -38,8 +38,6 @@
 
 #include "common.cuh"
 #include "ffn_stream.cuh"
-#include "gating.cuh"
-#include "route.cuh"
 
 namespace s2moe {
 
@@ -92,7 +90,6 @@ struct TcPlan {
     int stage_bytes;   // weight tile + token tiles, multiple of 1024
     int n1;            // tokens padded to 16 (phase-1 N)
     int tmem_cols;     // power of two >= 32
-    int n_acc;         // accumulator buffers in tensor memory (runs the MMA issuers may be ahead of the epilogue)
     int n_iss;         // MMA issuer warps (2, or 4 on the int4 path when the accumulators fit)
     int tab_bytes;
     int x_bytes;       // > 0: the hidden states stay resident in shared memory (all k-tiles)
@@ -102,22 +99,6 @@ struct TcPlan {
     int tok_off;       // offset of the token tiles inside a stage
     int kg;            // k-tiles per stage (1 for bf16 weights; 1, 2 or 4 for int4)
     int tokb;          // bytes of the token tiles of one k-tile
-    int fused;         // the kernel also routes and gates (one launch per layer)
-    int gate_bytes;    // fused: shared memory of the gating (staged logits and its tables)
-    int ksplit;        // fused: pieces of the contraction a router row is cut into
-};
-
-// what the fused layer kernel needs for its routing stage (unused by the two-launch form)
-struct TcRoute {
-    const void *hidden, *router, *sh_scale;     // [B][d] bf16, [E][d] router dtype, [d] or NULL
-    const float *conf;                          // [B] or NULL
-    int32_t *sel_idx;                           // outputs of the layer call
-    float *sel_w;
-    int32_t *n_unique;
-    double *lpart;                              // [ksplit][B][E (+1)] partial router logits
-    unsigned long long *gbar;                   // arrivals of all launches so far (never reset)
-    ZeroList zl;                                // what the kernel clears / copies before anything accumulates
-    int early;                                  // the experts of the tokens' largest logits may start before the gating
 };
 
 struct TcArgs {
@@ -125,38 +106,22 @@ struct TcArgs {
     Workspace ws;
     TcPlan plan;
     float *y;
-    float *pre;                       // [gate|up][slot][f_g] fp32 pre-activations (zeroed by the routing stage)
+    float *pre;                       // [gate|up][slot][f_g] fp32 pre-activations (zeroed by the routing kernel)
     __nv_bfloat16 *act_hi, *act_lo;   // [slot][f_g]
     int B;
-    TcRoute rt;
 };
 
-// warps of the fused kernel that run the gating while the layer starts: the four epilogue warps,
-// the three converter warps and the watcher (they have nothing to do before the first accumulator
-// is complete); their hardware barriers
-constexpr int kTcGateWarps = 8, kTcGateBar = 2;
-
-inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, bool fused = false)
+inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
 {
     TcPlan p{};
     const int G = sh.E + sh.n_sh;
     p.n_cta = n_sm;
     p.n1 = (B + 15) & ~15;
-    p.fused = fused ? 1 : 0;
-    if (fused) {
-        p.gate_bytes = (int)((8 * ((size_t)B * sh.E + 2 * (size_t)B) + gate_mem_bytes(sh.E, B, sh.k) + 64 + 15) & ~(size_t)15);   // logits, confidences, gate logits, tables
-        // a router row is cut into pieces so that the warps of all CTAs share the logit pass
-        const int rows = sh.E + 1, tgs = (B + 7) / 8, warps = n_sm * 11;
-        int ks = warps / (rows * tgs);
-        if (ks > 8) ks = 8;
-        if (ks > sh.d / 128) ks = sh.d / 128;
-        p.ksplit = ks < 1 ? 1 : ks;
-    }
     // token area of a stage: phase 1 = n1 rows of 128 bytes; phase 2 = per 8 slots their hi rows
     // (1 KiB) and right behind them their lo rows (a group never has more tokens than B)
     p.stage_bytes = kTcWTile + 2048 * ((B + 7) / 8);
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
-    p.tab_bytes = ((int)sizeof(TcGroup) * (G + 1) + 8 * n_slots + 4 * (G + 2) + p.gate_bytes + 1023) & ~1023;
+    p.tab_bytes = ((int)sizeof(TcGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
     // The ring is what keeps HBM busy (bytes in flight = stages x 16 KiB per SM, against a loaded
     // latency of 2-3 us), so shared memory goes to stages first: the hidden-state tiles stay
     // resident only if the ring reaches its maximum depth anyway, otherwise every stage fetches
@@ -166,17 +131,8 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, bool f
     p.stages = (kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes;
     if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
     p.n_iss = 2;
-    // accumulators: buffers x 2 issuers x up to 2 * n1 columns.  Two buffers keep the issuers busy while
-    // the epilogue drains; the fused kernel takes as many as tensor memory holds (up to 8), because
-    // there the accumulators of the early groups cannot be drained before the gating has finished
-    p.n_acc = 2;
-    if (fused) {
-        p.n_acc = 512 / (4 * p.n1);
-        if (p.n_acc > 8) p.n_acc = 8;
-        if (p.n_acc < 2) p.n_acc = 2;
-    }
     p.tmem_cols = 32;
-    while (p.tmem_cols < p.n_acc * 4 * p.n1) p.tmem_cols <<= 1;
+    while (p.tmem_cols < 8 * p.n1) p.tmem_cols <<= 1;   // 2 buffers x 2 issuers x up to 2 * n1 columns
     p.smem_bytes = p.tab_bytes + p.x_bytes + p.stages * p.stage_bytes + 1024;   // + slack to align to 1024
     p.tok_off = kTcWTile;
     p.kg = 1;
@@ -197,7 +153,6 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, bool f
         // a stage that is cheap to fetch, so as many issuers as the accumulators leave room for.
         p.n_iss = 16 * p.n1 <= kTcQ4ACol ? 4 : (8 * p.n1 <= kTcQ4ACol ? 2 : 1);
         p.tmem_cols = 512;
-        p.n_acc = 2;
         // The token tiles of a stage do not travel with its packed tiles: they are fetched into a
         // slot that belongs to the ring of dequantised tiles, just before they are used, so that a
         // stage is free again as soon as the dequantising warps have read it (its life decides
@@ -408,57 +363,12 @@ __device__ __forceinline__ void tc_ring_next(int &s, uint32_t &parity, int S)
     if (++s == S) { s = 0; parity ^= 1u; }
 }
 
-// ---- routing stage of the fused kernel ------------------------------------------------------
-
-// Router logits by the warps of the whole grid: a task is one router row (row E: the shared
-// experts' gate vector) x 8 tokens x one piece of the contraction, float64 accumulation; its
-// partial sums go to lpart[piece][token][row], which the gating adds up in a fixed order.
-template <int RT>
-__device__ __forceinline__ void tc_logit_tasks(const Shape &sh, int B, const TcRoute &rt, int ksplit, int gwarp, int n_gwarps,
-                                               int lane)
-{
-    const int d = sh.d, n_rows = sh.E + (rt.sh_scale ? 1 : 0), n_tg = (B + 7) >> 3;
-    const int len = ((d + 4 * ksplit - 1) / (4 * ksplit)) * 4;              // columns of a piece, a multiple of 4
-    const int n_tasks = n_rows * n_tg * ksplit;
-    const size_t rb = RT == DT_F32 ? 4 : 2;
-#pragma unroll 1
-    for (int task = gwarp; task < n_tasks; task += n_gwarps) {
-        const int row = task % n_rows, rest = task / n_rows, tg = rest % n_tg, piece = rest / n_tg;
-        const int c0 = piece * len, c1 = min(d, c0 + len), b0 = tg * 8;
-        const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(rt.router) + (size_t)row * d * rb
-                                         : reinterpret_cast<const uint8_t *>(rt.sh_scale);
-        double acc[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) acc[t] = 0.0;
-#pragma unroll 2
-        for (int c = c0 + lane * 4; c < c1; c += 128) {
-            float w[4], x[8][4];
-            load4_plain<RT>(wrow, c, w);
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const int bt = min(b0 + t, B - 1);           // past the batch: the last token again (not stored)
-                load4_plain<DT_BF16>(reinterpret_cast<const uint8_t *>(rt.hidden) + (size_t)bt * d * 2, c, x[t]);
-            }
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[t][i], acc[t]);
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const double v = warp_sum(acc[t]);
-            if (lane == t && b0 + t < B) rt.lpart[((size_t)piece * B + b0 + t) * n_rows + row] = v;
-        }
-    }
-}
-
 struct TcUnit {                        // plain ints: the single-thread roles read these on their critical path
     int phase, a, mat, rb, kt0, kt1;   // group slot, matrix (0 gate, 1 up, 2 down), row block, k-tile range
     int n;                             // MMA N: phase 1 tokens padded to 16; phase 2 16 per 8 slots (hi | lo)
+    int seg;                           // 0 / 1: phase 1 of wave 0 / 1, 2 / 3: phase 2 of wave 0 / 1
     int first, last;                   // first / last unit of an accumulation run (see the kernel)
-    int wave;                          // 0 / 1: the group belongs to the first / second wave
 };
-static_assert(sizeof(TcUnit) == 40, "layout");
 
 __device__ __forceinline__ TcUnit tc_decode(const TcGroup *groups, int n_active, int total1, int u, int d, int n1)
 {
@@ -509,140 +419,102 @@ struct TcMaps {
     CUtensorMap m[27];
 };
 
-// The share of one CTA in the eight segments of a layer (see the kernel): per segment the first
-// unit, the number of units and the half-unit trim bits.
-constexpr int kTcSegs = 8;
-struct TcShare {
-    int start[kTcSegs], cnt[kTcSegs], trim[kTcSegs];
-};
-
-// Every CTA takes one contiguous run of units of each segment (sizes differ by at most one; the
-// CTAs that get the extra unit rotate from segment to segment, so the totals differ by at most
-// one as well).  Where every unit of a projection has all its four k-tiles (contraction length a
-// multiple of 256) the segments are dealt in half units, so that the CTAs of a segment differ by
-// two k-tiles (0.75 us) instead of four: a share may then begin with the second half of a unit and
-// end with the first half of one (trim bits 1 and 2).  Measured at the OLMoE shape: 0.7 % of a
-// layer; dealing single k-tiles cuts more accumulation runs in two and gives it back.
-// bound[0..6]: the segments' boundaries in the numbering of tc_decode.
-__device__ __forceinline__ void tc_shares(const int (&bound)[kTcSegs + 1], bool halves1, bool halves2, int P, int cta, TcShare &out)
-{
-    int rot = 0;
-#pragma unroll
-    for (int sg = 0; sg < kTcSegs; ++sg) {
-        const bool halves = sg < 6 ? halves1 : halves2;
-        const int begin = bound[sg], n = bound[sg + 1] - bound[sg];
-        if (n <= 0) { out.cnt[sg] = 0; out.start[sg] = begin; out.trim[sg] = 0; continue; }
-        const int m = halves ? 2 : 1, n2 = n * m;
-        const int q = n2 / P, r = n2 - q * P;
-        int c = cta - rot;                             // (cta - rot) mod P without a division
-        if (c < 0) c += P;
-        const int cnt2 = q + (c < r ? 1 : 0), start2 = c * q + min(c, r);
-        const int u0 = halves ? start2 >> 1 : start2, u1 = halves ? (start2 + cnt2 - 1) >> 1 : start2 + cnt2 - 1;
-        out.cnt[sg] = cnt2 > 0 ? u1 - u0 + 1 : 0;
-        out.start[sg] = begin + u0;
-        out.trim[sg] = (halves && cnt2 > 0) ? ((start2 & 1) | (((start2 + cnt2) & 1) << 1)) : 0;
-        rot += r;
-        if (rot >= P) rot -= P;
-    }
-}
-
-// unit i of a CTA's sequence (segments in order)
-__device__ __forceinline__ TcUnit tc_unit_make(const TcShare &shr, const TcGroup *groups, int n_groups, int total1, int a_split,
-                                               int i, int d, int n1)
-{
-    // (static indices only: the shares stay in registers)
-    int seg = 0, j = i, start = shr.start[0], cnt = shr.cnt[0], trim = shr.trim[0];
-#pragma unroll
-    for (int sg = 1; sg < kTcSegs; ++sg)
-        if (seg == sg - 1 && j >= cnt) { j -= cnt; seg = sg; start = shr.start[sg]; cnt = shr.cnt[sg]; trim = shr.trim[sg]; }
-    TcUnit t = tc_decode(groups, n_groups, total1, start + j, d, n1);
-    const int K = t.phase == 1 ? d : groups[t.a].f;
-    if (j == 0 && (trim & 1)) t.kt0 += kTcKT / 2;            // the CTA before this one has the first half
-    if (j == cnt - 1 && (trim & 2)) t.kt1 -= kTcKT / 2;      // the next CTA has the second half
-    t.wave = t.a >= a_split ? 1 : 0;
-    t.first = (j == 0 || t.kt0 == 0) ? 1 : 0;
-    t.last = (j == cnt - 1 || t.kt1 == (K + 63) / 64) ? 1 : 0;
-    return t;
-}
-
-// FUSED: the kernel is the whole layer.  Its CTAs first clear what the layer accumulates into and
-// share the router's logit pass, meet once (a bounded grid-wide wait; one CTA per SM, all
-// resident), and then eight warps of every CTA run the gating for themselves, all on the same
-// numbers, while the producer and the MMA issuers already stream what needs no routing decision:
-// the shared experts, and the expert of every token's largest logit, which no bias of alpha <= 1
-// can push out of that token's top-k.  CTA 0 writes the layer's routing outputs.
-template <bool Q4, bool FUSED>
+template <bool Q4>
 __global__ void __launch_bounds__(Q4 ? kTcQ4Threads : kTcThreads, 1)
 ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[8], acc_empty[8], ep_bar, x_bar, cv_bar, conv_go[2];
+    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
     __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
     __shared__ uint32_t s_tmem;
-    __shared__ int s_flag, s_go;
+    __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
     __shared__ uint32_t s_umeta[kTcMaxUnits];      // what an MMA issuer needs of a unit, in one word (tc_unit_meta)
+    __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
     __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
-    // the unit tables come in three stages in the fused kernel: s_tab = 1 when this CTA's units of the
-    // first lot of early groups are decoded (s_nunits[0] units), 2 with the second lot (s_nunits[1]),
-    // 3 when everything is (s_nunits[2]); the two-launch form starts at 3
-    __shared__ volatile int s_tab;
-    __shared__ int s_nunits[3];
-    __shared__ TcShare s_share;
-    __shared__ int s_nact, s_split, s_total1;      // active groups, first group of wave 1 (s_nact: one wave), phase-1 units
-    __shared__ unsigned s_lot[3][8];               // fused: experts of the first and second early lot, all selected experts (bit words)
 
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
     const TcPlan &pl = p.plan;
     const int NI = Q4 ? p.plan.n_iss : 2;          // MMA issuers: a compile-time 2 on the bf16 path
-    const int NACC = FUSED ? p.plan.n_acc : 2;     // accumulator buffers: a compile-time 2 in the two-launch form
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // programmatic dependent launch: whatever is in front of this grid in the stream (the routing
-    // kernel of the two-launch form, the previous layer) must have finished before its results
-    // are read or this layer's buffers are cleared; the next kernel may be scheduled
+    // programmatic dependent launch: the routing kernel in front of this grid must have
+    // finished before its results are read; the next layer's routing kernel may be scheduled
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int n_active = ws.header[0];
     const int n_slots = p.B * sh.k + sh.n_sh * p.B;          // every token fills k routed slots
     const int G = sh.E + sh.n_sh;
-    const int S = pl.stages;
-    const int P = gridDim.x;
 
     TcGroup *groups = reinterpret_cast<TcGroup *>(tc_smem);
-    int *s_epfx = reinterpret_cast<int *>(tc_smem + sizeof(TcGroup) * (G + 1));     // [n_active + 1] activation elements in front of a group, in group order
-    int *s_slot_token = s_epfx + (G + 2);
-    float *s_slot_w = reinterpret_cast<float *>(s_slot_token + n_slots);
-    uint8_t *gate_area = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(s_slot_w + n_slots) + 15) & ~(uintptr_t)15);
+    const int tab_rest = pl.tab_bytes - (int)sizeof(TcGroup) * (G + 1);
+    int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(TcGroup) * (G + 1));
+    float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
     uint8_t *xres = tc_smem + pl.tab_bytes;
     xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
     uint8_t *ring = xres + pl.x_bytes;
     uint8_t *tokring = ring + (size_t)pl.stages * pl.stage_bytes;    // int4 only: token tiles, one slot per slot of dequantised tiles
 
+    // group table; stage prefixes follow from the active list alone (routed groups first)
+    const int U = ws.header[2];
     const int u1r = tc_units1(sh.f, sh.d), u2r = tc_units2(sh.f, sh.d);
     const int u1s = sh.n_sh ? tc_units1(sh.f_sh, sh.d) : 0, u2s = sh.n_sh ? tc_units2(sh.f_sh, sh.d) : 0;
-    // segments are dealt in half units where every unit has all its k-tiles; the int4 path needs whole units
-    const bool halves1 = !Q4 && sh.d % 256 == 0;
-    const bool halves2 = !Q4 && sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
-
+    // one round of global loads: the header above, the group table in its final form and the
+    // slot arrays, whose sizes are known without the header
+    for (int a = tid; a < G; a += blockDim.x) {
+        const uint4 r0 = ws.gtab[2 * a], r1 = ws.gtab[2 * a + 1];
+        if (a < n_active) {
+            TcGroup gr;
+            gr.group = (int)r0.x;
+            // offloaded experts: from here on the group id of a routed expert is the device slot its
+            // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
+            if (ws.slot_of && gr.group < sh.E) gr.group = __ldg(&ws.slot_of[gr.group]);
+            gr.T = (int)r0.y;
+            gr.off = (int)r0.z;
+            gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
+            gr.mask = (unsigned long long)r1.x | ((unsigned long long)r1.y << 32);
+            const int r = a < U ? a : U, s = a < U ? 0 : a - U;
+            gr.p1 = r * u1r + s * u1s;
+            gr.p2 = r * u2r + s * u2s;
+            groups[a] = gr;
+        }
+    }
+    for (int i = tid; i < n_slots; i += blockDim.x) {
+        s_slot_token[i] = ws.slot_token[i];
+        s_slot_w[i] = ws.slot_w[i];
+    }
+    const int total1 = U * u1r + sh.n_sh * u1s, total2 = U * u2r + sh.n_sh * u2s;
+    const int total = total1 + total2;
+    const int S = pl.stages;
+    const int P = gridDim.x;
     if (tid == 0) {
+        // wave 1 starts at the first group whose phase-1 units begin at or after that share
+        int sp = n_active;
+        if (n_active >= 2) {
+            sp = 1;
+            while (sp < n_active - 1) {
+                const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
+                if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)total1 * kTcSplitNum) break;
+                ++sp;
+            }
+        }
+        s_split = sp;
         s_ready[0] = 0;
         s_ready[1] = 0;
-        if (FUSED) s_tab = 0;
-        s_go = 1;
     }
     if (warp == 2) {
-        // barrier set-up, spread over a warp so that it runs beside the work of the others
+        // barrier set-up, spread over a warp so that it runs beside the table loads of the others
         if (lane < pl.stages) {
             mbar_init(&full_bar[lane], 1);
             mbar_init(&empty_bar[lane], Q4 ? kTcQ4DeqWarps : NI);   // one commit from each MMA issuer; int4: the dequantising warps
         }
-        if (lane < pl.n_acc) {
+        if (lane < 2) {
             mbar_init(&acc_full[lane], NI);
             mbar_init(&acc_empty[lane], 4);
+            mbar_init(&conv_go[lane], 4);
         }
-        if (lane < 2) mbar_init(&conv_go[lane], 4);
         if (Q4 && lane < pl.a_stages) {
             mbar_init(&a_full[lane], kTcQ4DeqWarps + 1);   // the dequantising warps and the producer's arrival with the token bytes
             mbar_init(&a_empty[lane], NI);
@@ -661,456 +533,78 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-
-    if constexpr (!FUSED) {
-        // the routing kernel has left the group table in its final form (routed groups in ascending
-        // order, the shared experts behind them) and the slot arrays, whose sizes are known
-        // without the header: one round of global loads
-        // the loads are issued first (each thread's first table entry and slot), what follows from the
-        // header alone is worked out while they are in flight
-        uint4 g0 = make_uint4(0u, 0u, 0u, 0u), g1 = g0;
-        if (tid < G) { g0 = ws.gtab[2 * tid]; g1 = ws.gtab[2 * tid + 1]; }
-        int st0 = 0;
-        float sw0 = 0.f;
-        if (tid < n_slots) { st0 = ws.slot_token[tid]; sw0 = ws.slot_w[tid]; }
-        const int n_active = ws.header[0], U = ws.header[2];
-        const int total1 = U * u1r + sh.n_sh * u1s, total2 = U * u2r + sh.n_sh * u2s;
-        // every thread works out the wave boundary and the CTA's shares for itself, so that nothing
-        // but the group table has to cross the barrier below: wave 1 starts at the first group whose
-        // phase-1 units begin at or after the wave share
-        int sp = n_active;
-        if (n_active >= 2) {
-            sp = 1;
-            while (sp < n_active - 1) {
-                const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
-                if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)total1 * kTcSplitNum) break;
-                ++sp;
-            }
-        }
-        TcShare shr;
-        int n_all = 0;
-        {
-            const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
-            const int split1 = sp < n_active ? r * u1r + q * u1s : total1, split2 = sp < n_active ? r * u2r + q * u2s : total2;
-            const int bound[kTcSegs + 1] = {0, 0, 0, 0, 0, split1, total1, total1 + split2, total1 + total2};    // no early segments
-            tc_shares(bound, halves1, halves2, P, (int)blockIdx.x, shr);
-            for (int sg = 0; sg < kTcSegs; ++sg) n_all += shr.cnt[sg];
-        }
-        for (int a = tid; a < G; a += blockDim.x) {
-            const uint4 r0 = a == tid ? g0 : ws.gtab[2 * a], r1 = a == tid ? g1 : ws.gtab[2 * a + 1];
-            if (a < n_active) {
-                TcGroup gr;
-                gr.group = (int)r0.x;
-                // offloaded experts: from here on the group id of a routed expert is the device slot its
-                // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
-                if (ws.slot_of && gr.group < sh.E) gr.group = __ldg(&ws.slot_of[gr.group]);
-                gr.T = (int)r0.y;
-                gr.off = (int)r0.z;
-                gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
-                gr.mask = (unsigned long long)r1.x | ((unsigned long long)r1.y << 32);
-                const int r = a < U ? a : U, q = a < U ? 0 : a - U;
-                gr.p1 = r * u1r + q * u1s;
-                gr.p2 = r * u2r + q * u2s;
-                groups[a] = gr;
-                // groups in slot order: the elements in front of a group are those of its first slot
-                s_epfx[a] = (int)act_offset(gr.off, p.B * sh.k, sh.f, sh.f_sh);
-            }
-        }
-        for (int i = tid; i < n_slots; i += blockDim.x) {
-            s_slot_token[i] = i == tid ? st0 : ws.slot_token[i];
-            s_slot_w[i] = i == tid ? sw0 : ws.slot_w[i];
-        }
-        if (tid == 0) {
-            s_split = sp;
-            s_nact = n_active;
-            s_total1 = total1;
-            s_epfx[n_active] = (int)((size_t)p.B * sh.k * sh.f + (size_t)sh.n_sh * p.B * sh.f_sh);
-            s_share = shr;
-            s_nunits[0] = 0;
-            s_nunits[1] = 0;
-            s_nunits[2] = n_all;
-            s_tab = 3;
-        }
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        // decoded once by all threads: the single-thread roles below then read a unit from shared
-        // memory instead of dividing
-        for (int i = tid; i < n_all && i < kTcMaxUnits; i += blockDim.x) {
-            const TcUnit t = tc_unit_make(shr, groups, n_active, total1, sp, i, sh.d, pl.n1);
-            s_units[i] = t;
-            s_umeta[i] = tc_unit_meta(t);
-        }
-        __syncthreads();
-    } else {
-        const TcRoute &rt = p.rt;
-        // ---- clear what the layer accumulates into (and, int4, leave the binary16 column-permuted
-        // copy of the hidden states): every CTA its share, all of it before the grid-wide meeting
-        {
-            const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + tid, gn = (unsigned long long)P * blockDim.x;
-#pragma unroll
-            for (int z = 0; z < 3; ++z) {
-                uint4 *q = reinterpret_cast<uint4 *>(rt.zl.ptr[z]);
-                for (unsigned long long i = gt; i < rt.zl.n16[z]; i += gn) q[i] = make_uint4(0u, 0u, 0u, 0u);
-            }
-            for (unsigned long long i = gt; i < rt.zl.perm_n16; i += gn) {
-                const uint4 v = rt.zl.perm_src[i];             // halves h0..h7 (bf16)
-                rt.zl.perm_dst[i] = make_uint4(bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x7632)),
-                                               bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x7632)));
-            }
-            if (Q4) asm volatile("fence.proxy.async.global;" ::: "memory");   // the copy is read by TMA copies of all CTAs
-        }
-        // ---- the logit pass, shared by the warps of all CTAs
-        {
-            const int nwarps = (int)blockDim.x >> 5;
-            if (sh.router_dtype == DT_F32) tc_logit_tasks<DT_F32>(sh, p.B, rt, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
-            else tc_logit_tasks<DT_BF16>(sh, p.B, rt, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
-        }
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        // ---- the meeting: every CTA adds one arrival to a counter that is never reset (all launches
-        // of a context have the same grid, so a launch ends on a multiple of the grid size) and
-        // waits, bounded, for that multiple.  A wait that gave up leaves nothing behind: the others
-        // still arrive.  The barriers on both sides extend the ordering to the block's threads.
-        if (tid == 0) {
-            unsigned long long t;
-            asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], 1;" : "=l"(t) : "l"(rt.gbar) : "memory");
-            const unsigned long long target = (t / (unsigned long long)P + 1ull) * (unsigned long long)P;
-            int ok = t + 1ull == target ? 1 : 0;
-            for (unsigned i = 0; i < kTcSpinLimit && !ok; ++i) {
-                unsigned long long v;
-                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(rt.gbar) : "memory");
-                if (v >= target) ok = 1;
-                else __nanosleep(32);
-            }
-            if (!ok) atomicExch(ws.status, ST_TICKET_TIMEOUT);
-            s_go = ok;
-        }
-        __syncthreads();
-    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
     const uint32_t tmem_base = s_tmem;
-    const bool go = s_go != 0;
-
-    // Eight segments in time order.  Phase 1 comes in up to three lots as the routing becomes known
-    // (fused kernel only: first the shared experts and the expert of every token's largest logit,
-    // then the experts that are in E* and among some token's first k, then the rest; the two-launch
-    // form has the last lot only), and every lot is cut in two at the group that brings it to the
-    // wave share, so that wherever the boundary between wave 0 and wave 1 finally falls it is a
-    // boundary between segments; then phase 2 of wave 0 and of wave 1.  Every segment is dealt over
-    // all CTAs.  Contiguous units are consecutive k-pieces of one 128-row block, so a CTA
+    const int a_split = s_split;
+    const int W = a_split < n_active ? 2 : 1;
+    // Four segments in time order: phase 1 of wave 0, of wave 1, phase 2 of wave 0, of wave 1.
+    // Every CTA takes one contiguous run of units of each segment (sizes differ by at most one;
+    // the CTAs that get the extra unit rotate from segment to segment, so the totals differ by at
+    // most one as well).  Contiguous units are consecutive k-pieces of one 128-row block, so a CTA
     // accumulates them in one TMEM accumulator and the epilogue runs once per run of k-pieces
     // instead of once per unit; only row blocks cut by a CTA boundary are reduced from two CTAs.
-    const bool gate_warp = (warp >= 2 && warp <= 5) || (warp >= 7 && warp <= 10);
-    // first phase-1 / phase-2 unit of the group at position a of the fused kernel's group order
-    // (the shared experts first, then routed experts)
-    auto p1_of = [&](int a) -> int { return a < sh.n_sh ? a * u1s : sh.n_sh * u1s + (a - sh.n_sh) * u1r; };
-    auto p2_of = [&](int a) -> int { return a < sh.n_sh ? a * u2s : sh.n_sh * u2s + (a - sh.n_sh) * u2r; };
-    // the group in [max(lo, 1), hi] whose first unit comes closest to the wave share of `total` (hi when
-    // the range is empty): where a lot of groups is cut in two
-    auto cut_at = [&](int lo, int hi, int total) -> int {
-        int best_a = hi;
-        long long best = -1;
-        for (int a = lo < 1 ? 1 : lo; a <= hi; ++a) {
-            long long dist = (long long)p1_of(a) * kTcSplitDen - (long long)total * kTcSplitNum;
-            if (dist < 0) dist = -dist;
-            if (best < 0 || dist < best) { best = dist; best_a = a; }
-        }
-        return best_a;
-    };
-    if (FUSED && go && gate_warp) {
-        const TcRoute &rt = p.rt;
-        const int gw = warp <= 5 ? warp - 2 : warp - 3;            // 0..7 inside the gating group
-        const GateGroup gg{gw * 32 + lane, kTcGateWarps * 32, kTcGateBar};
-        const int E = sh.E, B = p.B, k = sh.k, n_rows = E + (rt.sh_scale ? 1 : 0), n_routed = B * k;
-        const int EW = (E + 31) >> 5;                              // bit words of an expert set
-        double *s_l = reinterpret_cast<double *>(gate_area), *s_w = s_l + B * E, *s_gl = s_w + B;   // logits, confidences, gate logits
-        const GateMem gm = gate_mem_carve(s_gl + B, E, B, k);
-        const bool bias_on = sh.alpha > 0.0 && sh.cap < E && k < E;
-        // ---- stage the logits: the pieces of a row added in ascending order (all loads first)
-#pragma unroll 1
-        for (int i = gg.t; i < B * n_rows; i += gg.n) {
-            const int b = i / n_rows, r = i - b * n_rows;
-            double v[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = q < pl.ksplit ? __ldcg(&rt.lpart[((size_t)q * B + b) * n_rows + r]) : 0.0;
-            double acc = v[0];
-#pragma unroll
-            for (int q = 1; q < 8; ++q) acc += v[q];
-            if (r < E) s_l[b * E + r] = acc;
-            else s_gl[b] = acc;
-        }
-#pragma unroll 1
-        for (int b = gg.t; b < B; b += gg.n) s_w[b] = rt.conf ? (double)rt.conf[b] : 1.0;
-        if (gg.t < 24) s_lot[gg.t >> 3][gg.t & 7] = 0u;
-        for (int e = gg.t; e < E; e += gg.n) gm.star[e] = 0;
-        if (gg.t < 8) gm.star32[gg.t] = 0u;
-        gate_sync(gg);
-        // ---- first lot of early groups: the shared experts, and (alpha <= 1) every token's first
-        // expert in the order (logit descending, id ascending), which no bias can push out of its
-        // top-k: six warps; the other two find E* meanwhile
-        if (gw < 2) {
-            if (bias_on) gating_estar(sh, B, s_l, s_w, gm, gg.t, 64, kTcGateBar + 1);
-        } else if (rt.early) {
-#pragma unroll 1
-            for (int b = gw - 2; b < B; b += kTcGateWarps - 2) {
-                unsigned long long best = 0ull;
-                int be = 0;
-                for (int e = lane; e < E; e += 32) {
-                    const unsigned long long ke = dkey(s_l[b * E + e]);
-                    if (ke > best) { best = ke; be = e; }
-                }
-                const unsigned hb = warp_max_holders(best, best != 0ull);
-                const unsigned me = __reduce_min_sync(0xffffffffu, ((hb >> lane) & 1u) ? (unsigned)be : 0xffffffffu);
-                if (lane == 0) atomicOr(&s_lot[0][me >> 5], 1u << (me & 31));
-            }
-        }
-        gate_sync(gg);
-        // position of expert e among the members of a bit set
-        auto set_rank = [&](const unsigned *set, int e) -> int {
-            int r = __popc(set[e >> 5] & ((1u << (e & 31)) - 1u));
-            for (int w = 0; w < (e >> 5); ++w) r += __popc(set[w]);
-            return r;
+    const int split1 = W == 2 ? groups[a_split].p1 : total1;
+    const int split2 = W == 2 ? groups[a_split].p2 : total2;
+    // Where every unit of a projection has all its four k-tiles (contraction length a multiple of
+    // 256) the segments are dealt in half units, so that the CTAs of a segment differ by two
+    // k-tiles (0.75 us) instead of four: a share may then begin with the second half of a unit
+    // and end with the first half of one (trim bits 1 and 2).  Measured at the OLMoE shape: 0.7 %
+    // of a layer; dealing single k-tiles cuts more accumulation runs in two and gives it back.
+    // The int4 path needs whole units.
+    const bool halves1 = !Q4 && sh.d % 256 == 0;
+    const bool halves2 = !Q4 && sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
+    int my_start0, my_start1, my_start2, my_start3, my_cnt0, my_cnt1, my_cnt2, my_cnt3;
+    int my_trim0, my_trim1, my_trim2, my_trim3;
+    {
+        int rot = 0;
+        auto share = [&](int begin, int n, bool halves, int &start, int &cnt, int &trim) {
+            const int m = halves ? 2 : 1, n2 = n * m;
+            const int q = n2 / P, r = n2 - q * P;
+            int c = (int)blockIdx.x - rot;               // (blockIdx.x - rot) mod P without a division:
+            if (c < 0) c += P;                           // the four calls would otherwise chain four of them
+            const int cnt2 = q + (c < r ? 1 : 0), start2 = c * q + min(c, r);
+            const int u0 = halves ? start2 >> 1 : start2, u1 = halves ? (start2 + cnt2 - 1) >> 1 : start2 + cnt2 - 1;
+            cnt = cnt2 > 0 ? u1 - u0 + 1 : 0;
+            start = begin + u0;
+            trim = (halves && cnt2 > 0) ? ((start2 & 1) | (((start2 + cnt2) & 1) << 1)) : 0;
+            rot += r;
+            if (rot >= P) rot -= P;
         };
-        auto set_size = [&](const unsigned *set) -> int {
-            int n = 0;
-            for (int w = 0; w < EW; ++w) n += __popc(set[w]);
-            return n;
-        };
-        const int n_a = set_size(s_lot[0]);                        // experts of the first lot
-        {
-            // group entries of the first lot: the shared experts, then its experts in ascending order
-            for (int a = gg.t; a < sh.n_sh; a += gg.n) {
-                TcGroup gr{};
-                gr.group = E + a; gr.f = sh.f_sh; gr.p1 = a * u1s; gr.p2 = a * u2s;
-                groups[a] = gr;
-            }
-            for (int e = gg.t; e < E; e += gg.n) {
-                if ((s_lot[0][e >> 5] >> (e & 31)) & 1u) {
-                    const int r = set_rank(s_lot[0], e);
-                    TcGroup gr{};
-                    gr.group = e; gr.f = sh.f; gr.p1 = sh.n_sh * u1s + r * u1r; gr.p2 = sh.n_sh * u2s + r * u2r;
-                    groups[sh.n_sh + r] = gr;
-                }
-            }
-            if (gg.t == 0) {
-                const int e1 = p1_of(sh.n_sh + n_a), b1 = p1_of(cut_at(0, sh.n_sh + n_a, e1));
-                const int bound[kTcSegs + 1] = {0, b1, e1, e1, e1, e1, e1, e1, e1};
-                TcShare shr;
-                tc_shares(bound, halves1, halves2, P, (int)blockIdx.x, shr);
-                s_share = shr;
-                s_nunits[0] = shr.cnt[0] + shr.cnt[1];
-                // what a unit beyond the decoded table is made from (see unit_at): for now the early
-                // groups alone; the final values replace these once the groups are complete, and an
-                // early unit decodes the same from either
-                s_nact = sh.n_sh + n_a;
-                s_total1 = 0x7fffffff;
-                s_split = 0x7fffffff;
-            }
-        }
-        gate_sync(gg);
-        for (int i = gg.t; i < s_nunits[0] && i < kTcMaxUnits; i += gg.n) {
-            const TcUnit t = tc_unit_make(s_share, groups, sh.n_sh + n_a, 0x7fffffff, 0x7fffffff, i, sh.d, pl.n1);
-            s_units[i] = t;
-            s_umeta[i] = tc_unit_meta(t);
-        }
-        __threadfence_block();
-        gate_sync(gg);
-        if (gg.t == 0) s_tab = 1;
-        // ---- the gating, first part: E*, lambda_b, every token's first k experts by original logit
-        if (E <= 64) gating_part1<2>(sh, B, s_l, s_w, gg, gm, false, true, true);
-        else if (E <= 128) gating_part1<4>(sh, B, s_l, s_w, gg, gm, false, true, true);
-        else gating_part1<8>(sh, B, s_l, s_w, gg, gm, false, true, true);
-        // ---- second lot of early groups: an expert of E* that is among a token's first k stays in that
-        // token's top-k whatever the bias does to the others (at most its rank of them pass it), so
-        // E* intersected with the union of the tokens' first k can start now
-        if (bias_on && rt.early) {
-            const int J = E <= 64 ? 2 : (E <= 128 ? 4 : 8);
-            for (int i = gg.t; i < B * J; i += gg.n) {
-                const int j = i % J;
-                const unsigned wd = gm.topk[i] & gm.star32[j] & ~s_lot[0][j];
-                if (wd) atomicOr(&s_lot[1][j], wd);
-            }
-        }
-        gate_sync(gg);
-        const int n_b = set_size(s_lot[1]), n_early = sh.n_sh + n_a + n_b;
-        {
-            for (int e = gg.t; e < E; e += gg.n) {
-                if ((s_lot[1][e >> 5] >> (e & 31)) & 1u) {
-                    const int a = sh.n_sh + n_a + set_rank(s_lot[1], e);
-                    TcGroup gr{};
-                    gr.group = e; gr.f = sh.f; gr.p1 = sh.n_sh * u1s + (a - sh.n_sh) * u1r; gr.p2 = sh.n_sh * u2s + (a - sh.n_sh) * u2r;
-                    groups[a] = gr;
-                }
-            }
-            if (gg.t == 0) {
-                const int m1 = sh.n_sh + n_a, e1 = p1_of(m1), b1 = p1_of(cut_at(0, m1, e1));
-                const int e2 = p1_of(n_early), b3 = p1_of(cut_at(m1, n_early, e2));
-                const int bound[kTcSegs + 1] = {0, b1, e1, b3, e2, e2, e2, e2, e2};
-                TcShare shr;
-                tc_shares(bound, halves1, halves2, P, (int)blockIdx.x, shr);
-                s_share = shr;                         // (the first two segments come out as before)
-                s_nunits[1] = shr.cnt[0] + shr.cnt[1] + shr.cnt[2] + shr.cnt[3];
-            }
-        }
-        __threadfence_block();
-        gate_sync(gg);
-        if (gg.t == 0) s_nact = n_early;               // the second lot's groups are complete
-        for (int i = s_nunits[0] + gg.t; i < s_nunits[1] && i < kTcMaxUnits; i += gg.n) {
-            const TcUnit t = tc_unit_make(s_share, groups, n_early, 0x7fffffff, 0x7fffffff, i, sh.d, pl.n1);
-            s_units[i] = t;
-            s_umeta[i] = tc_unit_meta(t);
-        }
-        __threadfence_block();
-        gate_sync(gg);
-        if (gg.t == 0) s_tab = 2;
-        // ---- the gating, second part; CTA 0 also writes the call's outputs
-        const bool writer = blockIdx.x == 0;
-        if (E <= 64) gating_part2<2>(sh, B, s_l, gg, gm, writer ? rt.sel_idx : nullptr, writer ? rt.sel_w : nullptr, false);
-        else if (E <= 128) gating_part2<4>(sh, B, s_l, gg, gm, writer ? rt.sel_idx : nullptr, writer ? rt.sel_w : nullptr, false);
-        else gating_part2<8>(sh, B, s_l, gg, gm, writer ? rt.sel_idx : nullptr, writer ? rt.sel_w : nullptr, false);
-        // ---- the tables in their final form.  Group order: the early groups, then the other selected
-        // experts in ascending order; slots stay in expert order (routed first, then shared).
-        const int U = *gm.U, n_active = U + sh.n_sh;
-        {
-            // all selected experts as a bit set, one ballot per 32 experts
-            for (int e0 = gw * 32; e0 < E; e0 += kTcGateWarps * 32) {
-                const unsigned wd = __ballot_sync(0xffffffffu, e0 + lane < E && gm.cnt[e0 + lane] > 0);
-                if (lane == 0) s_lot[2][e0 >> 5] = wd;
-            }
-        }
-        gate_sync(gg);
-        const unsigned long long all = B >= 64 ? ~0ull : ((1ull << B) - 1ull);
-        for (int e = gg.t; e < E; e += gg.n) {
-            if (gm.cnt[e] == 0) continue;
-            const bool in_a = (s_lot[0][e >> 5] >> (e & 31)) & 1u, in_b = (s_lot[1][e >> 5] >> (e & 31)) & 1u;
-            int a;
-            if (in_a) a = sh.n_sh + set_rank(s_lot[0], e);
-            else if (in_b) a = sh.n_sh + n_a + set_rank(s_lot[1], e);
-            else {
-                // position among the selected experts outside both lots
-                int r = __popc(s_lot[2][e >> 5] & ~s_lot[0][e >> 5] & ~s_lot[1][e >> 5] & ((1u << (e & 31)) - 1u));
-                for (int w = 0; w < (e >> 5); ++w) r += __popc(s_lot[2][w] & ~s_lot[0][w] & ~s_lot[1][w]);
-                a = n_early + r;
-            }
-            TcGroup gr;
-            gr.group = e; gr.T = gm.cnt[e]; gr.off = gm.off[e]; gr.f = sh.f; gr.mask = gm.mask[e];
-            gr.p1 = sh.n_sh * u1s + (a - sh.n_sh) * u1r;
-            gr.p2 = sh.n_sh * u2s + (a - sh.n_sh) * u2r;
-            groups[a] = gr;
-        }
-        for (int a = gg.t; a < sh.n_sh; a += gg.n) {
-            TcGroup gr;
-            gr.group = E + a; gr.T = B; gr.off = n_routed + a * B; gr.f = sh.f_sh; gr.mask = all;
-            gr.p1 = a * u1s; gr.p2 = a * u2s;
-            groups[a] = gr;
-        }
-        const int total1 = sh.n_sh * u1s + U * u1r, total2 = sh.n_sh * u2s + U * u2r;
-        // The boundary between the waves: of the segment boundaries inside phase 1 (the cut and the end
-        // of either early lot, the cut of the rest) the one that comes closest to the wave share.
-        const int m1 = sh.n_sh + n_a, e1 = p1_of(m1), x_a = cut_at(0, m1, e1);
-        const int e2 = p1_of(n_early), x_b = cut_at(m1, n_early, e2);
-        const int x_r = cut_at(n_early, n_active, total1);
-        int sp = n_active;
-        {
-            const int cand[5] = {x_a, m1, x_b, n_early, x_r};
-            long long best = -1;
-#pragma unroll
-            for (int c = 0; c < 5; ++c) {
-                const int a = cand[c];
-                if (a < 1 || a > n_active - 1) continue;           // both waves keep at least one group
-                long long dist = (long long)p1_of(a) * kTcSplitDen - (long long)total1 * kTcSplitNum;
-                if (dist < 0) dist = -dist;
-                if (best < 0 || dist < best) { best = dist; sp = a; }
-            }
-        }
-        if (gg.t == 0) {
-            const int b5 = p1_of(x_r);
-            const int split2 = sp < n_active ? p2_of(sp) : total2;
-            const int bound[kTcSegs + 1] = {0, p1_of(x_a), e1, p1_of(x_b), e2, b5, total1, total1 + split2, total1 + total2};
-            TcShare shr;
-            tc_shares(bound, halves1, halves2, P, (int)blockIdx.x, shr);
-            s_share = shr;
-            int n = 0;
-            for (int sg = 0; sg < kTcSegs; ++sg) n += shr.cnt[sg];
-            s_nunits[2] = n;
-        }
-        __threadfence_block();
-        gate_sync(gg);
-        if (gg.t == 0) {                               // the groups are complete before their number grows
-            s_split = sp;
-            s_total1 = total1;
-            s_nact = n_active;
-        }
-        for (int i = s_nunits[1] + gg.t; i < s_nunits[2] && i < kTcMaxUnits; i += gg.n) {
-            const TcUnit t = tc_unit_make(s_share, groups, n_active, total1, sp, i, sh.d, pl.n1);
-            s_units[i] = t;
-            s_umeta[i] = tc_unit_meta(t);
-        }
-        __threadfence_block();
-        gate_sync(gg);
-        if (gg.t == 0) s_tab = 3;
-        // ---- what only these warps' later roles need: slots (tokens ascending inside an expert, the
-        // shared experts' slots behind the routed ones) and the groups' element ranges
-        for (int i = gg.t; i < n_routed; i += gg.n) {
-            const int b = i / k, e = gm.sel[i];
-            const int pos = gm.off[e] + __popcll(gm.mask[e] & ((1ull << b) - 1ull));
-            s_slot_token[pos] = b;
-            s_slot_w[pos] = gm.pw[i];
-        }
-        for (int i = gg.t; i < sh.n_sh * B; i += gg.n) {
-            const int b = i % B;
-            s_slot_token[n_routed + i] = b;
-            s_slot_w[n_routed + i] = rt.sh_scale ? (float)(1.0 / (1.0 + exp_once(-s_gl[b]))) : 1.0f;
-        }
-        if (gg.t == 0) {
-            int acc = 0;
-            for (int a = 0; a < n_active; ++a) { s_epfx[a] = acc; acc += groups[a].T * groups[a].f; }
-            s_epfx[n_active] = acc;
-        }
-        if (writer) {
-            // the layer's routing outputs and the bucketing arrays in the workspace (debug reads)
-            Workspace wsw = ws;
-            wsw.gtab = nullptr;
-            for (int b = gg.t; b < B; b += gg.n) ws.gate_logit[b] = s_gl[b];
-            for (int i = gg.t; i < B * E; i += gg.n) ws.logits[i] = s_l[i];
-            gate_sync(gg);
-            Shape shw = sh;
-            shw.plan = 3;
-            gating_writeout(shw, B, wsw, gm, rt.sh_scale ? 1 : 0, rt.n_unique, gg);
-        }
-        gate_sync(gg);
+        share(0, split1, halves1, my_start0, my_cnt0, my_trim0);
+        share(split1, total1 - split1, halves1, my_start1, my_cnt1, my_trim1);
+        share(total1, split2, halves2, my_start2, my_cnt2, my_trim2);
+        share(total1 + split2, total2 - split2, halves2, my_start3, my_cnt3, my_trim3);
     }
-
-    // The unit table as far as it is known to this thread, and a wait for more of it.  The
-    // two-launch form knows all its units from the start, and its single-thread roles loop on a
-    // register (a handful of instructions per unit in such a role cost about a hundred cycles).
-    int tab_seen = FUSED ? 0 : 3, n_known = FUSED ? 0 : s_nunits[2];
-    // 1: unit i exists, 0: the sequence has ended, -1: the wait for the tables gave up
-    auto more_units = [&](int i) -> int {
-        if constexpr (!FUSED) return i < n_known ? 1 : 0;
-        while (i >= n_known) {
-            if (tab_seen == 3) return 0;
-            bool ok = false;
-            for (unsigned spin = 0; spin < kTcSpinLimit; ++spin) {
-                if (s_tab > tab_seen) { ok = true; break; }
-                __nanosleep(40);
-            }
-            if (!ok) return -1;
-            tab_seen = s_tab;
-            __threadfence_block();
-            n_known = s_nunits[tab_seen - 1];
-        }
-        return 1;
+    const int n_units = my_cnt0 + my_cnt1 + my_cnt2 + my_cnt3;
+    auto unit_make = [&](int i) -> TcUnit {
+        int seg = 0, j = i, start = my_start0, cnt = my_cnt0, trim = my_trim0;
+        if (j >= cnt) { j -= cnt; seg = 1; start = my_start1; cnt = my_cnt1; trim = my_trim1; }
+        if (seg == 1 && j >= cnt) { j -= cnt; seg = 2; start = my_start2; cnt = my_cnt2; trim = my_trim2; }
+        if (seg == 2 && j >= cnt) { j -= cnt; seg = 3; start = my_start3; cnt = my_cnt3; trim = my_trim3; }
+        TcUnit t = tc_decode(groups, n_active, total1, start + j, sh.d, pl.n1);
+        const int K = t.phase == 1 ? sh.d : groups[t.a].f;
+        if (j == 0 && (trim & 1)) t.kt0 += kTcKT / 2;            // the CTA before this one has the first half
+        if (j == cnt - 1 && (trim & 2)) t.kt1 -= kTcKT / 2;      // the next CTA has the second half
+        t.seg = seg;
+        t.first = (j == 0 || t.kt0 == 0) ? 1 : 0;
+        t.last = (j == cnt - 1 || t.kt1 == (K + 63) / 64) ? 1 : 0;
+        return t;
     };
-    auto unit_at = [&](int i) -> TcUnit {
-        return i < kTcMaxUnits ? s_units[i] : tc_unit_make(s_share, groups, s_nact, s_total1, s_split, i, sh.d, pl.n1);
-    };
-    auto umeta_at = [&](int i) -> uint32_t { return i < kTcMaxUnits ? s_umeta[i] : tc_unit_meta(unit_at(i)); };
+    // decoded once by all threads: the single-thread roles below then read a unit from shared
+    // memory instead of dividing
+    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x) {
+        const TcUnit t = unit_make(i);
+        s_units[i] = t;
+        s_umeta[i] = tc_unit_meta(t);
+    }
+    __syncthreads();
+    auto unit_at = [&](int i) -> TcUnit { return i < kTcMaxUnits ? s_units[i] : unit_make(i); };
+    auto umeta_at = [&](int i) -> uint32_t { return i < kTcMaxUnits ? s_umeta[i] : tc_unit_meta(unit_make(i)); };
+    auto seg_of_unit = [&](int i) -> int { return i < n_units ? unit_at(i).seg : 4; };
 
-    if (!go) {
-        // the grid-wide meeting gave up (reported): nothing is started
-    } else if (warp == 0) {
+    if (warp == 0) {
         const uint64_t wpolicy = l2_evict_first_policy();
         // ------------------------------------------------------------------ TMA producer
         if (Q4 && lane == 0) {
@@ -1124,27 +618,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             constexpr int KG = kTcQ4KG;
             const int n_routed = p.B * sh.k;
             int pi = 0, ti = 0;                          // unit of each cursor
-            TcUnit pu{}, tu{};
-            bool pu_ok = false, tu_ok = false;           // the cursor's unit has been read from the table
-            int pkt = 0, tkt = 0;
+            TcUnit pu = unit_at(0), tu = pu;
+            int pkt = pu.kt0, tkt = pu.kt0;
             int s = 0, ta = 0;
             uint32_t ring_par = 1, t_par = 1;
             int ready_w = 0;
             unsigned idle = 0;
-            bool alive = true;
-            if (Q4 && FUSED) asm volatile("fence.proxy.async.global;" ::: "memory");   // the permuted hidden states were written by ordinary stores
+            bool alive = n_units > 0;
 
-            while (alive) {
-                if (pi >= n_known && ti >= n_known) {
-                    // both cursors have reached the end of what is decoded: more of the table, or the end
-                    const int m = more_units(pi);
-                    if (m < 0) { atomicExch(ws.status, ST_DEP_TIMEOUT); break; }
-                    if (m == 0) break;
-                }
-                if (!pu_ok && pi < n_known) { pu = unit_at(pi); pkt = pu.kt0; pu_ok = true; }
-                if (!tu_ok && ti < n_known) { tu = unit_at(ti); tkt = tu.kt0; tu_ok = true; }
+            while (alive && (pi < n_units || ti < n_units)) {
                 bool progress = false;
-                if (pu_ok && mbar_test(&empty_bar[s], ring_par)) {
+                if (pi < n_units && mbar_test(&empty_bar[s], ring_par)) {
 
                     const TcGroup &g = groups[pu.a];
                     const bool shared = g.group >= sh.E;
@@ -1160,12 +644,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     tma_load_2d(stage + KG * kTcQ4Packed, &maps.m[9 + mi], (pkt & ~3) * 2, row0, &full_bar[s]);
                     tc_ring_next(s, ring_par, S);
                     pkt += KG;
-                    if (pkt >= pu.kt1) { ++pi; pu_ok = false; }
+                    if (pkt >= pu.kt1 && ++pi < n_units) { pu = unit_at(pi); pkt = pu.kt0; }
                     progress = true;
 
                 }
-                if (tu_ok) {
-                    const int wv = tu.wave;
+                if (ti < n_units) {
+                    const int wv = tu.a >= a_split ? 1 : 0;
                     bool ready = tu.phase == 1 || wv < ready_w;
                     if (!ready && s_ready[wv]) {
                         // the activations of this wave are written: order them before the copies below
@@ -1192,7 +676,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         }
                         tc_ring_next(ta, t_par, pl.a_stages);
                         tkt += KG;
-                        if (tkt >= tu.kt1) { ++ti; tu_ok = false; }
+                        if (tkt >= tu.kt1 && ++ti < n_units) { tu = unit_at(ti); tkt = tu.kt0; }
                         progress = true;
 
                     }
@@ -1245,12 +729,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             int s = 0;                                   // ring slot of the next k-tile
             uint32_t ring_par = 1;                       // parity to wait for on its empty barrier
 
-            for (int i = 0; alive; ++i) {
-                const int m = more_units(i);
-                if (m <= 0) {
-                    if (m < 0) { atomicExch(ws.status, ST_DEP_TIMEOUT); alive = false; }
-                    break;
-                }
+            for (int i = 0; i < n_units && alive; ++i) {
+
                 const TcUnit t = unit_at(i);
                 const TcGroup &g = groups[t.a];
                 const bool shared = g.group >= sh.E;
@@ -1259,7 +739,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
                 const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared activation array
-                const int wv = t.wave;
+                const int wv = t.a >= a_split ? 1 : 0;
                 bool ready = t.phase == 1 || wv < ready_w;
                 if (!ready) {
                     // the pending tiles all belong to one wave (pend_wave); if that is an earlier wave than
@@ -1316,9 +796,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // and the epilogue adds the partial accumulators.
         const int half = warp == 1 ? 0 : (warp == 6 ? 1 : warp - (9 + kTcQ4DeqWarps));     // with one issuer (int4, many tokens): warp 1
         if (lane == 0 && half < NI) {
-            unsigned it = 0, ui = 0;
-            int buf = 0;                                 // accumulator buffer of the current run, and the parity
-            uint32_t buf_par = 1;                        // to wait for on its "drained" barrier
+            unsigned it = 0, ui = 0, run = 0;
             uint32_t acc = 0;
             bool alive = true;
             int s = 0;
@@ -1348,12 +826,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // int4: a unit is one stage; everything this thread needs of it is one word
                 uint32_t d_tmem = tmem_base + (uint32_t)(half * 2 * pl.n1), buf = 0, run_par = 1;
                 const uint32_t tok_slot = (uint32_t)kTcQ4KG * ((uint32_t)pl.tokb >> 4), tok_step1 = (uint32_t)pl.tokb >> 4;
-                for (;; ++ui) {
-                    const int m = more_units((int)ui);
-                    if (m <= 0) {
-                        if (m < 0) atomicExch(ws.status, ST_DEP_TIMEOUT);
-                        break;
-                    }
+                for (; (int)ui < n_units; ++ui) {
                     const uint32_t um = umeta_at((int)ui);
                     if (um & 1u) {
 
@@ -1393,16 +866,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 
                 }
             } else
-            for (; alive; ++ui) {
-                const int m = more_units((int)ui);
-                if (m <= 0) {
-                    if (m < 0) atomicExch(ws.status, ST_DEP_TIMEOUT);
-                    break;
-                }
+            for (; (int)ui < n_units && alive; ++ui) {
                 const TcUnit t = unit_at((int)ui);
+                const int buf = run & 1;
                 if (t.first) {
 
-                    if (!mbar_wait(&acc_empty[buf], buf_par)) {
+                    if (!mbar_wait(&acc_empty[buf], ((run >> 1) & 1u) ^ 1u)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         break;
                     }
@@ -1439,7 +908,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 }
                 if (alive && t.last) {
                     tc_commit(&acc_full[buf]);
-                    if (++buf == NACC) { buf = 0; buf_par ^= 1u; }
+                    ++run;
                 }
             }
 
@@ -1469,12 +938,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // contraction lengths are multiples of 256 here, so every unit is exactly one stage and
         // nothing of it has to be decoded
         {
-            for (int ui = 0; alive; ++ui, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
-                const int m = more_units(ui);
-                if (m <= 0) {
-                    if (m < 0 && lane == 0) atomicExch(ws.status, ST_DEP_TIMEOUT);
-                    break;
-                }
+            for (int ui = 0; ui < n_units && alive; ++ui, tc_ring_next(s, ring_par, S), tc_ring_next(ta, a_par, pl.a_stages)) {
 
                 const bool ok_full = mbar_wait(&full_bar[s], ring_par);
 
@@ -1549,7 +1013,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // polls the waves' second counters (all CTAs have written their slice of the activations)
         // and publishes them in shared memory, so that the producer never waits on global memory
         if (lane == 0) {
-            const int W = s_split < s_nact ? 2 : 1;
             for (int w = 0; w < W; ++w) {
                 bool ok = false;
                 for (unsigned i = 0; i < (1u << 21); ++i) {
@@ -1571,7 +1034,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         uint32_t ep_phase = 0;                         // running parity of cv_bar
         uint64_t *ep_bar_p = &cv_bar;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
-        const int n_active = s_nact, a_split = s_split, W = a_split < n_active ? 2 : 1;
+        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
 
         auto wave_convert = [&](int w) -> bool {
 
@@ -1590,20 +1053,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             __threadfence_block();                 // the counter was read with acquire by one thread of this barrier
 
             // pre holds a gate plane and an up plane, both indexed exactly like the activations
-            // (act_offset(slot) + row).  The wave's groups, one behind the other in group order, form
-            // one range of elements; this CTA converts a contiguous slice of it, four elements per
-            // thread and step (a group's elements are contiguous, the groups of a wave need not be)
-            // (in the two-launch form the groups are in slot order, so a wave is ONE range of elements)
-            const int g_lo = w == 0 ? 0 : a_split, g_hi = (w == 0 && W == 2) ? a_split : n_active;
-            const long long base = s_epfx[g_lo], n4 = ((long long)s_epfx[g_hi] - base) >> 2;
+            // (act_offset(slot) + row): this CTA converts a contiguous slice of the wave's range,
+            // four elements per thread and step
+            const long long w_lo = w == 0 ? 0 : el_split, w_hi = (w == 0 && W == 2) ? el_split : n_el;
+            const long long n4 = (w_hi - w_lo) >> 2;
             const long long lo4 = n4 * blockIdx.x / gridDim.x, hi4 = n4 * (blockIdx.x + 1) / gridDim.x;
-            const int a_first = FUSED ? g_lo : g_hi - 1;
-            for (int a = a_first; a < g_hi; ++a) {
-            const long long ga4 = FUSED ? ((long long)s_epfx[a] - base) >> 2 : 0, gb4 = FUSED ? ((long long)s_epfx[a + 1] - base) >> 2 : n4;
-            const long long qa = lo4 > ga4 ? lo4 : ga4, qb = hi4 < gb4 ? hi4 : gb4;
-            const long long abs0 = FUSED ? (long long)act_offset(groups[a].off, n_routed, sh.f, sh.f_sh) - 4 * ga4 : base;
-            for (long long q = qa + et; q < qb; q += 96) {
-                const long long i = abs0 + 4 * q;
+            for (long long q = lo4 + et; q < hi4; q += 96) {
+                const long long i = w_lo + 4 * q;
                 const float4 gv = __ldcg(reinterpret_cast<const float4 *>(p.pre + i));
                 const float4 uv = __ldcg(reinterpret_cast<const float4 *>(p.pre + n_el + i));
                 const float a0 = silu_mul(gv.x, uv.x), a1 = silu_mul(gv.y, uv.y), a2 = silu_mul(gv.z, uv.z),
@@ -1631,7 +1087,6 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
                 }
             }
-            }
             // the activations are read by TMA copies of other CTAs: proxy fence over global memory by
             // every writer, then one release at GPU scope behind the barrier of the converter warps
             asm volatile("fence.proxy.async.global;" ::: "memory");
@@ -1657,9 +1112,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;                        // TMEM lane quarter this warp may read
         const int et = tid - 64;                       // 0..127 among the epilogue threads
-        unsigned ui = 0;
-        int buf = 0;                                   // accumulator buffer of the next run to drain, and the parity
-        uint32_t buf_par = 0;                          // to wait for on its "complete" barrier
+        unsigned ui = 0, run = 0;
+        uint32_t ep_phase = 0;
         const int n_routed = p.B * sh.k;
         bool alive = true;
 
@@ -1667,23 +1121,24 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         const int n_routed_el = n_routed;   // (alias used below)
         (void)n_routed_el;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
-        const int n_units = s_nunits[2], W = s_split < s_nact ? 2 : 1;
-        const int a_split = s_split;
-        // (where the CTA's sequence stands in front of a unit: 0 in wave 0's first projection, 1 in
-        // wave 1's, 2 behind both: second projection, or the end)
+        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
         int next_arrive = 0;
         auto wave_arrive = [&](int w) -> bool {
             // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps,
             // whose first thread orders them (fence) before it arrives on the grid-wide counter, so
             // that no epilogue thread stalls on a fence
             __syncwarp();
-            if (lane == 0) mbar_arrive(&conv_go[w]);
+            if (lane == 0) {
+                mbar_arrive(&conv_go[w]);
+
+            }
             return true;
         };
         // called before every unit (and once at the end): hand a wave over once this CTA's phase-1
         // units of it are all done
-        auto service = [&](int stage) -> bool {
-            while (next_arrive < W && stage > next_arrive) {
+        auto service = [&](int upcoming_seg) -> bool {
+            const int seg_wave1 = W == 2 ? 1 : 2;        // first segment that lies after phase 1 of wave 0
+            while (next_arrive < W && upcoming_seg >= (next_arrive == 0 ? seg_wave1 : 2)) {
                 if (!wave_arrive(next_arrive)) return false;
                 ++next_arrive;
             }
@@ -1691,12 +1146,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         };
         {
             for (; (int)ui < n_units && alive; ++ui) {
+                if (!service(seg_of_unit((int)ui))) { alive = false; break; }
                 const TcUnit t = unit_at((int)ui);
-                if (!service(t.phase == 2 ? 2 : (t.a >= a_split ? 1 : 0))) { alive = false; break; }
                 if (!t.last) continue;                 // the run's accumulator is read after its last unit
                 const TcGroup &g = groups[t.a];
+                const int buf = run & 1;
 
-                if (!mbar_wait(&acc_full[buf], buf_par)) {
+                if (!mbar_wait(&acc_full[buf], (run >> 1) & 1u)) {
                     if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     alive = false;
                     break;
@@ -1755,10 +1211,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
-                if (++buf == NACC) { buf = 0; buf_par ^= 1u; }
+                ++run;
 
             }
-            if (alive && !service(2)) alive = false;
+            if (alive && !service(4)) alive = false;
         }
 
     }

@@ -16,6 +16,7 @@
 #include "expand.cuh"
 #include "ffn_tc.cuh"
 #include "route.cuh"
+#include "layer_tc.cuh"
 
 #include "expert_cache.h"
 
@@ -39,6 +40,7 @@ struct s2moe_ctx {
     size_t act_elems = 0;
     cudaLaunchAttribute pdl_attr{};
     bool use_pdl = true;                  // S2MOE_NO_PDL=1 in the environment turns it off
+    bool pdl_in_graph = false;            // S2MOE_PDL_IN_GRAPH=1: also under stream capture
     void *hperm = nullptr;                // int4 plan 3: column-permuted copy of the hidden states
     double *lpart = nullptr;              // fused layer kernel: partial router logits [piece][token][row]
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
@@ -183,7 +185,7 @@ cudaLaunchConfig_t pdl_config(s2moe_ctx *ctx, int grid, int block, size_t smem, 
     // (its kernel nodes already follow each other closely), so it is left out under capture
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     const bool capturing = cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone;
-    ctx->pdl_attr.val.programmaticStreamSerializationAllowed = (ctx->use_pdl && !capturing) ? 1 : 0;
+    ctx->pdl_attr.val.programmaticStreamSerializationAllowed = (ctx->use_pdl && (!capturing || ctx->pdl_in_graph)) ? 1 : 0;
     lc.attrs = &ctx->pdl_attr;
     lc.numAttrs = 1;
     return lc;
@@ -404,7 +406,7 @@ int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
         // CTAs than on a block of its own, and delays the first hand-over between the projections).
         // An offloaded context meets the host between routing and the experts: two launches.
         if (ctx->offload || ctx->tc_maps.empty()) return 0;
-        const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B, true);
+        const fused::TcPlan tp = fused::tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
         return tp.feasible ? 4 : 0;
     }
     if (want == 0 || want == 3) {
@@ -496,17 +498,20 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         if (rc != S2MOE_OK) return rc;
     }
     if (plan == 3 || plan == 4) {
-        const TcPlan tp = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B, plan == 4);
+        const TcPlan tp3 = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
+        const fused::TcPlan tp4 = plan == 4 ? fused::tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B) : fused::TcPlan{};
+        const bool q4 = plan == 4 ? tp4.q4 != 0 : tp3.q4 != 0;
+        const int tokb = plan == 4 ? tp4.tokb : tp3.tokb, kg = plan == 4 ? tp4.kg : tp3.kg;
         TcMaps maps = ctx->tc_maps[layer];
         const size_t n_routed = (size_t)B * sh.k;
         const uint64_t plane = (uint64_t)((const uint8_t *)ctx->act_lo - (const uint8_t *)ctx->act_hi);
         bool ok;
-        if (tp.q4) {
-            ok = make_map_ktiles(ctx, &maps.m[6], ctx->hperm, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp.tokb / 128, (uint32_t)tp.kg) &&
-                 make_map_hilo_ktiles(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane, (uint32_t)tp.kg);
+        if (q4) {
+            ok = make_map_ktiles(ctx, &maps.m[6], ctx->hperm, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tokb / 128, (uint32_t)kg) &&
+                 make_map_hilo_ktiles(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane, (uint32_t)kg);
             if (ok && sh.n_sh)
                 ok = make_map_hilo_ktiles(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B,
-                                          (uint64_t)sh.f_sh, plane, (uint32_t)tp.kg);
+                                          (uint64_t)sh.f_sh, plane, (uint32_t)kg);
         } else {
             ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
                  make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
@@ -514,12 +519,20 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
                 ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
         }
         if (!ok) return S2MOE_ECUDA;
-        TcArgs a;
-        a.sh = sh; a.ws = ctx->ws; a.plan = tp; a.y = out; a.pre = ctx->pre;
-        a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
-        a.rt = TcRoute{};
-        if (plan == 4) {
+        if (plan == 3) {
+            TcArgs a;
+            a.sh = sh; a.ws = ctx->ws; a.plan = tp3; a.y = out; a.pre = ctx->pre;
+            a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
+            LaunchScope scope(ctx, KC_TC, st);
+            cudaLaunchConfig_t lc = pdl_config(ctx, tp3.n_cta, q4 ? kTcQ4Threads : kTcThreads, tp3.smem_bytes, st);
+            if (q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true>, maps, a);
+            else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false>, maps, a);
+        } else {
+            fused::TcArgs a;
+            a.sh = sh; a.ws = ctx->ws; a.plan = tp4; a.y = out; a.pre = ctx->pre;
+            a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
             a.sh.plan = 3;
+            a.rt = fused::TcRoute{};
             a.rt.hidden = hidden; a.rt.router = lp.router; a.rt.sh_scale = lp.sh_scale; a.rt.conf = conf;
             a.rt.sel_idx = sel_idx; a.rt.sel_w = sel_w; a.rt.n_unique = n_unique;
             a.rt.lpart = ctx->lpart;
@@ -528,15 +541,10 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
             // the expert of a token's largest logit stays in its top-k under any bias of alpha <= 1
             const bool bias_on = sh.alpha > 0.0 && sh.cap < sh.E && sh.k < sh.E;
             a.rt.early = (!bias_on || sh.alpha <= 1.0) ? 1 : 0;
-        }
-        LaunchScope scope(ctx, plan == 4 ? KC_LAYER : KC_TC, st);
-        cudaLaunchConfig_t lc = pdl_config(ctx, tp.n_cta, tp.q4 ? kTcQ4Threads : kTcThreads, tp.smem_bytes, st);
-        if (plan == 4) {
-            if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true, true>, maps, a);
-            else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false, true>, maps, a);
-        } else {
-            if (tp.q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true, false>, maps, a);
-            else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false, false>, maps, a);
+            LaunchScope scope(ctx, KC_LAYER, st);
+            cudaLaunchConfig_t lc = pdl_config(ctx, tp4.n_cta, q4 ? kTcQ4Threads : kTcThreads, tp4.smem_bytes, st);
+            if (q4) cudaLaunchKernelEx(&lc, fused::layer_tc_kernel<true>, maps, a);
+            else cudaLaunchKernelEx(&lc, fused::layer_tc_kernel<false>, maps, a);
         }
     } else if (plan == 2) {
         StreamArgs a;
@@ -644,6 +652,8 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     {
         const char *no_pdl = std::getenv("S2MOE_NO_PDL");
         ctx->use_pdl = !(no_pdl && no_pdl[0] == '1');
+        const char *pg = std::getenv("S2MOE_PDL_IN_GRAPH");
+        ctx->pdl_in_graph = pg && pg[0] == '1';
     }
     if (e == cudaSuccess && ctx->plan != 1)
         e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStMaxSmem);
@@ -674,10 +684,10 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
             ctx->encode_tiled = fn;
             ctx->tc_maps.resize(config->n_layers);
             const bool q4 = sh.weight_dtype == DT_Q4B32;
-            bool ok = cudaFuncSetAttribute(ffn_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
-                      cudaFuncSetAttribute(ffn_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
-                      cudaFuncSetAttribute(ffn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
-                      cudaFuncSetAttribute(ffn_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
+            bool ok = cudaFuncSetAttribute(ffn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(ffn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(fused::layer_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess &&
+                      cudaFuncSetAttribute(fused::layer_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcMaxSmem) == cudaSuccess;
             // the int4 variant needs contraction lengths that are multiples of 256 (see tc_make_plan)
             if (q4 && (sh.d % 256 || sh.f % 256 || (sh.n_sh && sh.f_sh % 256))) ok = false;
             for (int l = 0; l < config->n_layers && ok; ++l) {
@@ -1074,7 +1084,7 @@ const char *s2moe_kernel_class_name(int32_t cls)
         case KC_DOWN: return "ffn_down_simple";
         case KC_STREAM: return "ffn_stream_kernel";
         case KC_TC: return "ffn_tc_kernel";
-        case KC_LAYER: return "ffn_tc_kernel/fused";
+        case KC_LAYER: return "layer_tc_kernel";
         default: return nullptr;
     }
 }
