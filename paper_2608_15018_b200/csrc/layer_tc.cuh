@@ -167,48 +167,6 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
 
 // ---- routing stage of the fused kernel ------------------------------------------------------
 
-// Router logits by the warps of the whole grid: a task is one router row (row E: the shared
-// experts' gate vector) x 8 tokens x one piece of the contraction, float64 accumulation; its
-// partial sums go to lpart[piece][token][row], which the gating adds up in a fixed order.
-template <int RT>
-__device__ __forceinline__ void lt_logit_tasks(const Shape &sh, int B, const TcRoute &rt, int ksplit, int gwarp, int n_gwarps,
-                                               int lane)
-{
-    const int d = sh.d, n_rows = sh.E + (rt.sh_scale ? 1 : 0), n_tg = (B + 7) >> 3;
-    const int len = ((d + 4 * ksplit - 1) / (4 * ksplit)) * 4;              // columns of a piece, a multiple of 4
-    const int n_tasks = n_rows * n_tg * ksplit;
-    const size_t rb = RT == DT_F32 ? 4 : 2;
-#pragma unroll 1
-    for (int task = gwarp; task < n_tasks; task += n_gwarps) {
-        const int row = task % n_rows, rest = task / n_rows, tg = rest % n_tg, piece = rest / n_tg;
-        const int c0 = piece * len, c1 = min(d, c0 + len), b0 = tg * 8;
-        const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(rt.router) + (size_t)row * d * rb
-                                         : reinterpret_cast<const uint8_t *>(rt.sh_scale);
-        double acc[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) acc[t] = 0.0;
-#pragma unroll 2
-        for (int c = c0 + lane * 4; c < c1; c += 128) {
-            float w[4], x[8][4];
-            load4_plain<RT>(wrow, c, w);
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const int bt = min(b0 + t, B - 1);           // past the batch: the last token again (not stored)
-                load4_plain<DT_BF16>(reinterpret_cast<const uint8_t *>(rt.hidden) + (size_t)bt * d * 2, c, x[t]);
-            }
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[t][i], acc[t]);
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const double v = warp_sum(acc[t]);
-            if (lane == t && b0 + t < B) rt.lpart[((size_t)piece * B + b0 + t) * n_rows + row] = v;
-        }
-    }
-}
-
 struct TcUnit {                        // plain ints: the single-thread roles read these on their critical path
     int phase, a, mat, rb, kt0, kt1;   // group slot, matrix (0 gate, 1 up, 2 down), row block, k-tile range
     int n;                             // MMA N: phase 1 tokens padded to 16; phase 2 16 per 8 slots (hi | lo)
@@ -422,8 +380,10 @@ layer_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // ---- the logit pass, shared by the warps of all CTAs
         {
             const int nwarps = (int)blockDim.x >> 5;
-            if (sh.router_dtype == DT_F32) lt_logit_tasks<DT_F32>(sh, p.B, rt, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
-            else lt_logit_tasks<DT_BF16>(sh, p.B, rt, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
+            if (sh.router_dtype == DT_F32)
+                route_logit_tasks<DT_BF16, DT_F32>(sh, p.B, rt.hidden, rt.router, rt.sh_scale, rt.lpart, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
+            else
+                route_logit_tasks<DT_BF16, DT_BF16>(sh, p.B, rt.hidden, rt.router, rt.sh_scale, rt.lpart, pl.ksplit, warp * P + (int)blockIdx.x, nwarps * P, lane);
         }
         tc_fence_before();
         __syncthreads();

@@ -118,7 +118,7 @@ __device__ __forceinline__ void gating_writeout(const Shape &sh, int B, const Wo
 template <int JE>
 __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
                                              int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
-                                             int32_t *__restrict__ n_unique, double *s_l)
+                                             int32_t *__restrict__ n_unique, double *s_l, int ksplit, const double *__restrict__ lpart)
 {
     __shared__ unsigned long long s_mask[kMaxExperts], s_gk[kMaxExperts];
     __shared__ double s_lam[kMaxTokens], s_zmax[kMaxTokens], s_den[kMaxTokens];
@@ -134,8 +134,26 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     gm.topk = reinterpret_cast<unsigned *>(s_sel);      // (the selection overwrites it: nobody reads it here)
     const GateGroup gg{(int)threadIdx.x, (int)blockDim.x, 0};
     double *s_w = s_l + B * sh.E;
+    if (ksplit > 0) {
+        // the pieces of a row added in ascending order (all loads first); the sums go back to the
+        // workspace, where the write-out (gate logits) and debug reads find them
+        const int n_rows = sh.E + has_gate;
 #pragma unroll 1
-    for (int i = gg.t; i < B * sh.E; i += gg.n) s_l[i] = __ldcg(&ws.logits[i]);
+        for (int i = gg.t; i < B * n_rows; i += gg.n) {
+            const int b = i / n_rows, r = i - b * n_rows;
+            double v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = q < ksplit ? __ldcg(&lpart[((size_t)q * B + b) * n_rows + r]) : 0.0;
+            double acc = v[0];
+#pragma unroll
+            for (int q = 1; q < 8; ++q) acc += v[q];
+            if (r < sh.E) { s_l[b * sh.E + r] = acc; ws.logits[b * sh.E + r] = acc; }
+            else ws.gate_logit[b] = acc;
+        }
+    } else {
+#pragma unroll 1
+        for (int i = gg.t; i < B * sh.E; i += gg.n) s_l[i] = __ldcg(&ws.logits[i]);
+    }
 #pragma unroll 1
     for (int b = gg.t; b < B; b += gg.n) s_w[b] = conf ? (double)conf[b] : 1.0;
     // (gating_group's first barrier orders these writes before the first read)
@@ -144,6 +162,12 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     gating_writeout(sh, B, ws, gm, has_gate, n_unique, gg);
 }
 
+constexpr int kRouteThreads = 512;
+constexpr int kRouteThreadsBig = 1024;
+constexpr int kRouteTok = 16;   // most tokens accumulated per pass
+
+// Buffers that the layer's later kernels accumulate into and that must start at zero; the
+// routing blocks clear them (16-byte units) so that no separate fill precedes the layer.
 // 4 consecutive elements of a plain (f32 / bf16) row starting at column c (c % 4 == 0)
 template <int DT>
 __device__ __forceinline__ void load4_plain(const void *row, int c, float (&v)[4])
@@ -157,11 +181,6 @@ __device__ __forceinline__ void load4_plain(const void *row, int c, float (&v)[4
     }
 }
 
-constexpr int kRouteThreads = 512;
-constexpr int kRouteTok = 16;   // most tokens accumulated per pass
-
-// Buffers that the layer's later kernels accumulate into and that must start at zero; the
-// routing blocks clear them (16-byte units) so that no separate fill precedes the layer.
 // two bf16 values -> two binary16 values (round to nearest; exact for magnitudes in [2^-14, 65504])
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t u)
 {
@@ -181,7 +200,54 @@ struct ZeroList {
     // logit pass: the tokens of a batch are split into this many groups, each with its own set of
     // row blocks (0 and 1: every row block takes all tokens)
     int groups;
+    // logit pass by warp tasks (larger batches): ksplit > 0 pieces of the contraction per router row,
+    // partial sums in lpart [piece][token][row] (see route_logit_tasks); 0: by row blocks
+    int ksplit;
+    double *lpart;
 };
+
+// Router logits by the warps of the whole grid: a task is one router row (row E: the shared
+// experts' gate vector) x 8 tokens x one piece of the contraction, float64 accumulation; its
+// partial sums go to lpart[piece][token][row], which the gating adds up in a fixed order.
+template <int ACT, int RT>
+__device__ __forceinline__ void route_logit_tasks(const Shape &sh, int B, const void *__restrict__ hidden,
+                                                  const void *__restrict__ router, const void *__restrict__ sh_scale,
+                                                  double *__restrict__ lpart, int ksplit, int gwarp, int n_gwarps, int lane)
+{
+    const int d = sh.d, n_rows = sh.E + (sh_scale ? 1 : 0), n_tg = (B + 7) >> 3;
+    const int len = ((d + 4 * ksplit - 1) / (4 * ksplit)) * 4;              // columns of a piece, a multiple of 4
+    const int n_tasks = n_rows * n_tg * ksplit;
+    const size_t rb = RT == DT_F32 ? 4 : 2, ab = ACT == DT_F32 ? 4 : 2;
+#pragma unroll 1
+    for (int task = gwarp; task < n_tasks; task += n_gwarps) {
+        const int row = task % n_rows, rest = task / n_rows, tg = rest % n_tg, piece = rest / n_tg;
+        const int c0 = piece * len, c1 = min(d, c0 + len), b0 = tg * 8;
+        const uint8_t *wrow = row < sh.E ? reinterpret_cast<const uint8_t *>(router) + (size_t)row * d * rb
+                                         : reinterpret_cast<const uint8_t *>(sh_scale);
+        double acc[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) acc[t] = 0.0;
+#pragma unroll 2
+        for (int c = c0 + lane * 4; c < c1; c += 128) {
+            float w[4], x[8][4];
+            load4_plain<RT>(wrow, c, w);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const int bt = min(b0 + t, B - 1);           // past the batch: the last token again (not stored)
+                load4_plain<ACT>(reinterpret_cast<const uint8_t *>(hidden) + (size_t)bt * d * ab, c, x[t]);
+            }
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[t] = fma((double)w[i], (double)x[t][i], acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const double v = warp_sum(acc[t]);
+            if (lane == t && b0 + t < B) lpart[((size_t)piece * B + b0 + t) * n_rows + row] = v;
+        }
+    }
+}
 
 // One pass of a router row over NT tokens b0 .. b0 + NT - 1 (indices past B - 1 repeat token
 // B - 1, so that every load is unconditional and issued before the first use).
@@ -229,11 +295,12 @@ __device__ __forceinline__ void route_pass(const Shape &sh, int B, int b0, const
 // Dynamic shared memory: max(B * E + B, 16 * kRouteTok) doubles.
 // JE: experts per lane in the gating (2, 4 or 8 for up to 64, 128, 256 experts): a kernel of its own
 // for each, so that the gating code of a launch is one straight piece
-template <int ACT, int RT, int JE>
-__global__ void __launch_bounds__(kRouteThreads)
-route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
-             const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
-             float *__restrict__ sel_w, int32_t *__restrict__ n_unique, ZeroList zl)
+// THREADS: kRouteThreads, or kRouteThreadsBig for the kernel of the larger batches (warp tasks only)
+template <int ACT, int RT, int JE, int THREADS>
+__device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspace &ws, const void *__restrict__ hidden,
+                                           const void *__restrict__ router, const void *__restrict__ sh_scale,
+                                           const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
+                                           float *__restrict__ sel_w, int32_t *__restrict__ n_unique, const ZeroList &zl)
 {
     extern __shared__ double s_dyn[];
     __shared__ int s_last;
@@ -250,12 +317,12 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
 #pragma unroll
     for (int z = 0; z < 3; ++z) {
         uint4 *p = reinterpret_cast<uint4 *>(zl.ptr[z]);
-        for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.n16[z];
-             i += (unsigned long long)gridDim.x * kRouteThreads)
+        for (unsigned long long i = (unsigned long long)blockIdx.x * THREADS + tid; i < zl.n16[z];
+             i += (unsigned long long)gridDim.x * THREADS)
             p[i] = make_uint4(0u, 0u, 0u, 0u);
     }
-    for (unsigned long long i = (unsigned long long)blockIdx.x * kRouteThreads + tid; i < zl.perm_n16;
-         i += (unsigned long long)gridDim.x * kRouteThreads) {
+    for (unsigned long long i = (unsigned long long)blockIdx.x * THREADS + tid; i < zl.perm_n16;
+         i += (unsigned long long)gridDim.x * THREADS) {
         const uint4 v = zl.perm_src[i];             // halves h0..h7 (bf16)
         zl.perm_dst[i] = make_uint4(bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.x, v.z, 0x7632)),
                                     bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x5410)), bf16x2_to_f16x2(__byte_perm(v.y, v.w, 0x7632)));
@@ -266,7 +333,17 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     // several sets of row blocks (as many as fit on the SMs beside each other), because a block
     // takes 16 tokens per pass and its passes run one after the other (B = 64: 22 us in one set).
     const int n_rows = sh.E + (sh_scale ? 1 : 0);
-    const int n_grp = zl.groups > 1 ? zl.groups : 1, n_arrive = n_rows * n_grp;
+    int n_arrive = 0;
+    if (zl.ksplit > 0) {
+        // larger batches: the logit pass as warp tasks over all blocks of the grid (a row block takes
+        // 16 tokens per pass and its passes run one after the other: 22 us at 64 tokens)
+        n_arrive = (int)gridDim.x;
+        route_logit_tasks<ACT, RT>(sh, B, hidden, router, sh_scale, zl.lpart, zl.ksplit, (tid >> 5) * (int)gridDim.x + (int)blockIdx.x,
+                                   (THREADS / 32) * (int)gridDim.x, tid & 31);
+        __syncthreads();
+    } else if constexpr (THREADS == kRouteThreads) {
+    const int n_grp = zl.groups > 1 ? zl.groups : 1;
+    n_arrive = n_rows * n_grp;
     if ((int)blockIdx.x >= n_arrive) return;
     const int row = (int)blockIdx.x % n_rows, grp = (int)blockIdx.x / n_rows, d = sh.d;
     const int tg = 4 * ((B + 4 * n_grp - 1) / (4 * n_grp));            // tokens per group, a multiple of 4
@@ -279,6 +356,7 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
         if (left > 8) { route_pass<ACT, RT, 16>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 16; }
         else if (left > 4) { route_pass<ACT, RT, 8>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 8; }
         else { route_pass<ACT, RT, 4>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 4; }
+    }
     }
     // Block 0 runs the gating once every row has arrived (its SM tends to be the same from layer
     // to layer, so part of the gating code is still in its instruction cache: measured 0.6 % of
@@ -314,7 +392,27 @@ route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, con
     }
     __syncthreads();
     if (!s_last) return;
-    gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn);
+    gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn, zl.ksplit, zl.lpart);
+}
+
+template <int ACT, int RT, int JE>
+__global__ void __launch_bounds__(kRouteThreads)
+route_kernel(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
+             const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
+             float *__restrict__ sel_w, int32_t *__restrict__ n_unique, ZeroList zl)
+{
+    route_body<ACT, RT, JE, kRouteThreads>(sh, B, ws, hidden, router, sh_scale, conf, sel_idx, sel_w, n_unique, zl);
+}
+
+// The same with twice the warps, for the larger batches (logit pass by warp tasks only): the gating
+// takes one warp per token, and at 64 tokens four passes of 16 warps were most of the kernel.
+template <int ACT, int RT, int JE>
+__global__ void __launch_bounds__(kRouteThreadsBig)
+route_kernel_big(Shape sh, int B, Workspace ws, const void *__restrict__ hidden, const void *__restrict__ router,
+                 const void *__restrict__ sh_scale, const float *__restrict__ conf, int32_t *__restrict__ sel_idx,
+                 float *__restrict__ sel_w, int32_t *__restrict__ n_unique, ZeroList zl)
+{
+    route_body<ACT, RT, JE, kRouteThreadsBig>(sh, B, ws, hidden, router, sh_scale, conf, sel_idx, sel_w, n_unique, zl);
 }
 
 }  // namespace s2moe

@@ -42,7 +42,8 @@ struct s2moe_ctx {
     bool use_pdl = true;                  // S2MOE_NO_PDL=1 in the environment turns it off
     bool pdl_in_graph = false;            // S2MOE_PDL_IN_GRAPH=1: also under stream capture
     void *hperm = nullptr;                // int4 plan 3: column-permuted copy of the hidden states
-    double *lpart = nullptr;              // fused layer kernel: partial router logits [piece][token][row]
+    double *lpart = nullptr;              // partial router logits [piece][token][row] (logit pass by warp tasks)
+    int route_task_from = 48;             // batches of this many tokens and more take the logit pass by warp tasks
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
@@ -210,17 +211,50 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
     // experts: 1.1 % of a layer at B = 8, 4.5 % at B = 16
     ZeroList zg = zl;
     zg.groups = 1;
+    zg.ksplit = 0;
+    zg.lpart = nullptr;
+    int grid;
+    const int task_from = ctx->route_task_from;
+    if (ctx->lpart && B >= task_from) {
+        // the logit pass as warp tasks: pieces of the contraction so that the warps of a full grid
+        // have about one task each
+        const int tgs = (B + 7) / 8, warps = ctx->n_sm * (kRouteThreadsBig / 32);
+        int ks = warps / (rows * tgs);
+        if (ks > 8) ks = 8;
+        if (ks > sh.d / 128) ks = sh.d / 128;
+        zg.ksplit = ks < 1 ? 1 : ks;
+        zg.lpart = ctx->lpart;
+        const int tasks = rows * tgs * zg.ksplit, blocks = (tasks + kRouteThreadsBig / 32 - 1) / (kRouteThreadsBig / 32);
+        grid = blocks < ctx->n_sm ? blocks : ctx->n_sm;
+        // more blocks (up to one per SM) when there is a lot to clear or copy
+        const unsigned long long want = (units + kRouteThreadsBig * 4 - 1) / (kRouteThreadsBig * 4);
+        if (want > (unsigned long long)grid) grid = (int)(want > (unsigned long long)ctx->n_sm ? (unsigned long long)ctx->n_sm : want);
+    } else {
     if (B > 4) {
         const int fit = ctx->n_sm / rows, want = (B + 3) / 4;
         zg.groups = fit < 1 ? 1 : (want < fit ? want : fit);
     }
-    int grid = rows * zg.groups;
+    grid = rows * zg.groups;
     if (units > (unsigned long long)rows * kRouteThreads * 4) {
         const unsigned long long want = (units + kRouteThreads * 4 - 1) / (kRouteThreads * 4);
         grid = (int)(want > (unsigned long long)ctx->n_sm ? (unsigned long long)ctx->n_sm : want);
         if (grid < rows * zg.groups) grid = rows * zg.groups;
     }
+    }
     LaunchScope scope(ctx, KC_ROUTER, st);
+    if (zg.ksplit > 0) {
+        cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreadsBig, route_smem(B, sh.E), st);
+        if (sh.E <= 64)
+            cudaLaunchKernelEx(&lc, route_kernel_big<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                               (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
+        else if (sh.E <= 128)
+            cudaLaunchKernelEx(&lc, route_kernel_big<ACT, RT, 4>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                               (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
+        else
+            cudaLaunchKernelEx(&lc, route_kernel_big<ACT, RT, 8>, sh, B, ctx->ws, hidden, (const void *)lp.router,
+                               (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
+        return;
+    }
     cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st);
     if (sh.E <= 64)
         cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
@@ -249,6 +283,9 @@ cudaError_t prepare_route_t(int bytes)
     cudaError_t e = cudaFuncSetAttribute(route_kernel<ACT, RT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<ACT, RT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel<ACT, RT, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel_big<ACT, RT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel_big<ACT, RT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(route_kernel_big<ACT, RT, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e;
 }
 
@@ -652,6 +689,8 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     {
         const char *no_pdl = std::getenv("S2MOE_NO_PDL");
         ctx->use_pdl = !(no_pdl && no_pdl[0] == '1');
+        const char *tf = std::getenv("S2MOE_ROUTE_TASKS_FROM");
+        if (tf && tf[0]) ctx->route_task_from = std::atoi(tf);
         const char *pg = std::getenv("S2MOE_PDL_IN_GRAPH");
         ctx->pdl_in_graph = pg && pg[0] == '1';
     }
