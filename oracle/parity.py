@@ -112,10 +112,13 @@ def check_layer(cfg: Config, w: Weights, hidden_raw: np.ndarray, conf: Optional[
 
 
 def check_bucketing(lists: dict, sel: np.ndarray, w: np.ndarray, n_experts: int, n_shared: int) -> None:
-    """Host-side validation of the bucketing arrays a layer call produced: offsets
-    are the exclusive scan of counts, every (token, choice) pair appears exactly once
-    under its expert with its mixing weight, tokens ascend inside an expert, and the
-    active list holds exactly the experts that have tokens."""
+    """Host-side validation of the bucketing arrays a layer call produced: the active
+    list holds exactly the groups that have tokens, the routed ones before the shared
+    ones (the order among the routed ones is the kernel's choice: not unique, so only
+    its validity is checked); walking that list, the groups' slot ranges follow each
+    other without gap or overlap from slot 0 on; every (token, choice) pair appears
+    exactly once under its expert with its mixing weight, and tokens ascend inside an
+    expert."""
     B, k = sel.shape
     counts = np.asarray(lists["counts"]); offsets = np.asarray(lists["offsets"])
     slot_token = np.asarray(lists["slot_token"]); slot_w = np.asarray(lists["slot_w"])
@@ -123,15 +126,22 @@ def check_bucketing(lists: dict, sel: np.ndarray, w: np.ndarray, n_experts: int,
     G = n_experts + n_shared
     assert lists["B"] == B and lists["n_slots"] == B * k + n_shared * B
     assert counts.shape[0] == G and offsets.shape[0] == G + 1
-    assert offsets[0] == 0 and np.array_equal(np.diff(offsets), counts)
     assert counts[:n_experts].sum() == B * k and np.all(counts[n_experts:] == B)
     assert lists["U"] == int((counts[:n_experts] > 0).sum())
-    assert active.tolist() == [g for g in range(G) if counts[g] > 0]
+    assert sorted(active.tolist()) == [g for g in range(G) if counts[g] > 0]
+    assert len(set(active.tolist())) == len(active)
+    routed = [g for g in active.tolist() if g < n_experts]
+    assert active.tolist() == routed + list(range(n_experts, G)), "shared groups close the active list, ascending"
+    at = 0
+    for g in active.tolist():
+        assert offsets[g] == at, f"group {g} starts at slot {offsets[g]}, expected {at}"
+        at += int(counts[g])
+    assert at == lists["n_slots"] and offsets[G] == at
     seen = set()
     for e in range(n_experts):
-        toks = slot_token[offsets[e]:offsets[e + 1]]
+        toks = slot_token[offsets[e]:offsets[e] + counts[e]]
         assert np.all(np.diff(toks) > 0), "tokens must ascend inside an expert"
-        for pos, b in zip(range(offsets[e], offsets[e + 1]), toks):
+        for pos, b in zip(range(offsets[e], offsets[e] + counts[e]), toks):
             j = np.nonzero(sel[b] == e)[0]
             assert len(j) == 1, f"slot {pos}: token {b} did not select expert {e}"
             assert slot_w[pos] == w[b, j[0]]
@@ -139,7 +149,7 @@ def check_bucketing(lists: dict, sel: np.ndarray, w: np.ndarray, n_experts: int,
     assert len(seen) == B * k
     for s in range(n_shared):
         g = n_experts + s
-        assert slot_token[offsets[g]:offsets[g + 1]].tolist() == list(range(B))
+        assert slot_token[offsets[g]:offsets[g] + counts[g]].tolist() == list(range(B))
 
 
 def from_workload(wl, tensors: dict):

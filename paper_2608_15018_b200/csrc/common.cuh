@@ -18,7 +18,7 @@ constexpr int kMaxShared = 4;
 enum : int { DT_F32 = 0, DT_BF16 = 1, DT_Q4B32 = 2 };
 
 // device status codes (non-zero: a bounded wait gave up)
-enum : int { ST_OK = 0, ST_MBAR_TIMEOUT = 1, ST_DEP_TIMEOUT = 2, ST_TICKET_TIMEOUT = 3 };
+enum : int { ST_OK = 0, ST_MBAR_TIMEOUT = 1, ST_DEP_TIMEOUT = 2, ST_TICKET_TIMEOUT = 3, ST_BAD_PLAN = 4 };
 
 struct LayerPtrs {
     const void *router;
@@ -61,6 +61,8 @@ struct Workspace {
     unsigned long long *tokmask;   // [E + n_sh] bit b set: token b is bucketed to the group
     uint4 *gtab;           // [n_active][2] {group, tokens, first slot, 0}, {mask lo, mask hi, 0, 0}: the
                            // active groups in their final form, or NULL when nobody reads it
+    int32_t *early;        // {flag, n, ids ...}: the experts whose first projection may start before the gating
+                           // has ended, published by the routing kernel (see gating_block), or NULL
     const int32_t *slot_of;  // [E] device slot that holds each routed expert's weights (expert offloading), or
                              // NULL: every expert is resident at its own index
 };

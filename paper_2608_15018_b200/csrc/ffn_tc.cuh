@@ -61,6 +61,7 @@ constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 K
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
 constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
 constexpr unsigned kTcSpinLimit = 1u << 22;
+constexpr int kTcMaxAcc = 8;                   // accumulator buffers in tensor memory (2 without the early start)
 constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
 // Share of the experts in wave 0.  A little more than half: the second projection of wave 0 is
 // what hides the hand-over of wave 1.  Measured again with the kernel as it stands, 16 layers of
@@ -99,6 +100,9 @@ struct TcPlan {
     int tok_off;       // offset of the token tiles inside a stage
     int kg;            // k-tiles per stage (1 for bf16 weights; 1, 2 or 4 for int4)
     int tokb;          // bytes of the token tiles of one k-tile
+    int rows1;         // rows of one hidden-state copy (bf16, one k-tile per stage)
+    int n_acc;         // accumulator buffers (a power of two; more than 2 only with the early start)
+    int early;         // the early start is possible for this shape (bf16 weights, units fit the table)
 };
 
 struct TcArgs {
@@ -109,9 +113,15 @@ struct TcArgs {
     float *pre;                       // [gate|up][slot][f_g] fp32 pre-activations (zeroed by the routing kernel)
     __nv_bfloat16 *act_hi, *act_lo;   // [slot][f_g]
     int B;
+    int early;                        // 1: early start (see the kernel)
 };
 
-inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
+// units of a group: phase 1 = 2 matrices x row blocks x k-pieces, phase 2 = row blocks x k-pieces
+__host__ __device__ __forceinline__ int tc_kpieces(int K) { return ((K + 63) / 64 + kTcKT - 1) / kTcKT; }
+__host__ __device__ __forceinline__ int tc_units1(int f_g, int d) { return 2 * ((f_g + 127) / 128) * tc_kpieces(d); }
+__host__ __device__ __forceinline__ int tc_units2(int f_g, int d) { return ((d + 127) / 128) * tc_kpieces(f_g); }
+
+inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, int bf16_kg = 2, bool early = false)
 {
     TcPlan p{};
     const int G = sh.E + sh.n_sh;
@@ -121,7 +131,7 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     // (1 KiB) and right behind them their lo rows (a group never has more tokens than B)
     p.stage_bytes = kTcWTile + 2048 * ((B + 7) / 8);
     p.stage_bytes = (p.stage_bytes + 1023) & ~1023;
-    p.tab_bytes = ((int)sizeof(TcGroup) * (G + 1) + 8 * n_slots + 1023) & ~1023;
+    p.tab_bytes = ((int)sizeof(TcGroup) * (G + 1 + sh.n_sh) + 8 * n_slots + 1023) & ~1023;
     // The ring is what keeps HBM busy (bytes in flight = stages x 16 KiB per SM, against a loaded
     // latency of 2-3 us), so shared memory goes to stages first: the hidden-state tiles stay
     // resident only if the ring reaches its maximum depth anyway, otherwise every stage fetches
@@ -137,7 +147,50 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     p.tok_off = kTcWTile;
     p.kg = 1;
     p.tokb = 2048 * ((B + 7) / 8);
-    p.feasible = p.stages >= 4 && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
+    p.rows1 = p.n1;    // the hidden-state k-tile of a stage in ONE copy (the producer is a single thread)
+    // bf16 weights: TWO k-tiles per ring stage where every contraction length is a multiple of 64
+    // (one weight copy of 32 KiB and one token copy per stage, one barrier round trip and five
+    // instead of six tensor-core instructions per issuer and 32 KiB): the producer and the MMA
+    // issuers are single threads, every instruction of theirs costs tens of cycles, and at
+    // 6 TB/s a 16 KiB k-tile has to leave an SM every 400 ns
+    if (bf16_kg == 2 && sh.weight_dtype == DT_BF16 && sh.d % 64 == 0 && sh.f % 64 == 0 && (sh.n_sh == 0 || sh.f_sh % 64 == 0)) {
+        p.kg = 2;
+        p.x_bytes = 0;
+        p.stage_bytes = (2 * kTcWTile + 2 * p.tokb + 1023) & ~1023;
+        p.tok_off = 2 * kTcWTile;
+        p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
+        if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
+        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + 1024;
+        if (p.stages < 3) {          // (large batches: back to one k-tile per stage)
+            p.kg = 1;
+            p.stage_bytes = (kTcWTile + p.tokb + 1023) & ~1023;
+            p.tok_off = kTcWTile;
+            p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
+            if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
+            p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + 1024;
+        }
+    }
+    p.n_acc = 2;
+    p.early = 0;
+    if (early && sh.weight_dtype == DT_BF16 && n_sm > 1) {
+        // Early start (see the kernel): one CTA less than SMs, because the SM that runs the gating is
+        // taken until the routing kernel ends and its CTA would start last with a full share; as many
+        // accumulators as tensor memory holds (the reductions of an early expert wait for the
+        // tables); and only where a CTA's units are sure to fit the table in shared memory.
+        const int P = n_sm - 1;
+        const long long worst = (long long)sh.E * (tc_units1(sh.f, sh.d) + tc_units2(sh.f, sh.d)) +
+                                (long long)sh.n_sh * (tc_units1(sh.f_sh, sh.d) + tc_units2(sh.f_sh, sh.d));
+        if (worst / P + 12 <= kTcMaxUnits) {
+            p.early = 1;
+            p.n_cta = P;
+            int nb = 8;
+            while (nb > 2 && nb * 4 * p.n1 > 512) nb >>= 1;
+            p.n_acc = nb;
+            p.tmem_cols = 32;
+            while (p.tmem_cols < nb * 4 * p.n1) p.tmem_cols <<= 1;
+        }
+    }
+    p.feasible = p.stages >= (p.kg == 2 ? 3 : 4) && B <= kMaxTokens && sh.weight_dtype == DT_BF16 && sh.act_dtype == DT_BF16 &&
                  sh.d % 64 == 0;
     if (sh.weight_dtype == DT_Q4B32) {
         // a stage holds the packed k-tiles and their unit's scales; the TMA copy of the scales
@@ -170,10 +223,6 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots)
     return p;
 }
 
-// units of a group: phase 1 = 2 matrices x row blocks x k-pieces, phase 2 = row blocks x k-pieces
-__host__ __device__ __forceinline__ int tc_kpieces(int K) { return ((K + 63) / 64 + kTcKT - 1) / kTcKT; }
-__host__ __device__ __forceinline__ int tc_units1(int f_g, int d) { return 2 * ((f_g + 127) / 128) * tc_kpieces(d); }
-__host__ __device__ __forceinline__ int tc_units2(int f_g, int d) { return ((d + 127) / 128) * tc_kpieces(f_g); }
 
 // ---- PTX helpers (tcgen05, TMA tensor copies) ------------------------------------------
 
@@ -199,6 +248,15 @@ __device__ __forceinline__ void tma_load_2d_stream(void *dst, const CUtensorMap 
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%3, %4}], [%2], %5;"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_stream(void *dst, const CUtensorMap *map, int x, int y, int z, uint64_t *bar,
+                                                   uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, uint64_t *bar)
@@ -425,13 +483,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2], ep_bar, x_bar, cv_bar, conv_go[2];
+    __shared__ __align__(8) uint64_t acc_full[kTcMaxAcc], acc_empty[kTcMaxAcc], ep_bar, x_bar, cv_bar, conv_go[2], tab_bar;
     __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
     __shared__ uint32_t s_umeta[kTcMaxUnits];      // what an MMA issuer needs of a unit, in one word (tc_unit_meta)
     __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
+    __shared__ int s_tab[2];                       // early start: units of the routed work of this CTA, active groups
     __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
 
     const Shape &sh = p.sh;
@@ -440,81 +499,19 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     const int NI = Q4 ? p.plan.n_iss : 2;          // MMA issuers: a compile-time 2 on the bf16 path
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // programmatic dependent launch: the routing kernel in front of this grid must have
-    // finished before its results are read; the next layer's routing kernel may be scheduled
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int n_active = ws.header[0];
-    const int n_slots = p.B * sh.k + sh.n_sh * p.B;          // every token fills k routed slots
-    const int G = sh.E + sh.n_sh;
-
-    TcGroup *groups = reinterpret_cast<TcGroup *>(tc_smem);
-    const int tab_rest = pl.tab_bytes - (int)sizeof(TcGroup) * (G + 1);
-    int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(TcGroup) * (G + 1));
-    float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
-    uint8_t *xres = tc_smem + pl.tab_bytes;
-    xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
-    uint8_t *ring = xres + pl.x_bytes;
-    uint8_t *tokring = ring + (size_t)pl.stages * pl.stage_bytes;    // int4 only: token tiles, one slot per slot of dequantised tiles
-
-    // group table; stage prefixes follow from the active list alone (routed groups first)
-    const int U = ws.header[2];
-    const int u1r = tc_units1(sh.f, sh.d), u2r = tc_units2(sh.f, sh.d);
-    const int u1s = sh.n_sh ? tc_units1(sh.f_sh, sh.d) : 0, u2s = sh.n_sh ? tc_units2(sh.f_sh, sh.d) : 0;
-    // one round of global loads: the header above, the group table in its final form and the
-    // slot arrays, whose sizes are known without the header
-    for (int a = tid; a < G; a += blockDim.x) {
-        const uint4 r0 = ws.gtab[2 * a], r1 = ws.gtab[2 * a + 1];
-        if (a < n_active) {
-            TcGroup gr;
-            gr.group = (int)r0.x;
-            // offloaded experts: from here on the group id of a routed expert is the device slot its
-            // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
-            if (ws.slot_of && gr.group < sh.E) gr.group = __ldg(&ws.slot_of[gr.group]);
-            gr.T = (int)r0.y;
-            gr.off = (int)r0.z;
-            gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
-            gr.mask = (unsigned long long)r1.x | ((unsigned long long)r1.y << 32);
-            const int r = a < U ? a : U, s = a < U ? 0 : a - U;
-            gr.p1 = r * u1r + s * u1s;
-            gr.p2 = r * u2r + s * u2s;
-            groups[a] = gr;
-        }
-    }
-    for (int i = tid; i < n_slots; i += blockDim.x) {
-        s_slot_token[i] = ws.slot_token[i];
-        s_slot_w[i] = ws.slot_w[i];
-    }
-    const int total1 = U * u1r + sh.n_sh * u1s, total2 = U * u2r + sh.n_sh * u2s;
-    const int total = total1 + total2;
-    const int S = pl.stages;
-    const int P = gridDim.x;
-    if (tid == 0) {
-        // wave 1 starts at the first group whose phase-1 units begin at or after that share
-        int sp = n_active;
-        if (n_active >= 2) {
-            sp = 1;
-            while (sp < n_active - 1) {
-                const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
-                if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)total1 * kTcSplitNum) break;
-                ++sp;
-            }
-        }
-        s_split = sp;
-        s_ready[0] = 0;
-        s_ready[1] = 0;
-    }
+    // Set-up that needs nothing of the routing kernel comes first: this grid is launched
+    // programmatically, so its CTAs may become resident while the routing kernel still runs
     if (warp == 2) {
         // barrier set-up, spread over a warp so that it runs beside the table loads of the others
         if (lane < pl.stages) {
             mbar_init(&full_bar[lane], 1);
             mbar_init(&empty_bar[lane], Q4 ? kTcQ4DeqWarps : NI);   // one commit from each MMA issuer; int4: the dequantising warps
         }
-        if (lane < 2) {
+        if (lane < kTcMaxAcc) {
             mbar_init(&acc_full[lane], NI);
             mbar_init(&acc_empty[lane], 4);
-            mbar_init(&conv_go[lane], 4);
         }
+        if (lane < 2) mbar_init(&conv_go[lane], 4);
         if (Q4 && lane < pl.a_stages) {
             mbar_init(&a_full[lane], kTcQ4DeqWarps + 1);   // the dequantising warps and the producer's arrival with the token bytes
             mbar_init(&a_empty[lane], NI);
@@ -523,6 +520,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             mbar_init(&ep_bar, 4);
             mbar_init(&x_bar, 1);
             mbar_init(&cv_bar, 3);
+            mbar_init(&tab_bar, 1);
+            s_ready[0] = 0;
+            s_ready[1] = 0;
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -533,20 +533,31 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = s_tmem;
-    const int a_split = s_split;
-    const int W = a_split < n_active ? 2 : 1;
-    // Four segments in time order: phase 1 of wave 0, of wave 1, phase 2 of wave 0, of wave 1.
-    // Every CTA takes one contiguous run of units of each segment (sizes differ by at most one;
-    // the CTAs that get the extra unit rotate from segment to segment, so the totals differ by at
-    // most one as well).  Contiguous units are consecutive k-pieces of one 128-row block, so a CTA
-    // accumulates them in one TMEM accumulator and the epilogue runs once per run of k-pieces
-    // instead of once per unit; only row blocks cut by a CTA boundary are reduced from two CTAs.
-    const int split1 = W == 2 ? groups[a_split].p1 : total1;
-    const int split2 = W == 2 ? groups[a_split].p2 : total2;
+    // Early start (bf16 weights, see tc_make_plan): this grid does not wait for the routing kernel
+    // as a whole.  The routing kernel publishes, before its gating, the experts that are certain
+    // to be selected; their first projection and that of the shared experts (the "pre-lot") is
+    // streamed while the gating runs.  Warps 7..10, idle until the first hand-over, wait for the
+    // routing kernel to end, build the tables of everything else and open tab_bar; the other
+    // roles pass that barrier when they have worked off their share of the pre-lot.
+    const bool EARLY = !Q4 && p.early != 0;
+    const int n_slots = p.B * sh.k + sh.n_sh * p.B;          // every token fills k routed slots
+    const int G = sh.E + sh.n_sh;
+    const int GP = G + 1;                                    // early start: provisional groups of the shared experts
+
+    TcGroup *groups = reinterpret_cast<TcGroup *>(tc_smem);
+    const int n_tab_groups = G + 1 + sh.n_sh;
+    const int tab_rest = pl.tab_bytes - (int)sizeof(TcGroup) * n_tab_groups;
+    int *s_slot_token = reinterpret_cast<int *>(tc_smem + sizeof(TcGroup) * n_tab_groups);
+    float *s_slot_w = reinterpret_cast<float *>(s_slot_token + tab_rest / 8);
+    uint8_t *xres = tc_smem + pl.tab_bytes;
+    xres = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(xres) + 1023) & ~(uintptr_t)1023);
+    uint8_t *ring = xres + pl.x_bytes;
+    uint8_t *tokring = ring + (size_t)pl.stages * pl.stage_bytes;    // int4 only: token tiles, one slot per slot of dequantised tiles
+
+    const int u1r = tc_units1(sh.f, sh.d), u2r = tc_units2(sh.f, sh.d);
+    const int u1s = sh.n_sh ? tc_units1(sh.f_sh, sh.d) : 0, u2s = sh.n_sh ? tc_units2(sh.f_sh, sh.d) : 0;
+    const int S = pl.stages;
+    const int P = gridDim.x;
     // Where every unit of a projection has all its four k-tiles (contraction length a multiple of
     // 256) the segments are dealt in half units, so that the CTAs of a segment differ by two
     // k-tiles (0.75 us) instead of four: a share may then begin with the second half of a unit
@@ -555,29 +566,106 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     // The int4 path needs whole units.
     const bool halves1 = !Q4 && sh.d % 256 == 0;
     const bool halves2 = !Q4 && sh.f % 256 == 0 && (sh.n_sh == 0 || sh.f_sh % 256 == 0);
-    int my_start0, my_start1, my_start2, my_start3, my_cnt0, my_cnt1, my_cnt2, my_cnt3;
-    int my_trim0, my_trim1, my_trim2, my_trim3;
-    {
-        int rot = 0;
-        auto share = [&](int begin, int n, bool halves, int &start, int &cnt, int &trim) {
-            const int m = halves ? 2 : 1, n2 = n * m;
-            const int q = n2 / P, r = n2 - q * P;
-            int c = (int)blockIdx.x - rot;               // (blockIdx.x - rot) mod P without a division:
-            if (c < 0) c += P;                           // the four calls would otherwise chain four of them
-            const int cnt2 = q + (c < r ? 1 : 0), start2 = c * q + min(c, r);
-            const int u0 = halves ? start2 >> 1 : start2, u1 = halves ? (start2 + cnt2 - 1) >> 1 : start2 + cnt2 - 1;
-            cnt = cnt2 > 0 ? u1 - u0 + 1 : 0;
-            start = begin + u0;
-            trim = (halves && cnt2 > 0) ? ((start2 & 1) | (((start2 + cnt2) & 1) << 1)) : 0;
-            rot += r;
-            if (rot >= P) rot -= P;
-        };
-        share(0, split1, halves1, my_start0, my_cnt0, my_trim0);
-        share(split1, total1 - split1, halves1, my_start1, my_cnt1, my_trim1);
-        share(total1, split2, halves2, my_start2, my_cnt2, my_trim2);
-        share(total1 + split2, total2 - split2, halves2, my_start3, my_cnt3, my_trim3);
+    // Every CTA takes one contiguous run of units of each segment (sizes differ by at most one;
+    // the CTAs that get the extra unit rotate from segment to segment, so the totals differ by at
+    // most one as well).
+    int rot = 0;
+    auto share = [&](int begin, int n, bool halves, int &start, int &cnt, int &trim) {
+        const int m = halves ? 2 : 1, n2 = n * m;
+        const int q = n2 / P, r = n2 - q * P;
+        int c = (int)blockIdx.x - rot;               // (blockIdx.x - rot) mod P without a division:
+        if (c < 0) c += P;                           // the calls would otherwise chain as many of them
+        const int cnt2 = q + (c < r ? 1 : 0), start2 = c * q + min(c, r);
+        const int u0 = halves ? start2 >> 1 : start2, u1 = halves ? (start2 + cnt2 - 1) >> 1 : start2 + cnt2 - 1;
+        cnt = cnt2 > 0 ? u1 - u0 + 1 : 0;
+        start = begin + u0;
+        trim = (halves && cnt2 > 0) ? ((start2 & 1) | (((start2 + cnt2) & 1) << 1)) : 0;
+        rot += r;
+        if (rot >= P) rot -= P;
+    };
+
+    // ---- the pre-lot (early start only)
+    int n_early = 0, n_pre = 0, pre_start = 0, pre_trim = 0;
+    if (EARLY) {
+        if (tid == 0) {
+            // bounded wait for the routing kernel's list (a release store behind everything that
+            // kernel clears; all its blocks are resident or done when this grid is scheduled)
+            int ok = 0;
+            for (unsigned i = 0; i < (1u << 21) && !ok; ++i) {
+                if (ld_acquire(ws.early) == 1) ok = 1;
+                else __nanosleep(40);
+            }
+            if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+            s_flag = ok;
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        n_early = s_flag ? __ldcg(ws.early + 1) : 0;
+        n_early = max(0, min(n_early, min(p.B, sh.E)));
+        const unsigned long long all = p.B >= 64 ? ~0ull : ((1ull << p.B) - 1ull);
+        // provisional groups: a shared expert's is complete (every token, slots known); an early
+        // routed expert's sits where its final entry will be (the early experts lead the active
+        // list in this order) and has only what the producer and the MMA issuers need
+        for (int j = tid; j < n_early + sh.n_sh; j += blockDim.x) {
+            TcGroup gr;
+            if (j < n_early) {
+                gr.mask = 0ull; gr.group = __ldcg(ws.early + 2 + j); gr.T = 0; gr.off = 0; gr.f = sh.f;
+                gr.p1 = sh.n_sh * u1s + j * u1r; gr.p2 = 0;
+                groups[j] = gr;
+            } else {
+                const int sx = j - n_early;
+                gr.mask = all; gr.group = sh.E + sx; gr.T = p.B; gr.off = p.B * sh.k + sx * p.B; gr.f = sh.f_sh;
+                gr.p1 = sx * u1s; gr.p2 = 0;
+                groups[GP + sx] = gr;
+            }
+        }
+        share(0, sh.n_sh * u1s + n_early * u1r, halves1, pre_start, n_pre, pre_trim);
+        if (n_pre > kTcMaxUnits) {                    // (the host leaves the early start off where this could happen)
+            if (tid == 0) atomicExch(ws.status, ST_BAD_PLAN);
+            n_pre = kTcMaxUnits;
+        }
     }
-    const int n_units = my_cnt0 + my_cnt1 + my_cnt2 + my_cnt3;
+    // unit i of this CTA's share of the pre-lot: shared experts first (their reductions need no table)
+    auto pre_unit_make = [&](int i) -> TcUnit {
+        const int u = pre_start + i, kt_all = (sh.d + 63) / 64;
+        TcUnit t;
+        int local, f_g;
+        if (u < sh.n_sh * u1s) { const int sx = u / u1s; t.a = GP + sx; local = u - sx * u1s; f_g = sh.f_sh; }
+        else { const int v = u - sh.n_sh * u1s, j = v / u1r; t.a = j; local = v - j * u1r; f_g = sh.f; }
+        const int kp = tc_kpieces(sh.d), rbs = (f_g + 127) / 128;
+        const int piece = local % kp, rest = local / kp;
+        t.phase = 1;
+        t.rb = rest % rbs;
+        t.mat = rest / rbs;
+        t.kt0 = piece * kTcKT;
+        t.kt1 = min(kt_all, t.kt0 + kTcKT);
+        t.n = pl.n1;
+        if (i == 0 && (pre_trim & 1)) t.kt0 += kTcKT / 2;
+        if (i == n_pre - 1 && (pre_trim & 2)) t.kt1 -= kTcKT / 2;
+        t.seg = 0;
+        t.first = (i == 0 || t.kt0 == 0) ? 1 : 0;
+        t.last = (i == n_pre - 1 || t.kt1 == kt_all) ? 1 : 0;
+        return t;
+    };
+    if (EARLY) {
+        for (int i = tid; i < n_pre; i += blockDim.x) {
+            const TcUnit t = pre_unit_make(i);
+            s_units[i] = t;
+            s_umeta[i] = tc_unit_meta(t);
+        }
+        __syncthreads();
+    }
+
+    // ---- the tables of the routed work: by every thread of the CTA (tt, tn = thread, threads; hardware
+    // barrier 0) or, with the early start, by warps 7..10 alone (barrier 1)
+    int n_active = 0, U = 0, total1 = 0, total2 = 0, a_split = 0, W = 1, n_main = 0;
+    int my_start0 = 0, my_start1 = 0, my_start2 = 0, my_start3 = 0, my_cnt0 = 0, my_cnt1 = 0, my_cnt2 = 0, my_cnt3 = 0;
+    int my_trim0 = 0, my_trim1 = 0, my_trim2 = 0, my_trim3 = 0;
+    // Four segments in time order: phase 1 of wave 0, of wave 1, phase 2 of wave 0, of wave 1.
+    // Contiguous units are consecutive k-pieces of one 128-row block, so a CTA accumulates them in
+    // one TMEM accumulator and the epilogue runs once per run of k-pieces instead of once per
+    // unit; only row blocks cut by a CTA boundary are reduced from two CTAs.
     auto unit_make = [&](int i) -> TcUnit {
         int seg = 0, j = i, start = my_start0, cnt = my_cnt0, trim = my_trim0;
         if (j >= cnt) { j -= cnt; seg = 1; start = my_start1; cnt = my_cnt1; trim = my_trim1; }
@@ -592,17 +680,108 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         t.last = (j == cnt - 1 || t.kt1 == (K + 63) / 64) ? 1 : 0;
         return t;
     };
-    // decoded once by all threads: the single-thread roles below then read a unit from shared
-    // memory instead of dividing
-    for (int i = tid; i < n_units && i < kTcMaxUnits; i += blockDim.x) {
-        const TcUnit t = unit_make(i);
-        s_units[i] = t;
-        s_umeta[i] = tc_unit_meta(t);
+    auto build_tables = [&](int tt, int tn, int bar_id) {
+        n_active = ws.header[0];
+        U = ws.header[2];
+        const int ne = EARLY ? n_early : 0;
+        // one round of global loads: the header above, the group table in its final form and the
+        // slot arrays, whose sizes are known without the header
+        for (int a = tt; a < G; a += tn) {
+            const uint4 r0 = ws.gtab[2 * a], r1 = ws.gtab[2 * a + 1];
+            if (a < n_active) {
+                TcGroup gr;
+                gr.group = (int)r0.x;
+                // offloaded experts: from here on the group id of a routed expert is the device slot its
+                // weights lie in (a slot index is below E as well, so shared groups stay recognisable)
+                if (ws.slot_of && gr.group < sh.E) gr.group = __ldg(&ws.slot_of[gr.group]);
+                gr.T = (int)r0.y;
+                gr.off = (int)r0.z;
+                gr.f = gr.group < sh.E ? sh.f : sh.f_sh;
+                gr.mask = (unsigned long long)r1.x | ((unsigned long long)r1.y << 32);
+                const int r = a < U ? a : U, s = a < U ? 0 : a - U;
+                // (early start: the first projection of the early and the shared experts is in the pre-lot)
+                gr.p1 = EARLY ? max(0, r - ne) * u1r : r * u1r + s * u1s;
+                gr.p2 = r * u2r + s * u2s;
+                // (the early experts must lead the final list in the order they were announced in)
+                if (EARLY && a < ne && groups[a].group != gr.group) atomicExch(ws.status, ST_BAD_PLAN);
+                groups[a] = gr;
+            }
+        }
+        for (int i = tt; i < n_slots; i += tn) {
+            s_slot_token[i] = ws.slot_token[i];
+            s_slot_w[i] = ws.slot_w[i];
+        }
+        total1 = EARLY ? max(0, U - ne) * u1r : U * u1r + sh.n_sh * u1s;
+        total2 = U * u2r + sh.n_sh * u2s;
+        if (tt == 0) {
+            // wave 1 starts at the first group whose first-projection units (pre-lot included) begin at
+            // or after that share of all of them
+            int sp = n_active;
+            if (n_active >= 2) {
+                sp = 1;
+                while (sp < n_active - 1) {
+                    const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
+                    if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)(U * u1r + sh.n_sh * u1s) * kTcSplitNum) break;
+                    ++sp;
+                }
+            }
+            s_split = sp;
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(tn) : "memory");
+        a_split = s_split;
+        W = a_split < n_active ? 2 : 1;
+        const int split1 = W == 2 ? groups[a_split].p1 : total1;
+        const int split2 = W == 2 ? groups[a_split].p2 : total2;
+        share(0, split1, halves1, my_start0, my_cnt0, my_trim0);
+        share(split1, total1 - split1, halves1, my_start1, my_cnt1, my_trim1);
+        share(total1, split2, halves2, my_start2, my_cnt2, my_trim2);
+        share(total1 + split2, total2 - split2, halves2, my_start3, my_cnt3, my_trim3);
+        n_main = my_cnt0 + my_cnt1 + my_cnt2 + my_cnt3;
+        if (EARLY && n_pre + n_main > kTcMaxUnits) {  // (see above: left off by the host)
+            if (tt == 0) atomicExch(ws.status, ST_BAD_PLAN);
+            n_main = kTcMaxUnits - n_pre;
+        }
+        // decoded once: the single-thread roles below then read a unit from shared memory instead
+        // of dividing
+        for (int i = tt; i < n_main && n_pre + i < kTcMaxUnits; i += tn) {
+            const TcUnit t = unit_make(i);
+            s_units[n_pre + i] = t;
+            s_umeta[n_pre + i] = tc_unit_meta(t);
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(tn) : "memory");
+    };
+    if (!EARLY) {
+        // programmatic dependent launch: the routing kernel in front of this grid must have
+        // finished before its results are read; the next layer's routing kernel may be scheduled
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        tc_fence_before();
+        build_tables(tid, (int)blockDim.x, 0);
+        tc_fence_after();
+    } else if (warp >= 7) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        build_tables(tid - 224, 128, 1);
+        if (tid == 224) {
+            s_tab[0] = n_main;
+            s_tab[1] = n_active;
+            mbar_arrive(&tab_bar);                    // (release: the tables are written)
+        }
     }
-    __syncthreads();
+    const uint32_t tmem_base = s_tmem;
+    // What a role knows of the tables: everything at once, or (early start) after tab_bar.  The
+    // roles keep their own copies (lim: units of this CTA known so far).
+    auto tables_wait = [&](int &lim, int &split, int &waves) -> bool {
+        if (!mbar_wait(&tab_bar, 0)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); return false; }
+        lim = n_pre + s_tab[0];
+        split = s_split;
+        waves = split < s_tab[1] ? 2 : 1;
+        return true;
+    };
+    const int n_units0 = EARLY ? n_pre : n_main;      // units known when the roles start
+    const int n_units = n_units0;                     // (the int4 roles: all of them)
     auto unit_at = [&](int i) -> TcUnit { return i < kTcMaxUnits ? s_units[i] : unit_make(i); };
     auto umeta_at = [&](int i) -> uint32_t { return i < kTcMaxUnits ? s_umeta[i] : tc_unit_meta(unit_make(i)); };
-    auto seg_of_unit = [&](int i) -> int { return i < n_units ? unit_at(i).seg : 4; };
 
     if (warp == 0) {
         const uint64_t wpolicy = l2_evict_first_policy();
@@ -706,6 +885,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             auto load_tokens2 = [&](int s, int kt, int srow, int shared, int tn) {
                 const CUtensorMap *am = &maps.m[shared ? 8 : 7];
                 uint8_t *op = ring + (size_t)s * pl.stage_bytes + pl.tok_off;
+                if (pl.kg == 2) {
+                    // one copy per 8 slots for both k-tiles: [hi | lo][k-tile][8 rows]
+                    for (int r = 0; r < tn / 2; r += 8) tma_load_4d(op + r * 512, am, 0, srow + r, kt, 0, &full_bar[s]);
+                    return;
+                }
                 // one copy per 8 slots: their hi rows (1 KiB) and, right behind them, their lo rows
                 for (int r = 0; r < tn / 2; r += 8) tma_load_3d(op + r * 256, am, kt * 64, srow + r, 0, &full_bar[s]);
             };
@@ -729,7 +913,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             int s = 0;                                   // ring slot of the next k-tile
             uint32_t ring_par = 1;                       // parity to wait for on its empty barrier
 
-            for (int i = 0; i < n_units && alive; ++i) {
+            int lim = n_units0, a_split_p = a_split, w_p = W;
+            bool tabs = !EARLY;
+            for (int i = 0; alive; ++i) {
+                if (i >= lim) {
+                    // (early start: the pre-lot is on its way; the rest needs the tables)
+                    if (tabs) break;
+                    tabs = true;
+                    if (!tables_wait(lim, a_split_p, w_p)) { alive = false; break; }
+                    if (i >= lim) break;
+                }
 
                 const TcUnit t = unit_at(i);
                 const TcGroup &g = groups[t.a];
@@ -739,7 +932,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
                 const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared activation array
-                const int wv = t.a >= a_split ? 1 : 0;
+                const int wv = t.a >= a_split_p ? 1 : 0;
                 bool ready = t.phase == 1 || wv < ready_w;
                 if (!ready) {
                     // the pending tiles all belong to one wave (pend_wave); if that is an earlier wave than
@@ -753,7 +946,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     }
                 }
 
-                for (int kt = t.kt0; kt < t.kt1 && alive; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
+                const int KGB = pl.kg;                     // k-tiles per stage (1 or 2)
+                for (int kt = t.kt0; kt < t.kt1 && alive; kt += KGB, ++it, tc_ring_next(s, ring_par, S)) {
                     if (!ready && pend_n == S) {
                         if (!wait_ready(wv)) { alive = false; break; }     // every slot waits for tokens
                         ready = true;
@@ -766,12 +960,30 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     }
 
                     uint8_t *stage = ring + (size_t)s * pl.stage_bytes;
+                    if (KGB == 2) {
+                        // both k-tiles of the stage in one weight copy (a k-tile past the end of the
+                        // contraction reads as zero) and one token copy (phase 2: one per 8 slots)
+                        const uint32_t op_bytes = t.phase == 1 ? 2u * (uint32_t)pl.tokb : 2u * (uint32_t)t.n * 128u;
+                        mbar_expect_tx(&full_bar[s], 2 * kTcWTile + op_bytes);
+                        tma_load_3d_stream(stage, &maps.m[9 + (shared ? 3 : 0) + t.mat], 0, row0, kt, &full_bar[s], wpolicy);
+                        if (t.phase == 1) {
+                            tma_load_3d(stage + pl.tok_off, &maps.m[6], 0, 0, kt, &full_bar[s]);
+                        } else if (ready) {
+                            load_tokens2(s, kt, srow, shared, t.n);
+                        } else {
+                            pend_stage[pend_n] = s; pend_kt[pend_n] = kt; pend_row[pend_n] = srow;
+                            pend_shared[pend_n] = shared; pend_tn[pend_n] = t.n;
+                            pend_wave = wv;
+                            ++pend_n;
+                        }
+                        continue;
+                    }
                     const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : (uint32_t)t.n * 128u) : (uint32_t)t.n * 128u;
                     mbar_expect_tx(&full_bar[s], kTcWTile + op_bytes);
                     tma_load_2d_stream(stage, wmap, kt * 64, row0, &full_bar[s], wpolicy);
                     if (t.phase == 1) {
                         if (!pl.x_bytes)
-                            for (int r = 0; r < t.n; r += 16)
+                            for (int r = 0; r < t.n; r += pl.rows1)
                                 tma_load_2d(stage + pl.tok_off + r * 128, &maps.m[6], kt * 64, r, &full_bar[s]);
                     } else if (ready) {
                         load_tokens2(s, kt, srow, shared, t.n);
@@ -807,7 +1019,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // all token tiles of the hidden states, once (this thread has nothing to issue before they land)
                 mbar_expect_tx(&x_bar, (uint32_t)pl.x_bytes);
                 for (int kt = 0; kt < (sh.d + 63) / 64; ++kt)
-                    for (int r = 0; r < pl.n1; r += 16)
+                    for (int r = 0; r < pl.n1; r += pl.rows1)
                         tma_load_2d(xres + ((size_t)kt * pl.n1 + r) * 128, &maps.m[6], kt * 64, r, &x_bar);
             }
             if (pl.x_bytes && !mbar_wait(&x_bar, 0)) {
@@ -818,6 +1030,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const uint32_t ks = 4u / (uint32_t)NI, koff = 2u * ks * (uint32_t)half;
             const uint32_t hi_std = (uint32_t)(tc_smem_desc(ring) >> 32);
             const uint32_t hi_p2 = Q4 ? (uint32_t)(tc_smem_desc_sbo(ring, (uint32_t)kTcQ4KG * 1024u) >> 32) : hi_std;
+            const uint32_t hi_p2k = (uint32_t)(tc_smem_desc_sbo(ring, 2048u) >> 32);     // bf16, two k-tiles per stage
+            const unsigned nbm = (unsigned)pl.n_acc - 1u, nbs = (unsigned)__ffs(pl.n_acc) - 1u;   // accumulator buffers: mask, log2
             const uint32_t ring_lo = (uint32_t)tc_smem_desc(ring) + koff, xres_lo = (uint32_t)tc_smem_desc(xres) + koff;
             const uint32_t tok_lo = (uint32_t)tc_smem_desc(tokring) + koff;
             const uint32_t a_tmem0 = tmem_base + (uint32_t)kTcQ4ACol + 4u * koff;     // 8 columns per K-step
@@ -866,12 +1080,18 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 
                 }
             } else
-            for (; (int)ui < n_units && alive; ++ui) {
+            for (int lim = n_units0, tabs = EARLY ? 0 : 1; alive; ++ui) {
+                if ((int)ui >= lim) {
+                    int sp_, w_;
+                    if (tabs) break;
+                    tabs = 1;
+                    if (!tables_wait(lim, sp_, w_) || (int)ui >= lim) break;
+                }
                 const TcUnit t = unit_at((int)ui);
-                const int buf = run & 1;
+                const int buf = run & nbm;
                 if (t.first) {
 
-                    if (!mbar_wait(&acc_empty[buf], ((run >> 1) & 1u) ^ 1u)) {
+                    if (!mbar_wait(&acc_empty[buf], ((run >> nbs) & 1u) ^ 1u)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
                         break;
                     }
@@ -883,7 +1103,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 // phase 2: every 16 columns are the hi rows and the lo rows of 8 slots; the epilogue
                 // adds the two halves
                 const uint32_t idesc = tc_idesc(t.n);
-                for (int kt = t.kt0; kt < t.kt1; ++kt, ++it, tc_ring_next(s, ring_par, S)) {
+                const int KGB = pl.kg;
+                for (int kt = t.kt0; kt < t.kt1; kt += KGB, ++it, tc_ring_next(s, ring_par, S)) {
 
                     if (!mbar_wait(&full_bar[s], ring_par)) {
                         atomicExch(ws.status, ST_MBAR_TIMEOUT);
@@ -893,7 +1114,20 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 
                     tc_fence_after();
 
-                    {
+                    if (KGB == 2) {
+                        // two weight k-tiles 16 KiB apart; their token tiles tokb apart (phase 1) or, per
+                        // 8 slots, [hi | lo][k-tile][8 rows]: 8-row groups 2 KiB apart, k-tiles 1 KiB
+                        const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
+                        const uint32_t b0 = a_lo + ((uint32_t)pl.tok_off >> 4);
+                        const bool p2 = t.phase == 2;
+                        const uint32_t b_step = p2 ? 64u : ((uint32_t)pl.tokb >> 4), b_hi = p2 ? hi_p2k : hi_std;
+#pragma unroll
+                        for (uint32_t g = 0; g < 2; ++g)
+                            for (uint32_t k = 0; k < ks; ++k) {
+                                tc_mma_bf16_parts(d_tmem, a_lo + g * (kTcWTile >> 4) + 2 * k, hi_std, b0 + g * b_step + 2 * k, b_hi, idesc, acc);
+                                acc = 1;
+                            }
+                    } else {
                         const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
                         const uint32_t b_lo = (t.phase == 1 && pl.x_bytes) ? xres_lo + (uint32_t)kt * ((uint32_t)pl.n1 * 8u)
                                                                            : a_lo + ((uint32_t)pl.tok_off >> 4);
@@ -959,12 +1193,19 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     sc[0] = *reinterpret_cast<const uint32_t *>(stage + KG * kTcQ4Packed + r * 16 + h * 4); sc[1] = 0;
                 }
                 const uint32_t a_slot = a_lane + (uint32_t)(ta * KG) * 32u;
+                // all packed chunks of this thread first: the stores to tensor memory below order
+                // memory accesses, so a load behind one of them would wait for it
+                uint4 pks[CP];
+#pragma unroll
+                for (int qi = 0; qi < CP; ++qi) {
+                    // the packed rows are swizzled over their own width by the TMA copy
+                    const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
+                    pks[qi] = *reinterpret_cast<const uint4 *>(prow + (((h * CP + qi) ^ sw) * 16));
+                }
 #pragma unroll
                 for (int qi = 0; qi < CP; ++qi) {
                     const int q = h * CP + qi;                         // chunk of 32 weights inside the stage
-                    // the packed rows are swizzled over their own width by the TMA copy
-                    const int sw = KG == 4 ? (r & 7) : (KG == 2 ? ((r >> 1) & 3) : ((r >> 2) & 1));
-                    const uint4 pk = *reinterpret_cast<const uint4 *>(prow + ((q ^ sw) * 16));
+                    const uint4 pk = pks[qi];
                     // the block's scale is binary16 already: both halves of a register
                     const uint32_t sc2u = __byte_perm(sc[qi >> 1], 0u, (qi & 1) ? 0x3232u : 0x1010u);
                     const __half2 sc2 = *reinterpret_cast<const __half2 *>(&sc2u);
@@ -1121,8 +1362,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         const int n_routed_el = n_routed;   // (alias used below)
         (void)n_routed_el;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
-        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
         int next_arrive = 0;
+        int lim = n_units0, a_split_e = a_split, w_e = W;
+        bool tabs = !EARLY;
+        const unsigned nbm = (unsigned)pl.n_acc - 1u, nbs = (unsigned)__ffs(pl.n_acc) - 1u;
+        (void)a_split_e;
         auto wave_arrive = [&](int w) -> bool {
             // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps,
             // whose first thread orders them (fence) before it arrives on the grid-wide counter, so
@@ -1137,22 +1381,33 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // called before every unit (and once at the end): hand a wave over once this CTA's phase-1
         // units of it are all done
         auto service = [&](int upcoming_seg) -> bool {
-            const int seg_wave1 = W == 2 ? 1 : 2;        // first segment that lies after phase 1 of wave 0
-            while (next_arrive < W && upcoming_seg >= (next_arrive == 0 ? seg_wave1 : 2)) {
+            const int seg_wave1 = w_e == 2 ? 1 : 2;      // first segment that lies after phase 1 of wave 0
+            while (next_arrive < w_e && upcoming_seg >= (next_arrive == 0 ? seg_wave1 : 2)) {
                 if (!wave_arrive(next_arrive)) return false;
                 ++next_arrive;
             }
             return true;
         };
         {
-            for (; (int)ui < n_units && alive; ++ui) {
-                if (!service(seg_of_unit((int)ui))) { alive = false; break; }
+            for (; alive; ++ui) {
+                if ((int)ui >= lim) {
+                    if (tabs) break;
+                    tabs = true;
+                    if (!tables_wait(lim, a_split_e, w_e)) { alive = false; break; }
+                    if ((int)ui >= lim) break;
+                }
                 const TcUnit t = unit_at((int)ui);
+                if (!service(t.seg)) { alive = false; break; }
                 if (!t.last) continue;                 // the run's accumulator is read after its last unit
+                if (!tabs && t.a < GP) {
+                    // an early routed expert of the pre-lot: its tokens and slots come with the tables
+                    tabs = true;
+                    if (!tables_wait(lim, a_split_e, w_e)) { alive = false; break; }
+                }
                 const TcGroup &g = groups[t.a];
-                const int buf = run & 1;
+                const int buf = run & nbm;
 
-                if (!mbar_wait(&acc_full[buf], (run >> 1) & 1u)) {
+                if (!mbar_wait(&acc_full[buf], (run >> nbs) & 1u)) {
                     if (lane == 0) atomicExch(ws.status, ST_MBAR_TIMEOUT);
                     alive = false;
                     break;

@@ -418,10 +418,32 @@ __device__ __forceinline__ void gating_part1(const Shape &sh, int B, const doubl
     gate_sync(gg);
 }
 
+// The expert with the largest original logit of token b (equal logits: the lower id), by one warp.
+template <int J>
+__device__ __forceinline__ int gate_top1(const Shape &sh, int b, const double *s_l, int lane)
+{
+    const unsigned full = 0xffffffffu;
+    unsigned long long best = 0ull;
+    int be = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+        const int e = lane + 32 * j;
+        if (e < sh.E) {
+            const unsigned long long kk = dkey(s_l[b * sh.E + e]);
+            if (kk > best) { best = kk; be = e; }          // (e ascends with j: the first of equal keys stays)
+        }
+    }
+    const unsigned hb = warp_max_holders(best, be != 0x7fffffff);
+    return (int)__reduce_min_sync(full, ((hb >> lane) & 1u) ? (unsigned)be : 0xffffffffu);
+}
+
+// early32 (or NULL): bit words of experts that go to the front of the active list and of the slot
+// order, ascending among themselves (every one of them must have been selected by some token); the
+// other active experts follow in ascending order.
 template <int J>
 __device__ __forceinline__ void gating_part2(const Shape &sh, int B, const double *__restrict__ s_l, const GateGroup gg,
                                              const GateMem gm, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
-                                             bool den_early)
+                                             bool den_early, const unsigned *early32 = nullptr)
 {
     const int tid = gg.t, nt = gg.n, warp = tid >> 5, lane = tid & 31, nw = nt >> 5;
     const int E = sh.E;
@@ -433,7 +455,7 @@ __device__ __forceinline__ void gating_part2(const Shape &sh, int B, const doubl
     // union, unique count, exclusive scan, list of active experts: warp 0, lane owns a run of experts
     if (tid < 32) {
         const int C = (E + 31) >> 5, e0 = lane * C;
-        int sum = 0, act = 0;
+        int sum = 0, act = 0, esum = 0, eact = 0;        // all experts of the run; the early ones among them
 #pragma unroll 1
         for (int i = 0; i < C; ++i) {
             const int e = e0 + i;
@@ -442,23 +464,35 @@ __device__ __forceinline__ void gating_part2(const Shape &sh, int B, const doubl
                 gm.cnt[e] = c;
                 sum += c;
                 act += c > 0;
+                if (early32 && ((early32[e >> 5] >> (e & 31)) & 1u)) { esum += c; eact += c > 0; }
             }
         }
-        int xs = sum, xa = act;
+        int xs = sum, xa = act, ys = esum, ya = eact;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int t = __shfl_up_sync(0xffffffffu, xs, o), u = __shfl_up_sync(0xffffffffu, xa, o);
             if (lane >= o) { xs += t; xa += u; }
+            if (early32) {
+                const int t2 = __shfl_up_sync(0xffffffffu, ys, o), u2 = __shfl_up_sync(0xffffffffu, ya, o);
+                if (lane >= o) { ys += t2; ya += u2; }
+            }
         }
-        int off = xs - sum, pos = xa - act;
+        // slots and list positions: the early experts first, then the rest
+        const int te = early32 ? __shfl_sync(0xffffffffu, ys, 31) : 0, ne = early32 ? __shfl_sync(0xffffffffu, ya, 31) : 0;
+        int eoff = ys - esum, epos = ya - eact;
+        int off = te + (xs - sum) - eoff, pos = ne + (xa - act) - epos;
 #pragma unroll 1
         for (int i = 0; i < C; ++i) {
             const int e = e0 + i;
             if (e < E) {
-                gm.off[e] = off;
-                gm.pos[e] = pos;
-                off += gm.cnt[e];
-                pos += gm.cnt[e] > 0;
+                const int c = gm.cnt[e];
+                if (early32 && ((early32[e >> 5] >> (e & 31)) & 1u)) {
+                    gm.off[e] = eoff; gm.pos[e] = epos;
+                    eoff += c; epos += c > 0;
+                } else {
+                    gm.off[e] = off; gm.pos[e] = pos;
+                    off += c; pos += c > 0;
+                }
             }
         }
         if (lane == 31) { gm.off[E] = xs; *gm.U = xa; }

@@ -118,9 +118,11 @@ __device__ __forceinline__ void gating_writeout(const Shape &sh, int B, const Wo
 template <int JE>
 __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Workspace &ws, const float *__restrict__ conf,
                                              int has_gate, int32_t *__restrict__ sel_idx, float *__restrict__ sel_w,
-                                             int32_t *__restrict__ n_unique, double *s_l, int ksplit, const double *__restrict__ lpart)
+                                             int32_t *__restrict__ n_unique, double *s_l, int ksplit, const double *__restrict__ lpart,
+                                             int early = 0)
 {
     __shared__ unsigned long long s_mask[kMaxExperts], s_gk[kMaxExperts];
+    __shared__ unsigned s_early32[8];
     __shared__ double s_lam[kMaxTokens], s_zmax[kMaxTokens], s_den[kMaxTokens];
     __shared__ int s_sel[kMaxTokens * kMaxTopK];
     __shared__ float s_pw[kMaxTokens * kMaxTopK];
@@ -156,9 +158,52 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
     }
 #pragma unroll 1
     for (int b = gg.t; b < B; b += gg.n) s_w[b] = conf ? (double)conf[b] : 1.0;
+    if (early) {
+        // The expert kernel is already resident (programmatic launch) and waits for this list: the
+        // experts whose first projection it may stream while the gating below still runs.  A token's
+        // first expert by original logit stays selected whatever E* turns out to be (the bias lifts
+        // an expert by at most alpha (l_(1) - l_(k+1)) <= l_(1) - l_(k+1), so only the other k - 1 of
+        // its first k can pass it), which the caller has checked for this layer's alpha (early == 2).
+        // These experts lead the active list and the slot order, ascending, so that the expert
+        // kernel knows their groups before it knows the others.
+        if (gg.t < 8) s_early32[gg.t] = 0u;
+        __syncthreads();                                  // the logits are staged, the words cleared
+        if (early == 2) {
+#pragma unroll 1
+            for (int b = gg.t >> 5; b < B; b += gg.n >> 5) {
+                const int e = gate_top1<JE>(sh, b, s_l, gg.t & 31);
+                if ((gg.t & 31) == 0) atomicOr(&s_early32[e >> 5], 1u << (e & 31));
+            }
+        }
+        __syncthreads();
+        if (gg.t < 32) {
+            const int lane = gg.t;
+            unsigned w = lane < 8 ? s_early32[lane] : 0u;
+            const int c = __popc(w);
+            int x = c;
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += t;
+            }
+            int at = x - c;
+            while (w) {
+                ws.early[2 + at++] = 32 * lane + __ffs(w) - 1;
+                w &= w - 1u;
+            }
+            const int total = __shfl_sync(0xffffffffu, x, 7);
+            __syncwarp();
+            if (lane == 0) {
+                ws.early[1] = total;
+                ws.header[6] = total;
+                __threadfence();
+                asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early), "r"(1) : "memory");
+            }
+        }
+    }
     // (gating_group's first barrier orders these writes before the first read)
     gating_part1<JE>(sh, B, s_l, s_w, gg, gm, true);
-    gating_part2<JE>(sh, B, s_l, gg, gm, sel_idx, sel_w, true);
+    gating_part2<JE>(sh, B, s_l, gg, gm, sel_idx, sel_w, true, early ? s_early32 : nullptr);
     gating_writeout(sh, B, ws, gm, has_gate, n_unique, gg);
 }
 
@@ -204,6 +249,9 @@ struct ZeroList {
     // partial sums in lpart [piece][token][row] (see route_logit_tasks); 0: by row blocks
     int ksplit;
     double *lpart;
+    // 1: the expert kernel behind this launch starts before the gating has ended (see gating_block);
+    // 2: the same, and every token's first expert by original logit is known to stay selected
+    int early;
 };
 
 // Router logits by the warps of the whole grid: a task is one router row (row E: the shared
@@ -309,6 +357,15 @@ __device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspa
     // layer's kernels, so it waits for them first; the FFN kernel that follows may come up now
     // and do its own set-up (both instructions do nothing in a plain launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (zl.early && blockIdx.x == 0) {
+        // the expert kernel of this layer polls this word from the moment it is scheduled, which is
+        // after every block of this grid has passed the next instruction: the flag is down by then
+        if (tid == 0) {
+            asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(ws.early), "r"(0) : "memory");
+            __threadfence();
+        }
+        __syncthreads();
+    }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // (block 0: where the arrival counter stood when the launch before had ended; see below)
     unsigned ticket_base = 0u;
@@ -344,7 +401,11 @@ __device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspa
     } else if constexpr (THREADS == kRouteThreads) {
     const int n_grp = zl.groups > 1 ? zl.groups : 1;
     n_arrive = n_rows * n_grp;
-    if ((int)blockIdx.x >= n_arrive) return;
+    // (early start of the expert kernel: it accumulates into what this grid clears as soon as the
+    // list above is out, so the blocks that only clear arrive on the counter as well)
+    if ((int)blockIdx.x >= n_arrive && !zl.early) return;
+    if (zl.early) n_arrive = (int)gridDim.x;
+    if ((int)blockIdx.x < n_rows * n_grp) {
     const int row = (int)blockIdx.x % n_rows, grp = (int)blockIdx.x / n_rows, d = sh.d;
     const int tg = 4 * ((B + 4 * n_grp - 1) / (4 * n_grp));            // tokens per group, a multiple of 4
     const int b_lo = min(B, grp * tg), b_hi = min(B, b_lo + tg);
@@ -358,6 +419,8 @@ __device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspa
         else { route_pass<ACT, RT, 4>(sh, B, b0, ws, row, wrow, hidden, s_dyn); b0 += 4; }
     }
     }
+    }
+    if (zl.early) __syncthreads();                        // all of this block's clearing, before its arrival
     // Block 0 runs the gating once every row has arrived (its SM tends to be the same from layer
     // to layer, so part of the gating code is still in its instruction cache: measured 0.6 % of
     // a layer against letting the last block to arrive do it).  Every block adds one arrival, with
@@ -392,7 +455,7 @@ __device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspa
     }
     __syncthreads();
     if (!s_last) return;
-    gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn, zl.ksplit, zl.lpart);
+    gating_block<JE>(sh, B, ws, conf, sh_scale ? 1 : 0, sel_idx, sel_w, n_unique, s_dyn, zl.ksplit, zl.lpart, zl.early);
 }
 
 template <int ACT, int RT, int JE>

@@ -44,6 +44,8 @@ struct s2moe_ctx {
     void *hperm = nullptr;                // int4 plan 3: column-permuted copy of the hidden states
     double *lpart = nullptr;              // partial router logits [piece][token][row] (logit pass by warp tasks)
     int route_task_from = 48;             // batches of this many tokens and more take the logit pass by warp tasks
+    bool early_start = true;              // bf16 tensor-core plan: the expert kernel starts under the gating (S2MOE_NO_EARLY=1: off)
+    int bf16_kg2_from = 32;               // batches of this many tokens and more: two k-tiles per ring stage (bf16)
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
@@ -174,7 +176,7 @@ int validate_layer(const s2moe_config *c, const s2moe_layer_weights *w)
 // Launch configuration with programmatic stream serialization: the kernel may start before
 // the one in front of it in the stream has finished; it calls griddepcontrol.wait before it
 // touches anything that kernel writes.  Only kernels that contain that wait are launched so.
-cudaLaunchConfig_t pdl_config(s2moe_ctx *ctx, int grid, int block, size_t smem, cudaStream_t st)
+cudaLaunchConfig_t pdl_config(s2moe_ctx *ctx, int grid, int block, size_t smem, cudaStream_t st, bool in_graph = false)
 {
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3((unsigned)grid);
@@ -183,10 +185,12 @@ cudaLaunchConfig_t pdl_config(s2moe_ctx *ctx, int grid, int block, size_t smem, 
     lc.stream = st;
     ctx->pdl_attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     // measured: plain stream launches gain about 4 % from it, a captured graph loses about 1 %
-    // (its kernel nodes already follow each other closely), so it is left out under capture
+    // (its kernel nodes already follow each other closely), so it is left out under capture unless
+    // the kernel does real work before its wait (in_graph: the expert kernel that starts under the
+    // gating, and the routing kernel in front of it)
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     const bool capturing = cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone;
-    ctx->pdl_attr.val.programmaticStreamSerializationAllowed = (ctx->use_pdl && (!capturing || ctx->pdl_in_graph)) ? 1 : 0;
+    ctx->pdl_attr.val.programmaticStreamSerializationAllowed = (ctx->use_pdl && (!capturing || ctx->pdl_in_graph || in_graph)) ? 1 : 0;
     lc.attrs = &ctx->pdl_attr;
     lc.numAttrs = 1;
     return lc;
@@ -243,7 +247,7 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
     }
     LaunchScope scope(ctx, KC_ROUTER, st);
     if (zg.ksplit > 0) {
-        cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreadsBig, route_smem(B, sh.E), st);
+        cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreadsBig, route_smem(B, sh.E), st, zl.early != 0);
         if (sh.E <= 64)
             cudaLaunchKernelEx(&lc, route_kernel_big<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
                                (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
@@ -255,7 +259,7 @@ void launch_route_t(s2moe_ctx *ctx, const Shape &sh, const LayerPtrs &lp, int B,
                                (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
         return;
     }
-    cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st);
+    cudaLaunchConfig_t lc = pdl_config(ctx, grid, kRouteThreads, route_smem(B, sh.E), st, zl.early != 0);
     if (sh.E <= 64)
         cudaLaunchKernelEx(&lc, route_kernel<ACT, RT, 2>, sh, B, ctx->ws, hidden, (const void *)lp.router,
                            (const void *)lp.sh_scale, conf, sel_idx, sel_w, n_unique, zg);
@@ -398,6 +402,21 @@ bool make_map_hilo(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uin
                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 weights as {64 columns, rows, k-tiles of 64 columns}, box = 64 x 128 x 2: two k-tiles of a
+// 128-row block in one copy, each a 16 KiB tile with the 128-byte swizzle
+bool make_map_w2(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols)
+{
+    if (!ctx->encode_tiled || !base || rows == 0 || cols % 64) return false;
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {cols * 2, 128};
+    const cuuint32_t box[3] = {64, 128, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return ((EncodeTiledFn)ctx->encode_tiled)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // int4 path: the hidden states as {64 columns, rows, k-tiles of 64 columns}, box = 64 x box_rows x kg:
 // the token tiles of kg consecutive k-tiles in one copy, each tile box_rows x 128 bytes
 bool make_map_ktiles(const s2moe_ctx *ctx, CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols,
@@ -447,7 +466,7 @@ int plan_for(const s2moe_ctx *ctx, int B, StPlan *out)
         return tp.feasible ? 4 : 0;
     }
     if (want == 0 || want == 3) {
-        const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B);
+        const TcPlan tp = tc_make_plan(s0, B, ctx->n_sm, B * s0.k + s0.n_sh * B, B >= ctx->bf16_kg2_from ? 2 : 1);
         if (tp.feasible && !ctx->tc_maps.empty()) return 3;
         if (want == 3) return 0;
     }
@@ -513,6 +532,11 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     if (plan == 0) return S2MOE_EINVAL;
     sh.plan = plan;
     sh.op_cap = pl.op_cap;
+    // tensor-core plan with bf16 weights: the expert kernel starts while the gating still runs, on the
+    // experts the routing kernel announces before it (not with offloaded experts: their weights are
+    // fetched between the two kernels)
+    const bool want_early = plan == 3 && ctx->early_start && ctx->use_pdl && !ctx->offload && sh.weight_dtype == DT_BF16;
+    const TcPlan tp3 = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B, B >= ctx->bf16_kg2_from ? 2 : 1, want_early);
     // what the FFN kernels accumulate into is cleared by the routing kernel's blocks
     ZeroList zl{};
     zl.ptr[0] = out;
@@ -529,13 +553,19 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
             zl.perm_n16 = (size_t)B * sh.d * 2 / 16;
         }
     }
+    if (plan == 3 && tp3.early) {
+        // a token's first expert by original logit stays selected for alpha < 1 (see gating_block);
+        // otherwise only the shared experts start early
+        const bool bias_on = sh.alpha > 0.0 && sh.cap < sh.E && sh.k < sh.E;
+        zl.early = (!bias_on || sh.alpha <= 0.999999) ? 2 : 1;
+    }
     if (plan != 4) launch_route(ctx, sh, lp, B, hidden, conf, sel_idx, sel_w, n_unique, zl, st);
     if (ctx->offload) {
         const int rc = fetch_experts(ctx, layer, st);
         if (rc != S2MOE_OK) return rc;
     }
     if (plan == 3 || plan == 4) {
-        const TcPlan tp3 = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B);
+
         const fused::TcPlan tp4 = plan == 4 ? fused::tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B) : fused::TcPlan{};
         const bool q4 = plan == 4 ? tp4.q4 != 0 : tp3.q4 != 0;
         const int tokb = plan == 4 ? tp4.tokb : tp3.tokb, kg = plan == 4 ? tp4.kg : tp3.kg;
@@ -549,8 +579,15 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
             if (ok && sh.n_sh)
                 ok = make_map_hilo_ktiles(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B,
                                           (uint64_t)sh.f_sh, plane, (uint32_t)kg);
+        } else if (plan == 3 && tp3.kg == 2) {
+            // two k-tiles per stage: the token tiles of both in one copy (see make_map_ktiles)
+            ok = make_map_ktiles(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp3.tokb / 128, 2) &&
+                 make_map_hilo_ktiles(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane, 2);
+            if (ok && sh.n_sh)
+                ok = make_map_hilo_ktiles(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B,
+                                          (uint64_t)sh.f_sh, plane, 2);
         } else {
-            ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, 16) &&
+            ok = make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, plan == 3 ? (uint32_t)tp3.rows1 : 16u) &&
                  make_map_hilo(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane);
             if (ok && sh.n_sh)
                 ok = make_map_hilo(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B, (uint64_t)sh.f_sh, plane);
@@ -559,9 +596,9 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
         if (plan == 3) {
             TcArgs a;
             a.sh = sh; a.ws = ctx->ws; a.plan = tp3; a.y = out; a.pre = ctx->pre;
-            a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B;
+            a.act_hi = ctx->act_hi; a.act_lo = ctx->act_lo; a.B = B; a.early = tp3.early;
             LaunchScope scope(ctx, KC_TC, st);
-            cudaLaunchConfig_t lc = pdl_config(ctx, tp3.n_cta, q4 ? kTcQ4Threads : kTcThreads, tp3.smem_bytes, st);
+            cudaLaunchConfig_t lc = pdl_config(ctx, tp3.n_cta, q4 ? kTcQ4Threads : kTcThreads, tp3.smem_bytes, st, tp3.early != 0);
             if (q4) cudaLaunchKernelEx(&lc, ffn_tc_kernel<true>, maps, a);
             else cudaLaunchKernelEx(&lc, ffn_tc_kernel<false>, maps, a);
         } else {
@@ -674,6 +711,7 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     const size_t o_up1 = take(4 * (size_t)(G + 2)), o_up2 = take(4 * (size_t)(G + 2));
     const size_t o_tm = take(8 * (size_t)G);
     const size_t o_gtab = take(32 * (size_t)(G + 1));
+    const size_t o_early = take(4 * (size_t)(kMaxTokens + 4));
     const size_t o_hperm = take(sh.weight_dtype == DT_Q4B32 ? 2 * (size_t)T * sh.d : 0);
     const size_t o_lpart = take(sizeof(double) * 8 * (size_t)T * (E + 1));
     const size_t o_sth = take(ab * (size_t)L * T * sh.d), o_stc = take(4 * (size_t)L * T);
@@ -689,10 +727,14 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     {
         const char *no_pdl = std::getenv("S2MOE_NO_PDL");
         ctx->use_pdl = !(no_pdl && no_pdl[0] == '1');
+        const char *kgv = std::getenv("S2MOE_BF16_KG2_FROM");
+        if (kgv && std::atoi(kgv) > 0) ctx->bf16_kg2_from = std::atoi(kgv);
         const char *tf = std::getenv("S2MOE_ROUTE_TASKS_FROM");
         if (tf && tf[0]) ctx->route_task_from = std::atoi(tf);
         const char *pg = std::getenv("S2MOE_PDL_IN_GRAPH");
         ctx->pdl_in_graph = pg && pg[0] == '1';
+        const char *ne = std::getenv("S2MOE_NO_EARLY");
+        ctx->early_start = !(ne && ne[0] == '1');
     }
     if (e == cudaSuccess && ctx->plan != 1)
         e = cudaFuncSetAttribute(ffn_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStMaxSmem);
@@ -709,6 +751,7 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
     ws.upfx1 = (int32_t *)(base + o_up1); ws.upfx2 = (int32_t *)(base + o_up2);
     ws.tokmask = (unsigned long long *)(base + o_tm);
     ws.gtab = (uint4 *)(base + o_gtab);
+    ws.early = (int32_t *)(base + o_early);
     ctx->hperm = base + o_hperm;
     ctx->lpart = (double *)(base + o_lpart);
     ctx->pre = (float *)(base + o_pre);
@@ -773,6 +816,17 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
                     ok = make_map(ctx, &m.m[3], lp.sh_gate, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
                          make_map(ctx, &m.m[4], lp.sh_up, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d, 128) &&
                          make_map(ctx, &m.m[5], lp.sh_down, (uint64_t)sh.n_sh * sh.d, (uint64_t)sh.f_sh, 128);
+                // the same matrices with two k-tiles per copy (maps 9..14), where every contraction
+                // length is a multiple of 64
+                if (ok && sh.d % 64 == 0 && sh.f % 64 == 0 && (sh.n_sh == 0 || sh.f_sh % 64 == 0)) {
+                    ok = make_map_w2(ctx, &m.m[9], lp.w_gate, (uint64_t)n_w_experts * sh.f, (uint64_t)sh.d) &&
+                         make_map_w2(ctx, &m.m[10], lp.w_up, (uint64_t)n_w_experts * sh.f, (uint64_t)sh.d) &&
+                         make_map_w2(ctx, &m.m[11], lp.w_down, (uint64_t)n_w_experts * sh.d, (uint64_t)sh.f);
+                    if (ok && sh.n_sh)
+                        ok = make_map_w2(ctx, &m.m[12], lp.sh_gate, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d) &&
+                             make_map_w2(ctx, &m.m[13], lp.sh_up, (uint64_t)sh.n_sh * sh.f_sh, (uint64_t)sh.d) &&
+                             make_map_w2(ctx, &m.m[14], lp.sh_down, (uint64_t)sh.n_sh * sh.d, (uint64_t)sh.f_sh);
+                }
             }
             if (!ok) ctx->tc_maps.clear();
         }
