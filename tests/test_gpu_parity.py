@@ -11,7 +11,7 @@ import torch
 from paper_2608_15018_b200 import binding, workloads
 from paper_2608_15018_b200.workloads import BF16, CONFIGS, F32, Q4B32
 
-from gpu_util import run_case, supports
+from gpu_util import check_outputs, run_case, supports
 
 pytestmark = pytest.mark.gpu
 
@@ -311,3 +311,54 @@ def test_128_expert_shapes(name, plan):
         rep, _ = run_case(wl, n_tokens=B, plan=plan)
         assert rep is not None and rep.tokens_checked == B
 
+
+
+@pytest.mark.parametrize("name,B", [("cfg2", 8), ("cfg3", 16), ("cfg5", 33), ("cfg5", 64)])
+def test_early_start_on_and_off(name, B, monkeypatch):
+    """bf16 tensor-core plan: by default the expert kernel starts while the gating still runs, on
+    the experts the routing kernel announces first (other slot order, other unit schedule); with
+    S2MOE_NO_EARLY=1 it waits for the routing kernel as a whole.  Both against the oracle, and the
+    discrete results against each other."""
+    wl = SMALL[name]
+    got = {}
+    for off in ("0", "1"):
+        monkeypatch.setenv("S2MOE_NO_EARLY", off)
+        rep, o = run_case(wl, n_tokens=B, sigma=0.7, plan=3)
+        assert rep.plan == 3
+        got[off] = o
+    assert torch.equal(got["0"].sel_idx, got["1"].sel_idx) and torch.equal(got["0"].n_unique, got["1"].n_unique)
+    assert torch.equal(got["0"].sel_w, got["1"].sel_w)
+
+
+def test_graph_replay_with_changing_inputs():
+    """A captured stack replayed on other inputs: the words the two kernels of a layer meet on (the
+    routing kernel's arrival counter, the early list and its flag) carry nothing over from one replay
+    to the next.  Every replay against the oracle."""
+    wl = SMALL["cfg5"]
+    L, B = 3, 16
+    m, T = _ctx(wl, L, 0)
+    dev = torch.device("cuda", 0)
+    H = torch.stack([workloads.hidden_states(wl, l, B, 0.5, dev) for l in range(L)])
+    C = torch.stack([workloads.confidences(wl, l, B, dev) for l in range(L)])
+    o = m.alloc_outputs(B, stack=True)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.verify_stack(H, C, o, stream=s)
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.verify_stack(H, C, o, stream=torch.cuda.current_stream())
+    for rep in range(4):
+        w = wl.with_(seed=wl.seed + 1000 * rep)
+        sigma = (0.1, 1.0, 0.5, 0.3)[rep]
+        H.copy_(torch.stack([workloads.hidden_states(w, l, B, sigma, dev) for l in range(L)]))
+        C.copy_(torch.stack([workloads.confidences(w, l, B, dev) for l in range(L)]))
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert m.device_status() == 0
+        for l in range(L):
+            ol = binding.LayerOutput(o.out[l], o.sel_idx[l], o.sel_w[l], o.n_unique[l:l + 1])
+            check_outputs(wl, T[l], H[l], C[l], ol)
+    m.close()
