@@ -61,8 +61,9 @@ struct Workspace {
     unsigned long long *tokmask;   // [E + n_sh] bit b set: token b is bucketed to the group
     uint4 *gtab;           // [n_active][2] {group, tokens, first slot, 0}, {mask lo, mask hi, 0, 0}: the
                            // active groups in their final form, or NULL when nobody reads it
-    int32_t *early;        // {flag, n, ids ...}: the experts whose first projection may start before the gating
-                           // has ended, published by the routing kernel (see gating_block), or NULL
+    int32_t *early;        // 8 words of 64 bits, {tag << 32 | bits of 32 experts}: the experts whose first projection
+                           // may start before the gating has ended, published by the routing kernel (see
+                           // gating_block), or NULL
     const int32_t *slot_of;  // [E] device slot that holds each routed expert's weights (expert offloading), or
                              // NULL: every expert is resident at its own index
 };

@@ -490,6 +490,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     __shared__ TcUnit s_units[kTcMaxUnits];
     __shared__ uint32_t s_umeta[kTcMaxUnits];      // what an MMA issuer needs of a unit, in one word (tc_unit_meta)
     __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
+    __shared__ unsigned s_early32[8];              // early start: the routing kernel's list of early experts, 32 per word
     __shared__ int s_tab[2];                       // early start: units of the routed work of this CTA, active groups
     __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
 
@@ -587,22 +588,32 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     // ---- the pre-lot (early start only)
     int n_early = 0, n_pre = 0, pre_start = 0, pre_trim = 0;
     if (EARLY) {
-        if (tid == 0) {
-            // bounded wait for the routing kernel's list (a release store behind everything that
-            // kernel clears; all its blocks are resident or done when this grid is scheduled)
-            int ok = 0;
-            for (unsigned i = 0; i < (1u << 21) && !ok; ++i) {
-                if (ld_acquire(ws.early) == 1) ok = 1;
-                else __nanosleep(40);
+        if (warp == 0) {
+            // bounded wait for the routing kernel's list: one tagged 64-bit word per 32 experts, each
+            // polled by a lane of its own (a release store behind everything that kernel clears; all
+            // its blocks are resident or done when this grid is scheduled)
+            const int nwords = (sh.E + 31) >> 5;
+            unsigned long long v = 0ull;
+            bool ok = false;
+            for (unsigned i = 0; i < (1u << 21); ++i) {
+                if (lane < nwords)
+                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(reinterpret_cast<const unsigned long long *>(ws.early) + lane) : "memory");
+                if (__all_sync(0xffffffffu, lane >= nwords || (v >> 32) == 1ull)) { ok = true; break; }
+                __nanosleep(20);
             }
-            if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
-            s_flag = ok;
+            if (lane < 8) s_early32[lane] = (ok && lane < nwords) ? (unsigned)v : 0u;
+            if (lane == 0) {
+                if (!ok) atomicExch(ws.status, ST_DEP_TIMEOUT);
+                s_flag = ok;
+            }
         }
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        n_early = s_flag ? __ldcg(ws.early + 1) : 0;
-        n_early = max(0, min(n_early, min(p.B, sh.E)));
+        unsigned ew[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { ew[q] = s_early32[q]; n_early += __popc(ew[q]); }
+        n_early = min(n_early, min(p.B, sh.E));
         const unsigned long long all = p.B >= 64 ? ~0ull : ((1ull << p.B) - 1ull);
         // provisional groups: a shared expert's is complete (every token, slots known); an early
         // routed expert's sits where its final entry will be (the early experts lead the active
@@ -610,7 +621,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         for (int j = tid; j < n_early + sh.n_sh; j += blockDim.x) {
             TcGroup gr;
             if (j < n_early) {
-                gr.mask = 0ull; gr.group = __ldcg(ws.early + 2 + j); gr.T = 0; gr.off = 0; gr.f = sh.f;
+                int rem = j, id = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {            // the j-th expert of the list
+                    const int c = __popc(ew[q]);
+                    if (rem >= 0 && rem < c) id = 32 * q + (int)__fns(ew[q], 0u, rem + 1);
+                    rem -= c;
+                }
+                gr.mask = 0ull; gr.group = id; gr.T = 0; gr.off = 0; gr.f = sh.f;
                 gr.p1 = sh.n_sh * u1s + j * u1r; gr.p2 = 0;
                 groups[j] = gr;
             } else {

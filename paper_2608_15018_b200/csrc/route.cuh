@@ -176,29 +176,13 @@ __device__ __forceinline__ void gating_block(const Shape &sh, int B, const Works
             }
         }
         __syncthreads();
-        if (gg.t < 32) {
-            const int lane = gg.t;
-            unsigned w = lane < 8 ? s_early32[lane] : 0u;
-            const int c = __popc(w);
-            int x = c;
-#pragma unroll
-            for (int o = 1; o < 8; o <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, x, o);
-                if (lane >= o) x += t;
-            }
-            int at = x - c;
-            while (w) {
-                ws.early[2 + at++] = 32 * lane + __ffs(w) - 1;
-                w &= w - 1u;
-            }
-            const int total = __shfl_sync(0xffffffffu, x, 7);
-            __syncwarp();
-            if (lane == 0) {
-                ws.early[1] = total;
-                ws.header[6] = total;
-                __threadfence();
-                asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early), "r"(1) : "memory");
-            }
+        // one 64-bit word per 32 experts: the bits of the early experts under a tag of 1 (the words
+        // were cleared before this grid let the expert kernel be scheduled), each released by itself,
+        // so that whoever polls a word has its part of the list with the same load
+        if (gg.t < ((sh.E + 31) >> 5)) {
+            const unsigned long long v = (1ull << 32) | (unsigned long long)s_early32[gg.t];
+            asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(reinterpret_cast<unsigned long long *>(ws.early) + gg.t), "l"(v)
+                         : "memory");
         }
     }
     // (gating_group's first barrier orders these writes before the first read)
@@ -358,10 +342,11 @@ __device__ __forceinline__ void route_body(const Shape &sh, int B, const Workspa
     // and do its own set-up (both instructions do nothing in a plain launch).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (zl.early && blockIdx.x == 0) {
-        // the expert kernel of this layer polls this word from the moment it is scheduled, which is
-        // after every block of this grid has passed the next instruction: the flag is down by then
-        if (tid == 0) {
-            asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(ws.early), "r"(0) : "memory");
+        // the expert kernel of this layer polls these words from the moment it is scheduled, which is
+        // after every block of this grid has passed the next instruction: they are cleared by then
+        if (tid < 8) {
+            asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(reinterpret_cast<unsigned long long *>(ws.early) + tid), "l"(0ull)
+                         : "memory");
             __threadfence();
         }
         __syncthreads();
