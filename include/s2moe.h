@@ -117,8 +117,11 @@ typedef struct {
     int32_t kernel_plan;   /* 0: automatic (plan 3 where it applies, else 2, else 1);
                               1: plain CUDA-core kernels (every format and batch size);
                               2: streaming mma.sync kernel (bf16 weights and activations);
-                              3: streaming tcgen05 kernel: bf16 activations with bf16 weights,
-                                 or with block-int4 weights when d_model, d_ff and
+                              3: streaming tcgen05 kernel: bf16 activations with bf16 weights
+                                 (the kernel then starts while the gating still runs, on the
+                                 shared experts and on every token's first expert by original
+                                 logit, which stays selected for alpha < 1: Sec. 4.2; not for
+                                 offloaded contexts), or with block-int4 weights when d_model, d_ff and
                                  d_ff_shared are multiples of 256 (the int4 values reach the
                                  tensor core as binary16 q * scale, rounded once: up to
                                  2^-12 relative per weight; block scales below 2^-17 lose
