@@ -154,19 +154,29 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, int bf
     p.rows1 = p.n1;    // the hidden-state k-tile of a stage in ONE copy (the producer is a single thread)
     // bf16 weights: TWO k-tiles per ring stage where every contraction length is a multiple of 64
     // (one weight copy of 32 KiB and one token copy per stage, one barrier round trip and five
-    // instead of six tensor-core instructions per issuer and 32 KiB): the producer and the MMA
-    // issuers are single threads, every instruction of theirs costs tens of cycles, and at
-    // 6 TB/s a 16 KiB k-tile has to leave an SM every 400 ns
+    // instead of six tensor-core instructions per issuer and 32 KiB).  The producer and the MMA
+    // issuers are single threads whose instructions cost tens of cycles each, and at 6 TB/s a
+    // 16 KiB k-tile has to leave an SM every 400 ns: with one k-tile per stage those loops are at
+    // their limit.  Measured (us per layer, one / two k-tiles per stage, resident hidden-state tiles
+    // in both where they fit): OLMoE shape 8 tokens 48.6 / 48.3, 16 tokens 55.7 / 53.6, 24 tokens
+    // 63.6 / 60.6; Qwen1.5-MoE shape 16 tokens 58.2 / 54.8; DeepSeek-V2-Lite shape 16 tokens 62.3 /
+    // 58.2, 64 tokens 121 / 109 (before the early start); a single token: 38.1 / 38.6, so the caller
+    // asks for it from two tokens on.  Three such stages beside the resident tiles beat five
+    // without them.
     if (bf16_kg == 2 && sh.weight_dtype == DT_BF16 && sh.d % 64 == 0 && sh.f % 64 == 0 && (sh.n_sh == 0 || sh.f_sh % 64 == 0)) {
         p.kg = 2;
-        p.x_bytes = 0;
         p.stage_bytes = (2 * kTcWTile + 2 * p.tokb + 1023) & ~1023;
         p.tok_off = 2 * kTcWTile;
-        p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
-        if (p.stages > kTcMaxStages) p.stages = kTcMaxStages;
-        p.smem_bytes = p.tab_bytes + p.stages * p.stage_bytes + 1024;
+        // (resident hidden-state tiles as above, if 3 of these stages fit beside them and no stage
+        // reaches past the last k-tile)
+        p.x_bytes = ((sh.d / 64) % 2 == 0) ? (sh.d / 64) * p.n1 * 128 : 0;
+        if ((kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes < 3) p.x_bytes = 0;
+        p.stages = (kTcMaxSmem - p.tab_bytes - 1024 - p.x_bytes) / p.stage_bytes;
+        if (p.stages > kTcRingDepth) p.stages = kTcRingDepth;
+        p.smem_bytes = p.tab_bytes + p.x_bytes + p.stages * p.stage_bytes + 1024;
         if (p.stages < 3) {          // (large batches: back to one k-tile per stage)
             p.kg = 1;
+            p.x_bytes = 0;
             p.stage_bytes = (kTcWTile + p.tokb + 1023) & ~1023;
             p.tok_off = kTcWTile;
             p.stages = (kTcMaxSmem - p.tab_bytes - 1024) / p.stage_bytes;
@@ -985,11 +995,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                     if (KGB == 2) {
                         // both k-tiles of the stage in one weight copy (a k-tile past the end of the
                         // contraction reads as zero) and one token copy (phase 2: one per 8 slots)
-                        const uint32_t op_bytes = t.phase == 1 ? 2u * (uint32_t)pl.tokb : 2u * (uint32_t)t.n * 128u;
+                        const uint32_t op_bytes = t.phase == 1 ? (pl.x_bytes ? 0u : 2u * (uint32_t)pl.tokb) : 2u * (uint32_t)t.n * 128u;
                         mbar_expect_tx(&full_bar[s], 2 * kTcWTile + op_bytes);
                         tma_load_3d_stream(stage, &maps.m[9 + (shared ? 3 : 0) + t.mat], 0, row0, kt, &full_bar[s], wpolicy);
                         if (t.phase == 1) {
-                            tma_load_3d(stage + pl.tok_off, &maps.m[6], 0, 0, kt, &full_bar[s]);
+                            if (!pl.x_bytes) tma_load_3d(stage + pl.tok_off, &maps.m[6], 0, 0, kt, &full_bar[s]);
                         } else if (ready) {
                             load_tokens2(s, kt, srow, shared, t.n);
                         } else {
@@ -1140,9 +1150,9 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                         // two weight k-tiles 16 KiB apart; their token tiles tokb apart (phase 1) or, per
                         // 8 slots, [hi | lo][k-tile][8 rows]: 8-row groups 2 KiB apart, k-tiles 1 KiB
                         const uint32_t a_lo = ring_lo + (uint32_t)s * ((uint32_t)pl.stage_bytes >> 4);
-                        const uint32_t b0 = a_lo + ((uint32_t)pl.tok_off >> 4);
-                        const bool p2 = t.phase == 2;
-                        const uint32_t b_step = p2 ? 64u : ((uint32_t)pl.tokb >> 4), b_hi = p2 ? hi_p2k : hi_std;
+                        const bool p2 = t.phase == 2, xr = !p2 && pl.x_bytes;       // (resident hidden-state tiles: n1 rows each)
+                        const uint32_t b0 = xr ? xres_lo + (uint32_t)kt * ((uint32_t)pl.n1 * 8u) : a_lo + ((uint32_t)pl.tok_off >> 4);
+                        const uint32_t b_step = p2 ? 64u : (xr ? (uint32_t)pl.n1 * 8u : ((uint32_t)pl.tokb >> 4)), b_hi = p2 ? hi_p2k : hi_std;
 #pragma unroll
                         for (uint32_t g = 0; g < 2; ++g)
                             for (uint32_t k = 0; k < ks; ++k) {

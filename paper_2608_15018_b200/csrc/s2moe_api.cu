@@ -45,7 +45,7 @@ struct s2moe_ctx {
     double *lpart = nullptr;              // partial router logits [piece][token][row] (logit pass by warp tasks)
     int route_task_from = 48;             // batches of this many tokens and more take the logit pass by warp tasks
     bool early_start = true;              // bf16 tensor-core plan: the expert kernel starts under the gating (S2MOE_NO_EARLY=1: off)
-    int bf16_kg2_from = 32;               // batches of this many tokens and more: two k-tiles per ring stage (bf16)
+    int bf16_kg2_from = 2;                // batches of this many tokens and more: two k-tiles per ring stage (bf16)
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
     void *encode_tiled = nullptr;         // cuTensorMapEncodeTiled, looked up through the runtime
@@ -581,7 +581,9 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
                                           (uint64_t)sh.f_sh, plane, (uint32_t)kg);
         } else if (plan == 3 && tp3.kg == 2) {
             // two k-tiles per stage: the token tiles of both in one copy (see make_map_ktiles)
-            ok = make_map_ktiles(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp3.tokb / 128, 2) &&
+            // (resident hidden-state tiles are loaded once, k-tile by k-tile, through the plain 2-D map)
+            ok = (tp3.x_bytes ? make_map(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp3.rows1)
+                              : make_map_ktiles(ctx, &maps.m[6], hidden, (uint64_t)B, (uint64_t)sh.d, (uint32_t)tp3.tokb / 128, 2)) &&
                  make_map_hilo_ktiles(ctx, &maps.m[7], ctx->act_hi, n_routed, (uint64_t)sh.f, plane, 2);
             if (ok && sh.n_sh)
                 ok = make_map_hilo_ktiles(ctx, &maps.m[8], ctx->act_hi + n_routed * sh.f, (uint64_t)sh.n_sh * B,
