@@ -63,15 +63,19 @@ constexpr int kTcKT = 4;                       // k-tiles (of 64) per unit: 64 K
 constexpr int kTcWTile = 128 * 128;            // bytes of one weight k-tile in shared memory
 constexpr int kTcMaxSmem = 232448 - 9216;      // dynamic shared memory; the rest is static (unit table, barriers)
 constexpr unsigned kTcSpinLimit = 1u << 22;
+constexpr int kTcMaxWaves = 3;                 // waves the experts are cut into at most (see the kernel)
 constexpr int kTcMaxAcc = 8;                   // accumulator buffers in tensor memory (2 without the early start)
 constexpr int kTcMaxUnits = 192;               // units of one CTA decoded once into shared memory
-// Share of the experts in wave 0.  A little more than half: the second projection of wave 0 is
-// what hides the hand-over of wave 1.  Measured again with the kernel as it stands, 16 layers of
-// the OLMoE-like shape: 0.7757 ms per step at 1/2, 0.7746 at 9/16, 0.7791 at 5/8, 0.7767 at 11/16,
-// 0.7830 at 3/4; 9/16 also takes 1 to 3 % off the shapes with shared experts and costs 0.7 % at
-// 64 tokens.
+// Share of the experts in wave 0 (by units of the first projection).  The second projection of
+// wave 0 is what hides the hand-over of wave 1, the first projection of wave 1 what hides that of
+// wave 0.  Measured with the kernel as it stands (early start, two k-tiles per stage), us per layer
+// at 6 / 7 / 8 / 9 / 10 / 11 sixteenths: OLMoE shape at 8 tokens 49.98 / 49.87 / 49.67 / 49.93 /
+// 49.94 / 50.41, DeepSeek-V2-Lite shape at 16 tokens 59.65 / 59.19 / 59.07 / 59.13 / 60.74 / 62.13,
+// Qwen1.5-MoE shape at 16 tokens 54.45 / 54.60 / 55.16 / 56.01 / 56.96 / 57.17; one wave: 52.8, 64.6,
+// 57.2; three waves (5 and 11, 4 and 10 sixteenths): 52.2 to 52.9 at the OLMoE shape (every
+// hand-over costs two grid-wide rounds and cuts accumulation runs), 58.6 to 58.8 at DeepSeek-V2-Lite.
 #ifndef S2MOE_SPLIT_NUM
-#define S2MOE_SPLIT_NUM 9
+#define S2MOE_SPLIT_NUM 7
 #define S2MOE_SPLIT_DEN 16
 #endif
 constexpr int kTcSplitNum = S2MOE_SPLIT_NUM, kTcSplitDen = S2MOE_SPLIT_DEN;
@@ -105,6 +109,7 @@ struct TcPlan {
     int rows1;         // rows of one hidden-state copy (bf16, one k-tile per stage)
     int n_acc;         // accumulator buffers (a power of two; more than 2 only with the early start)
     int early;         // the early start is possible for this shape (bf16 weights, units fit the table)
+    int split[2];      // where wave 1 and wave 2 begin, in 16ths of the first projection's units (16: no such wave)
 };
 
 struct TcArgs {
@@ -186,6 +191,8 @@ inline TcPlan tc_make_plan(const Shape &sh, int B, int n_sm, int n_slots, int bf
     }
     p.n_acc = 2;
     p.early = 0;
+    p.split[0] = kTcSplitNum * 16 / kTcSplitDen;
+    p.split[1] = 16;
     if (early && sh.weight_dtype == DT_BF16 && n_sm > 1) {
         // Early start (see the kernel): one CTA less than SMs, because the SM that runs the gating is
         // taken until the routing kernel ends and its CTA would start last with a full share; as many
@@ -497,16 +504,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 {
     extern __shared__ __align__(1024) uint8_t tc_smem[];
     __shared__ __align__(8) uint64_t full_bar[kTcMaxStages], empty_bar[kTcMaxStages];
-    __shared__ __align__(8) uint64_t acc_full[kTcMaxAcc], acc_empty[kTcMaxAcc], ep_bar, x_bar, cv_bar, conv_go[2], tab_bar;
+    __shared__ __align__(8) uint64_t acc_full[kTcMaxAcc], acc_empty[kTcMaxAcc], ep_bar, x_bar, cv_bar, conv_go[kTcMaxWaves], tab_bar;
     __shared__ __align__(8) uint64_t a_full[kTcMaxAStages], a_empty[kTcMaxAStages];   // int4: dequantised tiles
     __shared__ uint32_t s_tmem;
     __shared__ int s_flag;
     __shared__ TcUnit s_units[kTcMaxUnits];
     __shared__ uint32_t s_umeta[kTcMaxUnits];      // what an MMA issuer needs of a unit, in one word (tc_unit_meta)
-    __shared__ int s_split;                        // first active group of wave 1 (n_active: one wave)
+    __shared__ int s_split[2];                     // first active group of wave 1 and of wave 2 (n_active: no such wave)
     __shared__ unsigned s_early32[8];              // early start: the routing kernel's list of early experts, 32 per word
     __shared__ int s_tab[2];                       // early start: units of the routed work of this CTA, active groups
-    __shared__ volatile int s_ready[2];            // wave w's activations are written (set by the watcher warp)
+    __shared__ volatile int s_ready[kTcMaxWaves];  // wave w's activations are written (set by the watcher warp)
 
     const Shape &sh = p.sh;
     const Workspace &ws = p.ws;
@@ -526,7 +533,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             mbar_init(&acc_full[lane], NI);
             mbar_init(&acc_empty[lane], 4);
         }
-        if (lane < 2) mbar_init(&conv_go[lane], 4);
+        if (lane < kTcMaxWaves) mbar_init(&conv_go[lane], 4);
         if (Q4 && lane < pl.a_stages) {
             mbar_init(&a_full[lane], kTcQ4DeqWarps + 1);   // the dequantising warps and the producer's arrival with the token bytes
             mbar_init(&a_empty[lane], NI);
@@ -538,6 +545,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             mbar_init(&tab_bar, 1);
             s_ready[0] = 0;
             s_ready[1] = 0;
+            s_ready[2] = 0;
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -691,18 +699,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
 
     // ---- the tables of the routed work: by every thread of the CTA (tt, tn = thread, threads; hardware
     // barrier 0) or, with the early start, by warps 7..10 alone (barrier 1)
-    int n_active = 0, U = 0, total1 = 0, total2 = 0, a_split = 0, W = 1, n_main = 0;
-    int my_start0 = 0, my_start1 = 0, my_start2 = 0, my_start3 = 0, my_cnt0 = 0, my_cnt1 = 0, my_cnt2 = 0, my_cnt3 = 0;
-    int my_trim0 = 0, my_trim1 = 0, my_trim2 = 0, my_trim3 = 0;
-    // Four segments in time order: phase 1 of wave 0, of wave 1, phase 2 of wave 0, of wave 1.
+    int n_active = 0, U = 0, total1 = 0, total2 = 0, a_split = 0, a_split2 = 0, W = 1, n_main = 0;
+    int my_start[2 * kTcMaxWaves] = {0, 0, 0, 0, 0, 0}, my_cnt[2 * kTcMaxWaves] = {0, 0, 0, 0, 0, 0},
+        my_trim[2 * kTcMaxWaves] = {0, 0, 0, 0, 0, 0};
+    // 2 W segments in time order: phase 1 of waves 0 .. W - 1, then phase 2 of waves 0 .. W - 1.
     // Contiguous units are consecutive k-pieces of one 128-row block, so a CTA accumulates them in
     // one TMEM accumulator and the epilogue runs once per run of k-pieces instead of once per
     // unit; only row blocks cut by a CTA boundary are reduced from two CTAs.
     auto unit_make = [&](int i) -> TcUnit {
-        int seg = 0, j = i, start = my_start0, cnt = my_cnt0, trim = my_trim0;
-        if (j >= cnt) { j -= cnt; seg = 1; start = my_start1; cnt = my_cnt1; trim = my_trim1; }
-        if (seg == 1 && j >= cnt) { j -= cnt; seg = 2; start = my_start2; cnt = my_cnt2; trim = my_trim2; }
-        if (seg == 2 && j >= cnt) { j -= cnt; seg = 3; start = my_start3; cnt = my_cnt3; trim = my_trim3; }
+        int seg = 0, j = i;
+        while (seg < 2 * W - 1 && j >= my_cnt[seg]) { j -= my_cnt[seg]; ++seg; }
+        const int start = my_start[seg], cnt = my_cnt[seg], trim = my_trim[seg];
         TcUnit t = tc_decode(groups, n_active, total1, start + j, sh.d, pl.n1);
         const int K = t.phase == 1 ? sh.d : groups[t.a].f;
         if (j == 0 && (trim & 1)) t.kt0 += kTcKT / 2;            // the CTA before this one has the first half
@@ -746,29 +753,41 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         total1 = EARLY ? max(0, U - ne) * u1r : U * u1r + sh.n_sh * u1s;
         total2 = U * u2r + sh.n_sh * u2s;
         if (tt == 0) {
-            // wave 1 starts at the first group whose first-projection units (pre-lot included) begin at
-            // or after that share of all of them
-            int sp = n_active;
-            if (n_active >= 2) {
-                sp = 1;
-                while (sp < n_active - 1) {
-                    const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
-                    if ((long long)(r * u1r + q * u1s) * kTcSplitDen >= (long long)(U * u1r + sh.n_sh * u1s) * kTcSplitNum) break;
-                    ++sp;
+            // wave w starts at the first group whose first-projection units (pre-lot included) begin at
+            // or after its share of all of them (in 16ths: pl.split[w - 1]; 16: no such wave)
+            int sp = 0;
+            for (int w = 0; w < 2; ++w) {
+                if (pl.split[w] >= 16 || n_active < 2) sp = n_active;
+                else {
+                    if (sp < 1) sp = 1;
+                    if (w == 1 && sp < n_active) ++sp;   // (a wave has at least one group)
+                    while (sp < n_active - 1) {
+                        const int r = sp < U ? sp : U, q = sp < U ? 0 : sp - U;
+                        if ((long long)(r * u1r + q * u1s) * 16 >= (long long)(U * u1r + sh.n_sh * u1s) * pl.split[w]) break;
+                        ++sp;
+                    }
+                    if (sp > n_active) sp = n_active;
                 }
+                s_split[w] = sp;
             }
-            s_split = sp;
         }
         asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(tn) : "memory");
-        a_split = s_split;
-        W = a_split < n_active ? 2 : 1;
-        const int split1 = W == 2 ? groups[a_split].p1 : total1;
-        const int split2 = W == 2 ? groups[a_split].p2 : total2;
-        share(0, split1, halves1, my_start0, my_cnt0, my_trim0);
-        share(split1, total1 - split1, halves1, my_start1, my_cnt1, my_trim1);
-        share(total1, split2, halves2, my_start2, my_cnt2, my_trim2);
-        share(total1 + split2, total2 - split2, halves2, my_start3, my_cnt3, my_trim3);
-        n_main = my_cnt0 + my_cnt1 + my_cnt2 + my_cnt3;
+        a_split = s_split[0];
+        a_split2 = s_split[1];
+        W = 1 + (a_split < n_active ? 1 : 0) + (a_split2 < n_active ? 1 : 0);
+        {
+            // first unit of every wave in both projections
+            int b1[kTcMaxWaves + 1], b2[kTcMaxWaves + 1];
+            b1[0] = 0; b2[0] = 0;
+            b1[1] = a_split < n_active ? groups[a_split].p1 : total1;  b2[1] = a_split < n_active ? groups[a_split].p2 : total2;
+            b1[2] = a_split2 < n_active ? groups[a_split2].p1 : total1; b2[2] = a_split2 < n_active ? groups[a_split2].p2 : total2;
+            b1[W] = total1; b2[W] = total2;
+            n_main = 0;
+            for (int w = 0; w < W; ++w) share(b1[w], b1[w + 1] - b1[w], halves1, my_start[w], my_cnt[w], my_trim[w]);
+            for (int w = 0; w < W; ++w)
+                share(total1 + b2[w], b2[w + 1] - b2[w], halves2, my_start[W + w], my_cnt[W + w], my_trim[W + w]);
+            for (int g = 0; g < 2 * W; ++g) n_main += my_cnt[g];
+        }
         if (EARLY && n_pre + n_main > kTcMaxUnits) {  // (see above: left off by the host)
             if (tt == 0) atomicExch(ws.status, ST_BAD_PLAN);
             n_main = kTcMaxUnits - n_pre;
@@ -803,11 +822,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
     const uint32_t tmem_base = s_tmem;
     // What a role knows of the tables: everything at once, or (early start) after tab_bar.  The
     // roles keep their own copies (lim: units of this CTA known so far).
-    auto tables_wait = [&](int &lim, int &split, int &waves) -> bool {
+    auto tables_wait = [&](int &lim, int &split, int &split2, int &waves) -> bool {
         if (!mbar_wait(&tab_bar, 0)) { atomicExch(ws.status, ST_MBAR_TIMEOUT); return false; }
         lim = n_pre + s_tab[0];
-        split = s_split;
-        waves = split < s_tab[1] ? 2 : 1;
+        split = s_split[0];
+        split2 = s_split[1];
+        waves = 1 + (split < s_tab[1] ? 1 : 0) + (split2 < s_tab[1] ? 1 : 0);
         return true;
     };
     const int n_units0 = EARLY ? n_pre : n_main;      // units known when the roles start
@@ -945,14 +965,14 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             int s = 0;                                   // ring slot of the next k-tile
             uint32_t ring_par = 1;                       // parity to wait for on its empty barrier
 
-            int lim = n_units0, a_split_p = a_split, w_p = W;
+            int lim = n_units0, a_split_p = a_split, a_split2_p = a_split2, w_p = W;
             bool tabs = !EARLY;
             for (int i = 0; alive; ++i) {
                 if (i >= lim) {
                     // (early start: the pre-lot is on its way; the rest needs the tables)
                     if (tabs) break;
                     tabs = true;
-                    if (!tables_wait(lim, a_split_p, w_p)) { alive = false; break; }
+                    if (!tables_wait(lim, a_split_p, a_split2_p, w_p)) { alive = false; break; }
                     if (i >= lim) break;
                 }
 
@@ -964,7 +984,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 const int rows_per_e = t.mat == 2 ? sh.d : g.f;
                 const int row0 = e * rows_per_e + t.rb * 128;
                 const int srow = shared ? g.off - n_routed : g.off;   // row in the routed / shared activation array
-                const int wv = t.a >= a_split_p ? 1 : 0;
+                const int wv = (t.a >= a_split_p ? 1 : 0) + (t.a >= a_split2_p ? 1 : 0);
                 bool ready = t.phase == 1 || wv < ready_w;
                 if (!ready) {
                     // the pending tiles all belong to one wave (pend_wave); if that is an earlier wave than
@@ -1114,10 +1134,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             } else
             for (int lim = n_units0, tabs = EARLY ? 0 : 1; alive; ++ui) {
                 if ((int)ui >= lim) {
-                    int sp_, w_;
+                    int sp_, sp2_, w_;
                     if (tabs) break;
                     tabs = 1;
-                    if (!tables_wait(lim, sp_, w_) || (int)ui >= lim) break;
+                    if (!tables_wait(lim, sp_, sp2_, w_) || (int)ui >= lim) break;
                 }
                 const TcUnit t = unit_at((int)ui);
                 const int buf = run & nbm;
@@ -1307,7 +1327,11 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         uint32_t ep_phase = 0;                         // running parity of cv_bar
         uint64_t *ep_bar_p = &cv_bar;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
-        const long long el_split = W == 2 ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
+        long long el_b[kTcMaxWaves + 1];             // first element of every wave's activations
+        el_b[0] = 0;
+        el_b[1] = a_split < n_active ? (long long)act_offset(groups[a_split].off, n_routed, sh.f, sh.f_sh) : n_el;
+        el_b[2] = a_split2 < n_active ? (long long)act_offset(groups[a_split2].off, n_routed, sh.f, sh.f_sh) : n_el;
+        el_b[W] = n_el;
 
         auto wave_convert = [&](int w) -> bool {
 
@@ -1328,7 +1352,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             // pre holds a gate plane and an up plane, both indexed exactly like the activations
             // (act_offset(slot) + row): this CTA converts a contiguous slice of the wave's range,
             // four elements per thread and step
-            const long long w_lo = w == 0 ? 0 : el_split, w_hi = (w == 0 && W == 2) ? el_split : n_el;
+            const long long w_lo = el_b[w], w_hi = el_b[w + 1];
             const long long n4 = (w_hi - w_lo) >> 2;
             const long long lo4 = n4 * blockIdx.x / gridDim.x, hi4 = n4 * (blockIdx.x + 1) / gridDim.x;
             for (long long q = lo4 + et; q < hi4; q += 96) {
@@ -1395,10 +1419,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         (void)n_routed_el;
         const long long n_el = (long long)n_routed * sh.f + (long long)sh.n_sh * p.B * sh.f_sh;
         int next_arrive = 0;
-        int lim = n_units0, a_split_e = a_split, w_e = W;
+        int lim = n_units0, a_split_e = a_split, a_split2_e = a_split2, w_e = W;
         bool tabs = !EARLY;
         const unsigned nbm = (unsigned)pl.n_acc - 1u, nbs = (unsigned)__ffs(pl.n_acc) - 1u;
-        (void)a_split_e;
+        (void)a_split_e; (void)a_split2_e;
         auto wave_arrive = [&](int w) -> bool {
             // this CTA's phase-1 reductions of wave w are issued: hand over to the converter warps,
             // whose first thread orders them (fence) before it arrives on the grid-wide counter, so
@@ -1413,8 +1437,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         // called before every unit (and once at the end): hand a wave over once this CTA's phase-1
         // units of it are all done
         auto service = [&](int upcoming_seg) -> bool {
-            const int seg_wave1 = w_e == 2 ? 1 : 2;      // first segment that lies after phase 1 of wave 0
-            while (next_arrive < w_e && upcoming_seg >= (next_arrive == 0 ? seg_wave1 : 2)) {
+            // (segment w is phase 1 of wave w: it is done once a later segment comes up)
+            while (next_arrive < w_e && upcoming_seg > next_arrive) {
                 if (!wave_arrive(next_arrive)) return false;
                 ++next_arrive;
             }
@@ -1425,7 +1449,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 if ((int)ui >= lim) {
                     if (tabs) break;
                     tabs = true;
-                    if (!tables_wait(lim, a_split_e, w_e)) { alive = false; break; }
+                    if (!tables_wait(lim, a_split_e, a_split2_e, w_e)) { alive = false; break; }
                     if ((int)ui >= lim) break;
                 }
                 const TcUnit t = unit_at((int)ui);
@@ -1434,7 +1458,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 if (!tabs && t.a < GP) {
                     // an early routed expert of the pre-lot: its tokens and slots come with the tables
                     tabs = true;
-                    if (!tables_wait(lim, a_split_e, w_e)) { alive = false; break; }
+                    if (!tables_wait(lim, a_split_e, a_split2_e, w_e)) { alive = false; break; }
                 }
                 const TcGroup &g = groups[t.a];
                 const int buf = run & nbm;
@@ -1501,7 +1525,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
                 ++run;
 
             }
-            if (alive && !service(4)) alive = false;
+            if (alive && !service(2 * kTcMaxWaves)) alive = false;
         }
 
     }

@@ -45,6 +45,7 @@ struct s2moe_ctx {
     double *lpart = nullptr;              // partial router logits [piece][token][row] (logit pass by warp tasks)
     int route_task_from = 48;             // batches of this many tokens and more take the logit pass by warp tasks
     bool early_start = true;              // bf16 tensor-core plan: the expert kernel starts under the gating (S2MOE_NO_EARLY=1: off)
+    int wave_split[2] = {0, 16};          // S2MOE_WAVES=a,b: where waves 1 and 2 of the bf16 expert kernel begin (16ths; 0: the built-in)
     int bf16_kg2_from = 2;                // batches of this many tokens and more: two k-tiles per ring stage (bf16)
     float *pre = nullptr;                 // plan 3: fp32 pre-activations [gate|up][slot][f]
     std::vector<TcMaps> tc_maps;          // plan 3: per layer, weight maps filled at create
@@ -536,7 +537,8 @@ int verify_one(s2moe_ctx *ctx, int layer, int B, const void *hidden, const float
     // experts the routing kernel announces before it (not with offloaded experts: their weights are
     // fetched between the two kernels)
     const bool want_early = plan == 3 && ctx->early_start && ctx->use_pdl && !ctx->offload && sh.weight_dtype == DT_BF16;
-    const TcPlan tp3 = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B, B >= ctx->bf16_kg2_from ? 2 : 1, want_early);
+    TcPlan tp3 = tc_make_plan(sh, B, ctx->n_sm, B * sh.k + sh.n_sh * B, B >= ctx->bf16_kg2_from ? 2 : 1, want_early);
+    if (sh.weight_dtype == DT_BF16 && ctx->wave_split[0] > 0) { tp3.split[0] = ctx->wave_split[0]; tp3.split[1] = ctx->wave_split[1]; }
     // what the FFN kernels accumulate into is cleared by the routing kernel's blocks
     ZeroList zl{};
     zl.ptr[0] = out;
@@ -735,6 +737,11 @@ int create_impl(const s2moe_config *config, const s2moe_layer_weights *layers, i
         if (tf && tf[0]) ctx->route_task_from = std::atoi(tf);
         const char *pg = std::getenv("S2MOE_PDL_IN_GRAPH");
         ctx->pdl_in_graph = pg && pg[0] == '1';
+        const char *wv = std::getenv("S2MOE_WAVES");
+        if (wv && wv[0]) {
+            int a = 0, b = 16;
+            if (std::sscanf(wv, "%d,%d", &a, &b) >= 1 && a > 0 && a <= 16 && b >= a && b <= 16) { ctx->wave_split[0] = a; ctx->wave_split[1] = b; }
+        }
         const char *ne = std::getenv("S2MOE_NO_EARLY");
         ctx->early_start = !(ne && ne[0] == '1');
     }
