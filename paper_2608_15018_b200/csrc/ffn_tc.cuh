@@ -1355,33 +1355,46 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
             const long long w_lo = el_b[w], w_hi = el_b[w + 1];
             const long long n4 = (w_hi - w_lo) >> 2;
             const long long lo4 = n4 * blockIdx.x / gridDim.x, hi4 = n4 * (blockIdx.x + 1) / gridDim.x;
-            for (long long q = lo4 + et; q < hi4; q += 96) {
-                const long long i = w_lo + 4 * q;
-                const float4 gv = __ldcg(reinterpret_cast<const float4 *>(p.pre + i));
-                const float4 uv = __ldcg(reinterpret_cast<const float4 *>(p.pre + n_el + i));
-                const float a0 = silu_mul(gv.x, uv.x), a1 = silu_mul(gv.y, uv.y), a2 = silu_mul(gv.z, uv.z),
-                            a3 = silu_mul(gv.w, uv.w);
-                if (Q4) {
-                    // binary16 hi + lo parts (the int4 path's operand format).  Columns i .. i + 3 of
-                    // their group of 8 go to positions 0, 2, 4, 6 (first half of the group) or
-                    // 1, 3, 5, 7 (second half): the order the dequantised weights are in
-                    const __half2 h01 = __floats2half2_rn(a0, a1), h23 = __floats2half2_rn(a2, a3);
-                    const __half2 l01 = __floats2half2_rn(a0 - __low2float(h01), a1 - __high2float(h01));
-                    const __half2 l23 = __floats2half2_rn(a2 - __low2float(h23), a3 - __high2float(h23));
-                    const long long g8 = i & ~7ll;
-                    const int odd = (int)((i >> 2) & 1);
-                    __half *ph = reinterpret_cast<__half *>(p.act_hi) + g8 + odd, *pq = reinterpret_cast<__half *>(p.act_lo) + g8 + odd;
-                    ph[0] = __low2half(h01); ph[2] = __high2half(h01); ph[4] = __low2half(h23); ph[6] = __high2half(h23);
-                    pq[0] = __low2half(l01); pq[2] = __high2half(l01); pq[4] = __low2half(l23); pq[6] = __high2half(l23);
-                } else {
-                    const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
-                    const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
-                    const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
-                    uint2 hv, lv;
-                    hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
-                    lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
-                    *reinterpret_cast<uint2 *>(p.act_hi + i) = hv;
-                    *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
+            // eight loads in flight per thread (a slice is up to 13 passes of the 96 threads at 64 tokens:
+            // one pass at a time was 1 us of memory latency each, on the hand-over's critical path)
+            for (long long q0 = lo4 + et; q0 < hi4; q0 += 96 * 4) {
+                float4 gv[4], uv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const long long q = q0 + 96 * u, i = w_lo + 4 * q;
+                    if (q < hi4) {
+                        gv[u] = __ldcg(reinterpret_cast<const float4 *>(p.pre + i));
+                        uv[u] = __ldcg(reinterpret_cast<const float4 *>(p.pre + n_el + i));
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const long long q = q0 + 96 * u, i = w_lo + 4 * q;
+                    if (q >= hi4) continue;
+                    const float a0 = silu_mul(gv[u].x, uv[u].x), a1 = silu_mul(gv[u].y, uv[u].y), a2 = silu_mul(gv[u].z, uv[u].z),
+                                a3 = silu_mul(gv[u].w, uv[u].w);
+                    if (Q4) {
+                        // binary16 hi + lo parts (the int4 path's operand format).  Columns i .. i + 3 of
+                        // their group of 8 go to positions 0, 2, 4, 6 (first half of the group) or
+                        // 1, 3, 5, 7 (second half): the order the dequantised weights are in
+                        const __half2 h01 = __floats2half2_rn(a0, a1), h23 = __floats2half2_rn(a2, a3);
+                        const __half2 l01 = __floats2half2_rn(a0 - __low2float(h01), a1 - __high2float(h01));
+                        const __half2 l23 = __floats2half2_rn(a2 - __low2float(h23), a3 - __high2float(h23));
+                        const long long g8 = i & ~7ll;
+                        const int odd = (int)((i >> 2) & 1);
+                        __half *ph = reinterpret_cast<__half *>(p.act_hi) + g8 + odd, *pq = reinterpret_cast<__half *>(p.act_lo) + g8 + odd;
+                        ph[0] = __low2half(h01); ph[2] = __high2half(h01); ph[4] = __low2half(h23); ph[6] = __high2half(h23);
+                        pq[0] = __low2half(l01); pq[2] = __high2half(l01); pq[4] = __low2half(l23); pq[6] = __high2half(l23);
+                    } else {
+                        const __nv_bfloat162 h01 = __floats2bfloat162_rn(a0, a1), h23 = __floats2bfloat162_rn(a2, a3);
+                        const __nv_bfloat162 l01 = __floats2bfloat162_rn(a0 - __low2float(h01), a1 - __high2float(h01));
+                        const __nv_bfloat162 l23 = __floats2bfloat162_rn(a2 - __low2float(h23), a3 - __high2float(h23));
+                        uint2 hv, lv;
+                        hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+                        lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+                        *reinterpret_cast<uint2 *>(p.act_hi + i) = hv;
+                        *reinterpret_cast<uint2 *>(p.act_lo + i) = lv;
+                    }
                 }
             }
             // the activations are read by TMA copies of other CTAs: proxy fence over global memory by
