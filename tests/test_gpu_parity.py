@@ -330,12 +330,14 @@ def test_early_start_on_and_off(name, B, monkeypatch):
     assert torch.equal(got["0"].sel_w, got["1"].sel_w)
 
 
-def test_graph_replay_with_changing_inputs():
+@pytest.mark.parametrize("name,B", [("cfg5", 16), ("cfg2", 8), ("cfg5", 64)])
+def test_graph_replay_with_changing_inputs(name, B):
     """A captured stack replayed on other inputs: the words the two kernels of a layer meet on (the
-    routing kernel's arrival counter, the early list and its flag) carry nothing over from one replay
-    to the next.  Every replay against the oracle."""
-    wl = SMALL["cfg5"]
-    L, B = 3, 16
+    routing kernel's arrival counter, the early list and its tag) carry nothing over from one replay
+    to the next.  Every replay against the oracle.  (With and without shared experts; 64 tokens take
+    the routing kernel for large batches.)"""
+    wl = SMALL[name]
+    L = 3
     m, T = _ctx(wl, L, 0)
     dev = torch.device("cuda", 0)
     H = torch.stack([workloads.hidden_states(wl, l, B, 0.5, dev) for l in range(L)])
