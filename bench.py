@@ -294,7 +294,9 @@ def measure_stack(wl, B, sigma, L, plan, steps, warmup, dev, rank, world, peak, 
                     break
             graph_ms = statistics.median(graph_all)
             timed_path = (f"CUDA graph replay of one s2moe_verify_stack call per step; median of {reps} repeats of "
-                          f"{steps} steps ({done_s:.2f} s timed)")
+                          f"{steps} steps ({done_s:.2f} s timed); the graph keeps the programmatic launch edges, so with "
+                          f"bf16 weights the expert kernel of a layer starts while that layer's gating still runs "
+                          f"(the per-kernel durations of region B are taken with event pairs, which serialise the two)")
     except Exception as exc:  # pragma: no cover
         graph_ms = None
         print(f"graph replay skipped: {exc}", file=sys.stderr)
