@@ -643,13 +643,16 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs p)
         for (int j = tid; j < n_early + sh.n_sh; j += blockDim.x) {
             TcGroup gr;
             if (j < n_early) {
-                int rem = j, id = 0;
+                // the j-th expert of the list: its word first, then its bit by clearing the rem bits below it
+                int rem = j, wq = 0;
+                unsigned wbits = ew[0];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {            // the j-th expert of the list
+                for (int q = 0; q < 7; ++q) {
                     const int c = __popc(ew[q]);
-                    if (rem >= 0 && rem < c) id = 32 * q + (int)__fns(ew[q], 0u, rem + 1);
-                    rem -= c;
+                    if (wq == q && rem >= c) { rem -= c; wq = q + 1; wbits = ew[q + 1]; }
                 }
+                for (int t = 0; t < rem; ++t) wbits &= wbits - 1u;
+                const int id = 32 * wq + __ffs(wbits) - 1;
                 gr.mask = 0ull; gr.group = id; gr.T = 0; gr.off = 0; gr.f = sh.f;
                 gr.p1 = sh.n_sh * u1s + j * u1r; gr.p2 = 0;
                 groups[j] = gr;
